@@ -1,0 +1,187 @@
+/*
+ * compkv.h -- C ABI of the CompKV decode-step library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the decode hot path of compensation-aware block-sparse
+ * attention over a paged KV cache:
+ *   per-block summaries {|b|, mean key, grouped key variance, mean value}  (Sec. 4.1-4.2, Eq. 8)
+ *   -> per-query block score S_b = sum_g phat_{g,b} * sigma_hat^2_{g,b}    (Eq. 8-10)
+ *   -> mandatory blocks + stable top-k under a token budget                (Eq. 11)
+ *   -> exact attention on the selected blocks, block-mean compensation for
+ *      every other block, one shared softmax normaliser                    (Eq. 12)
+ * plus a dense decode attention over the same cache (Eq. 12 with every block selected).
+ *
+ * Conventions
+ *   - Every pointer documented "device" is device memory owned by the caller; "host" is
+ *     host memory.  The library allocates NO device memory: summaries and scratch live in
+ *     two caller-provided device buffers sized by ckv_query_sizes().  A ckv_ctx is a small
+ *     host object.
+ *   - All calls that take a stream enqueue work on it and return without synchronising
+ *     (ckv_step_host and ckv_read_status synchronise the stream before returning).
+ *   - Return value: 0 (CKV_OK) or a negative ckv_status.  Nothing throws or aborts.
+ *     Problems only the device can see (a page id outside the pool, a sequence that outgrew
+ *     its page table, a non-finite score) set a bit in a device status word and the
+ *     offending access is skipped; read it with ckv_read_status().
+ *   - One "unit" = one sequence x one KV head, with the G = num_q_heads / num_kv_heads query
+ *     heads that share it; a selected block set is shared by those G heads (Sec. 3.1).
+ *   - Blocks are cut from token 0 in fixed size block_size; the last block of a sequence may
+ *     be partial.  X_s = ceil(N_s / block_size) blocks in sequence s.
+ *
+ * Tensor layouts (row-major, innermost last)
+ *   K / V pools  [num_pages][num_kv_heads][page_size][head_dim]   kv_dtype (bf16, or fp32 in the debug layout)
+ *   page_table   [batch][max_pages_per_seq] int32, max_pages_per_seq = max_blocks_per_seq * block_size / page_size
+ *   seq_lens     [batch] int32
+ *   q, out       [batch][num_q_heads][head_dim]                   kv_dtype
+ *   k_new, v_new [batch][num_kv_heads][head_dim]                  kv_dtype
+ *   sel_ids      [batch][num_kv_heads][K_cap] int32, K_cap = budget_tokens / block_size, ascending, padded with -1
+ *   sel_cnt      [batch][num_kv_heads] int32
+ *   lse          [batch][num_q_heads] fp32 (natural log of the shared normaliser), may be NULL
+ */
+#ifndef COMPKV_H_
+#define COMPKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *ckv_stream;   /* a cudaStream_t */
+typedef struct ckv_ctx ckv_ctx;
+
+enum ckv_dtype { CKV_BF16 = 0, CKV_F32 = 1 };
+
+enum ckv_status {
+  CKV_OK = 0,
+  CKV_ERR_INVALID_ARG = -1,       /* NULL pointer, batch out of range, ... */
+  CKV_ERR_BAD_LAYOUT = -2,        /* a ckv_layout field outside what the kernels support */
+  CKV_ERR_BUDGET_TOO_SMALL = -3,  /* budget cannot hold the mandatory blocks (Eq. 11 needs K >= |F|) */
+  CKV_ERR_CAPACITY = -4,          /* a caller buffer is smaller than ckv_query_sizes() asks for */
+  CKV_ERR_CUDA = -5,              /* a CUDA runtime call failed; ckv_last_cuda_error() has the code */
+  CKV_ERR_TIMEOUT = -6            /* reserved: a bounded device-side wait ran out */
+};
+
+/* bits of the device status word */
+enum ckv_device_status {
+  CKV_DEV_BAD_PAGE = 1,     /* page table entry outside [0, num_pages): the page was skipped */
+  CKV_DEV_SEQ_FULL = 2,     /* append past max_blocks_per_seq * block_size: the token was dropped */
+  CKV_DEV_NONFINITE = 4     /* a block score was NaN/Inf: it was ranked as 0 */
+};
+
+typedef struct ckv_layout {
+  int32_t num_q_heads;        /* multiple of num_kv_heads; G = ratio in {1, 2, 4, 8} */
+  int32_t num_kv_heads;
+  int32_t head_dim;           /* 128 */
+  int32_t block_size;         /* 16, 32 or 64 tokens; multiple of page_size (Sec. 5.1 uses 16) */
+  int32_t page_size;          /* 16 */
+  int32_t var_groups;         /* r of Eq. 8: a power of two dividing head_dim/2, or head_dim */
+  int32_t group_layout;       /* coordinate groups of App. A.4: 0 = RoPE pair p is (2p, 2p+1), i.e. groups are
+                                 contiguous coordinate ranges; 1 = pair p is (p, p + head_dim/2) */
+  int32_t kv_dtype;           /* CKV_BF16, or CKV_F32 (debug layout: fp32 pools, q and out) */
+  int32_t max_batch;
+  int32_t max_blocks_per_seq; /* page-table row stride is max_blocks_per_seq * block_size / page_size */
+  int32_t num_pages;          /* pages in each pool; page ids are range-checked against it */
+  int32_t sink_blocks;        /* mandatory leading blocks (Sec. 4.2: 1) */
+  int32_t recent_blocks;      /* mandatory trailing blocks (Sec. 4.2: 2) */
+  float   sm_scale;           /* logit scale; 0 means 1/sqrt(head_dim) (Sec. 3.1) */
+} ckv_layout;
+
+/* Library version (major * 100 + minor). */
+int ckv_version(void);
+
+/* Human-readable name of a ckv_status (static storage). */
+const char *ckv_strerror(int status);
+
+/* cudaError_t of the last failed CUDA call made by this library on the calling thread (0 if none). */
+int ckv_last_cuda_error(void);
+
+/* Sizes in bytes of the two device buffers a context needs (Sec. 4.2: 2d + r + 1 scalars per
+ * block; the count |b| is implied by seq_lens, so 2d + r fp32 scalars are stored).
+ * stats_bytes: block summaries for max_batch sequences.  workspace_bytes: scratch for one
+ * decode step at max_batch (block log-weights, scores, split partials, host staging).
+ * Host-only; validates the layout (CKV_ERR_BAD_LAYOUT). */
+int ckv_query_sizes(const ckv_layout *layout, size_t *stats_bytes, size_t *workspace_bytes);
+
+/* Byte offsets, inside the stats buffer, of its three regions (the "selection region" holds
+ * mean keys and grouped variances, the "mean-values region" the mean values; Sec. 4.3):
+ *   kmean [max_batch][num_kv_heads][max_blocks_per_seq][head_dim] fp32
+ *   dbar  [max_batch][num_kv_heads][max_blocks_per_seq][var_groups] fp32
+ *   vmean [max_batch][num_kv_heads][max_blocks_per_seq][head_dim] fp32
+ * Host-only. */
+int ckv_stats_offsets(const ckv_layout *layout, size_t *kmean_off, size_t *dbar_off, size_t *vmean_off);
+
+/* Create a context over caller-owned device buffers (256-byte aligned, at least the sizes
+ * ckv_query_sizes() returned; the buffers must outlive the context).  Clears the device
+ * status word on `stream`.  *out receives a host object to be freed with ckv_destroy(). */
+int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, void *work_dev,
+               size_t work_bytes, ckv_stream stream, ckv_ctx **out);
+void ckv_destroy(ckv_ctx *ctx);
+
+/* Build the summaries of every block of `batch` prefilled sequences from the paged cache
+ * (Eq. 8 right half; Sec. 4.2): |b|, mean key, mean value and, per coordinate group, the
+ * population variance of the keys around the block mean (two passes, fp32 accumulation).
+ * Sequence s of this call uses summary rows of batch slot s.
+ * max_seq_len_host: an upper bound (host) on seq_lens[s], used only to size the grid. */
+int ckv_stats_build(ckv_ctx *ctx, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                    const int32_t *seq_lens, int batch, int max_seq_len_host, ckv_stream stream);
+
+/* Append one token per sequence (Sec. 4.2 "updated incrementally", App. D.1): writes
+ * k_new / v_new at position seq_lens[s] of the paged cache, recomputes the summary of the
+ * active (last) block from its resident tokens with the same arithmetic as ckv_stats_build
+ * (so build(N) + appends == build(N + m) bit for bit), leaves completed blocks untouched, and
+ * increments seq_lens[s].  The page table must already map the page of the new position. */
+int ckv_append(ckv_ctx *ctx, void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens,
+               const void *k_new, const void *v_new, int batch, ckv_stream stream);
+
+/* One compensated sparse decode step (Eq. 8-12) for `batch` sequences, one query token each.
+ *   budget_tokens: exact-read budget in tokens, mandatory blocks included (Sec. 5.1);
+ *                  K = budget_tokens / block_size blocks; K >= X_s selects every block of s,
+ *                  which makes the result dense attention.
+ *   out:     attention output, kv_dtype (fp32 accumulation, rounded once; App. D.1).
+ *   sel_ids: selected block ids per unit in position order; sel_cnt their number.
+ * The cache is read through page_table; summaries must be current (build / append).
+ * Returns CKV_ERR_BUDGET_TOO_SMALL when K < sink_blocks + recent_blocks and K * block_size <
+ * max_seq_len_host (some sequence could not hold its mandatory blocks). */
+int ckv_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_pool,
+               const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
+               int budget_tokens, void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt,
+               ckv_stream stream);
+
+/* ckv_decode with CUDA events recorded on `stream` between its four kernels (summary scan, score +
+ * top-k selection, exact attention on the selected blocks, merge).  Waits for the step to finish and
+ * writes the four durations in milliseconds to stage_ms_host[0..3] (host).  For measurement only. */
+int ckv_decode_profile(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_pool,
+                       const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
+                       int budget_tokens, void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt,
+                       ckv_stream stream, float *stage_ms_host);
+
+/* Dense decode attention over the whole paged cache (Sec. 3.1; Eq. 12 with S = all blocks),
+ * split along the sequence with a log-sum-exp merge.  Same tile code as the sparse path. */
+int ckv_dense_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_pool,
+                     const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
+                     void *out, float *lse, ckv_stream stream);
+
+/* Copy the block scores S_b of the last ckv_decode (Eq. 10) into dst (device),
+ * fp32 [batch][num_kv_heads][max_blocks_per_seq]; entries at or past X_s are unspecified.
+ * Mandatory blocks carry their score too (they are excluded from the ranking, not from Eq. 9). */
+int ckv_copy_scores(ckv_ctx *ctx, float *dst, int batch, ckv_stream stream);
+
+/* One whole decode step from HOST buffers: copies q, k_new, v_new to the device, runs
+ * ckv_append then ckv_decode, copies out / sel_ids / sel_cnt back and synchronises the stream.
+ * Host buffers should be pinned; device staging comes out of the workspace.  seq_lens (device)
+ * is incremented.  max_seq_len_host bounds the lengths AFTER the append. */
+int ckv_step_host(ckv_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
+                  void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens, int batch,
+                  int max_seq_len_host, int budget_tokens, void *out_host, int32_t *sel_ids_host,
+                  int32_t *sel_cnt_host, ckv_stream stream);
+
+/* Read and clear the device status word (bits of ckv_device_status); synchronises `stream`. */
+int ckv_read_status(ckv_ctx *ctx, int32_t *host_status, ckv_stream stream);
+
+/* Number of kernel launches the library has enqueued through this context so far. */
+int64_t ckv_launch_count(const ckv_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMPKV_H_ */

@@ -110,7 +110,9 @@ void ckvo_stats(const float *K, const float *V, int N, int d, int bs, int r, int
 }
 
 /* Scorer (Eq. 8 left half, Eq. 9, Eq. 10).  All outputs [G][X] except S [X].
- * sigma2_{g,b} = (1/d) sum_t (sum_{i in G_t} q_{g,i}^2) Dbar_{b,t}
+ * sigma2_{g,b} = scale^2 sum_t (sum_{i in G_t} q_{g,i}^2) Dbar_{b,t}
+ *                (Eq. 8 prints 1/d: App. A.4 obtains it from z - zbar = q (k - kbar)^T / sqrt(d), i.e. it is the
+ *                 squared logit scale, which is 1/d for the default scale)
  * zbar_{g,b}   = q_g . kbar_b * scale
  * phat_{g,b}   = |b| exp(zbar + sigma2/2) / sum_c |c| exp(zbar_c + sigma2_c/2)   (over all blocks)
  * S_b          = sum_g phat_{g,b} sigma2_{g,b}.
@@ -134,7 +136,7 @@ void ckvo_scores(const float *q, const int *cnt, const double *kmean, const doub
             zb[b] = acc * scale;
             double v = 0.0;
             for (int t = 0; t < r; ++t) v += w[t] * Dbar[(size_t)b * r + t];
-            s2[b] = v / d;
+            s2[b] = v * scale * scale;
             double l = log((double)cnt[b]) + zb[b] + (mass_order == 2 ? 0.5 * s2[b] : 0.0);
             ph[b] = l;
             if (l > m) m = l;

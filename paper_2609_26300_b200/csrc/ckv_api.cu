@@ -1,0 +1,304 @@
+// Host side of the C ABI declared in include/compkv.h: validation, buffer partitioning, launches.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "ckv_internal.cuh"
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+int check_layout(const ckv_layout *L) {
+  if (L == nullptr) return CKV_ERR_INVALID_ARG;
+  if (L->head_dim != CKV_D || L->page_size != CKV_PAGE) return CKV_ERR_BAD_LAYOUT;
+  if (L->num_kv_heads <= 0 || L->num_q_heads <= 0 || L->num_q_heads % L->num_kv_heads != 0) return CKV_ERR_BAD_LAYOUT;
+  const int G = L->num_q_heads / L->num_kv_heads;
+  if (G != 1 && G != 2 && G != 4 && G != 8) return CKV_ERR_BAD_LAYOUT;
+  if (L->block_size != 16 && L->block_size != 32 && L->block_size != 64) return CKV_ERR_BAD_LAYOUT;
+  if (!is_pow2(L->var_groups) || !(L->var_groups <= CKV_D / 2 || L->var_groups == CKV_D)) return CKV_ERR_BAD_LAYOUT;
+  if (L->group_layout != 0 && L->group_layout != 1) return CKV_ERR_BAD_LAYOUT;
+  if (L->kv_dtype != CKV_BF16 && L->kv_dtype != CKV_F32) return CKV_ERR_BAD_LAYOUT;
+  if (L->max_batch <= 0 || L->max_blocks_per_seq <= 0 || L->num_pages <= 0) return CKV_ERR_BAD_LAYOUT;
+  if ((long long)L->max_blocks_per_seq * L->block_size > (1ll << 30)) return CKV_ERR_BAD_LAYOUT;
+  if ((long long)L->max_batch * L->num_kv_heads > 65535) return CKV_ERR_BAD_LAYOUT;   // grid.y
+  if (L->sink_blocks < 0 || L->recent_blocks < 0) return CKV_ERR_BAD_LAYOUT;
+  if (!(L->sm_scale >= 0.f) || !isfinite(L->sm_scale)) return CKV_ERR_BAD_LAYOUT;
+  return CKV_OK;
+}
+
+struct Regions {
+  size_t kmean, dbar, vmean, stats_total;
+  size_t ls, scores, comp, attn, status, stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt, work_total;
+};
+
+Regions regions(const ckv_layout *L) {
+  Regions R;
+  const size_t units = (size_t)L->max_batch * L->num_kv_heads;
+  const size_t rows = units * L->max_blocks_per_seq;
+  const int G = L->num_q_heads / L->num_kv_heads;
+  const size_t esz = L->kv_dtype == CKV_BF16 ? 2 : 4;
+  size_t o = 0;
+  R.kmean = o; o = align_up(o + rows * CKV_D * 4, 256);
+  R.dbar = o;  o = align_up(o + rows * L->var_groups * 4, 256);
+  R.vmean = o; o = align_up(o + rows * CKV_D * 4, 256);
+  R.stats_total = o;
+  o = 0;
+  R.status = o; o = align_up(o + 256, 256);
+  R.ls = o;     o = align_up(o + rows * G * sizeof(float2), 256);
+  R.scores = o; o = align_up(o + rows * 4, 256);
+  R.comp = o;   o = align_up(o + units * CKV_MAX_CHUNKS * G * CKV_PART_STRIDE * 4, 256);
+  R.attn = o;   o = align_up(o + units * CKV_MAX_SPLITS * G * CKV_PART_STRIDE * 4, 256);
+  R.stage_q = o;    o = align_up(o + (size_t)L->max_batch * L->num_q_heads * CKV_D * esz, 256);
+  R.stage_knew = o; o = align_up(o + units * CKV_D * esz, 256);
+  R.stage_vnew = o; o = align_up(o + units * CKV_D * esz, 256);
+  R.stage_out = o;  o = align_up(o + (size_t)L->max_batch * L->num_q_heads * CKV_D * esz, 256);
+  R.stage_ids = o;  o = align_up(o + units * (size_t)L->max_blocks_per_seq * 4, 256);
+  R.stage_cnt = o;  o = align_up(o + units * 4, 256);
+  R.work_total = o;
+  return R;
+}
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return CKV_ERR_CUDA;
+}
+#define CKV_CUDA(expr)                                \
+  do {                                                \
+    cudaError_t e__ = (expr);                         \
+    if (e__ != cudaSuccess) return cuda_fail(e__);    \
+  } while (0)
+
+int check_step_args(const ckv_ctx *c, int batch, int max_len) {
+  if (c == nullptr) return CKV_ERR_INVALID_ARG;
+  if (batch <= 0 || batch > c->layout.max_batch) return CKV_ERR_INVALID_ARG;
+  if (max_len <= 0 || (long long)max_len > (long long)c->layout.max_blocks_per_seq * c->layout.block_size)
+    return CKV_ERR_INVALID_ARG;
+  return CKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ckv_version(void) { return 100; }
+
+const char *ckv_strerror(int status) {
+  switch (status) {
+    case CKV_OK: return "ok";
+    case CKV_ERR_INVALID_ARG: return "invalid argument";
+    case CKV_ERR_BAD_LAYOUT: return "unsupported layout";
+    case CKV_ERR_BUDGET_TOO_SMALL: return "budget smaller than the mandatory blocks";
+    case CKV_ERR_CAPACITY: return "caller buffer too small";
+    case CKV_ERR_CUDA: return "CUDA runtime error";
+    case CKV_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int ckv_last_cuda_error(void) { return g_last_cuda_error; }
+
+int ckv_query_sizes(const ckv_layout *layout, size_t *stats_bytes, size_t *workspace_bytes) {
+  const int st = check_layout(layout);
+  if (st != CKV_OK) return st;
+  if (stats_bytes == nullptr || workspace_bytes == nullptr) return CKV_ERR_INVALID_ARG;
+  const Regions R = regions(layout);
+  *stats_bytes = R.stats_total;
+  *workspace_bytes = R.work_total;
+  return CKV_OK;
+}
+
+int ckv_stats_offsets(const ckv_layout *layout, size_t *kmean_off, size_t *dbar_off, size_t *vmean_off) {
+  const int st = check_layout(layout);
+  if (st != CKV_OK) return st;
+  if (kmean_off == nullptr || dbar_off == nullptr || vmean_off == nullptr) return CKV_ERR_INVALID_ARG;
+  const Regions R = regions(layout);
+  *kmean_off = R.kmean;
+  *dbar_off = R.dbar;
+  *vmean_off = R.vmean;
+  return CKV_OK;
+}
+
+int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, void *work_dev, size_t work_bytes,
+               ckv_stream stream, ckv_ctx **out) {
+  const int st = check_layout(layout);
+  if (st != CKV_OK) return st;
+  if (stats_dev == nullptr || work_dev == nullptr || out == nullptr) return CKV_ERR_INVALID_ARG;
+  if (((uintptr_t)stats_dev & 255) != 0 || ((uintptr_t)work_dev & 255) != 0) return CKV_ERR_INVALID_ARG;
+  const Regions R = regions(layout);
+  if (stats_bytes < R.stats_total || work_bytes < R.work_total) return CKV_ERR_CAPACITY;
+  ckv_ctx *c = new (std::nothrow) ckv_ctx();
+  if (c == nullptr) return CKV_ERR_INVALID_ARG;
+  c->layout = *layout;
+  if (c->layout.sm_scale == 0.f) c->layout.sm_scale = 1.0f / sqrtf((float)layout->head_dim);
+  char *sb = (char *)stats_dev, *wb = (char *)work_dev;
+  CkvDev &P = c->dev;
+  P.Hq = layout->num_q_heads; P.Hkv = layout->num_kv_heads; P.G = P.Hq / P.Hkv;
+  P.bs = layout->block_size; P.ppb = layout->block_size / layout->page_size;
+  P.r = layout->var_groups; P.glayout = layout->group_layout;
+  P.max_blocks = layout->max_blocks_per_seq; P.max_pages_per_seq = P.max_blocks * P.ppb;
+  P.num_pages = layout->num_pages; P.sink = layout->sink_blocks; P.recent = layout->recent_blocks;
+  P.scale = c->layout.sm_scale;
+  P.kmean = (float *)(sb + R.kmean); P.dbar = (float *)(sb + R.dbar); P.vmean = (float *)(sb + R.vmean);
+  P.status = (int *)(wb + R.status);
+  P.ls = (float2 *)(wb + R.ls); P.scores = (float *)(wb + R.scores);
+  P.comp_part = (float *)(wb + R.comp); P.attn_part = (float *)(wb + R.attn);
+  c->work = wb; c->work_bytes = work_bytes;
+  c->stage_q = R.stage_q; c->stage_knew = R.stage_knew; c->stage_vnew = R.stage_vnew;
+  c->stage_out = R.stage_out; c->stage_ids = R.stage_ids; c->stage_cnt = R.stage_cnt;
+  c->launches = 0;
+  cudaError_t e = ckv_configure_kernels();
+  if (e == cudaSuccess) e = cudaMemsetAsync(P.status, 0, 256, (cudaStream_t)stream);
+  if (e != cudaSuccess) { delete c; return cuda_fail(e); }
+  *out = c;
+  return CKV_OK;
+}
+
+void ckv_destroy(ckv_ctx *ctx) { delete ctx; }
+
+int ckv_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                    const int32_t *seq_lens, int batch, int max_seq_len_host, ckv_stream stream) {
+  const int st = check_step_args(c, batch, max_seq_len_host);
+  if (st != CKV_OK) return st;
+  if (!k_pool || !v_pool || !page_table || !seq_lens) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(ckv_launch_stats_build(c, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host,
+                                  (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+int ckv_append(ckv_ctx *c, void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens,
+               const void *k_new, const void *v_new, int batch, ckv_stream stream) {
+  if (c == nullptr || batch <= 0 || batch > c->layout.max_batch) return CKV_ERR_INVALID_ARG;
+  if (!k_pool || !v_pool || !page_table || !seq_lens || !k_new || !v_new) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(ckv_launch_append(c, k_pool, v_pool, page_table, seq_lens, k_new, v_new, batch, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+namespace {
+
+// The four launches of a sparse decode step; ev (may be null) receives 5 events bracketing them.
+int decode_impl(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                const int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens, void *out, float *lse,
+                int32_t *sel_ids, int32_t *sel_cnt, cudaStream_t s, cudaEvent_t *ev) {
+  const int st = check_step_args(c, batch, max_seq_len_host);
+  if (st != CKV_OK) return st;
+  if (!q || !k_pool || !v_pool || !page_table || !seq_lens || !out || !sel_ids || !sel_cnt) return CKV_ERR_INVALID_ARG;
+  const ckv_layout &L = c->layout;
+  const int kcap = budget_tokens / L.block_size;
+  if (budget_tokens <= 0 || kcap <= 0) return CKV_ERR_BUDGET_TOO_SMALL;
+  if (kcap > L.max_blocks_per_seq) return CKV_ERR_INVALID_ARG;
+  if (kcap < L.sink_blocks + L.recent_blocks && (long long)kcap * L.block_size < max_seq_len_host)
+    return CKV_ERR_BUDGET_TOO_SMALL;
+  int n_chunks = 0, n_splits = 0;
+  if (ev) CKV_CUDA(cudaEventRecord(ev[0], s));
+  CKV_CUDA(ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, &n_chunks, s));
+  if (ev) CKV_CUDA(cudaEventRecord(ev[1], s));
+  CKV_CUDA(ckv_launch_select(c, seq_lens, batch, kcap, sel_ids, sel_cnt, s));
+  if (ev) CKV_CUDA(cudaEventRecord(ev[2], s));
+  CKV_CUDA(ckv_launch_attn(c, false, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, batch,
+                           max_seq_len_host, &n_splits, s));
+  if (ev) CKV_CUDA(cudaEventRecord(ev[3], s));
+  CKV_CUDA(ckv_launch_merge(c, false, seq_lens, sel_cnt, n_splits, n_chunks, batch, out, lse, s));
+  if (ev) CKV_CUDA(cudaEventRecord(ev[4], s));
+  return CKV_OK;
+}
+
+}  // namespace
+
+int ckv_decode(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
+               const int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens, void *out, float *lse,
+               int32_t *sel_ids, int32_t *sel_cnt, ckv_stream stream) {
+  return decode_impl(c, q, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, out, lse,
+                     sel_ids, sel_cnt, (cudaStream_t)stream, nullptr);
+}
+
+int ckv_decode_profile(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                       const int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens, void *out,
+                       float *lse, int32_t *sel_ids, int32_t *sel_cnt, ckv_stream stream, float *stage_ms_host) {
+  if (stage_ms_host == nullptr) return CKV_ERR_INVALID_ARG;
+  cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  int rc = CKV_OK;
+  for (int i = 0; i < 5 && rc == CKV_OK; ++i)
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  if (rc == CKV_OK)
+    rc = decode_impl(c, q, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, out, lse,
+                     sel_ids, sel_cnt, (cudaStream_t)stream, ev);
+  if (rc == CKV_OK && cudaEventSynchronize(ev[4]) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  for (int i = 0; i < 4 && rc == CKV_OK; ++i)
+    if (cudaEventElapsedTime(&stage_ms_host[i], ev[i], ev[i + 1]) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  for (int i = 0; i < 5; ++i)
+    if (ev[i]) cudaEventDestroy(ev[i]);
+  return rc;
+}
+
+int ckv_dense_decode(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                     const int32_t *seq_lens, int batch, int max_seq_len_host, void *out, float *lse,
+                     ckv_stream stream) {
+  const int st = check_step_args(c, batch, max_seq_len_host);
+  if (st != CKV_OK) return st;
+  if (!q || !k_pool || !v_pool || !page_table || !seq_lens || !out) return CKV_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int n_splits = 0;
+  CKV_CUDA(ckv_launch_attn(c, true, q, k_pool, v_pool, page_table, seq_lens, nullptr, nullptr, 0, batch,
+                           max_seq_len_host, &n_splits, s));
+  CKV_CUDA(ckv_launch_merge(c, true, seq_lens, nullptr, n_splits, 0, batch, out, lse, s));
+  return CKV_OK;
+}
+
+int ckv_copy_scores(ckv_ctx *c, float *dst, int batch, ckv_stream stream) {
+  if (c == nullptr || dst == nullptr || batch <= 0 || batch > c->layout.max_batch) return CKV_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)batch * c->layout.num_kv_heads * c->layout.max_blocks_per_seq * sizeof(float);
+  CKV_CUDA(cudaMemcpyAsync(dst, c->dev.scores, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+int ckv_step_host(ckv_ctx *c, const void *q_host, const void *k_new_host, const void *v_new_host, void *k_pool,
+                  void *v_pool, const int32_t *page_table, int32_t *seq_lens, int batch, int max_seq_len_host,
+                  int budget_tokens, void *out_host, int32_t *sel_ids_host, int32_t *sel_cnt_host,
+                  ckv_stream stream) {
+  const int st = check_step_args(c, batch, max_seq_len_host);
+  if (st != CKV_OK) return st;
+  if (!q_host || !k_new_host || !v_new_host || !out_host || !sel_ids_host || !sel_cnt_host) return CKV_ERR_INVALID_ARG;
+  const ckv_layout &L = c->layout;
+  const size_t esz = L.kv_dtype == CKV_BF16 ? 2 : 4;
+  const size_t q_bytes = (size_t)batch * L.num_q_heads * CKV_D * esz;
+  const size_t kv_bytes = (size_t)batch * L.num_kv_heads * CKV_D * esz;
+  const int kcap = budget_tokens / L.block_size;
+  if (kcap <= 0) return CKV_ERR_BUDGET_TOO_SMALL;
+  if (kcap > L.max_blocks_per_seq) return CKV_ERR_INVALID_ARG;
+  const size_t ids_bytes = (size_t)batch * L.num_kv_heads * kcap * 4;
+  const size_t cnt_bytes = (size_t)batch * L.num_kv_heads * 4;
+  cudaStream_t s = (cudaStream_t)stream;
+  void *dq = c->work + c->stage_q, *dk = c->work + c->stage_knew, *dv = c->work + c->stage_vnew;
+  void *dout = c->work + c->stage_out;
+  int32_t *dids = (int32_t *)(c->work + c->stage_ids), *dcnt = (int32_t *)(c->work + c->stage_cnt);
+  CKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
+  CKV_CUDA(cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+  CKV_CUDA(cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+  int r = ckv_append(c, k_pool, v_pool, page_table, seq_lens, dk, dv, batch, stream);
+  if (r != CKV_OK) return r;
+  r = ckv_decode(c, dq, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, dout, nullptr,
+                 dids, dcnt, stream);
+  if (r != CKV_OK) return r;
+  CKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s));
+  CKV_CUDA(cudaMemcpyAsync(sel_ids_host, dids, ids_bytes, cudaMemcpyDeviceToHost, s));
+  CKV_CUDA(cudaMemcpyAsync(sel_cnt_host, dcnt, cnt_bytes, cudaMemcpyDeviceToHost, s));
+  CKV_CUDA(cudaStreamSynchronize(s));
+  return CKV_OK;
+}
+
+int ckv_read_status(ckv_ctx *c, int32_t *host_status, ckv_stream stream) {
+  if (c == nullptr || host_status == nullptr) return CKV_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  CKV_CUDA(cudaMemcpyAsync(host_status, c->dev.status, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  CKV_CUDA(cudaMemsetAsync(c->dev.status, 0, sizeof(int32_t), s));
+  CKV_CUDA(cudaStreamSynchronize(s));
+  return CKV_OK;
+}
+
+int64_t ckv_launch_count(const ckv_ctx *c) { return c == nullptr ? 0 : c->launches; }
+
+}  // extern "C"

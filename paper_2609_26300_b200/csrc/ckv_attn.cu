@@ -1,0 +1,368 @@
+// Exact attention over a list of cache pages (split along the list), the removal of the selected
+// blocks' mean-compensation terms, and the final log-sum-exp merge (Eq. 12).
+//
+// Sparse mode: the page list of a unit is the pages of its selected blocks, in position order.
+// Dense mode: every page of the sequence (Eq. 12 with S = all blocks; Sec. 3.1).
+//
+// A CTA takes a contiguous slice of the list; each of its 8 warps takes every 8th page.  Within a
+// warp a token row (128 elements) is spread over the 16 lanes of a half warp (8 coordinates per
+// lane, one 16-byte load for bf16) and the two half warps take alternate rows.  QK^T partial sums
+// are reduced across the 16 lanes with a work-sharing shuffle tree, so that each lane ends up
+// owning the logits of one row for half of the heads and evaluates those exponentials only; the
+// probabilities go through a small shared-memory tile back to the lanes that hold the V rows.
+// Running maxima are kept per warp and only raised when exceeded by a slack (the partial
+// (m, l, acc) stays an exact representation of sum e^{z} v for any m).
+//
+// For every selected block the scan kernel has already added the block's mean term
+// |b| e^{zbar} vbar_b to the all-block compensation sum; here the same term is subtracted from the
+// exact partial, so that  merge = exact(S) + mean(all) - mean(S) = exact(S) + mean(not S).
+#include "ckv_internal.cuh"
+
+namespace {
+
+// Eight consecutive elements kept in their storage form (so a bf16 row costs 4 registers, not 8).
+template <typename T> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+  uint4 u;
+  __device__ __forceinline__ void load(const __nv_bfloat16 *p) { u = __ldg(reinterpret_cast<const uint4 *>(p)); }
+  __device__ __forceinline__ void zero() { u = make_uint4(0u, 0u, 0u, 0u); }
+  __device__ __forceinline__ void get(float (&o)[8]) const { bf16x8_to_float(u, o); }
+};
+template <> struct Raw8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float *p) {
+    a = __ldg(reinterpret_cast<const float4 *>(p)); b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+  }
+  __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
+  __device__ __forceinline__ void get(float (&o)[8]) const {
+    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+  }
+};
+
+template <int G, typename T, bool DENSE>
+__global__ void __launch_bounds__(256, (G <= 2) ? 2 : 1)
+ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool, const T *__restrict__ v_pool,
+                const int *__restrict__ page_table, const int *__restrict__ seq_lens,
+                const int *__restrict__ sel_ids, const int *__restrict__ sel_cnt, int kcap, int pages_per_split) {
+  constexpr int NV = 8 * G;                      // logits per lane before the reduction (8 rows x G heads)
+  constexpr int KEEP = (NV >= 16) ? NV / 16 : 1;  // logits per lane after it
+  constexpr int HSPLIT = (G >= 2) ? 2 : 1;        // a row's heads are shared by this many lanes
+  __shared__ float sq[G][CKV_D];
+  __shared__ __align__(16) float pbuf[8][CKV_PAGE][G];
+  __shared__ __align__(16) float red[8][G][CKV_PART_STRIDE];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, hw = lane >> 4, li = lane & 15;
+  const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
+  const int N = min(seq_lens[s], P.max_blocks * P.bs);
+  const int X = (N + P.bs - 1) / P.bs;
+  const int nsel = DENSE ? X : min(sel_cnt[unit], kcap);
+  const int total = DENSE ? (N + CKV_PAGE - 1) / CKV_PAGE : nsel * P.ppb;
+  const bool comp = !DENSE && nsel < X;
+  const int p0 = blockIdx.x * pages_per_split;
+  const int p1 = min(p0 + pages_per_split, total);
+  float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
+  if (p0 >= total) {
+    if (tid < G) { part[tid * CKV_PART_STRIDE] = -CUDART_INF_F; part[tid * CKV_PART_STRIDE + 1] = 0.f; }
+    return;
+  }
+
+  for (int idx = tid; idx < G * CKV_D; idx += 256)
+    sq[idx / CKV_D][idx % CKV_D] = to_float(q[((size_t)s * P.Hq + h * G) * CKV_D + idx]) * (P.scale * kLog2e);
+  __syncthreads();
+  float qr[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qr[g][i] = sq[g][8 * li + i];
+
+  float acc[G][8], m_ref[G], m_own[KEEP], l_own[KEEP];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    m_ref[g] = -CUDART_INF_F;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
+  }
+#pragma unroll
+  for (int jj = 0; jj < KEEP; ++jj) { m_own[jj] = -CUDART_INF_F; l_own[jj] = 0.f; }
+  // after the reduction this lane owns row (li / 2) of its half warp and heads [g_own0, g_own0 + KEEP)
+  const int g_own0 = (G >= 2) ? (li & 1) * KEEP : 0;
+  const int t_own = hw + 2 * (li >> 1);
+  const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
+  const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
+  const float *vmean = P.vmean + (size_t)unit * P.max_blocks * CKV_D;
+  bool bad = false;
+
+  for (int i = p0 + warp; i < p1; i += 8) {
+    int page, blk = 0;
+    if (DENSE) {
+      page = i;
+    } else {
+      blk = sel_ids[(size_t)unit * kcap + i / P.ppb];
+      if (blk < 0 || blk >= X) continue;
+      page = blk * P.ppb + i % P.ppb;
+    }
+    const int ntok = min(CKV_PAGE, N - page * CKV_PAGE);
+    if (ntok > 0) {
+      const int phys = pt_row[page];
+      if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
+      const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+      float sv[NV];
+      Raw8<T> kraw[8], vraw[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          kraw[j].load(k_pool + base + (size_t)t * CKV_D);
+          vraw[j].load(v_pool + base + (size_t)t * CKV_D);
+        } else {
+          kraw[j].zero();
+          vraw[j].zero();
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float kf[8];
+        kraw[j].get(kf);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          float z = 0.f;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) z = fmaf(qr[g][c], kf[c], z);
+          sv[j * G + g] = z;
+        }
+      }
+      reduce16<NV, KEEP>(sv, li);
+      // sv[0..KEEP): logits (log2 units) of row t_own for heads g_own0 + jj
+      const bool row_ok = t_own < ntok;
+      bool need = false;
+#pragma unroll
+      for (int jj = 0; jj < KEEP; ++jj) {
+        if (!row_ok) sv[jj] = -CUDART_INF_F;
+        need |= sv[jj] > m_own[jj] + CKV_RESCALE_SLACK;
+      }
+      if (__any_sync(0xffffffffu, need)) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          float cand = -CUDART_INF_F;
+#pragma unroll
+          for (int jj = 0; jj < KEEP; ++jj)
+            if (g_own0 + jj == g) cand = sv[jj];
+          cand = warp_max(cand);
+          if (cand > m_ref[g]) {
+            const float sc = exp2_diff(m_ref[g], cand);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc[g][c] *= sc;
+#pragma unroll
+            for (int jj = 0; jj < KEEP; ++jj)
+              if (g_own0 + jj == g) { l_own[jj] *= sc; m_own[jj] = cand; }
+            m_ref[g] = cand;
+          }
+        }
+      }
+      float pr[KEEP];
+#pragma unroll
+      for (int jj = 0; jj < KEEP; ++jj) {
+        pr[jj] = row_ok ? exp2f(sv[jj] - m_own[jj]) : 0.f;
+        // with G == 1 two lanes hold the same logit: only the even one counts it
+        if (G >= 2 || (li & 1) == 0) l_own[jj] += pr[jj];
+      }
+      float *prow = &pbuf[warp][t_own][g_own0];
+#pragma unroll
+      for (int jj = 0; jj < KEEP; ++jj) prow[jj] = pr[jj];
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float *pp = pbuf[warp][hw + 2 * j];
+        float vf[8];
+        vraw[j].get(vf);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const float pg = pp[g];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(pg, vf[c], acc[g][c]);
+        }
+      }
+      __syncwarp();
+    }
+    if (comp && (i % P.ppb) == 0) {
+      // take this block's mean term |b| e^{zbar} vbar_b back out (it is part of the all-block sum)
+      float zl2[G];
+      bool raise = false;
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float2 v = __ldg(ls + (size_t)blk * G + g);
+        zl2[g] = (v.x - 0.5f * v.y) * kLog2e;
+        raise |= zl2[g] > m_ref[g] + CKV_RESCALE_SLACK;
+      }
+      if (raise) {   // warp-uniform: every lane evaluates the same values
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          if (zl2[g] > m_ref[g]) {
+            const float sc = exp2_diff(m_ref[g], zl2[g]);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc[g][c] *= sc;
+#pragma unroll
+            for (int jj = 0; jj < KEEP; ++jj)
+              if (g_own0 + jj == g) { l_own[jj] *= sc; m_own[jj] = zl2[g]; }
+            m_ref[g] = zl2[g];
+          }
+        }
+      }
+      if (hw == 0) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li));
+        const float4 b4 = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li) + 1);
+        const float vb[8] = {a.x, a.y, a.z, a.w, b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const float wbar = exp2f(zl2[g] - m_ref[g]);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(-wbar, vb[c], acc[g][c]);
+#pragma unroll
+          for (int jj = 0; jj < KEEP; ++jj)
+            if (g_own0 + jj == g && li < HSPLIT) l_own[jj] -= wbar;
+        }
+      }
+    }
+  }
+  if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
+
+  // warp totals: both half warps share m_ref, so accumulators add directly
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[g][c] += __shfl_xor_sync(0xffffffffu, acc[g][c], 16);
+    float lg = 0.f;
+#pragma unroll
+    for (int jj = 0; jj < KEEP; ++jj)
+      if (g_own0 + jj == g) lg = l_own[jj];
+    lg = warp_sum(lg);
+    float *r = red[warp][g];
+    if (hw == 0) {
+      *reinterpret_cast<float4 *>(r + 4 + 8 * li) = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
+      *reinterpret_cast<float4 *>(r + 8 + 8 * li) = make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]);
+    }
+    if (lane == 0) { r[0] = m_ref[g]; r[1] = lg; }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < G * CKV_D; idx += 256) {
+    const int g = idx / CKV_D, c = idx % CKV_D;
+    float M = -CUDART_INF_F;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) M = fmaxf(M, red[w][g][0]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      const float sc = exp2_diff(red[w][g][0], M);
+      num = fmaf(red[w][g][4 + c], sc, num);
+      den = fmaf(red[w][g][1], sc, den);
+    }
+    part[g * CKV_PART_STRIDE + 4 + c] = num;
+    if (c == 0) { part[g * CKV_PART_STRIDE] = M; part[g * CKV_PART_STRIDE + 1] = den; }
+  }
+}
+
+// out_{g} = sum of all partials under one normaliser (Eq. 12).  One CTA per (sequence, query head),
+// one thread per output coordinate.
+template <typename T>
+__global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *__restrict__ seq_lens,
+                                                          const int *__restrict__ sel_cnt, int kcap, int n_splits,
+                                                          int n_chunks, bool dense, T *__restrict__ out,
+                                                          float *__restrict__ lse) {
+  const int hq = blockIdx.x, s = blockIdx.y, c = threadIdx.x;
+  const int G = P.G, unit = s * P.Hkv + hq / G, g = hq % G;
+  const int N = min(seq_lens[s], P.max_blocks * P.bs);
+  const int X = (N + P.bs - 1) / P.bs;
+  const bool comp = !dense && min(sel_cnt[unit], kcap) < X;
+  const float *ap = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS * G + g) * CKV_PART_STRIDE;
+  const float *cp = P.comp_part + ((size_t)unit * CKV_MAX_CHUNKS * G + g) * CKV_PART_STRIDE;
+  const size_t step = (size_t)G * CKV_PART_STRIDE;
+  float M = -CUDART_INF_F;
+  for (int i = 0; i < n_splits; ++i) M = fmaxf(M, ap[i * step]);
+  if (comp)
+    for (int i = 0; i < n_chunks; ++i) M = fmaxf(M, cp[i * step]);
+  float num = 0.f, den = 0.f;
+  for (int i = 0; i < n_splits; ++i) {
+    const float m = ap[i * step];
+    if (m == -CUDART_INF_F) continue;
+    const float sc = exp2f(m - M);
+    num = fmaf(ap[i * step + 4 + c], sc, num);
+    den = fmaf(ap[i * step + 1], sc, den);
+  }
+  if (comp)
+    for (int i = 0; i < n_chunks; ++i) {
+      const float m = cp[i * step];
+      if (m == -CUDART_INF_F) continue;
+      const float sc = exp2f(m - M);
+      num = fmaf(cp[i * step + 4 + c], sc, num);
+      den = fmaf(cp[i * step + 1], sc, den);
+    }
+  const size_t o = ((size_t)s * P.Hq + hq) * CKV_D + c;
+  store_out(out + o, N > 0 ? num / den : 0.f);
+  if (lse != nullptr && c == 0) lse[(size_t)s * P.Hq + hq] = N > 0 ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
+}
+
+template <int G, typename T>
+cudaError_t launch_gt(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
+                      const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt, int kcap,
+                      dim3 grid, int pps, cudaStream_t st) {
+  if (dense)
+    ckv_attn_kernel<G, T, true><<<grid, 256, 0, st>>>(c->dev, (const T *)q, (const T *)k_pool, (const T *)v_pool,
+                                                       page_table, seq_lens, sel_ids, sel_cnt, kcap, pps);
+  else
+    ckv_attn_kernel<G, T, false><<<grid, 256, 0, st>>>(c->dev, (const T *)q, (const T *)k_pool, (const T *)v_pool,
+                                                        page_table, seq_lens, sel_ids, sel_cnt, kcap, pps);
+  return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_g(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
+                     const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt, int kcap,
+                     dim3 grid, int pps, cudaStream_t st) {
+  if (c->layout.kv_dtype == CKV_BF16)
+    return launch_gt<G, __nv_bfloat16>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap,
+                                       grid, pps, st);
+  return launch_gt<G, float>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
+}
+
+}  // namespace
+
+cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
+                            const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
+                            int kcap, int batch, int max_len, int *n_splits_out, cudaStream_t st) {
+  const CkvDev &P = c->dev;
+  const int units = batch * P.Hkv;
+  const int xmax = (max_len + P.bs - 1) / P.bs;
+  const int total = dense ? (max_len + CKV_PAGE - 1) / CKV_PAGE : min(kcap, xmax) * P.ppb;
+  // about four CTAs per SM overall, at least one page per warp, at most CKV_MAX_SPLITS splits
+  int n_splits = (148 * 4 + units - 1) / units;
+  n_splits = max(1, min(n_splits, min(CKV_MAX_SPLITS, (total + 7) / 8)));
+  int pps = (total + n_splits - 1) / n_splits;
+  pps = (pps + 7) / 8 * 8;
+  n_splits = max(1, (total + pps - 1) / pps);
+  *n_splits_out = n_splits;
+  dim3 grid(n_splits, units);
+  c->launches++;
+  switch (P.G) {
+    case 1: return launch_g<1>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
+    case 2: return launch_g<2>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
+    case 4: return launch_g<4>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
+    case 8: return launch_g<8>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t ckv_launch_merge(ckv_ctx *c, bool dense, const int *seq_lens, const int *sel_cnt, int n_splits,
+                             int n_chunks, int batch, void *out, float *lse, cudaStream_t st) {
+  const CkvDev &P = c->dev;
+  dim3 grid(P.Hq, batch);
+  // kcap is only used to clamp sel_cnt; sel_cnt never exceeds it, so pass a large bound
+  const int kcap = 1 << 30;
+  if (c->layout.kv_dtype == CKV_BF16)
+    ckv_merge_kernel<__nv_bfloat16><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, kcap, n_splits, n_chunks, dense,
+                                                           (__nv_bfloat16 *)out, lse);
+  else
+    ckv_merge_kernel<float><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, kcap, n_splits, n_chunks, dense,
+                                                    (float *)out, lse);
+  c->launches++;
+  return cudaGetLastError();
+}

@@ -1,0 +1,150 @@
+// Internal declarations shared by the CompKV CUDA translation units (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "../../include/compkv.h"
+
+#define CKV_D 128             // head dimension the kernels are written for
+#define CKV_PAGE 16           // tokens per page
+#define CKV_PART_STRIDE 132   // floats per split partial: m, l, pad, pad, acc[128]
+#define CKV_MAX_CHUNKS 64     // scan partials per unit
+#define CKV_MAX_SPLITS 64     // attention partials per unit
+#define CKV_RESCALE_SLACK 16.0f  // log2 units: running maxima are only raised when exceeded by this much
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Everything a kernel needs to find its data; passed by value.
+struct CkvDev {
+  int Hq, Hkv, G, bs, ppb, r, glayout;
+  int max_blocks, max_pages_per_seq, num_pages, sink, recent;
+  float scale;
+  // block summaries (caller's stats buffer)
+  float *kmean, *dbar, *vmean;
+  // workspace
+  float2 *ls;        // [unit][max_blocks][G]  (log block weight estimate l_{g,b}, sigma_hat^2_{g,b})
+  float *scores;     // [unit][max_blocks]     S_b
+  float *comp_part;  // [unit][CKV_MAX_CHUNKS][G][CKV_PART_STRIDE]  all-block mean-compensation partials
+  float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials
+  int *status;       // device status word
+};
+
+struct ckv_ctx {
+  ckv_layout layout;
+  CkvDev dev;
+  char *work;
+  size_t work_bytes;
+  // host staging regions inside the workspace (ckv_step_host)
+  size_t stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt;
+  int64_t launches;
+};
+
+cudaError_t ckv_configure_kernels();
+
+// ---- launchers (one per translation unit) ---------------------------------------------------------
+cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int *page_table,
+                                   const int *seq_lens, int batch, int max_len, cudaStream_t st);
+cudaError_t ckv_launch_append(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
+                              const void *k_new, const void *v_new, int batch, cudaStream_t st);
+cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
+                            int *n_chunks_out, cudaStream_t st);
+cudaError_t ckv_launch_select(ckv_ctx *c, const int *seq_lens, int batch, int kcap, int *sel_ids, int *sel_cnt,
+                              cudaStream_t st);
+cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
+                            const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
+                            int kcap, int batch, int max_len, int *n_splits_out, cudaStream_t st);
+cudaError_t ckv_launch_merge(ckv_ctx *c, bool dense, const int *seq_lens, const int *sel_cnt, int n_splits,
+                             int n_chunks, int batch, void *out, float *lse, cudaStream_t st);
+
+// ---- device helpers -----------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void bf16x8_to_float(const uint4 &u, float (&o)[8]) {
+  o[0] = __uint_as_float(u.x << 16); o[1] = __uint_as_float(u.x & 0xffff0000u);
+  o[2] = __uint_as_float(u.y << 16); o[3] = __uint_as_float(u.y & 0xffff0000u);
+  o[4] = __uint_as_float(u.z << 16); o[5] = __uint_as_float(u.z & 0xffff0000u);
+  o[6] = __uint_as_float(u.w << 16); o[7] = __uint_as_float(u.w & 0xffff0000u);
+}
+
+// Eight consecutive elements as floats.  NC = read-only (non-coherent) path; use NC = false for
+// data the same kernel has just written.
+template <bool NC>
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&o)[8]) {
+  uint4 u;
+  if (NC) u = __ldg(reinterpret_cast<const uint4 *>(p));
+  else u = *reinterpret_cast<const uint4 *>(p);
+  bf16x8_to_float(u, o);
+}
+template <bool NC>
+__device__ __forceinline__ void load8(const float *p, float (&o)[8]) {
+  float4 a, b;
+  if (NC) { a = __ldg(reinterpret_cast<const float4 *>(p)); b = __ldg(reinterpret_cast<const float4 *>(p) + 1); }
+  else { a = *reinterpret_cast<const float4 *>(p); b = *(reinterpret_cast<const float4 *>(p) + 1); }
+  o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+}
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void store_out(float *p, float x) { *p = x; }
+__device__ __forceinline__ void store_out(__nv_bfloat16 *p, float x) { *p = __float2bfloat16_rn(x); }
+
+// Coordinate group of coordinate i (App. A.4 of the paper; see ckv_layout::group_layout).
+__device__ __forceinline__ int group_of(int i, int r, int glayout) {
+  if (r == CKV_D) return i;
+  if (glayout == 0) return i / (CKV_D / r);
+  const int half = CKV_D / 2;
+  const int p = i < half ? i : i - half;
+  return p / (half / r);
+}
+
+// Sum-reduce NV per-lane values across the 16 lanes of a half warp, sharing the work: while more
+// than KEEP values remain each step halves the count (a lane sends the half it gives up and keeps
+// the other), then the remaining steps are plain butterflies.  On return v[0..KEEP) hold complete
+// sums; the lane with half-warp index li owns original indices
+//   [ (li >> (4 - S)) * KEEP, +KEEP ),  S = log2(NV / KEEP) halving steps (S <= 4).
+template <int NV, int KEEP>
+__device__ __forceinline__ void reduce16(float (&v)[NV], int li) {
+  int n = NV;
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {
+    const int mask = 8 >> step;
+    if (n > KEEP) {
+      const int half = n / 2;
+      const bool up = (li & mask) != 0;
+#pragma unroll
+      for (int i = 0; i < NV / 2; ++i) {
+        if (i < half) {
+          const float send = up ? v[i] : v[i + half];
+          const float keep = up ? v[i + half] : v[i];
+          v[i] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
+        }
+      }
+      n = half;
+    } else {
+#pragma unroll
+      for (int i = 0; i < KEEP; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], mask);
+    }
+  }
+}
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+// exp2 of a difference that may involve -inf on either side without producing NaN.
+__device__ __forceinline__ float exp2_diff(float a, float b) {
+  return (a == -CUDART_INF_F) ? 0.0f : exp2f(a - b);
+}
+
+#endif  // __CUDACC__

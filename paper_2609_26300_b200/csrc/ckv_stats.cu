@@ -1,0 +1,185 @@
+// Block summaries: prefill-time build and per-token append (Sec. 4.1-4.2, Eq. 8 right half).
+//
+// One warp owns one block.  A token row (128 elements) is spread over the 16 lanes of a half
+// warp, 8 consecutive coordinates per lane (one 16-byte load for bf16); the two half warps take
+// alternate rows.  Means and squared deviations are accumulated in fp32 in two passes (mean
+// first, then deviations from it), the second pass re-reading the rows it just touched.
+// Build and append call the same routine, so their results are bit-identical.
+#include "ckv_internal.cuh"
+
+namespace {
+
+template <typename T, bool NC>
+__device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__restrict__ k_pool,
+                                                 const T *__restrict__ v_pool, const int *__restrict__ pt_row,
+                                                 int h, int b, int cnt, float *sq_smem, float *kmean_row,
+                                                 float *dbar_row, float *vmean_row, int lane) {
+  const int hw = lane >> 4, li = lane & 15;
+  float ks[8], vs[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { ks[i] = 0.f; vs[i] = 0.f; }
+  const int npages = (cnt + CKV_PAGE - 1) / CKV_PAGE;
+  bool bad = false;
+  for (int pg = 0; pg < npages; ++pg) {
+    const int phys = pt_row[b * P.ppb + pg];
+    if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
+    const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int t = hw + 2 * j;
+      if (t < ntok) {
+        float a[8], c[8];
+        load8<NC>(k_pool + base + (size_t)t * CKV_D, a);
+        load8<NC>(v_pool + base + (size_t)t * CKV_D, c);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+      }
+    }
+  }
+  const float fc = (float)cnt;
+  float km[8], sq[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
+    vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
+    km[i] = ks[i] / fc;
+    sq[i] = 0.f;
+  }
+  for (int pg = 0; pg < npages; ++pg) {
+    const int phys = pt_row[b * P.ppb + pg];
+    if (phys < 0 || phys >= P.num_pages) continue;
+    const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int t = hw + 2 * j;
+      if (t < ntok) {
+        float a[8];
+        load8<NC>(k_pool + base + (size_t)t * CKV_D, a);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], 16);
+  if (hw == 0) {
+    float4 *dst = reinterpret_cast<float4 *>(kmean_row + 8 * li);
+    dst[0] = make_float4(km[0], km[1], km[2], km[3]);
+    dst[1] = make_float4(km[4], km[5], km[6], km[7]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sq_smem[8 * li + i] = sq[i];
+  } else {
+    float4 *dst = reinterpret_cast<float4 *>(vmean_row + 8 * li);
+    dst[0] = make_float4(vs[0] / fc, vs[1] / fc, vs[2] / fc, vs[3] / fc);
+    dst[1] = make_float4(vs[4] / fc, vs[5] / fc, vs[6] / fc, vs[7] / fc);
+  }
+  __syncwarp();
+  // grouped variance: average of the per-coordinate population variances of each group (Eq. 8)
+  const int gs = CKV_D / P.r;
+  for (int t = lane; t < P.r; t += 32) {
+    float s = 0.f;
+    if (P.r == CKV_D) {
+      s = sq_smem[t];
+    } else if (P.glayout == 0) {
+      for (int i = 0; i < gs; ++i) s += sq_smem[t * gs + i];
+    } else {
+      const int hg = gs / 2;
+      for (int i = 0; i < hg; ++i) s += sq_smem[t * hg + i];
+      for (int i = 0; i < hg; ++i) s += sq_smem[CKV_D / 2 + t * hg + i];
+    }
+    dbar_row[t] = s / (fc * (float)gs);
+  }
+  __syncwarp();
+  if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) ckv_stats_build_kernel(CkvDev P, const T *__restrict__ k_pool,
+                                                              const T *__restrict__ v_pool,
+                                                              const int *__restrict__ page_table,
+                                                              const int *__restrict__ seq_lens) {
+  __shared__ float sq_smem[8][CKV_D];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
+  const int N = min(seq_lens[s], P.max_blocks * P.bs);
+  const int X = (N + P.bs - 1) / P.bs;
+  const int b = blockIdx.x * 8 + warp;
+  if (b >= X) return;
+  const int cnt = min(P.bs, N - b * P.bs);
+  const size_t row = (size_t)unit * P.max_blocks + b;
+  block_stats_warp<T, true>(P, k_pool, v_pool, page_table + (size_t)s * P.max_pages_per_seq, h, b, cnt,
+                            sq_smem[warp], P.kmean + row * CKV_D, P.dbar + row * P.r, P.vmean + row * CKV_D, lane);
+}
+
+// One CTA per sequence, one warp per KV head (looping when there are more heads than warps).
+template <typename T>
+__global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T *v_pool,
+                                                         const int *__restrict__ page_table, int *seq_lens,
+                                                         const T *__restrict__ k_new, const T *__restrict__ v_new) {
+  __shared__ float sq_smem[8][CKV_D];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int s = blockIdx.x;
+  const int N = seq_lens[s];
+  __syncthreads();   // every warp has read N before thread 0 may change it
+  if (N < 0 || N >= P.max_blocks * P.bs) {
+    if (threadIdx.x == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
+    return;
+  }
+  const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
+  const int page = N / CKV_PAGE, slot = N % CKV_PAGE;
+  const int phys = pt_row[page];
+  const bool ok = phys >= 0 && phys < P.num_pages;
+  const int b = N / P.bs, cnt = N + 1 - b * P.bs;
+  for (int h = warp; h < P.Hkv; h += nwarps) {
+    if (ok) {
+      // 16-byte pieces of the new row: lanes 0-15 copy K, lanes 16-31 copy V
+      constexpr int PIECES = (int)(CKV_D * sizeof(T) / 16);
+      const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + ((size_t)s * P.Hkv + h) * CKV_D);
+      uint4 *dst = reinterpret_cast<uint4 *>((lane < 16 ? k_pool : v_pool) +
+                                             (((size_t)phys * P.Hkv + h) * CKV_PAGE + slot) * CKV_D);
+      for (int i = lane & 15; i < PIECES; i += 16) dst[i] = src[i];
+    }
+    __syncwarp();
+    const size_t row = ((size_t)s * P.Hkv + h) * P.max_blocks + b;
+    block_stats_warp<T, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * CKV_D,
+                               P.dbar + row * P.r, P.vmean + row * CKV_D, lane);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) seq_lens[s] = N + 1;
+}
+
+}  // namespace
+
+cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int *page_table,
+                                   const int *seq_lens, int batch, int max_len, cudaStream_t st) {
+  const CkvDev &P = c->dev;
+  const int xmax = (max_len + P.bs - 1) / P.bs;
+  if (xmax <= 0 || batch <= 0) return cudaSuccess;
+  dim3 grid((xmax + 7) / 8, batch * P.Hkv);
+  if (c->layout.kv_dtype == CKV_BF16)
+    ckv_stats_build_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16 *)k_pool,
+                                                                (const __nv_bfloat16 *)v_pool, page_table, seq_lens);
+  else
+    ckv_stats_build_kernel<float><<<grid, 256, 0, st>>>(P, (const float *)k_pool, (const float *)v_pool, page_table,
+                                                        seq_lens);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+cudaError_t ckv_launch_append(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
+                              const void *k_new, const void *v_new, int batch, cudaStream_t st) {
+  const CkvDev &P = c->dev;
+  if (batch <= 0) return cudaSuccess;
+  const int threads = 32 * min(P.Hkv, 8);
+  if (c->layout.kv_dtype == CKV_BF16)
+    ckv_append_kernel<__nv_bfloat16><<<batch, threads, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
+                                                                page_table, seq_lens, (const __nv_bfloat16 *)k_new,
+                                                                (const __nv_bfloat16 *)v_new);
+  else
+    ckv_append_kernel<float><<<batch, threads, 0, st>>>(P, (float *)k_pool, (float *)v_pool, page_table, seq_lens,
+                                                        (const float *)k_new, (const float *)v_new);
+  c->launches++;
+  return cudaGetLastError();
+}

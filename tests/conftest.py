@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Build the CUDA library (nvcc cross-compiles without a GPU) and the oracle before any test."""
+    from oracle import compkv_oracle
+    from paper_2609_26300_b200 import build as ckv_build
+    compkv_oracle.build()
+    ckv_build.build()

@@ -1,0 +1,338 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Small cases compare every unit element by element; the full-size configurations compare
+sampled units (the oracle computes a unit in well under a second)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import compkv_oracle as O
+from paper_2609_26300_b200 import synth
+
+from helpers import (OUT_TOL, check_ids, check_stats, check_unit_decode, dev_q, rel_inf, setup, unit_inputs)
+
+pytestmark = pytest.mark.gpu
+
+TOY = synth.CONFIGS[1]
+
+
+def small(**kw):
+    base = dict(batch=2, num_q_heads=8, num_kv_heads=2, ctx=16 * 70 + 5, budget_tokens=16 * 12, needles=4,
+                outlier_dims=2, decode_steps=3, name="small")
+    base.update(kw)
+    return TOY.with_(**base)
+
+
+def all_units(w):
+    return [(s, h) for s in range(w.batch) for h in range(w.num_kv_heads)]
+
+
+def run_decode(d, budget, step=0, max_len=None):
+    q = dev_q(d, step)
+    out, lse, ids, cnt = d.ckv.decode(q, d.k_pool, d.v_pool, d.table, d.lens, max_len or d.max_len, budget)
+    scores = d.ckv.copy_scores(d.w.batch)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() == 0
+    return out, lse, ids, cnt, scores
+
+
+# ---- stats --------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("bs", [16, 32, 64])
+@pytest.mark.parametrize("r,layout", [(4, 1), (4, 0), (128, 1), (1, 1), (32, 0)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_stats_build(bs, r, layout, dtype):
+    w = small(block_size=bs, ctx_min=16 * 20 + 1, ctx=16 * 70 + 5)   # ragged lengths, partial last blocks
+    d = setup(w, dtype, var_groups=r, group_layout=layout)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    km, db, vm = d.ckv.stats_views()
+    lens = d.lens.cpu().numpy()
+    for s, h in all_units(w):
+        _, K, V = unit_inputs(w, s, h, int(lens[s]))
+        st = O.stats(K, V, bs, r, layout)
+        check_stats(st, km[s, h], db[s, h], vm[s, h], K, V)
+    assert d.ckv.read_status() == 0
+
+
+@pytest.mark.parametrize("bs", [16, 32])
+def test_append_equals_rebuild_bit_for_bit(bs):
+    steps = 40   # crosses block boundaries: a filled block, a rollover, a one-token block
+    w = small(block_size=bs, ctx=16 * 9 + 13, decode_steps=steps)
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    n0 = int(d.lens[0])
+    for t in range(steps):
+        k_new, v_new = synth.appended_rows(w, t)
+        d.ckv.append(d.k_pool, d.v_pool, d.table, d.lens,
+                     torch.from_numpy(k_new).to(d.dtype).cuda(), torch.from_numpy(v_new).to(d.dtype).cuda())
+    torch.cuda.synchronize()
+    assert d.lens.cpu().tolist() == [n0 + steps] * w.batch
+    km, db, vm = (t.clone() for t in d.ckv.stats_views())
+    # the appended rows are now in the cache: a fresh build over the longer cache must agree exactly
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, n0 + steps)
+    torch.cuda.synchronize()
+    km2, db2, vm2 = d.ckv.stats_views()
+    x = -(-(n0 + steps) // bs)
+    assert torch.equal(km[:, :, :x], km2[:, :, :x]) and torch.equal(db[:, :, :x], db2[:, :, :x])
+    assert torch.equal(vm[:, :, :x], vm2[:, :, :x])
+    for s, h in all_units(w):
+        _, K, V = unit_inputs(w, s, h, n0 + steps)
+        check_stats(O.stats(K, V, bs), km[s, h], db[s, h], vm[s, h], K, V)
+    assert d.ckv.read_status() == 0
+
+
+# ---- decode: small cases, every unit ------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (4, 2), (8, 2), (16, 2)])   # G = 1, 2, 4, 8
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_decode_small_all_group_sizes(hq, hkv, dtype):
+    w = small(num_q_heads=hq, num_kv_heads=hkv, ctx_min=16 * 30, ctx=16 * 70 + 5)
+    d = setup(w, dtype)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    lens = d.lens.cpu().numpy()
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, int(lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores)
+
+
+@pytest.mark.parametrize("bs,budget", [(32, 32 * 6), (64, 64 * 4), (16, 16 * 3), (16, 16 * 37)])
+@pytest.mark.parametrize("r,layout", [(4, 1), (128, 1), (8, 0)])
+def test_decode_small_block_sizes_and_groups(bs, budget, r, layout):
+    w = small(block_size=bs, budget_tokens=budget, ctx=16 * 90 + 7)
+    d = setup(w, var_groups=r, group_layout=layout)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, budget)
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, int(d.lens[s]), 0, budget, out, lse, ids, cnt, scores, var_groups=r,
+                          group_layout=layout)
+
+
+def test_decode_toy_config_fp32_and_bf16():
+    for dtype in (torch.float32, torch.bfloat16):
+        d = setup(TOY, dtype)
+        d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+        out, lse, ids, cnt, scores = run_decode(d, TOY.budget_tokens)
+        res = check_unit_decode(d, 0, 0, TOY.ctx, 0, TOY.budget_tokens, out, lse, ids, cnt, scores)
+        assert int(cnt[0, 0]) == 16
+
+
+def test_custom_scale_and_mandatory_counts():
+    w = small()
+    d = setup(w, sink=2, recent=3, sm_scale=0.05)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, int(d.lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores, sink=2, recent=3,
+                          scale=0.05)
+        got = ids[s, h, :int(cnt[s, h])].tolist()
+        x = -(-int(d.lens[s]) // 16)
+        assert got[:2] == [0, 1] and got[-3:] == [x - 3, x - 2, x - 1]
+
+
+# ---- special cases the method fixes -------------------------------------------------------------------------------------
+
+def test_select_all_equals_dense_kernel_and_oracle():
+    w = small(ctx=16 * 20 + 3, budget_tokens=16 * 32)
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, _ = run_decode(d, w.budget_tokens)
+    dout, dlse = d.ckv.dense_decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    x = 21
+    assert cnt.cpu().tolist() == [[x] * w.num_kv_heads] * w.batch
+    assert ids[0, 0, :x].tolist() == list(range(x)) and ids[0, 0, x:].tolist() == [-1] * (32 - x)
+    for s, h in all_units(w):
+        q, K, V = unit_inputs(w, s, h, int(d.lens[s]))
+        ref, ref_lse = O.dense(q, K, V)
+        G = w.group
+        for o, l in ((out, lse), (dout, dlse)):
+            assert rel_inf(o[s, h * G:(h + 1) * G].double().cpu().numpy(), ref) <= OUT_TOL[d.dtype]
+            assert np.abs(l[s, h * G:(h + 1) * G].double().cpu().numpy() - ref_lse).max() <= 1e-4
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_dense_decode_parity(dtype):
+    w = small(ctx_min=16 * 10, ctx=16 * 300 + 9, batch=3)
+    d = setup(w, dtype)
+    out, lse = d.ckv.dense_decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    G = w.group
+    for s, h in all_units(w):
+        q, K, V = unit_inputs(w, s, h, int(d.lens[s]))
+        ref, ref_lse = O.dense(q, K, V)
+        assert rel_inf(out[s, h * G:(h + 1) * G].double().cpu().numpy(), ref) <= OUT_TOL[dtype]
+        assert np.abs(lse[s, h * G:(h + 1) * G].double().cpu().numpy() - ref_lse).max() <= 1e-4
+    assert d.ckv.read_status() == 0
+
+
+def test_constant_key_blocks_make_any_selection_exact():
+    """Identical keys inside every block: mean compensation is exact, so the sparse output equals dense
+    attention whatever is selected (fp32 layout, tight tolerance)."""
+    w = small(batch=1, num_q_heads=4, num_kv_heads=1, ctx=16 * 40, decode_steps=0, needles=0, outlier_dims=0)
+    d = setup(w, torch.float32)
+    first = d.k_pool[:, :, :1, :].clone()
+    d.k_pool.copy_(first.expand_as(d.k_pool))
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, 16 * 5)
+    dout, dlse = d.ckv.dense_decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    assert int(cnt[0, 0]) == 5
+    assert float(scores[0, 0, :40].abs().max()) < 1e-9      # no within-block variance => zero scores
+    assert ids[0, 0, :5].tolist() == [0, 1, 2, 38, 39]       # all tied: lowest ids after the mandatory ones
+    assert rel_inf(out[0].double().cpu().numpy(), dout[0].double().cpu().numpy()) <= 1e-5
+    assert float((lse - dlse).abs().max()) <= 1e-5
+
+
+def test_exact_ties_go_to_lower_block_ids():
+    """Blocks with identical contents score identically on the GPU and in the oracle: stable order decides."""
+    w = small(batch=1, num_q_heads=4, num_kv_heads=1, ctx=16 * 64, decode_steps=0, needles=0, outlier_dims=0,
+              shuffle_pages=False)
+    d = setup(w)
+    # make blocks 8..39 copies of blocks 40..71 -> pairs of exactly tied scores (page == block, unshuffled)
+    d.k_pool[8:36] = d.k_pool[36:64]
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, 16 * 20)
+    sc = scores[0, 0, :64].cpu().numpy()
+    assert np.array_equal(sc[8:36], sc[36:64])
+    K = d.k_pool[:64, 0].float().reshape(-1, 128).cpu().numpy()
+    V = d.v_pool[:64, 0].float().reshape(-1, 128).cpu().numpy()
+    q = synth.queries(w)[0]
+    st = O.stats(K, V, 16)
+    osc = O.scores(q, st)
+    assert np.array_equal(osc.S[8:36], osc.S[36:64])
+    ref_ids = O.select(osc.S, 20)
+    got = ids[0, 0, :int(cnt[0, 0])].cpu().numpy()
+    check_ids(got, ref_ids, osc.S, 20)
+    # among an exactly tied pair the lower id must be the one taken (or both)
+    for b in range(8, 36):
+        if (b + 28) in got:
+            assert b in got
+
+
+# ---- edge cases ---------------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 47, 48, 49])
+def test_tiny_sequences(n):
+    w = small(batch=1, ctx=n, decode_steps=0, needles=0, budget_tokens=16 * 3)
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, 16 * 3)
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, n, 0, 16 * 3, out, lse, ids, cnt, scores)
+    dout, _ = d.ckv.dense_decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    G = w.group
+    q, K, V = unit_inputs(w, 0, 1, n)
+    assert rel_inf(dout[0, G:2 * G].double().cpu().numpy(), O.dense(q, K, V)[0]) <= OUT_TOL[d.dtype]
+
+
+def test_empty_sequence_in_batch():
+    w = small(batch=2, decode_steps=0)
+    d = setup(w)
+    d.lens[1] = 0
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    assert cnt[1].tolist() == [0] * w.num_kv_heads and bool((ids[1] == -1).all())
+    assert float(out[1].float().abs().max()) == 0.0
+    for h in range(w.num_kv_heads):
+        check_unit_decode(d, 0, h, int(d.lens[0]), 0, w.budget_tokens, out, lse, ids, cnt, scores)
+
+
+def test_budget_errors_and_argument_checks():
+    from paper_2609_26300_b200 import binding
+    w = small(decode_steps=0)
+    d = setup(w)
+    q = dev_q(d)
+    with pytest.raises(binding.CompKVError) as e:
+        d.ckv.decode(q, d.k_pool, d.v_pool, d.table, d.lens, d.max_len, 16 * 2)    # K = 2 < 3 mandatory blocks
+    assert e.value.status == binding.CKV_ERR_BUDGET_TOO_SMALL
+    with pytest.raises(binding.CompKVError) as e:
+        d.ckv.decode(q, d.k_pool, d.v_pool, d.table, d.lens, 10 ** 8, 16 * 8)      # longer than the layout allows
+    assert e.value.status == binding.CKV_ERR_INVALID_ARG
+    with pytest.raises(binding.CompKVError):
+        binding.CompKV(12, 4, 1, 8, 8)                                              # G = 3 unsupported
+    with pytest.raises(binding.CompKVError):
+        binding.CompKV(8, 2, 1, 8, 8, block_size=48)
+
+
+def test_bad_page_id_sets_status_and_does_not_fault():
+    w = small(batch=1, decode_steps=0)
+    d = setup(w)
+    from paper_2609_26300_b200 import binding
+    d.table[0, 5] = d.k_pool.shape[0] + 7      # outside the pool: must be skipped, not dereferenced
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() & binding.CKV_DEV_BAD_PAGE
+    d.ckv.dense_decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() & binding.CKV_DEV_BAD_PAGE
+    assert d.ckv.read_status() == 0            # reading clears it
+
+
+def test_append_past_capacity_sets_status():
+    from paper_2609_26300_b200 import binding
+    w = small(batch=1, ctx=16 * 4, decode_steps=0)
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    z = torch.zeros(1, w.num_kv_heads, 128, dtype=d.dtype, device="cuda")
+    d.ckv.append(d.k_pool, d.v_pool, d.table, d.lens, z, z)       # table has room for exactly ctx tokens
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() & binding.CKV_DEV_SEQ_FULL
+    assert int(d.lens[0]) == 16 * 4
+
+
+# ---- decode steps with appends ----------------------------------------------------------------------------------------
+
+def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False):
+    w = d.w
+    n0 = d.lens.cpu().numpy().copy()
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    for t in range(steps):
+        k_new, v_new = synth.appended_rows(w, t)
+        q = synth.queries(w, t)
+        max_len = d.max_len + t + 1
+        if use_host_call:
+            kcap = budget // w.block_size
+            hq = torch.from_numpy(q).to(d.dtype).pin_memory()
+            hk = torch.from_numpy(k_new).to(d.dtype).pin_memory(); hv = torch.from_numpy(v_new).to(d.dtype).pin_memory()
+            ho = torch.empty(w.batch, w.num_q_heads, 128, dtype=d.dtype).pin_memory()
+            hi = torch.empty(w.batch, w.num_kv_heads, kcap, dtype=torch.int32).pin_memory()
+            hc = torch.empty(w.batch, w.num_kv_heads, dtype=torch.int32).pin_memory()
+            d.ckv.step_host(hq, hk, hv, d.k_pool, d.v_pool, d.table, d.lens, max_len, budget, ho, hi, hc)
+            out, ids, cnt = ho, hi, hc
+            lse = None
+        else:
+            d.ckv.append(d.k_pool, d.v_pool, d.table, d.lens, torch.from_numpy(k_new).to(d.dtype).cuda(),
+                         torch.from_numpy(v_new).to(d.dtype).cuda())
+            out, lse, ids, cnt = d.ckv.decode(torch.from_numpy(q).to(d.dtype).cuda(), d.k_pool, d.v_pool, d.table,
+                                              d.lens, max_len, budget)
+        if t in check_steps:
+            scores = d.ckv.copy_scores(w.batch)
+            torch.cuda.synchronize()
+            for s, h in sample_units:
+                if lse is None:   # the host call returns no lse: compare outputs and ids only
+                    G = w.group
+                    qq, K, V = unit_inputs(w, s, h, int(n0[s]) + t + 1, t)
+                    st = O.stats(K, V, w.block_size)
+                    sc = O.scores(qq, st)
+                    ref_ids = O.select(sc.S, budget // w.block_size)
+                    got = ids[s, h, :int(cnt[s, h])].numpy()
+                    same = check_ids(got, ref_ids, sc.S, budget // w.block_size)
+                    ref, _ = O.sparse(qq, K, V, st, ref_ids if same else got)
+                    assert rel_inf(out[s, h * G:(h + 1) * G].double().numpy(), ref) <= OUT_TOL[d.dtype]
+                else:
+                    check_unit_decode(d, s, h, int(n0[s]) + t + 1, t, budget, out, lse, ids, cnt, scores)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() == 0
+    assert np.array_equal(d.lens.cpu().numpy(), n0 + steps)
+
+
+def test_decode_loop_small_with_appends():
+    w = small(ctx_min=16 * 30 + 1, ctx=16 * 60, decode_steps=36)
+    d = setup(w)
+    decode_loop(d, 36, w.budget_tokens, set(range(36)), all_units(w))
+
+
+def test_decode_loop_through_host_buffer_call():
+    w = small(ctx=16 * 50 + 15, decode_steps=20)
+    d = setup(w)
+    decode_loop(d, 20, w.budget_tokens, {0, 1, 2, 16, 17, 19}, all_units(w), use_host_call=True)
