@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the CompKV decode step (append + compensated sparse decode) at 128K context.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload: benchmark configs[2] -- Llama-3-8B-shaped layer, batch 4, 32 query / 8 KV heads,
+head_dim 128, bf16 paged KV, 131072 prefilled tokens per sequence, block size 16, budget 2048
+tokens; every step appends one token per sequence (summary update) and decodes one query.
+Seeded synthetic inputs.  One JSON line on stdout (rank 0).
+
+A "step" is ckv_append + ckv_decode (summary update, summary scan, scoring + top-k, exact attention
+on the selected blocks, compensation merge).  The one-off prefill summary build and the dense
+baseline are timed separately and reported in the same line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "sparse decode-attn us/step at 128K ctx (append + decode, batch 4)"
+UNIT = "us/step"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+PAPER_CONTEXT = {"speedup_vs_full": 6.85, "hardware": "NVIDIA H100 80GB HBM3, CPU-offload pipeline, batch 1",
+                 "setting": "128K endpoint, budget 512, r=4 (1.456 ms vs 9.966 ms)", "note": "context only"}
+# DRAM traffic per algorithmic byte of the summary-scan kernel, from the committed ncu capture
+# (profiles/): None until a capture has been summarised.
+SCAN_TRAFFIC_RATIO = None
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period: float = 0.002):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def workload(total_steps: int):
+    from paper_2609_26300_b200 import synth
+    return synth.CONFIGS[3].with_(decode_steps=total_steps)
+
+
+def step_inputs(w, n_steps: int):
+    """Per-step queries and appended rows as numpy arrays [steps][...] (bf16 values in float32)."""
+    from paper_2609_26300_b200 import synth
+    q = np.stack([synth.queries(w, t) for t in range(n_steps)])
+    k_new = np.zeros((n_steps, w.batch, w.num_kv_heads, w.head_dim), np.float32)
+    v_new = np.zeros_like(k_new)
+    for s in range(w.batch):
+        for h in range(w.num_kv_heads):
+            kt, vt = synth.unit_tail(w, s, h)
+            k_new[:, s, h] = kt[:n_steps]
+            v_new[:, s, h] = vt[:n_steps]
+    return q, k_new, v_new
+
+
+def oracle_sample_setup(w):
+    """Inputs of the oracle's sample: every KV head of sequence 0, prefill + the appended rows."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import compkv_oracle as O
+    from paper_2609_26300_b200 import synth
+    heads = list(range(w.num_kv_heads))
+    cores = min(os.cpu_count() or 1, len(heads))
+    with ThreadPoolExecutor(cores) as ex:
+        kv = list(ex.map(lambda h: synth.unit_kv(w, 0, h), heads))
+        n0 = int(synth.seq_lens(w)[0])
+        stats = list(ex.map(lambda i: O.stats(kv[i][0][:n0], kv[i][1][:n0], w.block_size, w.var_groups), heads))
+    return kv, stats, n0, cores
+
+
+def oracle_step(w, kv, stats, n0, cores, step: int):
+    """One oracle decode step (summary update, scores, selection, compensated attention) on the sample units.
+    Returns wall seconds; stats are advanced in place."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import compkv_oracle as O
+    from paper_2609_26300_b200 import synth
+    q = synth.queries(w, step)[0]
+    n = n0 + step + 1
+    G = w.group
+
+    def one(h):
+        K, V = kv[h][0][:n], kv[h][1][:n]
+        stats[h] = O.append(stats[h], K, V)
+        O.decode_unit(q[h * G:(h + 1) * G], K, V, stats[h], w.budget_tokens)
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(cores) as ex:
+        list(ex.map(one, range(len(kv))))
+    return time.perf_counter() - t0
+
+
+def required_bytes(w, lens, sel_tokens_per_unit):
+    """Bytes one decode step must read: every block summary once, plus K and V of the selected tokens."""
+    stats = 0
+    for n in lens:
+        x = -(-int(n) // w.block_size)
+        stats += w.num_kv_heads * x * (2 * w.head_dim * 4 + 4 * w.var_groups)
+    sel = int(np.sum(sel_tokens_per_unit)) * 2 * w.head_dim * 2
+    return stats, sel
+
+
+def reference_arm(args):
+    """Times the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from oracle import compkv_oracle as O  # noqa: F401
+    w = workload(args.warmup + args.steps)
+    kv, stats, n0, cores = oracle_sample_setup(w)
+    scale = w.batch   # the sample is one of `batch` equally sized sequences
+    for t in range(args.warmup):
+        oracle_step(w, kv, stats, n0, cores, t)
+    times = [oracle_step(w, kv, stats, n0, cores, args.warmup + t) for t in range(args.steps)]
+    us = float(np.mean(times)) * 1e6 * scale
+    sample = ("CPU oracle (fp64, plain C) decode step on the %d KV heads of sequence 0 (1 of %d sequences), "
+              "wall time x %d" % (w.num_kv_heads, w.batch, scale))
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "configs[2] llama8b_128k_b4: batch 4, 32q/8kv heads, d128, ctx 131072, "
+                                   "block 16, budget 2048", "sample": sample},
+            "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--profile-steps", type=int, default=48)
+    ap.add_argument("--e2e-steps", type=int, default=48)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+
+    import torch
+    from paper_2609_26300_b200 import binding, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    W, K, KP, KE = max(args.warmup, 3), args.steps, args.profile_steps, args.e2e_steps
+    total = W + K + KP + KE + W
+    w = workload(total)
+    dev = torch.device("cuda", local)
+
+    # ---- inputs: every rank holds a full replica of the workload (the path does not shard) ----
+    k_pool, v_pool, table, lens = synth.make_pools(w, threads=min(8, os.cpu_count() or 1))
+    q_np, kn_np, vn_np = step_inputs(w, total)
+    max_blocks = synth.pages_per_seq(w)
+    ckv = binding.CompKV(w.num_q_heads, w.num_kv_heads, w.batch, max_blocks, k_pool.shape[0],
+                         block_size=w.block_size, var_groups=w.var_groups, device=str(dev))
+    k_pool, v_pool, table, lens = (t.to(dev) for t in (k_pool, v_pool, table, lens))
+    q_all = torch.from_numpy(q_np).to(torch.bfloat16).to(dev)
+    kn_all = torch.from_numpy(kn_np).to(torch.bfloat16).to(dev)
+    vn_all = torch.from_numpy(vn_np).to(torch.bfloat16).to(dev)
+    n0 = int(lens.max())
+    max_len = n0 + total
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    outputs = ckv.alloc_outputs(w.batch, w.budget_tokens)
+
+    def l2_flush():
+        flush.zero_()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- prefill summary build (timed separately) ----
+    build_ms = []
+    for i in range(5):
+        l2_flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); ckv.stats_build(k_pool, v_pool, table, lens, n0); e1.record()
+        torch.cuda.synchronize()
+        build_ms.append(e0.elapsed_time(e1))
+    build_us = float(np.median(build_ms[2:])) * 1e3
+    build_bytes = sum(int(n) for n in lens.tolist()) * w.num_kv_heads * 2 * w.head_dim * 2 + \
+        required_bytes(w, lens.tolist(), 0)[0]
+
+    # ---- one step as a CUDA graph over static input buffers ----
+    sq, sk, sv = q_all[0].clone(), kn_all[0].clone(), vn_all[0].clone()
+    step = 0
+
+    def eager_step(t):
+        ckv.append(k_pool, v_pool, table, lens, kn_all[t], vn_all[t])
+        ckv.decode(q_all[t], k_pool, v_pool, table, lens, max_len, w.budget_tokens, outputs)
+
+    for _ in range(W):           # untimed eager warm-up (also pages in the kernels before capture)
+        eager_step(step); step += 1
+    torch.cuda.synchronize()
+    launches0 = ckv.launch_count()
+    graph = torch.cuda.CUDAGraph()
+    sq.copy_(q_all[step]); sk.copy_(kn_all[step]); sv.copy_(vn_all[step])
+    with torch.cuda.graph(graph):
+        ckv.append(k_pool, v_pool, table, lens, sk, sv)
+        ckv.decode(sq, k_pool, v_pool, table, lens, max_len, w.budget_tokens, outputs)
+    launches_per_step = ckv.launch_count() - launches0
+    # capture does not execute: seq_lens is unchanged, the captured step runs on replay
+
+    def graph_step(t, ev=None):
+        sq.copy_(q_all[t]); sk.copy_(kn_all[t]); sv.copy_(vn_all[t])
+        l2_flush()
+        if ev is not None:
+            ev[0].record()
+        graph.replay()
+        if ev is not None:
+            ev[1].record()
+
+    for _ in range(W):
+        graph_step(step); step += 1
+    sync_all()
+    sampler = ClockSampler(local)
+    sampler.start()
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    t_wall0 = time.perf_counter()
+    for i in range(K):
+        graph_step(step, events[i]); step += 1
+    sync_all()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    step_ms = np.array([a.elapsed_time(b) for a, b in events])
+    ms_per_step = float(step_ms.mean())
+    sel_cnt = outputs[3].cpu().numpy()
+    lens_now = lens.cpu().numpy()
+    stats_b, sel_b = required_bytes(w, lens_now, sel_cnt * w.block_size)
+    assert ckv.read_status() == 0
+
+    # ---- per-kernel durations (events between the launches), L2 flushed before each step ----
+    stage = np.zeros((KP, 5))
+    for i in range(KP):
+        l2_flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); ckv.append(k_pool, v_pool, table, lens, kn_all[step], vn_all[step]); e1.record()
+        _, ms = ckv.decode_profile(q_all[step], k_pool, v_pool, table, lens, max_len, w.budget_tokens, outputs)
+        stage[i, 0] = e0.elapsed_time(e1)
+        stage[i, 1:] = ms
+        step += 1
+    stage_us = stage[KP // 4:].mean(0) * 1e3
+    scan_us = float(stage_us[1])
+
+    # ---- dense decode attention over the same cache ----
+    dense_ms = []
+    dout = torch.empty_like(outputs[0])
+    for i in range(12):
+        l2_flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); ckv.dense_decode(q_all[step - 1], k_pool, v_pool, table, lens, max_len, dout, outputs[1]); e1.record()
+        torch.cuda.synchronize()
+        dense_ms.append(e0.elapsed_time(e1))
+    dense_us = float(np.median(dense_ms[3:])) * 1e3
+    dense_bytes = int(lens_now.sum()) * w.num_kv_heads * 2 * w.head_dim * 2
+
+    # ---- end to end from pinned host buffers through ckv_step_host ----
+    kcap = w.budget_tokens // w.block_size
+    hq = torch.from_numpy(q_np).to(torch.bfloat16).pin_memory()
+    hk = torch.from_numpy(kn_np).to(torch.bfloat16).pin_memory()
+    hv = torch.from_numpy(vn_np).to(torch.bfloat16).pin_memory()
+    ho = torch.empty(w.batch, w.num_q_heads, w.head_dim, dtype=torch.bfloat16).pin_memory()
+    hi = torch.empty(w.batch, w.num_kv_heads, kcap, dtype=torch.int32).pin_memory()
+    hc = torch.empty(w.batch, w.num_kv_heads, dtype=torch.int32).pin_memory()
+    e2e_s = []
+    for i in range(KE):
+        l2_flush()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ckv.step_host(hq[step], hk[step], hv[step], k_pool, v_pool, table, lens, max_len, w.budget_tokens, ho, hi, hc)
+        e2e_s.append(time.perf_counter() - t0)
+        step += 1
+    e2e_us = float(np.mean(e2e_s[KE // 4:])) * 1e6
+    h2d = hq[0].numel() * 2 + hk[0].numel() * 2 + hv[0].numel() * 2
+    d2h = ho.numel() * 2 + hi.numel() * 4 + hc.numel() * 4
+    assert ckv.read_status() == 0
+
+    # ---- max over ranks ----
+    vals = torch.tensor([ms_per_step, e2e_us, scan_us, dense_us], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    ms_per_step, e2e_us, scan_us, dense_us = (float(x) for x in vals.tolist())
+    us_per_step = ms_per_step * 1e3
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    peak, peak_kind = measured_peak()
+    req = stats_b + sel_b
+    step_gbs = req / (us_per_step * 1e-6) / 1e9
+    scan_gbs = stats_b / (scan_us * 1e-6) / 1e9
+    line = {
+        "metric": METRIC, "value": us_per_step, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "configs[2] llama8b_128k_b4: batch 4, 32q/8kv heads, d128, ctx 131072 (+ appended "
+                               "tokens), block 16, budget 2048, r=4, fp32 summaries, bf16 paged KV",
+                   "step": "ckv_append + ckv_decode replayed as one CUDA graph; CUDA events around each replay",
+                   "l2": "flushed between steps (256 MiB memset outside the events); per-step inputs exceed L2",
+                   "replicas": "every rank runs the whole workload (the path does not shard)",
+                   "kv_storage": "bf16", "seed": w.seed},
+        "tokens_per_s": world * w.batch / (us_per_step * 1e-6),
+        "required_bytes_per_step": req, "hbm_gbs": step_gbs,
+        "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS, "frac_of_%s_peak" % peak_kind: step_gbs / peak,
+        "dense_us": dense_us, "dense_gbs": dense_bytes / (dense_us * 1e-6) / 1e9,
+        "speedup_vs_dense": dense_us / us_per_step,
+        "stages_us": {"append": float(stage_us[0]), "scan": float(stage_us[1]), "select": float(stage_us[2]),
+                      "attention": float(stage_us[3]), "merge": float(stage_us[4]),
+                      "note": "eager launches with events between kernels; their sum exceeds the graph replay"},
+        "stats_build": {"us": build_us, "gbs": build_bytes / (build_us * 1e-6) / 1e9, "bytes": build_bytes},
+        "roofline": {"kernel": "ckv_scan_kernel", "bound": "hbm", "achieved": scan_gbs, "peak": peak,
+                     "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": scan_gbs / peak,
+                     "algorithmic_bytes": stats_b,
+                     "traffic": None if SCAN_TRAFFIC_RATIO is None else SCAN_TRAFFIC_RATIO * stats_b},
+        "clocks": clocks,
+        "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "call": "ckv_step_host (pinned host q/k_new/v_new in, out/sel_ids/sel_cnt back, stream sync)"},
+        "gpu_launches": int(launches_per_step * K),
+        "wall_s_timed_region": t_wall,
+        "paper_context": PAPER_CONTEXT,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        kv, stats, n0s, cores = oracle_sample_setup(w)
+        reps = 6
+        oracle_step(w, kv, stats, n0s, cores, 0)
+        ts = [oracle_step(w, kv, stats, n0s, cores, 1 + i) for i in range(reps)]
+        cpu_us = float(np.mean(ts)) * 1e6 * w.batch
+        line["cpu_baseline"] = {"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": "oracle decode step (summary update, scores, top-k, compensated attention) "
+                                          "on the %d KV heads of sequence 0, %d steps, wall time x %d sequences"
+                                          % (w.num_kv_heads, reps, w.batch)}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -65,7 +65,8 @@ enum ckv_status {
 enum ckv_device_status {
   CKV_DEV_BAD_PAGE = 1,     /* page table entry outside [0, num_pages): the page was skipped */
   CKV_DEV_SEQ_FULL = 2,     /* append past max_blocks_per_seq * block_size: the token was dropped */
-  CKV_DEV_NONFINITE = 4     /* a block score was NaN/Inf: it was ranked as 0 */
+  CKV_DEV_NONFINITE = 4,    /* a block score was NaN/Inf: it was ranked as 0 */
+  CKV_DEV_TIMEOUT = 8       /* a bounded wait inside a kernel ran out: the step's results are invalid */
 };
 
 typedef struct ckv_layout {
@@ -169,7 +170,8 @@ int ckv_copy_scores(ckv_ctx *ctx, float *dst, int batch, ckv_stream stream);
 /* One whole decode step from HOST buffers: copies q, k_new, v_new to the device, runs
  * ckv_append then ckv_decode, copies out / sel_ids / sel_cnt back and synchronises the stream.
  * Host buffers should be pinned; device staging comes out of the workspace.  seq_lens (device)
- * is incremented.  max_seq_len_host bounds the lengths AFTER the append. */
+ * is incremented.  max_seq_len_host bounds the lengths AFTER the append.  The id staging area holds
+ * max_blocks_per_seq ids per unit: budget_tokens / block_size beyond that is CKV_ERR_INVALID_ARG. */
 int ckv_step_host(ckv_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
                   void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens, int batch,
                   int max_seq_len_host, int budget_tokens, void *out_host, int32_t *sel_ids_host,

@@ -37,7 +37,10 @@ class ckv_layout(ctypes.Structure):
 class CompKVError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
-        super().__init__("%s failed: %s (status %d)" % (what, strerror(status), status))
+        extra = ""
+        if status == CKV_ERR_CUDA:
+            extra = ", cudaError %d" % load().ckv_last_cuda_error()
+        super().__init__("%s failed: %s (status %d%s)" % (what, strerror(status), status, extra))
 
 
 _lib = None

@@ -50,7 +50,7 @@ Regions regions(const ckv_layout *L) {
   R.status = o; o = align_up(o + 256, 256);
   R.ls = o;     o = align_up(o + rows * G * sizeof(float2), 256);
   R.scores = o; o = align_up(o + rows * 4, 256);
-  R.comp = o;   o = align_up(o + units * CKV_MAX_CHUNKS * G * CKV_PART_STRIDE * 4, 256);
+  R.comp = o;   o = align_up(o + (units + CKV_MAX_SCAN_CTAS) * G * CKV_PART_STRIDE * 4, 256);
   R.attn = o;   o = align_up(o + units * CKV_MAX_SPLITS * G * CKV_PART_STRIDE * 4, 256);
   R.stage_q = o;    o = align_up(o + (size_t)L->max_batch * L->num_q_heads * CKV_D * esz, 256);
   R.stage_knew = o; o = align_up(o + units * CKV_D * esz, 256);
@@ -151,6 +151,10 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   c->stage_out = R.stage_out; c->stage_ids = R.stage_ids; c->stage_cnt = R.stage_cnt;
   c->launches = 0;
   cudaError_t e = ckv_configure_kernels();
+  if (e == cudaSuccess) e = ckv_configure_scan(c);
+  int dev_id = 0;
+  if (e == cudaSuccess) e = cudaGetDevice(&dev_id);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev_id);
   if (e == cudaSuccess) e = cudaMemsetAsync(P.status, 0, 256, (cudaStream_t)stream);
   if (e != cudaSuccess) { delete c; return cuda_fail(e); }
   *out = c;
@@ -189,19 +193,18 @@ int decode_impl(ckv_ctx *c, const void *q, const void *k_pool, const void *v_poo
   const ckv_layout &L = c->layout;
   const int kcap = budget_tokens / L.block_size;
   if (budget_tokens <= 0 || kcap <= 0) return CKV_ERR_BUDGET_TOO_SMALL;
-  if (kcap > L.max_blocks_per_seq) return CKV_ERR_INVALID_ARG;
   if (kcap < L.sink_blocks + L.recent_blocks && (long long)kcap * L.block_size < max_seq_len_host)
     return CKV_ERR_BUDGET_TOO_SMALL;
-  int n_chunks = 0, n_splits = 0;
+  int scan_grid = 0, n_splits = 0;
   if (ev) CKV_CUDA(cudaEventRecord(ev[0], s));
-  CKV_CUDA(ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, &n_chunks, s));
+  CKV_CUDA(ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, &scan_grid, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[1], s));
-  CKV_CUDA(ckv_launch_select(c, seq_lens, batch, kcap, sel_ids, sel_cnt, s));
+  CKV_CUDA(ckv_launch_select(c, seq_lens, batch, kcap, scan_grid, sel_ids, sel_cnt, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[2], s));
   CKV_CUDA(ckv_launch_attn(c, false, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, batch,
                            max_seq_len_host, &n_splits, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[3], s));
-  CKV_CUDA(ckv_launch_merge(c, false, seq_lens, sel_cnt, n_splits, n_chunks, batch, out, lse, s));
+  CKV_CUDA(ckv_launch_merge(c, false, seq_lens, sel_cnt, n_splits, scan_grid, batch, out, lse, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[4], s));
   return CKV_OK;
 }

@@ -262,40 +262,77 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
 }
 
 // out_{g} = sum of all partials under one normaliser (Eq. 12).  One CTA per (sequence, query head),
-// one thread per output coordinate.
+// one thread per output coordinate.  Partials: the unit's attention splits and, unless every block
+// was selected, the scan partials of the CTAs whose tile range touched the unit (entries c + unit for
+// c in [c_first, c_last], recomputed here from the same tile arithmetic the scan uses).
+constexpr int kMergeMax = CKV_MAX_SPLITS + CKV_MAX_SCAN_CTAS;
+
 template <typename T>
 __global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *__restrict__ seq_lens,
-                                                          const int *__restrict__ sel_cnt, int kcap, int n_splits,
-                                                          int n_chunks, bool dense, T *__restrict__ out,
+                                                          const int *__restrict__ sel_cnt, int n_splits,
+                                                          int scan_grid, int units, bool dense, T *__restrict__ out,
                                                           float *__restrict__ lse) {
+  __shared__ float s_scale[kMergeMax];
+  __shared__ float s_l[kMergeMax];
+  __shared__ const float *s_ptr[kMergeMax];
+  __shared__ float s_wmax[CKV_D / 32];
+  __shared__ int s_cfirst, s_ccount;
   const int hq = blockIdx.x, s = blockIdx.y, c = threadIdx.x;
   const int G = P.G, unit = s * P.Hkv + hq / G, g = hq % G;
-  const int N = min(seq_lens[s], P.max_blocks * P.bs);
+  const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
   const int X = (N + P.bs - 1) / P.bs;
-  const bool comp = !dense && min(sel_cnt[unit], kcap) < X;
-  const float *ap = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS * G + g) * CKV_PART_STRIDE;
-  const float *cp = P.comp_part + ((size_t)unit * CKV_MAX_CHUNKS * G + g) * CKV_PART_STRIDE;
-  const size_t step = (size_t)G * CKV_PART_STRIDE;
-  float M = -CUDART_INF_F;
-  for (int i = 0; i < n_splits; ++i) M = fmaxf(M, ap[i * step]);
-  if (comp)
-    for (int i = 0; i < n_chunks; ++i) M = fmaxf(M, cp[i * step]);
-  float num = 0.f, den = 0.f;
-  for (int i = 0; i < n_splits; ++i) {
-    const float m = ap[i * step];
-    if (m == -CUDART_INF_F) continue;
-    const float sc = exp2f(m - M);
-    num = fmaf(ap[i * step + 4 + c], sc, num);
-    den = fmaf(ap[i * step + 1], sc, den);
-  }
-  if (comp)
-    for (int i = 0; i < n_chunks; ++i) {
-      const float m = cp[i * step];
-      if (m == -CUDART_INF_F) continue;
-      const float sc = exp2f(m - M);
-      num = fmaf(cp[i * step + 4 + c], sc, num);
-      den = fmaf(cp[i * step + 1], sc, den);
+  const bool comp = !dense && sel_cnt[unit] < X;
+  if (c == 0) {
+    int cfirst = 0, ccount = 0;
+    if (comp) {
+      long long T = 0, T0 = 0;
+      for (int u = 0; u < units; ++u) {
+        const int n = max(min(seq_lens[u / P.Hkv], P.max_blocks * P.bs), 0);
+        const int tiles = ((n + P.bs - 1) / P.bs + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE;
+        if (u == unit) T0 = T;
+        T += tiles;
+      }
+      const long long tpc = (T + scan_grid - 1) / scan_grid;
+      const int my_tiles = (X + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE;
+      cfirst = (int)(T0 / tpc);
+      ccount = (int)((T0 + my_tiles - 1) / tpc) - cfirst + 1;
     }
+    s_cfirst = cfirst; s_ccount = ccount;
+  }
+  __syncthreads();
+  const int n_comp = s_ccount;
+  const int n = n_splits + n_comp;
+  const size_t step = (size_t)G * CKV_PART_STRIDE;
+  const float *ap = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS * G + g) * CKV_PART_STRIDE;
+  const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * G + g) * CKV_PART_STRIDE;
+  float mloc = -CUDART_INF_F;
+  for (int i = c; i < n; i += CKV_D) {
+    const float *p = i < n_splits ? ap + (size_t)i * step : cp + (size_t)(i - n_splits) * step;
+    const float m = p[0];
+    s_ptr[i] = p; s_scale[i] = m; s_l[i] = p[1];
+    mloc = fmaxf(mloc, m);
+  }
+  mloc = warp_max(mloc);
+  if ((c & 31) == 0) s_wmax[c >> 5] = mloc;
+  __syncthreads();
+  float M = s_wmax[0];
+#pragma unroll
+  for (int w = 1; w < CKV_D / 32; ++w) M = fmaxf(M, s_wmax[w]);
+  for (int i = c; i < n; i += CKV_D) s_scale[i] = exp2_diff(s_scale[i], M);
+  __syncthreads();
+  float num = 0.f, den = 0.f;
+  int i = 0;
+  for (; i + 4 <= n; i += 4) {   // four independent loads in flight
+    const float a0 = s_ptr[i][4 + c], a1 = s_ptr[i + 1][4 + c], a2 = s_ptr[i + 2][4 + c], a3 = s_ptr[i + 3][4 + c];
+    num = fmaf(a0, s_scale[i], num); num = fmaf(a1, s_scale[i + 1], num);
+    num = fmaf(a2, s_scale[i + 2], num); num = fmaf(a3, s_scale[i + 3], num);
+    den = fmaf(s_l[i], s_scale[i], den); den = fmaf(s_l[i + 1], s_scale[i + 1], den);
+    den = fmaf(s_l[i + 2], s_scale[i + 2], den); den = fmaf(s_l[i + 3], s_scale[i + 3], den);
+  }
+  for (; i < n; ++i) {
+    if (s_scale[i] != 0.f) num = fmaf(s_ptr[i][4 + c], s_scale[i], num);
+    den = fmaf(s_l[i], s_scale[i], den);
+  }
   const size_t o = ((size_t)s * P.Hq + hq) * CKV_D + c;
   store_out(out + o, N > 0 ? num / den : 0.f);
   if (lse != nullptr && c == 0) lse[(size_t)s * P.Hq + hq] = N > 0 ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
@@ -352,16 +389,15 @@ cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k
 }
 
 cudaError_t ckv_launch_merge(ckv_ctx *c, bool dense, const int *seq_lens, const int *sel_cnt, int n_splits,
-                             int n_chunks, int batch, void *out, float *lse, cudaStream_t st) {
+                             int scan_grid, int batch, void *out, float *lse, cudaStream_t st) {
   const CkvDev &P = c->dev;
   dim3 grid(P.Hq, batch);
-  // kcap is only used to clamp sel_cnt; sel_cnt never exceeds it, so pass a large bound
-  const int kcap = 1 << 30;
+  const int units = batch * P.Hkv;
   if (c->layout.kv_dtype == CKV_BF16)
-    ckv_merge_kernel<__nv_bfloat16><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, kcap, n_splits, n_chunks, dense,
+    ckv_merge_kernel<__nv_bfloat16><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, n_splits, scan_grid, units, dense,
                                                            (__nv_bfloat16 *)out, lse);
   else
-    ckv_merge_kernel<float><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, kcap, n_splits, n_chunks, dense,
+    ckv_merge_kernel<float><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, n_splits, scan_grid, units, dense,
                                                     (float *)out, lse);
   c->launches++;
   return cudaGetLastError();

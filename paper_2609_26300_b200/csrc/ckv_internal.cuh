@@ -11,7 +11,8 @@
 #define CKV_D 128             // head dimension the kernels are written for
 #define CKV_PAGE 16           // tokens per page
 #define CKV_PART_STRIDE 132   // floats per split partial: m, l, pad, pad, acc[128]
-#define CKV_MAX_CHUNKS 64     // scan partials per unit
+#define CKV_SCAN_TILE 16      // blocks per scan tile
+#define CKV_MAX_SCAN_CTAS 512 // persistent scan grid is capped at this many CTAs
 #define CKV_MAX_SPLITS 64     // attention partials per unit
 #define CKV_RESCALE_SLACK 16.0f  // log2 units: running maxima are only raised when exceeded by this much
 
@@ -28,7 +29,7 @@ struct CkvDev {
   // workspace
   float2 *ls;        // [unit][max_blocks][G]  (log block weight estimate l_{g,b}, sigma_hat^2_{g,b})
   float *scores;     // [unit][max_blocks]     S_b
-  float *comp_part;  // [unit][CKV_MAX_CHUNKS][G][CKV_PART_STRIDE]  all-block mean-compensation partials
+  float *comp_part;  // [scan CTA + unit][G][CKV_PART_STRIDE]  all-block mean-compensation partials
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials
   int *status;       // device status word
 };
@@ -41,9 +42,12 @@ struct ckv_ctx {
   // host staging regions inside the workspace (ckv_step_host)
   size_t stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt;
   int64_t launches;
+  int sm_count;
 };
 
-cudaError_t ckv_configure_kernels();
+cudaError_t ckv_configure_kernels();   // selection kernel attributes
+cudaError_t ckv_configure_scan(const ckv_ctx *c);   // scan kernel attributes
+int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len);
 
 // ---- launchers (one per translation unit) ---------------------------------------------------------
 cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int *page_table,
@@ -51,14 +55,14 @@ cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v
 cudaError_t ckv_launch_append(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
                               const void *k_new, const void *v_new, int batch, cudaStream_t st);
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
-                            int *n_chunks_out, cudaStream_t st);
-cudaError_t ckv_launch_select(ckv_ctx *c, const int *seq_lens, int batch, int kcap, int *sel_ids, int *sel_cnt,
-                              cudaStream_t st);
+                            int *grid_out, cudaStream_t st);
+cudaError_t ckv_launch_select(ckv_ctx *c, const int *seq_lens, int batch, int kcap, int scan_grid, int *sel_ids,
+                              int *sel_cnt, cudaStream_t st);
 cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                             const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
                             int kcap, int batch, int max_len, int *n_splits_out, cudaStream_t st);
 cudaError_t ckv_launch_merge(ckv_ctx *c, bool dense, const int *seq_lens, const int *sel_cnt, int n_splits,
-                             int n_chunks, int batch, void *out, float *lse, cudaStream_t st);
+                             int scan_grid, int batch, void *out, float *lse, cudaStream_t st);
 
 // ---- device helpers -----------------------------------------------------------------------------------
 #ifdef __CUDACC__

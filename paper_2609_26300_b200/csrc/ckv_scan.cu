@@ -1,7 +1,7 @@
-// Summary scan: one streaming pass over every block summary of a unit (Eq. 8-9 and the
-// compensation sums of Eq. 12).
+// Summary scan: one streaming pass over every block summary (Eq. 8-9 and the compensation sums
+// of Eq. 12), as a persistent, bulk-copy-pipelined kernel.
 //
-// For every block b and query head g of the unit the pass computes
+// For every block b and query head g of a unit the pass computes
 //   zbar_{g,b}        = q_g . kbar_b * scale                      (block-mean logit, Sec. 4.1)
 //   sigma_hat^2_{g,b} = scale^2 sum_t w_{g,t} Dbar_{b,t}         (Eq. 8 with 1/d = scale^2, w_{g,t} = sum_{i in G_t} q_{g,i}^2)
 //   l_{g,b}           = log|b| + zbar + sigma_hat^2 / 2           (log of the numerator of Eq. 9)
@@ -11,214 +11,383 @@
 // are taken out again by the attention kernel.  That way kbar, Dbar and vbar are each read
 // from HBM exactly once per decode step.
 //
-// Mapping: 16 lanes share one block row (128 fp32 = 32 float4; lane li takes float4 li and li+16,
-// so each load instruction of a half warp covers 256 contiguous bytes); a warp does two blocks at
-// a time and the 8 warps of a CTA cover 16 consecutive blocks per iteration.  Each lane keeps its
-// 8 coordinates of q (all G heads) and of the G output accumulators in registers.
+// Schedule: the summaries of all units are cut into tiles of 16 consecutive blocks (16 KB of mean
+// keys + 16 KB of mean values + the variances); the tiles, in (unit, position) order, are split
+// into one contiguous range per CTA and the grid is one CTA per SM.  A producer thread streams the
+// CTA's tiles into a ring of shared-memory stages with cp.async.bulk, completion on mbarriers;
+// eight consumer warps take two blocks each per tile.  A CTA writes one partial per unit it
+// touched; partial (CTA c, unit u) lives in entry c + u, which is unique because the (c, u)
+// pairs that occur form a monotone staircase.
+//
+// Consumer mapping: 16 lanes share one block row (128 fp32 = 32 float4; lane li takes float4 li and
+// li + 16, conflict-free in shared memory); each lane keeps its 8 coordinates of q (all G heads) and
+// of the G output accumulators in registers.
 #include "ckv_internal.cuh"
+#include "ckv_pipe.cuh"
 
 namespace {
+
+using namespace ckv_pipe;
 
 template <int G> struct Log2 { static constexpr int v = 1 + Log2<G / 2>::v; };
 template <> struct Log2<1> { static constexpr int v = 0; };
 
+constexpr int TB = CKV_SCAN_TILE;   // blocks per tile
+constexpr int kMaxStages = 8;
+constexpr int kThreads = 256;       // 8 warps, all consumers; thread 0 also issues the bulk copies
+constexpr int kLag = 2;             // a stage is refilled two tiles after it was consumed
+
+struct UnitInfo { int N, X, tiles; };
+
+__device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *__restrict__ seq_lens, int u) {
+  UnitInfo ui;
+  ui.N = min(seq_lens[u / P.Hkv], P.max_blocks * P.bs);
+  ui.N = max(ui.N, 0);
+  ui.X = (ui.N + P.bs - 1) / P.bs;
+  ui.tiles = (ui.X + TB - 1) / TB;
+  return ui;
+}
+
 template <int G, typename QT>
-__global__ void __launch_bounds__(256, (G <= 4) ? 2 : 1)
-ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_lens, int chunk) {
+__global__ void __launch_bounds__(kThreads, 1)
+ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_lens, int units, int stages) {
   constexpr int SH = 4 - Log2<G>::v;   // lane (g << SH) of a half warp owns head g after the reduction
+  extern __shared__ __align__(128) float stage_mem[];
+  __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
   __shared__ float sq[G][CKV_D];
   __shared__ __align__(16) float sw[CKV_D][G];
   __shared__ __align__(16) float red[8][G][CKV_PART_STRIDE];
+  __shared__ int s_u0, s_tl0, s_count, s_abort, s_issued, s_consumed;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 4, li = lane & 15;
-  const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
-  const int N = min(seq_lens[s], P.max_blocks * P.bs);
-  const int X = (N + P.bs - 1) / P.bs;
-  const int c0 = blockIdx.x * chunk;
-  const int c1 = min(c0 + chunk, X);
-  float *part = P.comp_part + ((size_t)unit * CKV_MAX_CHUNKS + blockIdx.x) * G * CKV_PART_STRIDE;
-  if (c0 >= X) {   // nothing here: leave an empty partial
-    if (tid < G) { part[tid * CKV_PART_STRIDE] = -CUDART_INF_F; part[tid * CKV_PART_STRIDE + 1] = 0.f; }
-    return;
-  }
+  const bool dbar_bulk = P.r >= 4;   // smaller rows cannot keep the 16-byte alignment bulk copies need
+  const int stage_floats = TB * 2 * CKV_D + (dbar_bulk ? TB * P.r : 0);
 
-  for (int idx = tid; idx < G * CKV_D; idx += 256)
-    sq[idx / CKV_D][idx % CKV_D] = to_float(q[((size_t)s * P.Hq + h * G) * CKV_D + idx]);
-  __syncthreads();
-  for (int idx = tid; idx < P.r * G; idx += 256) {
-    const int t = idx / G, g = idx % G;
-    float w = 0.f;
-    for (int i = 0; i < CKV_D; ++i)
-      if (group_of(i, P.r, P.glayout) == t) w = fmaf(sq[g][i], sq[g][i], w);
-    sw[t][g] = w;
-  }
-  __syncthreads();
-
-  float qr[G][8];
-#pragma unroll
-  for (int g = 0; g < G; ++g)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      qr[g][i] = sq[g][4 * li + i] * P.scale;
-      qr[g][4 + i] = sq[g][64 + 4 * li + i] * P.scale;
-    }
-
-  const size_t row0 = (size_t)unit * P.max_blocks;
-  const float4 *km4 = reinterpret_cast<const float4 *>(P.kmean + row0 * CKV_D);
-  const float4 *vm4 = reinterpret_cast<const float4 *>(P.vmean + row0 * CKV_D);
-  const float *db = P.dbar + row0 * P.r;
-  float2 *ls = P.ls + row0 * G;
-
-  float acc[G][8], m_ref[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    m_ref[g] = -CUDART_INF_F;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
-  }
-  float m_my = -CUDART_INF_F, l_my = 0.f;
-  const int myg = li >> SH;
-  const float log_bs = logf((float)P.bs);
-  const float log_last = logf((float)(N - (X - 1) * P.bs));
-  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
-
-  int b = c0 + warp * 2 + gid;
-  float4 k0 = zero4, k1 = zero4, v0 = zero4, v1 = zero4;
-  if (b < c1) {
-    k0 = __ldg(km4 + (size_t)b * 32 + li); k1 = __ldg(km4 + (size_t)b * 32 + 16 + li);
-    v0 = __ldg(vm4 + (size_t)b * 32 + li); v1 = __ldg(vm4 + (size_t)b * 32 + 16 + li);
-  }
-  for (int base = c0; base < c1; base += 16) {
-    const bool valid = b < c1;
-    const float kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
-    const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    const int bn = b + 16;
-    if (bn < c1) {   // prefetch the next rows while this one is being reduced
-      k0 = __ldg(km4 + (size_t)bn * 32 + li); k1 = __ldg(km4 + (size_t)bn * 32 + 16 + li);
-      v0 = __ldg(vm4 + (size_t)bn * 32 + li); v1 = __ldg(vm4 + (size_t)bn * 32 + 16 + li);
-    }
-    float red_v[2 * G];
-#pragma unroll
-    for (int g = 0; g < G; ++g) { red_v[2 * g] = 0.f; red_v[2 * g + 1] = 0.f; }
-    if (valid) {
-      for (int t = li; t < P.r; t += 16) {
-        const float dv = __ldg(db + (size_t)b * P.r + t);
-#pragma unroll
-        for (int g = 0; g < G; ++g) red_v[2 * g + 1] = fmaf(sw[t][g], dv, red_v[2 * g + 1]);
+  if (tid == 0) {
+    long long T = 0;
+    for (int u = 0; u < units; ++u) T += unit_info(P, seq_lens, u).tiles;
+    const long long tpc = (T + gridDim.x - 1) / gridDim.x;
+    const long long first = (long long)blockIdx.x * tpc;
+    long long cnt = T - first;
+    if (cnt > tpc) cnt = tpc;
+    if (cnt < 0) cnt = 0;
+    int u0 = 0, tl0 = 0;
+    if (cnt > 0) {
+      long long accum = 0;
+      for (int u = 0; u < units; ++u) {
+        const int t = unit_info(P, seq_lens, u).tiles;
+        if (first < accum + t) { u0 = u; tl0 = (int)(first - accum); break; }
+        accum += t;
       }
     }
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float z = 0.f;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) z = fmaf(qr[g][i], kk[i], z);
-      red_v[2 * g] = z;
-    }
-    reduce16<2 * G, 2>(red_v, li);
-    const float zbar = red_v[0];
-    const float sig = red_v[1] * (P.scale * P.scale);   // Eq. 8's 1/d is the squared logit scale
-    const float logc = (b == X - 1) ? log_last : log_bs;
-    const float ell = logc + zbar + 0.5f * sig;
-    if (valid && (li & ((1 << SH) - 1)) == 0) ls[(size_t)b * G + myg] = make_float2(ell, sig);
-    // compensation weight of this block for head myg: |b| e^{zbar}, in log2 units
-    const float zl2 = valid ? (zbar + logc) * kLog2e : -CUDART_INF_F;
-    if (__any_sync(0xffffffffu, zl2 > m_my + CKV_RESCALE_SLACK)) {
+    s_u0 = u0; s_tl0 = tl0; s_count = (int)cnt; s_abort = 0; s_issued = 0; s_consumed = 0;
+    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], 8); }
+    fence_barrier_init();
+  }
+  __syncthreads();
+  const int count = s_count;
+  if (count == 0) return;   // uniform: this CTA has no tiles
+
+  {
+    // ---------------- consumers ----------------
+    float qr[G][8], acc[G][8], m_ref[G];
+    float m_my = -CUDART_INF_F, l_my = 0.f, lp_my = 0.f;   // lp: sum of e^{l - m}, the normaliser of Eq. 9
+    const int myg = li >> SH;
+    const float log_bs = logf((float)P.bs);
+    float log_last = 0.f;
+    int u = s_u0, tl = s_tl0, cur = -1;
+    UnitInfo ui = unit_info(P, seq_lens, u);
+    float2 *ls = nullptr;
+    const float *db = nullptr;
+    bool aborted = false;
+    // producer state (thread 0 only): next tile to issue and its position in the walk
+    int p_next = 0, p_u = u, p_tl = tl;
+    UnitInfo p_ui = ui;
+    auto issue_next = [&]() {
+      const int st = p_next % stages, k = p_next / stages;
+      if (k >= 1 && !mbar_wait(&empty_bar[st], (k - 1) & 1)) {
+        atomicOr(P.status, CKV_DEV_TIMEOUT);
+        *(volatile int *)&s_abort = 1;
+        return;
+      }
+      const int b0 = p_tl * TB;
+      const int nb = min(TB, p_ui.X - b0);
+      const size_t row = (size_t)p_u * P.max_blocks + b0;
+      float *sk = stage_mem + (size_t)st * stage_floats;
+      float *sv = sk + TB * CKV_D;
+      const uint32_t kbytes = (uint32_t)nb * CKV_D * 4;
+      const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
+      mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
+      bulk_g2s(sk, P.kmean + row * CKV_D, kbytes, &full_bar[st]);
+      bulk_g2s(sv, P.vmean + row * CKV_D, kbytes, &full_bar[st]);
+      if (dbar_bulk) bulk_g2s(sv + TB * CKV_D, P.dbar + row * P.r, dbytes, &full_bar[st]);
+      *(volatile int *)&s_issued = ++p_next;
+      if (++p_tl == p_ui.tiles) {
+        p_tl = 0;
+        do { ++p_u; } while (p_u < units && (p_ui = unit_info(P, seq_lens, p_u)).tiles == 0);
+      }
+    };
+    if (tid == 0)
+      for (int i = 0; i < stages - kLag && i < count; ++i) issue_next();
+
+    auto flush = [&](int unit_done) {
+      // fold the two half warps, then the 8 warps, into one partial per head of `unit_done`
 #pragma unroll
       for (int g = 0; g < G; ++g) {
-        const float cand = __shfl_sync(0xffffffffu, zl2, (lane & 16) | (g << SH));
-        if (cand > m_ref[g]) {
-          const float sc = exp2_diff(m_ref[g], cand);
+        const float mo = __shfl_xor_sync(0xffffffffu, m_ref[g], 16);
+        const float mn = fmaxf(m_ref[g], mo);
+        const float sc = exp2_diff(m_ref[g], mn);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) acc[g][i] *= sc;
-          if (myg == g) { l_my *= sc; m_my = cand; }
-          m_ref[g] = cand;
+        for (int i = 0; i < 8; ++i) {
+          const float a = acc[g][i] * sc;
+          acc[g][i] = a + __shfl_xor_sync(0xffffffffu, a, 16);
+        }
+        float lg = (myg == g) ? l_my * sc : 0.f;
+        float lpg = (myg == g) ? lp_my * sc : 0.f;
+        lg += __shfl_xor_sync(0xffffffffu, lg, 16);
+        lpg += __shfl_xor_sync(0xffffffffu, lpg, 16);
+        if (myg == g) { l_my = lg; lp_my = lpg; }
+        m_ref[g] = mn;
+      }
+      if (gid == 0) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          float *r = red[warp][g];
+          *reinterpret_cast<float4 *>(r + 4 + 4 * li) = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
+          *reinterpret_cast<float4 *>(r + 4 + 64 + 4 * li) = make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]);
+          if (li == (g << SH)) { r[0] = m_ref[g]; r[1] = l_my; r[2] = lp_my; }
         }
       }
-    }
-    const float wt = valid ? exp2f(zl2 - m_my) : 0.f;
-    l_my += wt;
+      named_barrier(1, kThreads);
+      float *part = P.comp_part + (size_t)(blockIdx.x + unit_done) * G * CKV_PART_STRIDE;
+      for (int idx = tid; idx < G * CKV_D; idx += kThreads) {
+        const int g = idx / CKV_D, i = idx % CKV_D;
+        float M = -CUDART_INF_F;
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const float wg = __shfl_sync(0xffffffffu, wt, (lane & 16) | (g << SH));
+        for (int w = 0; w < 8; ++w) M = fmaxf(M, red[w][g][0]);
+        float num = 0.f, den = 0.f, denp = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[g][i] = fmaf(wg, vv[i], acc[g][i]);
-    }
-    b = bn;
-  }
+        for (int w = 0; w < 8; ++w) {
+          const float sc = exp2_diff(red[w][g][0], M);
+          num = fmaf(red[w][g][4 + i], sc, num);
+          den = fmaf(red[w][g][1], sc, den);
+          denp = fmaf(red[w][g][2], sc, denp);
+        }
+        part[g * CKV_PART_STRIDE + 4 + i] = num;
+        if (i == 0) {
+          part[g * CKV_PART_STRIDE] = M; part[g * CKV_PART_STRIDE + 1] = den; part[g * CKV_PART_STRIDE + 2] = denp;
+        }
+      }
+      named_barrier(1, kThreads);
+    };
 
-  // fold the two half warps, then the 8 warps, into one partial per head
+    for (int it = 0; it < count; ++it) {
+      if (u != cur) {
+        if (cur >= 0) flush(cur);
+        // per-unit setup: the unit's queries, their per-group squared norms, fresh accumulators
+        const int s = u / P.Hkv, h = u % P.Hkv;
+        for (int idx = tid; idx < G * CKV_D; idx += kThreads)
+          sq[idx / CKV_D][idx % CKV_D] = to_float(q[((size_t)s * P.Hq + h * G) * CKV_D + idx]);
+        named_barrier(1, kThreads);
+        for (int idx = tid; idx < P.r * G; idx += kThreads) {
+          const int t = idx / G, g = idx % G;
+          float w = 0.f;
+          for (int i = 0; i < CKV_D; ++i)
+            if (group_of(i, P.r, P.glayout) == t) w = fmaf(sq[g][i], sq[g][i], w);
+          sw[t][g] = w;
+        }
+        named_barrier(1, kThreads);
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const float mo = __shfl_xor_sync(0xffffffffu, m_ref[g], 16);
-    const float mn = fmaxf(m_ref[g], mo);
-    const float sc = exp2_diff(m_ref[g], mn);
+        for (int g = 0; g < G; ++g) {
+          m_ref[g] = -CUDART_INF_F;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float a = acc[g][i] * sc;
-      acc[g][i] = a + __shfl_xor_sync(0xffffffffu, a, 16);
+          for (int i = 0; i < 4; ++i) {
+            qr[g][i] = sq[g][4 * li + i] * P.scale;
+            qr[g][4 + i] = sq[g][64 + 4 * li + i] * P.scale;
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
+        }
+        m_my = -CUDART_INF_F; l_my = 0.f; lp_my = 0.f;
+        log_last = logf((float)(ui.N - (ui.X - 1) * P.bs));
+        const size_t row0 = (size_t)u * P.max_blocks;
+        ls = P.ls + row0 * G;
+        db = P.dbar + row0 * P.r;
+        cur = u;
+      }
+      const int st = it % stages;
+      if (tid == 0 && p_next < count && !*(volatile int *)&s_abort) issue_next();
+      // a wait that runs out marks the step invalid; the walk (and its barriers) still runs to the end
+      if (!aborted && *(volatile int *)&s_abort) aborted = true;
+      if (!aborted && !mbar_wait(&full_bar[st], (it / stages) & 1)) {
+        atomicOr(P.status, CKV_DEV_TIMEOUT);
+        *(volatile int *)&s_abort = 1;
+        aborted = true;
+      }
+      aborted = __any_sync(0xffffffffu, aborted);
+      if (aborted) {
+        if (++tl == ui.tiles) {
+          tl = 0;
+          do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+        }
+        continue;
+      }
+      const float *sk = stage_mem + (size_t)st * stage_floats;
+      const float *sv = sk + TB * CKV_D;
+      const float *sd = sv + TB * CKV_D;
+      const int b0 = tl * TB;
+      const int nb = min(TB, ui.X - b0);
+      const int bl = warp * 2 + gid;
+      const int b = b0 + bl;
+      const bool valid = bl < nb;
+      float4 k0 = *reinterpret_cast<const float4 *>(sk + bl * CKV_D + 4 * li);
+      float4 k1 = *reinterpret_cast<const float4 *>(sk + bl * CKV_D + 64 + 4 * li);
+      float4 v0 = *reinterpret_cast<const float4 *>(sv + bl * CKV_D + 4 * li);
+      float4 v1 = *reinterpret_cast<const float4 *>(sv + bl * CKV_D + 64 + 4 * li);
+      if (nb < TB && !valid) {   // rows past the unit's last block hold stale bytes
+        k0 = k1 = v0 = v1 = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      const float kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
+      const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+      float red_v[2 * G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) { red_v[2 * g] = 0.f; red_v[2 * g + 1] = 0.f; }
+      if (valid) {
+        for (int t = li; t < P.r; t += 16) {
+          const float dv = dbar_bulk ? sd[bl * P.r + t] : __ldg(db + (size_t)b * P.r + t);
+#pragma unroll
+          for (int g = 0; g < G; ++g) red_v[2 * g + 1] = fmaf(sw[t][g], dv, red_v[2 * g + 1]);
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float z = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) z = fmaf(qr[g][i], kk[i], z);
+        red_v[2 * g] = z;
+      }
+      reduce16<2 * G, 2>(red_v, li);
+      const float zbar = red_v[0];
+      const float sig = red_v[1] * (P.scale * P.scale);   // Eq. 8's 1/d is the squared logit scale
+      const float logc = (b == ui.X - 1) ? log_last : log_bs;
+      const float ell = logc + zbar + 0.5f * sig;
+      if (valid && (li & ((1 << SH) - 1)) == 0) ls[(size_t)b * G + myg] = make_float2(ell, sig);
+      // compensation weight of this block for head myg: |b| e^{zbar}, in log2 units
+      const float zl2 = valid ? (zbar + logc) * kLog2e : -CUDART_INF_F;
+      if (__any_sync(0xffffffffu, zl2 > m_my + CKV_RESCALE_SLACK)) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const float cand = __shfl_sync(0xffffffffu, zl2, (lane & 16) | (g << SH));
+          if (cand > m_ref[g]) {
+            const float sc = exp2_diff(m_ref[g], cand);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[g][i] *= sc;
+            if (myg == g) { l_my *= sc; lp_my *= sc; m_my = cand; }
+            m_ref[g] = cand;
+          }
+        }
+      }
+      const float wt = valid ? exp2f(zl2 - m_my) : 0.f;
+      l_my += wt;
+      lp_my = fmaf(wt, exp2f(0.5f * kLog2e * sig), lp_my);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float wg = __shfl_sync(0xffffffffu, wt, (lane & 16) | (g << SH));
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[g][i] = fmaf(wg, vv[i], acc[g][i]);
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&empty_bar[st]);
+        if (warp == 0) *(volatile int *)&s_consumed = it + 1;
+      }
+      if (++tl == ui.tiles) {
+        tl = 0;
+        do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+      }
     }
-    float lg = (myg == g) ? l_my * sc : 0.f;
-    lg += __shfl_xor_sync(0xffffffffu, lg, 16);
-    if (myg == g) l_my = lg;
-    m_ref[g] = mn;
-  }
-  if (gid == 0) {
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float *r = red[warp][g];
-      *reinterpret_cast<float4 *>(r + 4 + 4 * li) = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
-      *reinterpret_cast<float4 *>(r + 4 + 64 + 4 * li) = make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]);
-      if (li == (g << SH)) { r[0] = m_ref[g]; r[1] = l_my; }
-    }
+    if (cur >= 0) flush(cur);
   }
   __syncthreads();
-  for (int idx = tid; idx < G * CKV_D; idx += 256) {
-    const int g = idx / CKV_D, i = idx % CKV_D;
-    float M = -CUDART_INF_F;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) M = fmaxf(M, red[w][g][0]);
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-      const float sc = exp2_diff(red[w][g][0], M);
-      num = fmaf(red[w][g][4 + i], sc, num);
-      den = fmaf(red[w][g][1], sc, den);
-    }
-    part[g * CKV_PART_STRIDE + 4 + i] = num;
-    if (i == 0) { part[g * CKV_PART_STRIDE] = M; part[g * CKV_PART_STRIDE + 1] = den; }
+  if (s_abort && tid == 0) {
+    // leave no bulk copy in flight into this CTA's shared memory: wait (bounded) for every issued fill
+    for (int it = s_consumed; it < s_issued; ++it) mbar_wait(&full_bar[it % stages], (it / stages) & 1);
   }
 }
 
-template <int G>
-cudaError_t launch_g(ckv_ctx *c, const void *q, const int *seq_lens, dim3 grid, int chunk, cudaStream_t st) {
-  if (c->layout.kv_dtype == CKV_BF16)
-    ckv_scan_kernel<G, __nv_bfloat16><<<grid, 256, 0, st>>>(c->dev, (const __nv_bfloat16 *)q, seq_lens, chunk);
-  else
-    ckv_scan_kernel<G, float><<<grid, 256, 0, st>>>(c->dev, (const float *)q, seq_lens, chunk);
+struct ScanCfg { int stages; size_t smem; };
+
+ScanCfg scan_cfg(const CkvDev &P, int G) {
+  const size_t stage_bytes = (size_t)TB * 2 * CKV_D * 4 + (P.r >= 4 ? (size_t)TB * P.r * 4 : 0);
+  const size_t fixed = (size_t)G * CKV_D * 4 + (size_t)CKV_D * G * 4 + (size_t)8 * G * CKV_PART_STRIDE * 4 + 1024;
+  const size_t budget = 220 * 1024 - fixed;
+  int stages = (int)(budget / stage_bytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) stages = 2;
+  return ScanCfg{stages, stages * stage_bytes};
+}
+
+template <int G, typename QT>
+cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, cudaStream_t st) {
+  const ScanCfg cfg = scan_cfg(c->dev, G);
+  ckv_scan_kernel<G, QT><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
   return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_g(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, cudaStream_t st) {
+  if (c->layout.kv_dtype == CKV_BF16) return launch_gt<G, __nv_bfloat16>(c, q, seq_lens, units, grid, st);
+  return launch_gt<G, float>(c, q, seq_lens, units, grid, st);
+}
+
+template <int G, typename QT>
+cudaError_t configure_gt(const ckv_ctx *c) {
+  return cudaFuncSetAttribute(ckv_scan_kernel<G, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)scan_cfg(c->dev, G).smem);
+}
+
+template <int G>
+cudaError_t configure_g(const ckv_ctx *c) {
+  if (c->layout.kv_dtype == CKV_BF16) return configure_gt<G, __nv_bfloat16>(c);
+  return configure_gt<G, float>(c);
 }
 
 }  // namespace
 
-cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
-                            int *n_chunks_out, cudaStream_t st) {
+// Opt in to the dynamic shared memory this context's scan instantiation needs, on the current device.
+cudaError_t ckv_configure_scan(const ckv_ctx *c) {
+  switch (c->dev.G) {
+    case 1: return configure_g<1>(c);
+    case 2: return configure_g<2>(c);
+    case 4: return configure_g<4>(c);
+    case 8: return configure_g<8>(c);
+  }
+  return cudaErrorInvalidValue;
+}
+
+// Grid size the scan uses for a step (one persistent CTA per SM, never more CTAs than tiles).
+int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
+  const CkvDev &P = c->dev;
+  const int xmax = (max_len + P.bs - 1) / P.bs;
+  const long long tiles = (long long)batch * P.Hkv * ((xmax + TB - 1) / TB);
+  long long grid = c->sm_count;
+  if (grid > CKV_MAX_SCAN_CTAS) grid = CKV_MAX_SCAN_CTAS;
+  if (grid > tiles) grid = tiles;
+  return (int)(grid < 1 ? 1 : grid);
+}
+
+cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len, int *grid_out,
+                            cudaStream_t st) {
   const CkvDev &P = c->dev;
   const int units = batch * P.Hkv;
-  const int xmax = (max_len + P.bs - 1) / P.bs;
-  // about four CTAs per SM overall, at least 32 blocks per CTA, at most CKV_MAX_CHUNKS chunks per unit
-  int n_chunks = (148 * 4 + units - 1) / units;
-  n_chunks = max(1, min(n_chunks, min(CKV_MAX_CHUNKS, (xmax + 31) / 32)));
-  int chunk = (xmax + n_chunks - 1) / n_chunks;
-  chunk = (chunk + 15) / 16 * 16;
-  n_chunks = (xmax + chunk - 1) / chunk;
-  *n_chunks_out = n_chunks;
-  dim3 grid(n_chunks, units);
+  const int grid = ckv_scan_grid(c, batch, max_len);
+  *grid_out = grid;
   c->launches++;
   switch (P.G) {
-    case 1: return launch_g<1>(c, q, seq_lens, grid, chunk, st);
-    case 2: return launch_g<2>(c, q, seq_lens, grid, chunk, st);
-    case 4: return launch_g<4>(c, q, seq_lens, grid, chunk, st);
-    case 8: return launch_g<8>(c, q, seq_lens, grid, chunk, st);
+    case 1: return launch_g<1>(c, q, seq_lens, units, grid, st);
+    case 2: return launch_g<2>(c, q, seq_lens, units, grid, st);
+    case 4: return launch_g<4>(c, q, seq_lens, units, grid, st);
+    case 8: return launch_g<8>(c, q, seq_lens, units, grid, st);
   }
   return cudaErrorInvalidValue;
 }

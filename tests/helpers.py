@@ -86,8 +86,13 @@ def check_stats(st: O.Stats, kmean, dbar, vmean, K: np.ndarray, V: np.ndarray) -
 
 def check_scores(gpu_scores: np.ndarray, sc: O.Scores) -> None:
     ref = sc.S
+    got = gpu_scores[:len(ref)]
+    assert np.all(np.isfinite(got)) and np.all(got >= 0.0)
+    if ref.max() == 0.0:            # no within-block variance anywhere: every score is exactly zero
+        assert np.all(got == 0.0)
+        return
     big = ref >= 1e-30 * ref.max()
-    rel = np.abs(gpu_scores[:len(ref)][big] - ref[big]) / ref[big]
+    rel = np.abs(got[big] - ref[big]) / ref[big]
     assert rel.max() <= SCORE_RTOL, "score mismatch %.3g" % rel.max()
 
 

@@ -1,0 +1,101 @@
+"""GPU parity at the full sizes of the five benchmark configurations, on sampled units (the oracle
+computes one unit at a time), in the launch configuration the bench times (CUDA-graph replay of
+append + decode where the configuration has decode steps)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import compkv_oracle as O
+from paper_2609_26300_b200 import synth
+from paper_2609_26300_b200.runner import GraphStep
+
+from helpers import OUT_TOL, check_stats, check_unit_decode, dev_q, rel_inf, setup, unit_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config2_llama_32k():
+    w = synth.CONFIGS[2]
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt = d.ckv.decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len, w.budget_tokens)
+    scores = d.ckv.copy_scores(w.batch)
+    dout, dlse = d.ckv.dense_decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() == 0
+    assert cnt.cpu().tolist() == [[64] * 8]
+    km, db, vm = d.ckv.stats_views()
+    G = w.group
+    for h in (0, 3, 7):
+        check_unit_decode(d, 0, h, w.ctx, 0, w.budget_tokens, out, lse, ids, cnt, scores)
+        q, K, V = unit_inputs(w, 0, h, w.ctx)
+        check_stats(O.stats(K, V, 16), km[0, h], db[0, h], vm[0, h], K, V)
+        ref, _ = O.dense(q, K, V)
+        assert rel_inf(dout[0, h * G:(h + 1) * G].double().cpu().numpy(), ref) <= OUT_TOL[d.dtype]
+
+
+def test_config3_llama_128k_batch4_64_decode_steps():
+    w = synth.CONFIGS[3]
+    d = setup(w)
+    n0 = w.ctx
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, n0)
+    step = GraphStep(d.ckv, d.k_pool, d.v_pool, d.table, d.lens, n0 + w.decode_steps, w.budget_tokens, w.batch)
+    check_steps = {0, 1, 15, 16, 17, 31, 32, 63}
+    sample = [(0, 0), (3, 5)]
+    for t in range(w.decode_steps):
+        k_new, v_new = synth.appended_rows(w, t)
+        step.set_inputs(torch.from_numpy(synth.queries(w, t)).bfloat16().cuda(),
+                        torch.from_numpy(k_new).bfloat16().cuda(), torch.from_numpy(v_new).bfloat16().cuda())
+        out, lse, ids, cnt = step.replay()
+        if t in check_steps:
+            scores = d.ckv.copy_scores(w.batch)
+            torch.cuda.synchronize()
+            assert cnt.cpu().tolist() == [[128] * 8] * 4
+            for s, h in sample:
+                check_unit_decode(d, s, h, n0 + t + 1, t, w.budget_tokens, out, lse, ids, cnt, scores)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() == 0
+    assert d.lens.cpu().tolist() == [n0 + 64] * 4
+    # summaries after 64 appends equal the oracle's over the longer cache
+    km, db, vm = d.ckv.stats_views()
+    for s, h in sample:
+        _, K, V = unit_inputs(w, s, h, n0 + 64)
+        check_stats(O.stats(K, V, 16), km[s, h], db[s, h], vm[s, h], K, V)
+
+
+def test_config4_qwen_ragged_batch16_group8():
+    w = synth.CONFIGS[4]
+    d = setup(w)
+    lens = d.lens.cpu().numpy()
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt = d.ckv.decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len, w.budget_tokens)
+    scores = d.ckv.copy_scores(w.batch)
+    dout, _ = d.ckv.dense_decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() == 0
+    assert bool((cnt == 64).all())
+    G = w.group
+    for s, h in [(int(lens.argmin()), 1), (int(lens.argmax()), 6), (5, 0), (11, 3)]:
+        check_unit_decode(d, s, h, int(lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores)
+        q, K, V = unit_inputs(w, s, h, int(lens[s]))
+        ref, _ = O.dense(q, K, V)
+        assert rel_inf(dout[s, h * G:(h + 1) * G].double().cpu().numpy(), ref) <= OUT_TOL[d.dtype]
+
+
+@pytest.mark.parametrize("bs", synth.SWEEP_BLOCK_SIZES)
+def test_config5_sweep_128k(bs):
+    w = synth.CONFIGS[5].with_(block_size=bs)
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    h = 2
+    q, K, V = unit_inputs(w, 0, h, w.ctx)
+    km, db, vm = d.ckv.stats_views()
+    check_stats(O.stats(K, V, bs), km[0, h], db[0, h], vm[0, h], K, V)
+    for budget in synth.SWEEP_BUDGETS:
+        out, lse, ids, cnt = d.ckv.decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len, budget)
+        scores = d.ckv.copy_scores(w.batch)
+        torch.cuda.synchronize()
+        assert cnt.cpu().tolist() == [[budget // bs] * 8]
+        check_unit_decode(d, 0, h, w.ctx, 0, budget, out, lse, ids, cnt, scores)
+    assert d.ckv.read_status() == 0

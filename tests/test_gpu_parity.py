@@ -204,7 +204,7 @@ def test_exact_ties_go_to_lower_block_ids():
     got = ids[0, 0, :int(cnt[0, 0])].cpu().numpy()
     check_ids(got, ref_ids, osc.S, 20)
     # among an exactly tied pair the lower id must be the one taken (or both)
-    for b in range(8, 36):
+    for b in range(8, 34):          # 62 and 63 (= 34 + 28, 35 + 28) are mandatory, so start the pairs below them
         if (b + 28) in got:
             assert b in got
 
