@@ -17,43 +17,34 @@
 // |b| e^{zbar} vbar_b to the all-block compensation sum; here the same term is subtracted from the
 // exact partial, so that  merge = exact(S) + mean(all) - mean(S) = exact(S) + mean(not S).
 #include "ckv_internal.cuh"
+#include "ckv_pipe.cuh"
 
 namespace {
 
-// Eight consecutive elements kept in their storage form (so a bf16 row costs 4 registers, not 8).
-template <typename T> struct Raw8;
-template <> struct Raw8<__nv_bfloat16> {
-  uint4 u;
-  __device__ __forceinline__ void load(const __nv_bfloat16 *p) { u = __ldg(reinterpret_cast<const uint4 *>(p)); }
-  __device__ __forceinline__ void zero() { u = make_uint4(0u, 0u, 0u, 0u); }
-  __device__ __forceinline__ void get(float (&o)[8]) const { bf16x8_to_float(u, o); }
-};
-template <> struct Raw8<float> {
-  float4 a, b;
-  __device__ __forceinline__ void load(const float *p) {
-    a = __ldg(reinterpret_cast<const float4 *>(p)); b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
-  }
-  __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
-  __device__ __forceinline__ void get(float (&o)[8]) const {
-    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
-  }
-};
+using namespace ckv_pipe;
+
+constexpr int kMaxBuf = 4;                       // page buffers per warp
+constexpr int kPageElems = CKV_PAGE * CKV_D;     // elements of one head's K (or V) page
 
 template <int G, typename T, bool DENSE>
-__global__ void __launch_bounds__(256, (G <= 2) ? 2 : 1)
+__global__ void __launch_bounds__(256, (DENSE || G > 4) ? 1 : 2)
 ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool, const T *__restrict__ v_pool,
                 const int *__restrict__ page_table, const int *__restrict__ seq_lens,
-                const int *__restrict__ sel_ids, const int *__restrict__ sel_cnt, int kcap, int pages_per_split) {
+                const int *__restrict__ sel_ids, const int *__restrict__ sel_cnt, int kcap, int pages_per_split,
+                int nbuf) {
   constexpr int NV = 8 * G;                      // logits per lane before the reduction (8 rows x G heads)
   constexpr int KEEP = (NV >= 16) ? NV / 16 : 1;  // logits per lane after it
   constexpr int HSPLIT = (G >= 2) ? 2 : 1;        // a row's heads are shared by this many lanes
+  extern __shared__ __align__(128) unsigned char pg_mem[];   // [8 warps][nbuf][K page | V page]
+  __shared__ __align__(8) uint64_t bars[8][kMaxBuf];
+  __shared__ int meta[8][kMaxBuf][4];             // physical page (or -1), valid tokens, block id, list index
   __shared__ float sq[G][CKV_D];
   __shared__ __align__(16) float pbuf[8][CKV_PAGE][G];
   __shared__ __align__(16) float red[8][G][CKV_PART_STRIDE];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, hw = lane >> 4, li = lane & 15;
   const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
-  const int N = min(seq_lens[s], P.max_blocks * P.bs);
+  const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
   const int X = (N + P.bs - 1) / P.bs;
   const int nsel = DENSE ? X : min(sel_cnt[unit], kcap);
   const int total = DENSE ? (N + CKV_PAGE - 1) / CKV_PAGE : nsel * P.ppb;
@@ -66,9 +57,56 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
     return;
   }
 
+  T *wbuf = reinterpret_cast<T *>(pg_mem) + (size_t)warp * nbuf * 2 * kPageElems;
+  uint64_t *wbar = bars[warp];
+  if (lane == 0) {
+    for (int b = 0; b < nbuf; ++b) mbar_init(&wbar[b], 1);
+    fence_barrier_init();
+  }
   for (int idx = tid; idx < G * CKV_D; idx += 256)
     sq[idx / CKV_D][idx % CKV_D] = to_float(q[((size_t)s * P.Hq + h * G) * CKV_D + idx]) * (P.scale * kLog2e);
   __syncthreads();
+
+  const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
+  const int pshift = P.ppb == 1 ? 0 : (P.ppb == 2 ? 1 : 2);
+  const int n_mine = (p1 - p0 - warp + 7) >> 3;   // this warp's pages: list index p0 + warp + 8 n
+  bool bad = false;
+
+  // lane 0: resolve list entry n to a physical page and start its copy into buffer n % nbuf
+  auto issue = [&](int n, int b) {
+    const int i = p0 + warp + 8 * n;
+    int phys = -1, ntok = 0, blk = -1, page = i;
+    bool ok = true;
+    if (!DENSE) {
+      blk = sel_ids[(size_t)unit * kcap + (i >> pshift)];
+      ok = blk >= 0 && blk < X;
+      if (!ok) blk = -1;
+      page = (blk << pshift) + (i & (P.ppb - 1));
+    }
+    if (ok) {
+      ntok = min(CKV_PAGE, N - page * CKV_PAGE);
+      if (ntok > 0) {
+        phys = pt_row[page];
+        if (phys < 0 || phys >= P.num_pages) { phys = -1; bad = true; }
+      } else {
+        ntok = 0;
+      }
+    }
+    meta[warp][b][0] = phys; meta[warp][b][1] = ntok; meta[warp][b][2] = blk; meta[warp][b][3] = i;
+    if (phys >= 0) {
+      const uint32_t bytes = (uint32_t)ntok * CKV_D * sizeof(T);
+      const size_t src = ((size_t)phys * P.Hkv + h) * kPageElems;
+      T *dst = wbuf + (size_t)b * 2 * kPageElems;
+      mbar_arrive_expect_tx(&wbar[b], 2 * bytes);
+      bulk_g2s(dst, k_pool + src, bytes, &wbar[b]);
+      bulk_g2s(dst + kPageElems, v_pool + src, bytes, &wbar[b]);
+    }
+  };
+  int issued = 0;
+  if (lane == 0)
+    for (; issued < nbuf && issued < n_mine; ++issued) issue(issued, issued);
+  __syncwarp();
+
   float qr[G][8];
 #pragma unroll
   for (int g = 0; g < G; ++g)
@@ -87,48 +125,38 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
   // after the reduction this lane owns row (li / 2) of its half warp and heads [g_own0, g_own0 + KEEP)
   const int g_own0 = (G >= 2) ? (li & 1) * KEEP : 0;
   const int t_own = hw + 2 * (li >> 1);
-  const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
   const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
   const float *vmean = P.vmean + (size_t)unit * P.max_blocks * CKV_D;
-  bool bad = false;
+  uint32_t phase_bits = 0;   // bit b: parity of the next completion of buffer b
+  bool aborted = false;
+  int n_abort = 0;
 
-  for (int i = p0 + warp; i < p1; i += 8) {
-    int page, blk = 0;
-    if (DENSE) {
-      page = i;
-    } else {
-      blk = sel_ids[(size_t)unit * kcap + i / P.ppb];
-      if (blk < 0 || blk >= X) continue;
-      page = blk * P.ppb + i % P.ppb;
+  for (int n = 0, b = 0; n < n_mine; ++n) {
+    const int phys = meta[warp][b][0], ntok = meta[warp][b][1], blk = meta[warp][b][2], i = meta[warp][b][3];
+    if (phys >= 0 && !aborted) {
+      if (!mbar_wait(&wbar[b], (phase_bits >> b) & 1)) {
+        atomicOr(P.status, CKV_DEV_TIMEOUT);
+        aborted = true;
+      }
+      aborted = __any_sync(0xffffffffu, aborted);
+      if (aborted) n_abort = n;
     }
-    const int ntok = min(CKV_PAGE, N - page * CKV_PAGE);
-    if (ntok > 0) {
-      const int phys = pt_row[page];
-      if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
-      const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+    if (phys >= 0 && !aborted) {
+      phase_bits ^= 1u << b;
+      const T *kp = wbuf + (size_t)b * 2 * kPageElems + 8 * li;
+      const T *vp = kp + kPageElems;
       float sv[NV];
-      Raw8<T> kraw[8], vraw[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int t = hw + 2 * j;
-        if (t < ntok) {
-          kraw[j].load(k_pool + base + (size_t)t * CKV_D);
-          vraw[j].load(v_pool + base + (size_t)t * CKV_D);
-        } else {
-          kraw[j].zero();
-          vraw[j].zero();
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
         float kf[8];
-        kraw[j].get(kf);
+        load8<false>(kp + t * CKV_D, kf);
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           float z = 0.f;
 #pragma unroll
           for (int c = 0; c < 8; ++c) z = fmaf(qr[g][c], kf[c], z);
-          sv[j * G + g] = z;
+          sv[j * G + g] = (t < ntok) ? z : 0.f;   // rows past the last token hold stale bytes
         }
       }
       reduce16<NV, KEEP>(sv, li);
@@ -172,56 +200,71 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
       __syncwarp();
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const float *pp = pbuf[warp][hw + 2 * j];
-        float vf[8];
-        vraw[j].get(vf);
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          const float *pp = pbuf[warp][t];
+          float vf[8];
+          load8<false>(vp + t * CKV_D, vf);
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-          const float pg = pp[g];
+          for (int g = 0; g < G; ++g) {
+            const float pg = pp[g];
 #pragma unroll
-          for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(pg, vf[c], acc[g][c]);
-        }
-      }
-      __syncwarp();
-    }
-    if (comp && (i % P.ppb) == 0) {
-      // take this block's mean term |b| e^{zbar} vbar_b back out (it is part of the all-block sum)
-      float zl2[G];
-      bool raise = false;
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const float2 v = __ldg(ls + (size_t)blk * G + g);
-        zl2[g] = (v.x - 0.5f * v.y) * kLog2e;
-        raise |= zl2[g] > m_ref[g] + CKV_RESCALE_SLACK;
-      }
-      if (raise) {   // warp-uniform: every lane evaluates the same values
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-          if (zl2[g] > m_ref[g]) {
-            const float sc = exp2_diff(m_ref[g], zl2[g]);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) acc[g][c] *= sc;
-#pragma unroll
-            for (int jj = 0; jj < KEEP; ++jj)
-              if (g_own0 + jj == g) { l_own[jj] *= sc; m_own[jj] = zl2[g]; }
-            m_ref[g] = zl2[g];
+            for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(pg, vf[c], acc[g][c]);
           }
         }
       }
-      if (hw == 0) {
-        const float4 a = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li));
-        const float4 b4 = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li) + 1);
-        const float vb[8] = {a.x, a.y, a.z, a.w, b4.x, b4.y, b4.z, b4.w};
+      if (comp && (i & (P.ppb - 1)) == 0) {
+        // take this block's mean term |b| e^{zbar} vbar_b back out (it is part of the all-block sum)
+        float zl2[G];
+        bool raise = false;
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-          const float wbar = exp2f(zl2[g] - m_ref[g]);
+          const float2 v = __ldg(ls + (size_t)blk * G + g);
+          zl2[g] = (v.x - 0.5f * v.y) * kLog2e;
+          raise |= zl2[g] > m_ref[g] + CKV_RESCALE_SLACK;
+        }
+        if (raise) {   // warp-uniform: every lane evaluates the same values
 #pragma unroll
-          for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(-wbar, vb[c], acc[g][c]);
+          for (int g = 0; g < G; ++g) {
+            if (zl2[g] > m_ref[g]) {
+              const float sc = exp2_diff(m_ref[g], zl2[g]);
 #pragma unroll
-          for (int jj = 0; jj < KEEP; ++jj)
-            if (g_own0 + jj == g && li < HSPLIT) l_own[jj] -= wbar;
+              for (int c = 0; c < 8; ++c) acc[g][c] *= sc;
+#pragma unroll
+              for (int jj = 0; jj < KEEP; ++jj)
+                if (g_own0 + jj == g) { l_own[jj] *= sc; m_own[jj] = zl2[g]; }
+              m_ref[g] = zl2[g];
+            }
+          }
+        }
+        if (hw == 0) {
+          const float4 a = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li));
+          const float4 b4 = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li) + 1);
+          const float vb[8] = {a.x, a.y, a.z, a.w, b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const float wbar_g = exp2f(zl2[g] - m_ref[g]);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc[g][c] = fmaf(-wbar_g, vb[c], acc[g][c]);
+#pragma unroll
+            for (int jj = 0; jj < KEEP; ++jj)
+              if (g_own0 + jj == g && li < HSPLIT) l_own[jj] -= wbar_g;
+          }
         }
       }
+    }
+    // the buffer is free: order this warp's shared-memory reads before the next bulk copy into it
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0 && !aborted && issued < n_mine) { issue(issued, b); ++issued; }
+    __syncwarp();
+    if (++b == nbuf) b = 0;
+  }
+  if (aborted && lane == 0) {
+    // leave no bulk copy in flight into this warp's buffers
+    for (int n = n_abort; n < issued; ++n) {
+      const int b = n % nbuf;
+      if (meta[warp][b][0] >= 0) mbar_wait(&wbar[b], (phase_bits >> b) & 1);
     }
   }
   if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
@@ -282,22 +325,10 @@ __global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *_
   const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
   const int X = (N + P.bs - 1) / P.bs;
   const bool comp = !dense && sel_cnt[unit] < X;
-  if (c == 0) {
+  if (c < 32) {
     int cfirst = 0, ccount = 0;
-    if (comp) {
-      long long T = 0, T0 = 0;
-      for (int u = 0; u < units; ++u) {
-        const int n = max(min(seq_lens[u / P.Hkv], P.max_blocks * P.bs), 0);
-        const int tiles = ((n + P.bs - 1) / P.bs + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE;
-        if (u == unit) T0 = T;
-        T += tiles;
-      }
-      const long long tpc = (T + scan_grid - 1) / scan_grid;
-      const int my_tiles = (X + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE;
-      cfirst = (int)(T0 / tpc);
-      ccount = (int)((T0 + my_tiles - 1) / tpc) - cfirst + 1;
-    }
-    s_cfirst = cfirst; s_ccount = ccount;
+    if (comp) unit_scan_slots(P, seq_lens, units, unit, scan_grid, c, cfirst, ccount);
+    if (c == 0) { s_cfirst = cfirst; s_ccount = ccount; }
   }
   __syncthreads();
   const int n_comp = s_ccount;
@@ -338,16 +369,35 @@ __global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *_
   if (lse != nullptr && c == 0) lse[(size_t)s * P.Hq + hq] = N > 0 ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
 }
 
+// Static shared memory of the attention kernel (query tile, probability tile, warp partials, barriers).
+inline size_t attn_static_smem(int G) {
+  return (size_t)G * CKV_D * 4 + (size_t)8 * CKV_PAGE * G * 4 + (size_t)8 * G * CKV_PART_STRIDE * 4 + 1024;
+}
+inline size_t attn_page_pair_bytes(const ckv_ctx *c) {
+  return (size_t)2 * kPageElems * (c->layout.kv_dtype == CKV_BF16 ? 2 : 4);
+}
+// Page buffers per warp: one for the sparse list (a warp owns one or two pages), as many as fit (up to 3) for dense.
+inline int attn_nbuf(const ckv_ctx *c, bool dense, int pps) {
+  const size_t per_buf = 8 * attn_page_pair_bytes(c);
+  const size_t room = 220 * 1024 - attn_static_smem(c->dev.G);
+  int fit = (int)(room / per_buf);
+  if (fit < 1) fit = 1;
+  int want = dense ? 3 : (pps > 8 ? 2 : 1);
+  return want < fit ? want : fit;
+}
+
 template <int G, typename T>
 cudaError_t launch_gt(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                       const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt, int kcap,
                       dim3 grid, int pps, cudaStream_t st) {
+  const int nbuf = attn_nbuf(c, dense, pps);
+  const size_t smem = (size_t)nbuf * 8 * attn_page_pair_bytes(c);
   if (dense)
-    ckv_attn_kernel<G, T, true><<<grid, 256, 0, st>>>(c->dev, (const T *)q, (const T *)k_pool, (const T *)v_pool,
-                                                       page_table, seq_lens, sel_ids, sel_cnt, kcap, pps);
+    ckv_attn_kernel<G, T, true><<<grid, 256, smem, st>>>(c->dev, (const T *)q, (const T *)k_pool, (const T *)v_pool,
+                                                          page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, nbuf);
   else
-    ckv_attn_kernel<G, T, false><<<grid, 256, 0, st>>>(c->dev, (const T *)q, (const T *)k_pool, (const T *)v_pool,
-                                                        page_table, seq_lens, sel_ids, sel_cnt, kcap, pps);
+    ckv_attn_kernel<G, T, false><<<grid, 256, smem, st>>>(c->dev, (const T *)q, (const T *)k_pool, (const T *)v_pool,
+                                                           page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, nbuf);
   return cudaGetLastError();
 }
 
@@ -361,7 +411,32 @@ cudaError_t launch_g(ckv_ctx *c, bool dense, const void *q, const void *k_pool, 
   return launch_gt<G, float>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
 }
 
+template <int G, typename T>
+cudaError_t configure_gt(const ckv_ctx *c) {
+  const int smem = (int)(220 * 1024 - attn_static_smem(G));
+  cudaError_t e = cudaFuncSetAttribute(ckv_attn_kernel<G, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(ckv_attn_kernel<G, T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  return e;
+}
+template <int G>
+cudaError_t configure_g(const ckv_ctx *c) {
+  if (c->layout.kv_dtype == CKV_BF16) return configure_gt<G, __nv_bfloat16>(c);
+  return configure_gt<G, float>(c);
+}
+
 }  // namespace
+
+// Opt in to the dynamic shared memory this context's attention instantiations need, on the current device.
+cudaError_t ckv_configure_attn(const ckv_ctx *c) {
+  switch (c->dev.G) {
+    case 1: return configure_g<1>(c);
+    case 2: return configure_g<2>(c);
+    case 4: return configure_g<4>(c);
+    case 8: return configure_g<8>(c);
+  }
+  return cudaErrorInvalidValue;
+}
 
 cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                             const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,

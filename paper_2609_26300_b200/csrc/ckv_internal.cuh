@@ -11,7 +11,7 @@
 #define CKV_D 128             // head dimension the kernels are written for
 #define CKV_PAGE 16           // tokens per page
 #define CKV_PART_STRIDE 132   // floats per split partial: m, l, pad, pad, acc[128]
-#define CKV_SCAN_TILE 16      // blocks per scan tile
+#define CKV_SCAN_TILE 32      // blocks per scan tile
 #define CKV_MAX_SCAN_CTAS 512 // persistent scan grid is capped at this many CTAs
 #define CKV_MAX_SPLITS 64     // attention partials per unit
 #define CKV_RESCALE_SLACK 16.0f  // log2 units: running maxima are only raised when exceeded by this much
@@ -47,6 +47,7 @@ struct ckv_ctx {
 
 cudaError_t ckv_configure_kernels();   // selection kernel attributes
 cudaError_t ckv_configure_scan(const ckv_ctx *c);   // scan kernel attributes
+cudaError_t ckv_configure_attn(const ckv_ctx *c);   // attention kernel attributes
 int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len);
 
 // ---- launchers (one per translation unit) ---------------------------------------------------------
@@ -135,6 +136,34 @@ __device__ __forceinline__ void reduce16(float (&v)[NV], int li) {
   }
 }
 
+// Two fp32 values in one 64-bit register pair, for the packed fp32 instructions of sm_100.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// d = a * b + c on both halves (one instruction).
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x with the hardware approximation (relative error about 2^-22; -inf gives 0).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ float warp_max(float x) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
@@ -149,6 +178,30 @@ __device__ __forceinline__ float warp_sum(float x) {
 // exp2 of a difference that may involve -inf on either side without producing NaN.
 __device__ __forceinline__ float exp2_diff(float a, float b) {
   return (a == -CUDART_INF_F) ? 0.0f : exp2f(a - b);
+}
+
+// Which scan partials belong to `unit`: the scan cuts all units' summaries into tiles of CKV_SCAN_TILE
+// blocks, gives CTA c the tiles [c * tpc, (c + 1) * tpc) and stores its partial for unit u in entry
+// c + u.  Must be called by all 32 lanes of a warp; every lane gets the result.
+__device__ __forceinline__ void unit_scan_slots(const CkvDev &P, const int *__restrict__ seq_lens, int units, int unit,
+                                                int scan_grid, int lane, int &cfirst, int &ccount) {
+  const int batch = units / P.Hkv, s = unit / P.Hkv, h = unit % P.Hkv;
+  unsigned tot = 0, before = 0, mine = 0;
+  for (int i = lane; i < batch; i += 32) {
+    const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
+    const unsigned t = (unsigned)(((n + P.bs - 1) / P.bs + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE);
+    tot += t;
+    if (i < s) before += t;
+    if (i == s) mine = t;
+  }
+  tot = __reduce_add_sync(0xffffffffu, tot);
+  before = __reduce_add_sync(0xffffffffu, before);
+  mine = __reduce_add_sync(0xffffffffu, mine);
+  const long long T = (long long)tot * P.Hkv;
+  const long long T0 = (long long)before * P.Hkv + (long long)h * mine;
+  const long long tpc = max((T + scan_grid - 1) / scan_grid, 1ll);
+  cfirst = (int)(T0 / tpc);
+  ccount = mine == 0 ? 0 : (int)((T0 + mine - 1) / tpc) - cfirst + 1;
 }
 
 #endif  // __CUDACC__

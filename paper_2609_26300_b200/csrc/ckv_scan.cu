@@ -34,10 +34,19 @@ template <> struct Log2<1> { static constexpr int v = 0; };
 
 constexpr int TB = CKV_SCAN_TILE;   // blocks per tile
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 256;       // 8 warps, all consumers; thread 0 also issues the bulk copies
-constexpr int kLag = 2;             // a stage is refilled two tiles after it was consumed
+constexpr int NP = TB / 16;          // row pairs a consumer warp takes per tile
+constexpr int kConsumers = 256;     // 8 consumer warps
+constexpr int kThreads = kConsumers + 32;   // plus one producer warp (a single thread of it issues the bulk copies)
+constexpr int kMaxUnits = 1024;     // sequence lengths are staged in shared memory up to this many sequences
 
 struct UnitInfo { int N, X, tiles; };
+
+// Tiles of one sequence's units: from the staged table, or recomputed for sequences beyond it.
+__device__ __forceinline__ int seq_tiles(const int *s_tiles, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
+  if (i < kMaxUnits) return s_tiles[i];
+  const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
+  return ((n + P.bs - 1) / P.bs + TB - 1) / TB;
+}
 
 __device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *__restrict__ seq_lens, int u) {
   UnitInfo ui;
@@ -58,14 +67,22 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
   __shared__ __align__(16) float sw[CKV_D][G];
   __shared__ __align__(16) float red[8][G][CKV_PART_STRIDE];
   __shared__ int s_u0, s_tl0, s_count, s_abort, s_issued, s_consumed;
+  __shared__ int s_tiles[kMaxUnits];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 4, li = lane & 15;
   const bool dbar_bulk = P.r >= 4;   // smaller rows cannot keep the 16-byte alignment bulk copies need
   const int stage_floats = TB * 2 * CKV_D + (dbar_bulk ? TB * P.r : 0);
 
+  // tiles per unit from the sequence lengths (staged in shared memory: one parallel load, no serial global reads)
+  const int batch = units / P.Hkv;
+  for (int i = tid; i < batch && i < kMaxUnits; i += kThreads) {
+    const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
+    s_tiles[i] = ((n + P.bs - 1) / P.bs + TB - 1) / TB;
+  }
+  __syncthreads();
   if (tid == 0) {
     long long T = 0;
-    for (int u = 0; u < units; ++u) T += unit_info(P, seq_lens, u).tiles;
+    for (int sq_i = 0; sq_i < batch; ++sq_i) T += (long long)seq_tiles(s_tiles, seq_lens, P, sq_i) * P.Hkv;
     const long long tpc = (T + gridDim.x - 1) / gridDim.x;
     const long long first = (long long)blockIdx.x * tpc;
     long long cnt = T - first;
@@ -74,10 +91,14 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     int u0 = 0, tl0 = 0;
     if (cnt > 0) {
       long long accum = 0;
-      for (int u = 0; u < units; ++u) {
-        const int t = unit_info(P, seq_lens, u).tiles;
-        if (first < accum + t) { u0 = u; tl0 = (int)(first - accum); break; }
-        accum += t;
+      for (int sq_i = 0; sq_i < batch; ++sq_i) {
+        const long long t = seq_tiles(s_tiles, seq_lens, P, sq_i);
+        if (t > 0 && first < accum + t * P.Hkv) {
+          const long long off = first - accum;
+          u0 = sq_i * P.Hkv + (int)(off / t); tl0 = (int)(off % t);
+          break;
+        }
+        accum += t * P.Hkv;
       }
     }
     s_u0 = u0; s_tl0 = tl0; s_count = (int)cnt; s_abort = 0; s_issued = 0; s_consumed = 0;
@@ -88,47 +109,52 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
   const int count = s_count;
   if (count == 0) return;   // uniform: this CTA has no tiles
 
-  {
+  if (warp == 8) {
+    // ---------------- producer: one thread streams the CTA's tiles into the ring ----------------
+    if (lane == 0) {
+      int u = s_u0, tl = s_tl0, st = 0;
+      uint32_t phase = 0;            // parity of the empty-barrier phase the next refill of stage `st` waits for
+      UnitInfo ui = unit_info(P, seq_lens, u);
+      for (int it = 0; it < count; ++it) {
+        if (it >= stages && !mbar_wait(&empty_bar[st], phase)) {
+          atomicOr(P.status, CKV_DEV_TIMEOUT);
+          *(volatile int *)&s_abort = 1;
+        }
+        if (*(volatile int *)&s_abort) break;
+        const int b0 = tl * TB;
+        const int nb = min(TB, ui.X - b0);
+        const size_t row = (size_t)u * P.max_blocks + b0;
+        float *sk = stage_mem + (size_t)st * stage_floats;
+        float *sv = sk + TB * CKV_D;
+        const uint32_t kbytes = (uint32_t)nb * CKV_D * 4;
+        const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
+        mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
+        bulk_g2s(sk, P.kmean + row * CKV_D, kbytes, &full_bar[st]);
+        bulk_g2s(sv, P.vmean + row * CKV_D, kbytes, &full_bar[st]);
+        if (dbar_bulk) bulk_g2s(sv + TB * CKV_D, P.dbar + row * P.r, dbytes, &full_bar[st]);
+        *(volatile int *)&s_issued = it + 1;
+        if (++st == stages) { st = 0; if (it >= stages) phase ^= 1; }
+        if (++tl == ui.tiles) {
+          tl = 0;
+          do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+        }
+      }
+    }
+  } else {
     // ---------------- consumers ----------------
-    float qr[G][8], acc[G][8], m_ref[G];
+    f32x2 qr[G][4], acc[G][4];   // this lane's 8 coordinates (4 pairs) of every head's query and accumulator
+    float m_ref[G], wown[4];
     float m_my = -CUDART_INF_F, l_my = 0.f, lp_my = 0.f;   // lp: sum of e^{l - m}, the normaliser of Eq. 9
+    const bool r4 = P.r == 4 && dbar_bulk;   // the default r: the owner lane evaluates Eq. 8 by itself
     const int myg = li >> SH;
     const float log_bs = logf((float)P.bs);
     float log_last = 0.f;
-    int u = s_u0, tl = s_tl0, cur = -1;
+    int u = s_u0, tl = s_tl0, cur = -1, st = 0;
+    uint32_t phase = 0;              // parity of the full-barrier phase of stage `st` this pass over the ring
     UnitInfo ui = unit_info(P, seq_lens, u);
     float2 *ls = nullptr;
     const float *db = nullptr;
     bool aborted = false;
-    // producer state (thread 0 only): next tile to issue and its position in the walk
-    int p_next = 0, p_u = u, p_tl = tl;
-    UnitInfo p_ui = ui;
-    auto issue_next = [&]() {
-      const int st = p_next % stages, k = p_next / stages;
-      if (k >= 1 && !mbar_wait(&empty_bar[st], (k - 1) & 1)) {
-        atomicOr(P.status, CKV_DEV_TIMEOUT);
-        *(volatile int *)&s_abort = 1;
-        return;
-      }
-      const int b0 = p_tl * TB;
-      const int nb = min(TB, p_ui.X - b0);
-      const size_t row = (size_t)p_u * P.max_blocks + b0;
-      float *sk = stage_mem + (size_t)st * stage_floats;
-      float *sv = sk + TB * CKV_D;
-      const uint32_t kbytes = (uint32_t)nb * CKV_D * 4;
-      const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
-      mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
-      bulk_g2s(sk, P.kmean + row * CKV_D, kbytes, &full_bar[st]);
-      bulk_g2s(sv, P.vmean + row * CKV_D, kbytes, &full_bar[st]);
-      if (dbar_bulk) bulk_g2s(sv + TB * CKV_D, P.dbar + row * P.r, dbytes, &full_bar[st]);
-      *(volatile int *)&s_issued = ++p_next;
-      if (++p_tl == p_ui.tiles) {
-        p_tl = 0;
-        do { ++p_u; } while (p_u < units && (p_ui = unit_info(P, seq_lens, p_u)).tiles == 0);
-      }
-    };
-    if (tid == 0)
-      for (int i = 0; i < stages - kLag && i < count; ++i) issue_next();
 
     auto flush = [&](int unit_done) {
       // fold the two half warps, then the 8 warps, into one partial per head of `unit_done`
@@ -138,9 +164,13 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         const float mn = fmaxf(m_ref[g], mo);
         const float sc = exp2_diff(m_ref[g], mn);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float a = acc[g][i] * sc;
-          acc[g][i] = a + __shfl_xor_sync(0xffffffffu, a, 16);
+        for (int i = 0; i < 4; ++i) {
+          float a0, a1;
+          unpack2(acc[g][i], a0, a1);
+          a0 *= sc; a1 *= sc;
+          a0 += __shfl_xor_sync(0xffffffffu, a0, 16);
+          a1 += __shfl_xor_sync(0xffffffffu, a1, 16);
+          acc[g][i] = pack2(a0, a1);
         }
         float lg = (myg == g) ? l_my * sc : 0.f;
         float lpg = (myg == g) ? lp_my * sc : 0.f;
@@ -153,14 +183,17 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           float *r = red[warp][g];
-          *reinterpret_cast<float4 *>(r + 4 + 4 * li) = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
-          *reinterpret_cast<float4 *>(r + 4 + 64 + 4 * li) = make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]);
+          float a[8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) unpack2(acc[g][i], a[2 * i], a[2 * i + 1]);
+          *reinterpret_cast<float4 *>(r + 4 + 4 * li) = make_float4(a[0], a[1], a[2], a[3]);
+          *reinterpret_cast<float4 *>(r + 4 + 64 + 4 * li) = make_float4(a[4], a[5], a[6], a[7]);
           if (li == (g << SH)) { r[0] = m_ref[g]; r[1] = l_my; r[2] = lp_my; }
         }
       }
-      named_barrier(1, kThreads);
+      named_barrier(1, kConsumers);
       float *part = P.comp_part + (size_t)(blockIdx.x + unit_done) * G * CKV_PART_STRIDE;
-      for (int idx = tid; idx < G * CKV_D; idx += kThreads) {
+      for (int idx = tid; idx < G * CKV_D; idx += kConsumers) {
         const int g = idx / CKV_D, i = idx % CKV_D;
         float M = -CUDART_INF_F;
 #pragma unroll
@@ -178,7 +211,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
           part[g * CKV_PART_STRIDE] = M; part[g * CKV_PART_STRIDE + 1] = den; part[g * CKV_PART_STRIDE + 2] = denp;
         }
       }
-      named_barrier(1, kThreads);
+      named_barrier(1, kConsumers);
     };
 
     for (int it = 0; it < count; ++it) {
@@ -186,28 +219,30 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         if (cur >= 0) flush(cur);
         // per-unit setup: the unit's queries, their per-group squared norms, fresh accumulators
         const int s = u / P.Hkv, h = u % P.Hkv;
-        for (int idx = tid; idx < G * CKV_D; idx += kThreads)
+        for (int idx = tid; idx < G * CKV_D; idx += kConsumers)
           sq[idx / CKV_D][idx % CKV_D] = to_float(q[((size_t)s * P.Hq + h * G) * CKV_D + idx]);
-        named_barrier(1, kThreads);
-        for (int idx = tid; idx < P.r * G; idx += kThreads) {
+        named_barrier(1, kConsumers);
+        for (int idx = tid; idx < P.r * G; idx += kConsumers) {
           const int t = idx / G, g = idx % G;
           float w = 0.f;
           for (int i = 0; i < CKV_D; ++i)
             if (group_of(i, P.r, P.glayout) == t) w = fmaf(sq[g][i], sq[g][i], w);
           sw[t][g] = w;
         }
-        named_barrier(1, kThreads);
+        named_barrier(1, kConsumers);
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           m_ref[g] = -CUDART_INF_F;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            qr[g][i] = sq[g][4 * li + i] * P.scale;
-            qr[g][4 + i] = sq[g][64 + 4 * li + i] * P.scale;
+          for (int i = 0; i < 2; ++i) {
+            qr[g][i] = pack2(sq[g][4 * li + 2 * i] * P.scale, sq[g][4 * li + 2 * i + 1] * P.scale);
+            qr[g][2 + i] = pack2(sq[g][64 + 4 * li + 2 * i] * P.scale, sq[g][64 + 4 * li + 2 * i + 1] * P.scale);
           }
 #pragma unroll
-          for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
+          for (int i = 0; i < 4; ++i) acc[g][i] = pack2(0.f, 0.f);
         }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) wown[t] = r4 ? sw[t][myg] * (P.scale * P.scale) : 0.f;
         m_my = -CUDART_INF_F; l_my = 0.f; lp_my = 0.f;
         log_last = logf((float)(ui.N - (ui.X - 1) * P.bs));
         const size_t row0 = (size_t)u * P.max_blocks;
@@ -215,17 +250,16 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         db = P.dbar + row0 * P.r;
         cur = u;
       }
-      const int st = it % stages;
-      if (tid == 0 && p_next < count && !*(volatile int *)&s_abort) issue_next();
       // a wait that runs out marks the step invalid; the walk (and its barriers) still runs to the end
       if (!aborted && *(volatile int *)&s_abort) aborted = true;
-      if (!aborted && !mbar_wait(&full_bar[st], (it / stages) & 1)) {
+      if (!aborted && !mbar_wait(&full_bar[st], phase)) {
         atomicOr(P.status, CKV_DEV_TIMEOUT);
         *(volatile int *)&s_abort = 1;
         aborted = true;
       }
       aborted = __any_sync(0xffffffffu, aborted);
       if (aborted) {
+        if (++st == stages) { st = 0; phase ^= 1; }
         if (++tl == ui.tiles) {
           tl = 0;
           do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
@@ -237,70 +271,123 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
       const float *sd = sv + TB * CKV_D;
       const int b0 = tl * TB;
       const int nb = min(TB, ui.X - b0);
-      const int bl = warp * 2 + gid;
-      const int b = b0 + bl;
-      const bool valid = bl < nb;
-      float4 k0 = *reinterpret_cast<const float4 *>(sk + bl * CKV_D + 4 * li);
-      float4 k1 = *reinterpret_cast<const float4 *>(sk + bl * CKV_D + 64 + 4 * li);
-      float4 v0 = *reinterpret_cast<const float4 *>(sv + bl * CKV_D + 4 * li);
-      float4 v1 = *reinterpret_cast<const float4 *>(sv + bl * CKV_D + 64 + 4 * li);
-      if (nb < TB && !valid) {   // rows past the unit's last block hold stale bytes
-        k0 = k1 = v0 = v1 = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-      const float kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
-      const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-      float red_v[2 * G];
+      // this warp's NP row pairs of the tile: rows warp * 2 NP + 2 p + gid; the pairs are independent
+      // chains the compiler interleaves
+      int bl[NP];
+      bool valid[NP];
+      f32x2 kk[NP][4], vv[NP][4];
 #pragma unroll
-      for (int g = 0; g < G; ++g) { red_v[2 * g] = 0.f; red_v[2 * g + 1] = 0.f; }
-      if (valid) {
-        for (int t = li; t < P.r; t += 16) {
-          const float dv = dbar_bulk ? sd[bl * P.r + t] : __ldg(db + (size_t)b * P.r + t);
+      for (int p = 0; p < NP; ++p) {
+        bl[p] = warp * (2 * NP) + 2 * p + gid;
+        valid[p] = bl[p] < nb;
+        const float4 k0 = *reinterpret_cast<const float4 *>(sk + bl[p] * CKV_D + 4 * li);
+        const float4 k1 = *reinterpret_cast<const float4 *>(sk + bl[p] * CKV_D + 64 + 4 * li);
+        const float4 v0 = *reinterpret_cast<const float4 *>(sv + bl[p] * CKV_D + 4 * li);
+        const float4 v1 = *reinterpret_cast<const float4 *>(sv + bl[p] * CKV_D + 64 + 4 * li);
+        kk[p][0] = pack2(k0.x, k0.y); kk[p][1] = pack2(k0.z, k0.w); kk[p][2] = pack2(k1.x, k1.y); kk[p][3] = pack2(k1.z, k1.w);
+        vv[p][0] = pack2(v0.x, v0.y); vv[p][1] = pack2(v0.z, v0.w); vv[p][2] = pack2(v1.x, v1.y); vv[p][3] = pack2(v1.z, v1.w);
+        if (nb < TB && !valid[p]) {   // rows past the unit's last block hold stale bytes
 #pragma unroll
-          for (int g = 0; g < G; ++g) red_v[2 * g + 1] = fmaf(sw[t][g], dv, red_v[2 * g + 1]);
+          for (int i = 0; i < 4; ++i) { kk[p][i] = pack2(0.f, 0.f); vv[p][i] = pack2(0.f, 0.f); }
         }
       }
+      float zbar[NP], sig[NP];
+      if (r4) {
+        // r = 4: reduce the G mean logits only; the owner lane of a head evaluates sigma_hat^2 from the
+        // block's four group variances (one 16-byte read) with its head's weights held in registers
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float z = 0.f;
+        for (int p = 0; p < NP; ++p) {
+          float zr[G];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) z = fmaf(qr[g][i], kk[i], z);
-        red_v[2 * g] = z;
+          for (int g = 0; g < G; ++g) {
+            f32x2 z2 = mul2(qr[g][0], kk[p][0]);
+#pragma unroll
+            for (int i = 1; i < 4; ++i) z2 = fma2(qr[g][i], kk[p][i], z2);
+            float z0, z1;
+            unpack2(z2, z0, z1);
+            zr[g] = z0 + z1;
+          }
+          reduce16<G, 1>(zr, li);
+          const float4 dv = *reinterpret_cast<const float4 *>(sd + bl[p] * 4);
+          zbar[p] = zr[0];
+          sig[p] = fmaf(wown[0], dv.x, fmaf(wown[1], dv.y, fmaf(wown[2], dv.z, wown[3] * dv.w)));
+        }
+      } else {
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+          float red_v[2 * G];
+#pragma unroll
+          for (int g = 0; g < G; ++g) red_v[2 * g + 1] = 0.f;
+          if (valid[p]) {
+            for (int t = li; t < P.r; t += 16) {
+              const float dv = dbar_bulk ? sd[bl[p] * P.r + t] : __ldg(db + (size_t)(b0 + bl[p]) * P.r + t);
+#pragma unroll
+              for (int g = 0; g < G; ++g) red_v[2 * g + 1] = fmaf(sw[t][g], dv, red_v[2 * g + 1]);
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            f32x2 z2 = mul2(qr[g][0], kk[p][0]);
+#pragma unroll
+            for (int i = 1; i < 4; ++i) z2 = fma2(qr[g][i], kk[p][i], z2);
+            float z0, z1;
+            unpack2(z2, z0, z1);
+            red_v[2 * g] = z0 + z1;
+          }
+          reduce16<2 * G, 2>(red_v, li);
+          zbar[p] = red_v[0];
+          sig[p] = red_v[1] * (P.scale * P.scale);   // Eq. 8's 1/d is the squared logit scale
+        }
       }
-      reduce16<2 * G, 2>(red_v, li);
-      const float zbar = red_v[0];
-      const float sig = red_v[1] * (P.scale * P.scale);   // Eq. 8's 1/d is the squared logit scale
-      const float logc = (b == ui.X - 1) ? log_last : log_bs;
-      const float ell = logc + zbar + 0.5f * sig;
-      if (valid && (li & ((1 << SH) - 1)) == 0) ls[(size_t)b * G + myg] = make_float2(ell, sig);
-      // compensation weight of this block for head myg: |b| e^{zbar}, in log2 units
-      const float zl2 = valid ? (zbar + logc) * kLog2e : -CUDART_INF_F;
-      if (__any_sync(0xffffffffu, zl2 > m_my + CKV_RESCALE_SLACK)) {
+      float zl2[NP];
+      bool raise = false;
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-          const float cand = __shfl_sync(0xffffffffu, zl2, (lane & 16) | (g << SH));
-          if (cand > m_ref[g]) {
-            const float sc = exp2_diff(m_ref[g], cand);
+      for (int p = 0; p < NP; ++p) {
+        const int b = b0 + bl[p];
+        const float logc = (b == ui.X - 1) ? log_last : log_bs;
+        const float ell = logc + zbar[p] + 0.5f * sig[p];
+        if (valid[p] && (li & ((1 << SH) - 1)) == 0) ls[(size_t)b * G + myg] = make_float2(ell, sig[p]);
+        // compensation weight of this block for head myg: |b| e^{zbar}, in log2 units
+        zl2[p] = valid[p] ? (zbar[p] + logc) * kLog2e : -CUDART_INF_F;
+        raise |= zl2[p] > m_my + CKV_RESCALE_SLACK;
+      }
+      if (__any_sync(0xffffffffu, raise)) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[g][i] *= sc;
-            if (myg == g) { l_my *= sc; lp_my *= sc; m_my = cand; }
-            m_ref[g] = cand;
+        for (int p = 0; p < NP; ++p) {
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const float cand = __shfl_sync(0xffffffffu, zl2[p], (lane & 16) | (g << SH));
+            if (cand > m_ref[g]) {
+              const float sc = exp2_diff(m_ref[g], cand);
+              const f32x2 sc2 = pack2(sc, sc);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) acc[g][i] = mul2(acc[g][i], sc2);
+              if (myg == g) { l_my *= sc; lp_my *= sc; m_my = cand; }
+              m_ref[g] = cand;
+            }
           }
         }
       }
-      const float wt = valid ? exp2f(zl2 - m_my) : 0.f;
-      l_my += wt;
-      lp_my = fmaf(wt, exp2f(0.5f * kLog2e * sig), lp_my);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const float wg = __shfl_sync(0xffffffffu, wt, (lane & 16) | (g << SH));
+      for (int p = 0; p < NP; ++p) {
+        // rows past the end contribute nothing (their shared-memory bytes are stale, and m_my may still be -inf)
+        const float wt = valid[p] ? fast_exp2(zl2[p] - m_my) : 0.f;
+        l_my += wt;
+        if (valid[p]) lp_my = fmaf(wt, fast_exp2(0.5f * kLog2e * sig[p]), lp_my);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[g][i] = fmaf(wg, vv[i], acc[g][i]);
+        for (int g = 0; g < G; ++g) {
+          const float wg = __shfl_sync(0xffffffffu, wt, (lane & 16) | (g << SH));
+          const f32x2 w2 = pack2(wg, wg);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) acc[g][i] = fma2(w2, vv[p][i], acc[g][i]);
+        }
       }
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(&empty_bar[st]);
         if (warp == 0) *(volatile int *)&s_consumed = it + 1;
       }
+      if (++st == stages) { st = 0; phase ^= 1; }
       if (++tl == ui.tiles) {
         tl = 0;
         do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);

@@ -70,18 +70,10 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   }
 
   // ---- normalisers of Eq. 9 from the scan partials of this unit (entries c + unit, c in [cfirst, cfirst + ccount)) ----
-  if (tid == 0) {
-    long long T = 0, T0 = 0;
-    for (int u = 0; u < units; ++u) {
-      const int n = max(min(seq_lens[u / P.Hkv], P.max_blocks * P.bs), 0);
-      const int tiles = ((n + P.bs - 1) / P.bs + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE;
-      if (u == unit) T0 = T;
-      T += tiles;
-    }
-    const long long tpc = (T + scan_grid - 1) / scan_grid;
-    const int my_tiles = (X + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE;
-    s_cfirst = (int)(T0 / tpc);
-    s_ccount = (int)((T0 + my_tiles - 1) / tpc) - s_cfirst + 1;
+  if (warp == 0) {
+    int cfirst, ccount;
+    unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
+    if (lane == 0) { s_cfirst = cfirst; s_ccount = ccount; }
   }
   __syncthreads();
   if (warp < G) {
@@ -105,16 +97,38 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   for (int g = 0; g < G; ++g) { Mg[g] = s_M[g]; iL[g] = s_invL[g]; }
   const bool cached = X <= kSmemKeys;
   bool nonfinite = false;
-  for (int b = tid; b < X; b += kThreads) {
-    float sc = 0.f;
+  // four blocks per thread at a time, so that their loads are in flight together
+  for (int base = 0; base < X; base += 4 * kThreads) {
+    float2 v[4][G];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const float2 v = ls[(size_t)b * G + g];
-      sc = fmaf(exp2f(fmaf(v.x, kLog2e, -Mg[g])) * iL[g], v.y, sc);
+    for (int j = 0; j < 4; ++j) {
+      const int b = base + j * kThreads + tid;
+      if (b < X) {
+        if (G >= 2) {
+          const float4 *p4 = reinterpret_cast<const float4 *>(ls + (size_t)b * G);
+#pragma unroll
+          for (int g = 0; g < G / 2; ++g) {
+            const float4 t = p4[g];
+            v[j][2 * g] = make_float2(t.x, t.y);
+            v[j][2 * g + 1] = make_float2(t.z, t.w);
+          }
+        } else {
+          v[j][0] = ls[b];
+        }
+      }
     }
-    if (!(sc >= 0.f) || sc > 3.0e38f) { nonfinite = true; sc = 0.f; }
-    scores[b] = sc;
-    if (cached) skeys[b] = __float_as_uint(sc);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int b = base + j * kThreads + tid;
+      if (b < X) {
+        float sc = 0.f;
+#pragma unroll
+        for (int g = 0; g < G; ++g) sc = fmaf(fast_exp2(fmaf(v[j][g].x, kLog2e, -Mg[g])) * iL[g], v[j][g].y, sc);
+        if (!(sc >= 0.f) || sc > 3.0e38f) { nonfinite = true; sc = 0.f; }
+        scores[b] = sc;
+        if (cached) skeys[b] = __float_as_uint(sc);
+      }
+    }
   }
   if (nonfinite) atomicOr(P.status, CKV_DEV_NONFINITE);
   __syncthreads();   // scores[] written by this CTA are read back below (same CTA: visible after the barrier)
