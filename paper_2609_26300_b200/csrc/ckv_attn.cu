@@ -219,7 +219,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
         bool raise = false;
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-          const float2 v = __ldg(ls + (size_t)blk * G + g);
+          const float2 v = __ldg(ls + (size_t)g * P.max_blocks + blk);
           zl2[g] = (v.x - 0.5f * v.y) * kLog2e;
           raise |= zl2[g] > m_ref[g] + CKV_RESCALE_SLACK;
         }

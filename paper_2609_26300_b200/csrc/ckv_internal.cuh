@@ -27,7 +27,7 @@ struct CkvDev {
   // block summaries (caller's stats buffer)
   float *kmean, *dbar, *vmean;
   // workspace
-  float2 *ls;        // [unit][max_blocks][G]  (log block weight estimate l_{g,b}, sigma_hat^2_{g,b})
+  float2 *ls;        // [unit][G][max_blocks]  (log block weight estimate l_{g,b}, sigma_hat^2_{g,b})
   float *scores;     // [unit][max_blocks]     S_b
   float *comp_part;  // [scan CTA + unit][G][CKV_PART_STRIDE]  all-block mean-compensation partials
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials

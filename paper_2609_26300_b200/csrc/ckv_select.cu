@@ -104,17 +104,8 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
     for (int j = 0; j < 4; ++j) {
       const int b = base + j * kThreads + tid;
       if (b < X) {
-        if (G >= 2) {
-          const float4 *p4 = reinterpret_cast<const float4 *>(ls + (size_t)b * G);
 #pragma unroll
-          for (int g = 0; g < G / 2; ++g) {
-            const float4 t = p4[g];
-            v[j][2 * g] = make_float2(t.x, t.y);
-            v[j][2 * g + 1] = make_float2(t.z, t.w);
-          }
-        } else {
-          v[j][0] = ls[b];
-        }
+        for (int g = 0; g < G; ++g) v[j][g] = ls[(size_t)g * P.max_blocks + b];   // head-major: coalesced per head
       }
     }
 #pragma unroll
