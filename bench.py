@@ -232,10 +232,14 @@ def main():
     n0 = int(lens.max())
     max_len = n0 + total
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    clean = torch.zeros(64 << 20, dtype=torch.float32, device=dev)
     outputs = ckv.alloc_outputs(w.batch, w.budget_tokens)
 
     def l2_flush():
+        # write a buffer larger than L2, then read another one: L2 ends up holding clean lines of neither
+        # the cache nor the summaries, so the timed step neither hits in L2 nor pays for dirty write-backs
         flush.zero_()
+        clean.sum()
 
     def sync_all():
         torch.cuda.synchronize()
@@ -372,7 +376,7 @@ def main():
         "config": {"workload": "configs[2] llama8b_128k_b4: batch 4, 32q/8kv heads, d128, ctx 131072 (+ appended "
                                "tokens), block 16, budget 2048, r=4, fp32 summaries, bf16 paged KV",
                    "step": "ckv_append + ckv_decode replayed as one CUDA graph; CUDA events around each replay",
-                   "l2": "flushed between steps (256 MiB memset outside the events); per-step inputs exceed L2",
+                   "l2": "flushed between steps (256 MiB memset then 256 MiB read, outside the events); per-step inputs exceed L2",
                    "replicas": "every rank runs the whole workload (the path does not shard)",
                    "kv_storage": "bf16", "seed": w.seed},
         "tokens_per_s": world * w.batch / (us_per_step * 1e-6),

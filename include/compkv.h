@@ -97,7 +97,7 @@ const char *ckv_strerror(int status);
 int ckv_last_cuda_error(void);
 
 /* Sizes in bytes of the two device buffers a context needs (Sec. 4.2: 2d + r + 1 scalars per
- * block; the count |b| is implied by seq_lens, so 2d + r fp32 scalars are stored).
+ * block; the count |b| is implied by seq_lens, so 2d + r 32-bit scalars are stored).
  * stats_bytes: block summaries for max_batch sequences.  workspace_bytes: scratch for one
  * decode step at max_batch (block log-weights, scores, split partials, host staging).
  * Host-only; validates the layout (CKV_ERR_BAD_LAYOUT). */
@@ -105,10 +105,12 @@ int ckv_query_sizes(const ckv_layout *layout, size_t *stats_bytes, size_t *works
 
 /* Byte offsets, inside the stats buffer, of its three regions (the "selection region" holds
  * mean keys and grouped variances, the "mean-values region" the mean values; Sec. 4.3):
- *   kmean [max_batch][num_kv_heads][max_blocks_per_seq][head_dim] fp32
+ *   kmean [max_batch][num_kv_heads][max_blocks_per_seq] rows of 512 bytes
  *   dbar  [max_batch][num_kv_heads][max_blocks_per_seq][var_groups] fp32
- *   vmean [max_batch][num_kv_heads][max_blocks_per_seq][head_dim] fp32
- * Host-only. */
+ *   vmean [max_batch][num_kv_heads][max_blocks_per_seq] rows of 512 bytes
+ * A mean-key / mean-value row holds its 128 entries as split bf16 pairs (hi = bf16(x),
+ * lo = bf16(x - hi): 32 bits per entry, relative error <= 2^-18) in a bank-swizzled chunk
+ * order private to the kernels; use ckv_stats_export() to read summaries.  Host-only. */
 int ckv_stats_offsets(const ckv_layout *layout, size_t *kmean_off, size_t *dbar_off, size_t *vmean_off);
 
 /* Create a context over caller-owned device buffers (256-byte aligned, at least the sizes
@@ -125,6 +127,11 @@ void ckv_destroy(ckv_ctx *ctx);
  * max_seq_len_host: an upper bound (host) on seq_lens[s], used only to size the grid. */
 int ckv_stats_build(ckv_ctx *ctx, const void *k_pool, const void *v_pool, const int32_t *page_table,
                     const int32_t *seq_lens, int batch, int max_seq_len_host, ckv_stream stream);
+
+/* Write the summaries of `batch` sequences as plain fp32 arrays (device):
+ *   kmean, vmean [batch][num_kv_heads][max_blocks_per_seq][head_dim], dbar [...][var_groups].
+ * Rows at or past X_s are unspecified.  For inspection and tests. */
+int ckv_stats_export(ckv_ctx *ctx, int batch, float *kmean, float *dbar, float *vmean, ckv_stream stream);
 
 /* Append one token per sequence (Sec. 4.2 "updated incrementally", App. D.1): writes
  * k_new / v_new at position seq_lens[s] of the paged cache, recomputes the summary of the

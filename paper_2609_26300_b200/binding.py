@@ -22,7 +22,7 @@ CKV_ERR_CAPACITY, CKV_ERR_CUDA, CKV_ERR_TIMEOUT = -4, -5, -6
 CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE = 1, 2, 4
 
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
-           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_append", "ckv_decode", "ckv_decode_profile", "ckv_dense_decode",
+           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_decode_profile", "ckv_dense_decode",
            "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
 
 
@@ -68,6 +68,7 @@ def load() -> ctypes.CDLL:
     lib.ckv_destroy.argtypes = [vp]
     lib.ckv_destroy.restype = None
     lib.ckv_stats_build.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp]
+    lib.ckv_stats_export.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.ckv_decode.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.ckv_decode_profile.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp,
@@ -78,7 +79,7 @@ def load() -> ctypes.CDLL:
     lib.ckv_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
     lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_launch_count.restype = ctypes.c_int64
-    for name in ("ckv_query_sizes", "ckv_stats_offsets", "ckv_create", "ckv_stats_build", "ckv_append",
+    for name in ("ckv_query_sizes", "ckv_stats_offsets", "ckv_create", "ckv_stats_build", "ckv_stats_export", "ckv_append",
                  "ckv_decode", "ckv_decode_profile", "ckv_dense_decode", "ckv_copy_scores", "ckv_step_host", "ckv_read_status"):
         getattr(lib, name).restype = i32
     _lib = lib
@@ -151,17 +152,17 @@ class CompKV:
         except Exception:
             pass
 
-    # ---- views ------------------------------------------------------------------------------------------
-    def stats_views(self):
-        """(kmean, dbar, vmean) fp32 views into the stats buffer, [max_batch][kv_heads][max_blocks][...]."""
+    # ---- summaries ----------------------------------------------------------------------------------------
+    def export_stats(self, batch: Optional[int] = None):
+        """ckv_stats_export: (kmean, dbar, vmean) as fp32 tensors [batch][kv_heads][max_blocks][...]."""
         L = self.layout
-        ko, do, vo = stats_offsets(L)
-        rows = L.max_batch * L.num_kv_heads * L.max_blocks_per_seq
-        f = self.stats.view(torch.float32)
-        shape = (L.max_batch, L.num_kv_heads, L.max_blocks_per_seq)
-        km = f[ko // 4: ko // 4 + rows * L.head_dim].view(*shape, L.head_dim)
-        db = f[do // 4: do // 4 + rows * L.var_groups].view(*shape, L.var_groups)
-        vm = f[vo // 4: vo // 4 + rows * L.head_dim].view(*shape, L.head_dim)
+        batch = batch or L.max_batch
+        shape = (batch, L.num_kv_heads, L.max_blocks_per_seq)
+        km = torch.empty(*shape, L.head_dim, dtype=torch.float32, device=self.device)
+        db = torch.empty(*shape, L.var_groups, dtype=torch.float32, device=self.device)
+        vm = torch.empty(*shape, L.head_dim, dtype=torch.float32, device=self.device)
+        _check(self.lib.ckv_stats_export(self._ctx, batch, _ptr(km), _ptr(db), _ptr(vm), _stream()),
+               "ckv_stats_export")
         return km, db, vm
 
     # ---- C ABI calls --------------------------------------------------------------------------------------

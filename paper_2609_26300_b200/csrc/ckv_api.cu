@@ -50,7 +50,7 @@ Regions regions(const ckv_layout *L) {
   R.status = o; o = align_up(o + 256, 256);
   R.ls = o;     o = align_up(o + rows * G * sizeof(float2), 256);
   R.scores = o; o = align_up(o + rows * 4, 256);
-  R.comp = o;   o = align_up(o + (units + CKV_MAX_SCAN_CTAS) * G * CKV_PART_STRIDE * 4, 256);
+  R.comp = o;   o = align_up(o + (units + CKV_MAX_SCAN_CTAS) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE * 4, 256);
   R.attn = o;   o = align_up(o + units * CKV_MAX_SPLITS * G * CKV_PART_STRIDE * 4, 256);
   R.stage_q = o;    o = align_up(o + (size_t)L->max_batch * L->num_q_heads * CKV_D * esz, 256);
   R.stage_knew = o; o = align_up(o + units * CKV_D * esz, 256);
@@ -142,7 +142,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.max_blocks = layout->max_blocks_per_seq; P.max_pages_per_seq = P.max_blocks * P.ppb;
   P.num_pages = layout->num_pages; P.sink = layout->sink_blocks; P.recent = layout->recent_blocks;
   P.scale = c->layout.sm_scale;
-  P.kmean = (float *)(sb + R.kmean); P.dbar = (float *)(sb + R.dbar); P.vmean = (float *)(sb + R.vmean);
+  P.kmean = (__nv_bfloat16 *)(sb + R.kmean); P.dbar = (float *)(sb + R.dbar); P.vmean = (__nv_bfloat16 *)(sb + R.vmean);
   P.status = (int *)(wb + R.status);
   P.ls = (float2 *)(wb + R.ls); P.scores = (float *)(wb + R.scores);
   P.comp_part = (float *)(wb + R.comp); P.attn_part = (float *)(wb + R.attn);
@@ -171,6 +171,13 @@ int ckv_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const in
   if (!k_pool || !v_pool || !page_table || !seq_lens) return CKV_ERR_INVALID_ARG;
   CKV_CUDA(ckv_launch_stats_build(c, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host,
                                   (cudaStream_t)stream));
+  return CKV_OK;
+}
+
+int ckv_stats_export(ckv_ctx *c, int batch, float *kmean, float *dbar, float *vmean, ckv_stream stream) {
+  if (c == nullptr || batch <= 0 || batch > c->layout.max_batch) return CKV_ERR_INVALID_ARG;
+  if (!kmean || !dbar || !vmean) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(ckv_launch_stats_export(c, batch, kmean, dbar, vmean, (cudaStream_t)stream));
   return CKV_OK;
 }
 

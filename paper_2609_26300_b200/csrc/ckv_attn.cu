@@ -126,7 +126,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
   const int g_own0 = (G >= 2) ? (li & 1) * KEEP : 0;
   const int t_own = hw + 2 * (li >> 1);
   const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
-  const float *vmean = P.vmean + (size_t)unit * P.max_blocks * CKV_D;
+  const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * CKV_ROW_ELEMS;
   uint32_t phase_bits = 0;   // bit b: parity of the next completion of buffer b
   bool aborted = false;
   int n_abort = 0;
@@ -238,9 +238,8 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
           }
         }
         if (hw == 0) {
-          const float4 a = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li));
-          const float4 b4 = __ldg(reinterpret_cast<const float4 *>(vmean + (size_t)blk * CKV_D + 8 * li) + 1);
-          const float vb[8] = {a.x, a.y, a.z, a.w, b4.x, b4.y, b4.z, b4.w};
+          float vb[8];
+          load_split8(vmean + (size_t)blk * CKV_ROW_ELEMS, li, blk, vb);
 #pragma unroll
           for (int g = 0; g < G; ++g) {
             const float wbar_g = exp2f(zl2[g] - m_ref[g]);
@@ -308,7 +307,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
 // one thread per output coordinate.  Partials: the unit's attention splits and, unless every block
 // was selected, the scan partials of the CTAs whose tile range touched the unit (entries c + unit for
 // c in [c_first, c_last], recomputed here from the same tile arithmetic the scan uses).
-constexpr int kMergeMax = CKV_MAX_SPLITS + CKV_MAX_SCAN_CTAS;
+constexpr int kMergeMax = CKV_MAX_SPLITS + CKV_MAX_SCAN_CTAS * CKV_SCAN_WARPS;
 
 template <typename T>
 __global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *__restrict__ seq_lens,
@@ -331,11 +330,11 @@ __global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *_
     if (c == 0) { s_cfirst = cfirst; s_ccount = ccount; }
   }
   __syncthreads();
-  const int n_comp = s_ccount;
+  const int n_comp = s_ccount * CKV_SCAN_WARPS;
   const int n = n_splits + n_comp;
   const size_t step = (size_t)G * CKV_PART_STRIDE;
   const float *ap = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS * G + g) * CKV_PART_STRIDE;
-  const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * G + g) * CKV_PART_STRIDE;
+  const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * CKV_SCAN_WARPS * G + g) * CKV_PART_STRIDE;
   float mloc = -CUDART_INF_F;
   for (int i = c; i < n; i += CKV_D) {
     const float *p = i < n_splits ? ap + (size_t)i * step : cp + (size_t)(i - n_splits) * step;

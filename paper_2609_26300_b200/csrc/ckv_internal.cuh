@@ -10,9 +10,11 @@
 
 #define CKV_D 128             // head dimension the kernels are written for
 #define CKV_PAGE 16           // tokens per page
+#define CKV_ROW_ELEMS 256     // bf16 elements of one mean-key / mean-value summary row (128 hi halves + 128 lo halves)
 #define CKV_PART_STRIDE 132   // floats per split partial: m, l, pad, pad, acc[128]
 #define CKV_SCAN_TILE 32      // blocks per scan tile
-#define CKV_MAX_SCAN_CTAS 512 // persistent scan grid is capped at this many CTAs
+#define CKV_SCAN_WARPS 8       // consumer warps of a scan CTA, each with a partial of its own
+#define CKV_MAX_SCAN_CTAS 160 // persistent scan grid is capped at this many CTAs
 #define CKV_MAX_SPLITS 64     // attention partials per unit
 #define CKV_RESCALE_SLACK 16.0f  // log2 units: running maxima are only raised when exceeded by this much
 
@@ -24,12 +26,13 @@ struct CkvDev {
   int Hq, Hkv, G, bs, ppb, r, glayout;
   int max_blocks, max_pages_per_seq, num_pages, sink, recent;
   float scale;
-  // block summaries (caller's stats buffer)
-  float *kmean, *dbar, *vmean;
+  // block summaries (caller's stats buffer): mean keys / mean values as split-bf16 rows (see store_split8), variances fp32
+  __nv_bfloat16 *kmean, *vmean;   // [unit][max_blocks][CKV_ROW_ELEMS]
+  float *dbar;                    // [unit][max_blocks][r]
   // workspace
   float2 *ls;        // [unit][G][max_blocks]  (log block weight estimate l_{g,b}, sigma_hat^2_{g,b})
   float *scores;     // [unit][max_blocks]     S_b
-  float *comp_part;  // [scan CTA + unit][G][CKV_PART_STRIDE]  all-block mean-compensation partials
+  float *comp_part;  // [(scan CTA + unit) * CKV_SCAN_WARPS + warp][G][CKV_PART_STRIDE]  all-block mean-compensation partials
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials
   int *status;       // device status word
 };
@@ -53,6 +56,7 @@ int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len);
 // ---- launchers (one per translation unit) ---------------------------------------------------------
 cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int *page_table,
                                    const int *seq_lens, int batch, int max_len, cudaStream_t st);
+cudaError_t ckv_launch_stats_export(ckv_ctx *c, int batch, float *kmean, float *dbar, float *vmean, cudaStream_t st);
 cudaError_t ckv_launch_append(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
                               const void *k_new, const void *v_new, int batch, cudaStream_t st);
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
@@ -96,6 +100,40 @@ __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 __device__ __forceinline__ void store_out(float *p, float x) { *p = x; }
 __device__ __forceinline__ void store_out(__nv_bfloat16 *p, float x) { *p = __float2bfloat16_rn(x); }
+
+// Summary rows.  A mean key / mean value entry x is stored as two bf16, hi = bf16(x) and lo = bf16(x - hi): the same
+// 32 bits as an fp32, relative error at most 2^-18, and directly usable as tensor-core operands (x * y is evaluated
+// as hi * y + lo * y).  A row of 128 entries is 512 bytes: sixteen 16-byte chunks of hi halves (8 coordinates each),
+// then sixteen chunks of lo halves.  Inside every group of 8 chunks the chunk order is XORed with (block index & 7),
+// so that a matrix load touching one chunk column of 8 consecutive rows hits 8 different bank groups.
+__device__ __forceinline__ int swz_chunk(int chunk, int block) { return chunk ^ (block & 7); }
+
+__device__ __forceinline__ void store_split8(__nv_bfloat16 *row, int chunk, int block, const float (&x)[8]) {
+  uint32_t hi[4], lo[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(x[2 * i]), h1 = __float2bfloat16_rn(x[2 * i + 1]);
+    const __nv_bfloat16 l0 = __float2bfloat16_rn(x[2 * i] - __bfloat162float(h0));
+    const __nv_bfloat16 l1 = __float2bfloat16_rn(x[2 * i + 1] - __bfloat162float(h1));
+    hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+    lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+  }
+  const int p = swz_chunk(chunk, block) * 8;
+  *reinterpret_cast<uint4 *>(row + p) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+  *reinterpret_cast<uint4 *>(row + CKV_D + p) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+}
+
+// The eight entries of one chunk, hi + lo, as floats.
+__device__ __forceinline__ void load_split8(const __nv_bfloat16 *row, int chunk, int block, float (&x)[8]) {
+  const int p = swz_chunk(chunk, block) * 8;
+  const uint4 h = __ldg(reinterpret_cast<const uint4 *>(row + p));
+  const uint4 l = __ldg(reinterpret_cast<const uint4 *>(row + CKV_D + p));
+  float a[8], b[8];
+  bf16x8_to_float(h, a);
+  bf16x8_to_float(l, b);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) x[i] = a[i] + b[i];
+}
 
 // Coordinate group of coordinate i (App. A.4 of the paper; see ckv_layout::group_layout).
 __device__ __forceinline__ int group_of(int i, int r, int glayout) {

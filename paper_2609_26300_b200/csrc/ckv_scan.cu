@@ -1,28 +1,30 @@
 // Summary scan: one streaming pass over every block summary (Eq. 8-9 and the compensation sums
-// of Eq. 12), as a persistent, bulk-copy-pipelined kernel.
+// of Eq. 12), as a persistent, bulk-copy-pipelined, tensor-core kernel.
 //
 // For every block b and query head g of a unit the pass computes
 //   zbar_{g,b}        = q_g . kbar_b * scale                      (block-mean logit, Sec. 4.1)
 //   sigma_hat^2_{g,b} = scale^2 sum_t w_{g,t} Dbar_{b,t}         (Eq. 8 with 1/d = scale^2, w_{g,t} = sum_{i in G_t} q_{g,i}^2)
 //   l_{g,b}           = log|b| + zbar + sigma_hat^2 / 2           (log of the numerator of Eq. 9)
-// and stores (l, sigma_hat^2) for the selection kernel, together with per-CTA partials of the
-// normaliser of Eq. 9.  In the same pass it accumulates the mean-compensation terms of Eq. 12 over
-// ALL blocks,  sum_b |b| e^{zbar} vbar_b  and  sum_b |b| e^{zbar},  as online-softmax partials; the
-// terms of the blocks that end up selected are taken out again by the attention kernel.  That way
-// kbar, Dbar and vbar are each read from HBM exactly once per decode step.
+// and stores (l, sigma_hat^2) for the selection kernel, together with partials of the normaliser of
+// Eq. 9.  In the same pass it accumulates the mean-compensation terms of Eq. 12 over ALL blocks,
+// sum_b |b| e^{zbar} vbar_b  and  sum_b |b| e^{zbar},  as online-softmax partials; the terms of the
+// blocks that end up selected are taken out again by the attention kernel.  That way kbar, Dbar and
+// vbar are each read from HBM exactly once per decode step.
+//
+// The two contractions are the GQA-grouped Q Kbar^T and W Vbar tiles, on mma.sync.m16n8k16 (bf16 in,
+// fp32 accumulate): heads are the M dimension (G <= 8 rows of 16 used), 8 blocks the N dimension of
+// Q Kbar^T, whose accumulator layout is the A-operand layout of W Vbar.  The summaries are stored as
+// split bf16 pairs (hi + lo), so x * y is hi * y + lo * y with no conversion instructions; the weights
+// w = |b| e^{zbar - m} are split the same way (three products per tile: hi hi, lo hi, hi lo).
 //
 // Schedule: the summaries of all units are cut into tiles of 32 consecutive blocks; the tiles, in
 // (unit, position) order, are split into one contiguous range per CTA and the grid is one CTA per
-// SM.  A producer warp streams the CTA's tiles into a ring of shared-memory stages with
-// cp.async.bulk (mean-key rows one copy each, so that they land with a padded row stride), completion
-// on mbarriers.  Eight consumer warps work on a tile in three phases separated by named barriers:
-//   1. mean logits: each thread takes one block (one padded row, conflict-free) and a pair of heads over
-//      a slice of the 128 coordinates, the query slice coming from shared memory as a broadcast;
-//   2. one thread per (block, head): variance projection, l, the running maximum of the tile, the
-//      compensation weight |b| e^{zbar - m}; weights go to shared memory;
-//   3. accumulation: a warp takes a mean-value row, each lane four coordinates of all G heads.
-// A CTA writes one partial per unit it touched; partial (CTA c, unit u) lives in entry c + u, which
-// is unique because the (c, u) pairs that occur form a monotone staircase.
+// SM.  A producer thread streams the CTA's tiles into a ring of shared-memory stages with
+// cp.async.bulk (two 16 KB copies and the variances per tile), completion on mbarriers.  Each of the
+// eight consumer warps takes every eighth half tile (16 blocks) on its own -- there is no CTA-wide
+// barrier in the loop -- with a per-warp running maximum that is only raised when exceeded by a
+// slack.  A warp writes one partial per unit its CTA touched; partial (CTA c, warp w, unit u) lives
+// in entry (c + u) * 8 + w, unique because the (c, u) pairs that occur form a monotone staircase.
 #include "ckv_internal.cuh"
 #include "ckv_pipe.cuh"
 
@@ -30,12 +32,12 @@ namespace {
 
 using namespace ckv_pipe;
 
-constexpr int TB = CKV_SCAN_TILE;   // blocks per tile (32: one block per lane in phase 1)
-constexpr int KROW = CKV_D + 4;     // padded mean-key row (floats): rows 8 apart share banks, a quarter warp does not
+constexpr int TB = CKV_SCAN_TILE;   // blocks per tile
 constexpr int kMaxStages = 8;
-constexpr int kConsumers = 256;     // 8 consumer warps
-constexpr int kThreads = kConsumers + 32;   // plus the producer warp
-constexpr int kMaxUnits = 1024;     // sequence lengths are staged in shared memory up to this many sequences
+constexpr int kConsumerWarps = CKV_SCAN_WARPS;
+constexpr int kThreads = kConsumerWarps * 32 + 32;   // plus the producer warp
+constexpr int kMaxSeqs = 1024;      // sequence lengths are staged in shared memory up to this many sequences
+constexpr int kRowBytes = CKV_ROW_ELEMS * 2;
 
 struct UnitInfo { int N, X, tiles; };
 
@@ -47,48 +49,59 @@ __device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *__rest
   return ui;
 }
 
-// Tiles of one sequence's units: from the staged table, or recomputed for sequences beyond it.
 __device__ __forceinline__ int seq_tiles(const int *s_tiles, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
-  if (i < kMaxUnits) return s_tiles[i];
+  if (i < kMaxSeqs) return s_tiles[i];
   const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
   return ((n + P.bs - 1) / P.bs + TB - 1) / TB;
 }
 
-// Phase-1 work split: HP heads per thread, the 128 coordinates cut into QD slices, so that the
-// (head group, slice) tasks are a multiple of the 8 consumer warps.
-template <int G> struct P1Cfg {
-  static constexpr int HP = G >= 2 ? 2 : 1;
-  static constexpr int HG = G / HP;                       // head groups
-  static constexpr int QD = (HG >= 2) ? 4 : 8;            // coordinate slices
-  static constexpr int TASKS = HG * QD;                   // warp tasks per tile: 8 (G <= 4) or 16 (G = 8)
-  static constexpr int SLICE = CKV_D / QD;                // coordinates per slice
-};
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr) : "memory");
+}
+// D(16x8) = A(16x16) B(16x8) + C with only rows 0..7 of A in use (a1 = a3 = 0): d0, d1 accumulate in place, the
+// two results of the unused rows go to scratch outputs and take zero as their C, so they chain nothing.
+__device__ __forceinline__ void mma_rows8(float &d0, float &d1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  float x, y;
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %5}, {%7, %8}, "
+               "{%0, %1, %9, %9};"
+               : "+f"(d0), "+f"(d1), "=f"(x), "=f"(y)
+               : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+}
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+template <typename QT> struct QSplit { static constexpr bool value = false; };
+template <> struct QSplit<float> { static constexpr bool value = true; };
 
 template <int G, typename QT>
 __global__ void __launch_bounds__(kThreads, 1)
 ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_lens, int units, int stages) {
-  using C1 = P1Cfg<G>;
-  extern __shared__ __align__(128) float stage_mem[];
+  constexpr bool QS = QSplit<QT>::value;   // fp32 queries are split into hi + lo like the summaries
+  extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
-  __shared__ __align__(16) float sq[G][CKV_D];           // the unit's queries, scaled
-  __shared__ __align__(16) float sw[CKV_D][G];           // w_{g,t} * scale^2
-  __shared__ __align__(16) float zpart[C1::QD][G][TB];   // phase 1 -> 2: partial mean logits
-  __shared__ __align__(16) float2 wbuf[2][TB][G];        // phase 2 -> 3: compensation weights, each stored twice (w, w)
-  __shared__ __align__(8) float2 s_scale[2][G];          // phase 2 -> 3: accumulator rescale factors (s, s), 1 unless the
-                                                         // running maximum moved; both double-buffered by tile parity
-  __shared__ float s_mref[G];                            // flush: the heads' running maxima
-  __shared__ __align__(16) float red[G][CKV_D];          // flush: sum of the warps' accumulators
-  __shared__ float s_l[8][G], s_lp[8][G];
-  __shared__ int s_u0, s_tl0, s_count, s_abort, s_issued, s_consumed;
-  __shared__ int s_tiles[kMaxUnits];
+  __shared__ int s_u0, s_tl0, s_count, s_ulast, s_abort, s_issued;
+  __shared__ int s_tiles[kMaxSeqs];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool dbar_bulk = P.r >= 4;   // smaller rows cannot keep the 16-byte alignment bulk copies need
-  const int stage_floats = TB * KROW + TB * CKV_D + (dbar_bulk ? TB * P.r : 0);
+  const bool r4 = P.r == 4;          // the default: the variance projection is four FMAs on one 16-byte read
+  const int stage_bytes = TB * 2 * kRowBytes + (dbar_bulk ? TB * P.r * 4 : 0);
+  // per-warp w_{g,t} table for r != 4, behind the ring
+  float *sw_all = reinterpret_cast<float *>(stage_mem + (size_t)stages * stage_bytes);
 
-  // tiles per unit from the sequence lengths (staged in shared memory: one parallel load, no serial global reads)
+  // rows past a unit's last block are never copied: clear the ring once so that they hold zeros or old summaries,
+  // never arbitrary bit patterns (a NaN times a zero weight would poison the accumulators)
+  for (int i = tid; i < stages * stage_bytes / 16; i += kThreads) reinterpret_cast<uint4 *>(stage_mem)[i] = make_uint4(0u, 0u, 0u, 0u);
+  fence_proxy_async();
   const int batch = units / P.Hkv;
-  for (int i = tid; i < batch && i < kMaxUnits; i += kThreads) {
+  for (int i = tid; i < batch && i < kMaxSeqs; i += kThreads) {
     const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
     s_tiles[i] = ((n + P.bs - 1) / P.bs + TB - 1) / TB;
   }
@@ -101,147 +114,179 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     long long cnt = T - first;
     if (cnt > tpc) cnt = tpc;
     if (cnt < 0) cnt = 0;
-    int u0 = 0, tl0 = 0;
+    int u0 = 0, tl0 = 0, ulast = 0;
     if (cnt > 0) {
       long long accum = 0;
+      bool have_first = false;
       for (int i = 0; i < batch; ++i) {
         const long long t = seq_tiles(s_tiles, seq_lens, P, i);
-        if (t > 0 && first < accum + t * P.Hkv) {
-          const long long off = first - accum;
-          u0 = i * P.Hkv + (int)(off / t); tl0 = (int)(off % t);
-          break;
+        if (t > 0) {
+          if (!have_first && first < accum + t * P.Hkv) {
+            const long long off = first - accum;
+            u0 = i * P.Hkv + (int)(off / t); tl0 = (int)(off % t);
+            have_first = true;
+          }
+          if (first + cnt - 1 < accum + t * P.Hkv) {
+            ulast = i * P.Hkv + (int)((first + cnt - 1 - accum) / t);
+            break;
+          }
         }
         accum += t * P.Hkv;
       }
     }
-    s_u0 = u0; s_tl0 = tl0; s_count = (int)cnt; s_abort = 0; s_issued = 0; s_consumed = 0;
-    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], 8); }
+    s_u0 = u0; s_tl0 = tl0; s_ulast = ulast; s_count = (int)cnt; s_abort = 0; s_issued = 0;
+    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], 2); }
     fence_barrier_init();
   }
   __syncthreads();
   const int count = s_count;
   if (count == 0) return;   // uniform: this CTA has no tiles
 
-  if (warp == 8) {
-    // ---------------- producer warp: streams the CTA's tiles into the ring ----------------
-    int u = s_u0, tl = s_tl0, st = 0;
-    uint32_t phase = 0;            // parity of the empty-barrier phase the next refill of stage `st` waits for
-    UnitInfo ui = unit_info(P, seq_lens, u);
-    for (int it = 0; it < count; ++it) {
-      int stop = 0;
-      if (lane == 0) {
+  if (warp == kConsumerWarps) {
+    // ---------------- producer: one thread streams the CTA's tiles into the ring ----------------
+    if (lane == 0) {
+      int u = s_u0, tl = s_tl0, st = 0;
+      uint32_t phase = 0;            // parity of the empty-barrier phase the next refill of stage `st` waits for
+      UnitInfo ui = unit_info(P, seq_lens, u);
+      for (int it = 0; it < count; ++it) {
         if (it >= stages && !mbar_wait(&empty_bar[st], phase)) {
           atomicOr(P.status, CKV_DEV_TIMEOUT);
           *(volatile int *)&s_abort = 1;
         }
-        stop = *(volatile int *)&s_abort;
-      }
-      if (__shfl_sync(0xffffffffu, stop, 0)) break;
-      const int b0 = tl * TB;
-      const int nb = min(TB, ui.X - b0);
-      const size_t row = (size_t)u * P.max_blocks + b0;
-      float *sk = stage_mem + (size_t)st * stage_floats;
-      float *sv = sk + TB * KROW;
-      const uint32_t kbytes = (uint32_t)nb * CKV_D * 4;
-      const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
-      if (lane == 0) mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
-      __syncwarp();
-      if (lane < nb) bulk_g2s(sk + lane * KROW, P.kmean + (row + lane) * CKV_D, CKV_D * 4, &full_bar[st]);
-      if (lane == 0) {
-        bulk_g2s(sv, P.vmean + row * CKV_D, kbytes, &full_bar[st]);
-        if (dbar_bulk) bulk_g2s(sv + TB * CKV_D, P.dbar + row * P.r, dbytes, &full_bar[st]);
+        if (*(volatile int *)&s_abort) break;
+        const int b0 = tl * TB;
+        const int nb = min(TB, ui.X - b0);
+        const size_t row = (size_t)u * P.max_blocks + b0;
+        unsigned char *sk = stage_mem + (size_t)st * stage_bytes;
+        unsigned char *sv = sk + TB * kRowBytes;
+        const uint32_t kbytes = (uint32_t)nb * kRowBytes;
+        const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
+        mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
+        bulk_g2s(sk, P.kmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st]);
+        bulk_g2s(sv, P.vmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st]);
+        if (dbar_bulk) bulk_g2s(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, &full_bar[st]);
         *(volatile int *)&s_issued = it + 1;
-      }
-      if (++st == stages) { st = 0; if (it >= stages) phase ^= 1; }
-      if (++tl == ui.tiles) {
-        tl = 0;
-        do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+        if (++st == stages) { st = 0; if (it >= stages) phase ^= 1; }
+        if (++tl == ui.tiles) {
+          tl = 0;
+          do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+        }
       }
     }
   } else {
-    // ---------------- consumers ----------------
-    // phase 1 role: block = lane; task = (head group, coordinate slice)
-    // phase 2 role: one (block, head) per thread; a head's 32 blocks sit in one warp, so its tile maximum is a
-    // warp reduction and the (l, sigma^2) stores of the head-major layout coalesce
-    const bool p2 = warp < G;              // phase 2: warp g owns head g, lane = block of the tile
-    const int p2_bl = lane, p2_g = warp;
-    // phase 3 role: rows warp, warp + 8, ...; this lane's four coordinates of all heads
-    f32x2 acc[G][2];
-    float m_ref = -CUDART_INF_F, l_acc = 0.f, lp_acc = 0.f;   // phase-2 state of head p2_g (same m_ref in every thread of a head)
+    // ---------------- consumer warps: half tile j = warp, warp + 8, ... of the CTA's range ----------------
+    const int head = lane >> 2, qd = lane & 3;   // this thread's accumulator row (head) and column pair
+    const bool hv = head < G;
+    uint32_t qa[8][2], qb[QS ? 8 : 1][2];        // A fragments of the unit's queries (rows 0..7), per 16-coordinate step
+    float acc[16][2];                            // W Vbar accumulator: head `head`, coordinates 8 t + 2 qd + {0, 1}
+    float m_ref = -CUDART_INF_F, l_acc = 0.f, lp_acc = 0.f;
     float wown[4] = {0.f, 0.f, 0.f, 0.f};
-    const bool r4 = P.r == 4 && dbar_bulk;   // the default r: the variance projection is four FMAs on one 16-byte read
+    float *sw = sw_all + (size_t)warp * P.r * G;   // [t][g], r != 4 only
     const float log_bs = logf((float)P.bs);
     float log_last = 0.f;
-    int u = s_u0, tl = s_tl0, cur = -1, st = 0;
-    uint32_t phase = 0;              // parity of the full-barrier phase of stage `st` this pass over the ring
+    const int ulast = s_ulast;
+    int u = s_u0, tl = s_tl0, cur = -1, next_empty = s_u0;
     UnitInfo ui = unit_info(P, seq_lens, u);
     float2 *ls = nullptr;
     const float *db = nullptr;
     bool aborted = false;
 
-    auto flush = [&](int unit_done) {
-      // all warps share m_ref, so their accumulators add directly (shared-memory atomics: this runs once per unit)
-      for (int idx = tid; idx < G * CKV_D; idx += kConsumers) red[idx / CKV_D][idx % CKV_D] = 0.f;
-      named_barrier(1, kConsumers);
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float a0, a1, a2, a3;
-        unpack2(acc[g][0], a0, a1);
-        unpack2(acc[g][1], a2, a3);
-        atomicAdd(&red[g][4 * lane], a0); atomicAdd(&red[g][4 * lane + 1], a1);
-        atomicAdd(&red[g][4 * lane + 2], a2); atomicAdd(&red[g][4 * lane + 3], a3);
-      }
-      if (p2) {
-        // l and lp of head p2_g: sum over the lanes of its warp
-        const float l = warp_sum(l_acc), lp = warp_sum(lp_acc);
-        if (lane == 0) { s_l[0][p2_g] = l; s_lp[0][p2_g] = lp; s_mref[p2_g] = m_ref; }
-      }
-      named_barrier(1, kConsumers);
-      float *part = P.comp_part + (size_t)(blockIdx.x + unit_done) * G * CKV_PART_STRIDE;
-      for (int idx = tid; idx < G * CKV_D; idx += kConsumers) {
-        const int g = idx / CKV_D, i = idx % CKV_D;
-        part[g * CKV_PART_STRIDE + 4 + i] = red[g][i];
-        if (i == 0) {
-          part[g * CKV_PART_STRIDE] = s_mref[g];
-          part[g * CKV_PART_STRIDE + 1] = s_l[0][g];
-          part[g * CKV_PART_STRIDE + 2] = s_lp[0][g];
+    auto write_partial = [&](int unit_id, bool real) {
+      float *part = P.comp_part + ((size_t)(blockIdx.x + unit_id) * kConsumerWarps + warp) * G * CKV_PART_STRIDE;
+      if (!real) {
+        if (lane < G) {
+          part[lane * CKV_PART_STRIDE] = -CUDART_INF_F;
+          part[lane * CKV_PART_STRIDE + 1] = 0.f;
+          part[lane * CKV_PART_STRIDE + 2] = 0.f;
         }
+        return;
       }
-      named_barrier(1, kConsumers);
+      // l and lp: sum over the four lanes that share the head
+      float l = l_acc, lp = lp_acc;
+      l += __shfl_xor_sync(0xffffffffu, l, 1); l += __shfl_xor_sync(0xffffffffu, l, 2);
+      lp += __shfl_xor_sync(0xffffffffu, lp, 1); lp += __shfl_xor_sync(0xffffffffu, lp, 2);
+      if (hv) {
+        float *pg = part + head * CKV_PART_STRIDE;
+#pragma unroll
+        for (int t = 0; t < 16; ++t)
+          *reinterpret_cast<float2 *>(pg + 4 + 8 * t + 2 * qd) = make_float2(acc[t][0], acc[t][1]);
+        if (qd == 0) { pg[0] = m_ref; pg[1] = l; pg[2] = lp; }
+      }
+    };
+    // units of this CTA's range that this warp never worked on still need an (empty) partial
+    auto fill_empty_upto = [&](int upto) {
+      for (; next_empty < upto; ++next_empty)
+        if (unit_info(P, seq_lens, next_empty).tiles > 0) write_partial(next_empty, false);
     };
 
-    for (int it = 0; it < count; ++it) {
+    // advance the walk to this warp's first tile
+    int it = warp >> 1;
+    const int half = warp & 1;
+    for (int k = 0; k < it && k < count; ++k) {
+      if (++tl == ui.tiles) {
+        tl = 0;
+        do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+      }
+    }
+    for (; it < count; it += kConsumerWarps / 2) {
       if (u != cur) {
-        if (cur >= 0) flush(cur);
-        // per-unit setup: the unit's queries (scaled), their per-group squared norms, fresh accumulators
+        if (cur >= 0) { write_partial(cur, true); next_empty = cur + 1; }
+        fill_empty_upto(u);
+        // per-unit setup: query fragments, variance weights, fresh accumulators
         const int s = u / P.Hkv, h = u % P.Hkv;
-        for (int idx = tid; idx < G * CKV_D; idx += kConsumers)
-          sq[idx / CKV_D][idx % CKV_D] = to_float(q[((size_t)s * P.Hq + h * G) * CKV_D + idx]);
-        named_barrier(1, kConsumers);
-        for (int idx = tid; idx < P.r * G; idx += kConsumers) {
-          const int t = idx / G, g = idx % G;
-          float w = 0.f;
-          for (int i = 0; i < CKV_D; ++i)
-            if (group_of(i, P.r, P.glayout) == t) w = fmaf(sq[g][i], sq[g][i], w);
-          sw[t][g] = w * (P.scale * P.scale);   // Eq. 8's 1/d is the squared logit scale
-        }
-        named_barrier(1, kConsumers);
-        for (int idx = tid; idx < G * CKV_D; idx += kConsumers) sq[idx / CKV_D][idx % CKV_D] *= P.scale;
-        if (r4 && p2) {
+        const QT *qrow = q + ((size_t)s * P.Hq + h * G + (hv ? head : 0)) * CKV_D;
 #pragma unroll
-          for (int t = 0; t < 4; ++t) wown[t] = sw[t][p2_g];
+        for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const int c0 = 16 * ks + 8 * hh + 2 * qd;
+            const float x0 = hv ? to_float(qrow[c0]) : 0.f, x1 = hv ? to_float(qrow[c0 + 1]) : 0.f;
+            qa[ks][hh] = pack_bf16(x0, x1);
+            if (QS) qb[QS ? ks : 0][hh] = pack_bf16(x0 - bf16_round(x0), x1 - bf16_round(x1));
+          }
+        }
+        if (r4) {
+          // w_{g,t} for this thread's head: every lane of the quad sums all 128 coordinates (once per unit)
+          float wsum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            float x[8];
+            load8<true>(qrow + 8 * c, x);
+            float s8 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) s8 = fmaf(x[i], x[i], s8);
+            // an aligned run of 8 coordinates lies in one group for r = 4 (groups are runs of 32 or 16)
+            const int t = P.glayout == 0 ? (8 * c) / 32 : ((8 * c) % 64) / 16;
+            wsum[0] += t == 0 ? s8 : 0.f; wsum[1] += t == 1 ? s8 : 0.f;
+            wsum[2] += t == 2 ? s8 : 0.f; wsum[3] += t == 3 ? s8 : 0.f;
+          }
+          if (!hv) { wsum[0] = wsum[1] = wsum[2] = wsum[3] = 0.f; }
+#pragma unroll
+          for (int t = 0; t < 4; ++t) wown[t] = wsum[t] * (P.scale * P.scale);   // Eq. 8's 1/d is the squared logit scale
+        } else {
+          __syncwarp();
+          for (int idx = lane; idx < P.r * G; idx += 32) {
+            const int t = idx / G, g = idx % G;
+            const QT *qg = q + ((size_t)s * P.Hq + h * G + g) * CKV_D;
+            float w = 0.f;
+            for (int i = 0; i < CKV_D; ++i)
+              if (group_of(i, P.r, P.glayout) == t) { const float x = to_float(qg[i]); w = fmaf(x, x, w); }
+            sw[idx] = w * (P.scale * P.scale);
+          }
+          __syncwarp();
         }
 #pragma unroll
-        for (int g = 0; g < G; ++g) { acc[g][0] = pack2(0.f, 0.f); acc[g][1] = pack2(0.f, 0.f); }
+        for (int t = 0; t < 16; ++t) { acc[t][0] = 0.f; acc[t][1] = 0.f; }
         m_ref = -CUDART_INF_F; l_acc = 0.f; lp_acc = 0.f;
         log_last = logf((float)(ui.N - (ui.X - 1) * P.bs));
         const size_t row0 = (size_t)u * P.max_blocks;
         ls = P.ls + row0 * G;   // [head][block] within the unit
         db = P.dbar + row0 * P.r;
         cur = u;
-        named_barrier(1, kConsumers);
       }
-      // a wait that runs out marks the step invalid; the walk (and its barriers) still runs to the end
+      const int st = it % stages;
+      const uint32_t phase = (uint32_t)(it / stages) & 1u;
+      // a wait that runs out marks the step invalid; the walk still runs to the end
       if (!aborted) {
         bool fail = *(volatile int *)&s_abort != 0;
         if (!fail && !mbar_wait(&full_bar[st], phase)) {
@@ -251,146 +296,156 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         }
         aborted = __any_sync(0xffffffffu, fail);
       }
-      const float *sk = stage_mem + (size_t)st * stage_floats;
-      const float *sv = sk + TB * KROW;
-      const float *sd = sv + TB * CKV_D;
       const int b0 = tl * TB;
       const int nb = min(TB, ui.X - b0);
+      const int rb = half * 16;          // first row of this warp's half tile
+      if (!aborted && rb < nb) {
+        const uint32_t sk = smem_u32(stage_mem + (size_t)st * stage_bytes);
+        const uint32_t sv = sk + TB * kRowBytes;
+        const float *sd = reinterpret_cast<const float *>(stage_mem + (size_t)st * stage_bytes + 2 * TB * kRowBytes);
 
-      // ---- phase 1: partial mean logits, thread = (block lane, head group, coordinate slice) ----
-      if (!aborted) {
+        // ---- Z^T = Q Kbar^T: heads x 16 blocks (two n-tiles of 8 blocks), hi and lo planes into one accumulator ----
+        float z[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        {
+          // ldmatrix lane roles: matrix lane / 8 -> 8-coordinate chunk, row lane % 8
+          const int lrow = lane & 7, lmat = lane >> 3;
 #pragma unroll
-        for (int task = warp; task < C1::TASKS; task += 8) {
-          const int hg = task % C1::HG, qd = task / C1::HG;
-          const float *krow = sk + lane * KROW + qd * C1::SLICE;
-          f32x2 za[C1::HP], zb[C1::HP];
+          for (int nt = 0; nt < 2; ++nt) {
+            const int r = rb + nt * 8 + lrow;
+            const uint32_t rowaddr = sk + r * kRowBytes;
 #pragma unroll
-          for (int hh = 0; hh < C1::HP; ++hh) { za[hh] = pack2(0.f, 0.f); zb[hh] = pack2(0.f, 0.f); }
-#pragma unroll
-          for (int c = 0; c < C1::SLICE; c += 4) {
-            // 16-byte loads as two packed pairs: no repacking between the load and the packed FMA
-            const ulonglong2 k2 = *reinterpret_cast<const ulonglong2 *>(krow + c);
-#pragma unroll
-            for (int hh = 0; hh < C1::HP; ++hh) {
-              const ulonglong2 q2 = *reinterpret_cast<const ulonglong2 *>(&sq[hg * C1::HP + hh][qd * C1::SLICE + c]);
-              za[hh] = fma2(q2.x, k2.x, za[hh]);
-              zb[hh] = fma2(q2.y, k2.y, zb[hh]);
+            for (int j = 0; j < 4; ++j) {   // two 16-coordinate steps per ldmatrix.x4
+              const uint32_t coff = (uint32_t)swz_chunk(4 * j + lmat, r) * 16;
+              uint32_t bh[4], bl[4];
+              ldmatrix_x4(bh, rowaddr + coff);
+              ldmatrix_x4(bl, rowaddr + 256 + coff);
+              mma_rows8(z[nt][0], z[nt][1], qa[2 * j][0], qa[2 * j][1], bh[0], bh[1]);
+              mma_rows8(z[nt][0], z[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bh[2], bh[3]);
+              mma_rows8(z[nt][0], z[nt][1], qa[2 * j][0], qa[2 * j][1], bl[0], bl[1]);
+              mma_rows8(z[nt][0], z[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bl[2], bl[3]);
+              if (QS) {
+                mma_rows8(z[nt][0], z[nt][1], qb[QS ? 2 * j : 0][0], qb[QS ? 2 * j : 0][1], bh[0], bh[1]);
+                mma_rows8(z[nt][0], z[nt][1], qb[QS ? 2 * j + 1 : 0][0], qb[QS ? 2 * j + 1 : 0][1], bh[2], bh[3]);
+              }
             }
           }
-#pragma unroll
-          for (int hh = 0; hh < C1::HP; ++hh) {
-            float a0, a1, b0f, b1f;
-            unpack2(za[hh], a0, a1);
-            unpack2(zb[hh], b0f, b1f);
-            zpart[qd][hg * C1::HP + hh][lane] = (a0 + a1) + (b0f + b1f);
-          }
         }
-      }
-      named_barrier(2, kConsumers);
 
-      // ---- phase 2: per (block, head) ----
-      float zl2 = -CUDART_INF_F, sig = 0.f;
-      bool valid = false;
-      if (p2 && !aborted) {
-        valid = p2_bl < nb;
-        float zbar = 0.f;
+        // ---- per (head, block): variance projection, l, running maximum, compensation weight ----
+        float zl2[2][2], sig[2][2], wt[2][2];
+        bool val[2][2];
+        float tmax = -CUDART_INF_F;
 #pragma unroll
-        for (int qd = 0; qd < C1::QD; ++qd) zbar += zpart[qd][p2_g][p2_bl];
-        if (valid) {
-          if (r4) {
-            const float4 dv = *reinterpret_cast<const float4 *>(sd + p2_bl * 4);
-            sig = fmaf(wown[0], dv.x, fmaf(wown[1], dv.y, fmaf(wown[2], dv.z, wown[3] * dv.w)));
-          } else {
-            for (int t = 0; t < P.r; ++t) {
-              const float dv = dbar_bulk ? sd[p2_bl * P.r + t] : __ldg(db + (size_t)(b0 + p2_bl) * P.r + t);
-              sig = fmaf(sw[t][p2_g], dv, sig);
+        for (int nt = 0; nt < 2; ++nt) {
+          const int r0 = rb + nt * 8 + 2 * qd;     // this thread's two blocks of the n-tile: rows r0, r0 + 1
+          float ell[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int r = r0 + e, b = b0 + r;
+            val[nt][e] = hv && r < nb;
+            float sg = 0.f;
+            if (val[nt][e]) {
+              if (r4) {
+                const float4 dv = *reinterpret_cast<const float4 *>(sd + r * 4);
+                sg = fmaf(wown[0], dv.x, fmaf(wown[1], dv.y, fmaf(wown[2], dv.z, wown[3] * dv.w)));
+              } else {
+                for (int t = 0; t < P.r; ++t) {
+                  const float dv = dbar_bulk ? sd[r * P.r + t] : __ldg(db + (size_t)b * P.r + t);
+                  sg = fmaf(sw[t * G + head], dv, sg);
+                }
+              }
             }
+            sig[nt][e] = sg;
+            const float zbar = z[nt][e] * P.scale;
+            const float logc = (b == ui.X - 1) ? log_last : log_bs;
+            ell[e] = logc + zbar + 0.5f * sg;
+            zl2[nt][e] = val[nt][e] ? (zbar + logc) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
+            tmax = fmaxf(tmax, zl2[nt][e]);
           }
-          const int b = b0 + p2_bl;
-          const float logc = (b == ui.X - 1) ? log_last : log_bs;
-          ls[(size_t)p2_g * P.max_blocks + b] = make_float2(logc + zbar + 0.5f * sig, sig);
-          zl2 = (zbar + logc) * kLog2e;   // log2 of the compensation weight |b| e^{zbar}
+          // 8-byte stores: a head's row of (l, sigma^2) pairs starts at head * max_blocks, which may be odd
+          float2 *lrow = ls + (size_t)head * P.max_blocks + b0 + r0;
+          if (val[nt][0]) lrow[0] = make_float2(ell[0], sig[nt][0]);
+          if (val[nt][1]) lrow[1] = make_float2(ell[1], sig[nt][1]);
         }
-        // the running maximum is only raised when the tile's maximum exceeds it by a slack: weights stay below 2^slack
-        const float tm = warp_max(zl2);
-        float sc = 1.f;
-        if (tm > m_ref + CKV_RESCALE_SLACK) {
-          sc = exp2_diff(m_ref, tm);
-          m_ref = tm;
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        if (tmax > m_ref + CKV_RESCALE_SLACK) {   // the running maximum is only raised when exceeded by a slack
+          const float sc = exp2_diff(m_ref, tmax);
+          m_ref = tmax;
           l_acc *= sc; lp_acc *= sc;
+#pragma unroll
+          for (int t = 0; t < 16; ++t) { acc[t][0] *= sc; acc[t][1] *= sc; }
         }
-        if (lane == 0) s_scale[it & 1][p2_g] = make_float2(sc, sc);
-        const float wt = valid ? fast_exp2(zl2 - m_ref) : 0.f;
-        wbuf[it & 1][p2_bl][p2_g] = make_float2(wt, wt);
-        l_acc += wt;
-        lp_acc = fmaf(wt, fast_exp2(0.5f * kLog2e * sig), lp_acc);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
-      }
-      named_barrier(2, kConsumers);
+        uint32_t wh[2], wl[2];   // A fragments of the weights: k = blocks 2 qd + {0, 1} (+ 8), hi and lo halves
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            wt[nt][e] = val[nt][e] ? fast_exp2(zl2[nt][e] - m_ref) : 0.f;
+            l_acc += wt[nt][e];
+            lp_acc = fmaf(wt[nt][e], fast_exp2(0.5f * kLog2e * sig[nt][e]), lp_acc);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
+          }
+          wh[nt] = pack_bf16(wt[nt][0], wt[nt][1]);
+          wl[nt] = pack_bf16(wt[nt][0] - bf16_round(wt[nt][0]), wt[nt][1] - bf16_round(wt[nt][1]));
+        }
 
-      // ---- phase 3: acc_g += w_{g,b} vbar_b, a warp per row, four coordinates per lane ----
-      if (!aborted) {
-        const f32x2 *scp = reinterpret_cast<const f32x2 *>(s_scale[it & 1]);
+        // ---- acc += W Vbar: heads x 128 coordinates, k = this half tile's 16 blocks ----
+        {
+          // ldmatrix.trans lane roles: matrix lane / 8 -> (block half, coordinate chunk parity), row lane % 8
+          const int r = rb + ((lane >> 3) & 1) * 8 + (lane & 7);
+          const uint32_t rowaddr = sv + r * kRowBytes;
+          const int cpar = lane >> 4;
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-          const f32x2 sc2 = scp[g];
-          acc[g][0] = mul2(acc[g][0], sc2);
-          acc[g][1] = mul2(acc[g][1], sc2);
-        }
-#pragma unroll
-        for (int j = 0; j < TB / 8; ++j) {
-          const int bl = warp + 8 * j;
-          if (bl < nb) {   // rows past the unit's last block hold stale bytes
-            const ulonglong2 v2 = *reinterpret_cast<const ulonglong2 *>(sv + bl * CKV_D + 4 * lane);
-            const f32x2 *wp = reinterpret_cast<const f32x2 *>(wbuf[it & 1][bl]);
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-              const f32x2 w2 = wp[g];
-              acc[g][0] = fma2(w2, v2.x, acc[g][0]);
-              acc[g][1] = fma2(w2, v2.y, acc[g][1]);
-            }
+          for (int t2 = 0; t2 < 8; ++t2) {   // two 8-coordinate n-tiles per ldmatrix.x4
+            const uint32_t coff = (uint32_t)swz_chunk(2 * t2 + cpar, r) * 16;
+            uint32_t vh[4], vl[4];
+            ldmatrix_x4_trans(vh, rowaddr + coff);
+            ldmatrix_x4_trans(vl, rowaddr + 256 + coff);
+            mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vh[0], vh[1]);
+            mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wl[0], wl[1], vh[0], vh[1]);
+            mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vl[0], vl[1]);
+            mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vh[2], vh[3]);
+            mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wl[0], wl[1], vh[2], vh[3]);
+            mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vl[2], vl[3]);
           }
         }
       }
-      // the stage is free once every warp has read its rows (the weights are double-buffered, so the next
-      // tile's phase 2 may start while slower warps are still here)
       __syncwarp();
-      if (lane == 0 && !aborted) {
-        mbar_arrive(&empty_bar[st]);
-        if (warp == 0) *(volatile int *)&s_consumed = it + 1;
-      }
-      if (++st == stages) { st = 0; phase ^= 1; }
-      if (++tl == ui.tiles) {
-        tl = 0;
-        do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+      if (lane == 0 && !aborted) mbar_arrive(&empty_bar[st]);
+      for (int k = 0; k < kConsumerWarps / 2 && u < units; ++k) {
+        if (++tl == ui.tiles) {
+          tl = 0;
+          do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+        }
       }
     }
-    if (cur >= 0) flush(cur);
+    if (cur >= 0) { write_partial(cur, true); next_empty = cur + 1; }
+    fill_empty_upto(ulast + 1);
   }
   __syncthreads();
   if (s_abort && tid == 0) {
     // leave no bulk copy in flight into this CTA's shared memory: wait (bounded) for every issued fill
-    for (int it = s_consumed; it < s_issued; ++it) mbar_wait(&full_bar[it % stages], (it / stages) & 1);
+    // (a completed phase is seen as complete again, so waiting on consumed stages returns at once)
+    const int issued = s_issued;
+    for (int it = max(issued - stages, 0); it < issued; ++it) mbar_wait(&full_bar[it % stages], (it / stages) & 1);
   }
 }
 
 struct ScanCfg { int stages; size_t smem; };
 
-template <int G>
-ScanCfg scan_cfg(const CkvDev &P) {
-  using C1 = P1Cfg<G>;
-  const size_t stage_bytes = ((size_t)TB * KROW + (size_t)TB * CKV_D + (P.r >= 4 ? (size_t)TB * P.r : 0)) * 4;
-  const size_t fixed = (size_t)G * CKV_D * 4 + (size_t)CKV_D * G * 4 + (size_t)C1::QD * TB * G * 4 + (size_t)TB * G * 4 +
-                       (size_t)G * CKV_D * 4 + (size_t)kMaxUnits * 4 + 2048;
-  const size_t budget = 224 * 1024 - fixed;
+ScanCfg scan_cfg(const CkvDev &P, int G) {
+  const size_t stage_bytes = (size_t)TB * 2 * kRowBytes + (P.r >= 4 ? (size_t)TB * P.r * 4 : 0);
+  const size_t sw_bytes = P.r == 4 ? 0 : (size_t)kConsumerWarps * P.r * G * 4;
+  const size_t budget = 220 * 1024 - 8 * 1024 - sw_bytes;   // static shared memory stays below 8 KB
   int stages = (int)(budget / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) stages = 2;
-  return ScanCfg{stages, stages * stage_bytes};
+  return ScanCfg{stages, stages * stage_bytes + sw_bytes};
 }
 
 template <int G, typename QT>
 cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, cudaStream_t st) {
-  const ScanCfg cfg = scan_cfg<G>(c->dev);
+  const ScanCfg cfg = scan_cfg(c->dev, G);
   ckv_scan_kernel<G, QT><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
   return cudaGetLastError();
 }
@@ -404,7 +459,7 @@ cudaError_t launch_g(ckv_ctx *c, const void *q, const int *seq_lens, int units, 
 template <int G, typename QT>
 cudaError_t configure_gt(const ckv_ctx *c) {
   return cudaFuncSetAttribute(ckv_scan_kernel<G, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)scan_cfg<G>(c->dev).smem);
+                              (int)scan_cfg(c->dev, G).smem);
 }
 
 template <int G>

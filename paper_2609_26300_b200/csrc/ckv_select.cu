@@ -77,13 +77,14 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   }
   __syncthreads();
   if (warp < G) {
-    const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * G + warp) * CKV_PART_STRIDE;
+    const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * CKV_SCAN_WARPS * G + warp) * CKV_PART_STRIDE;
     const size_t step = (size_t)G * CKV_PART_STRIDE;
+    const int n_part = s_ccount * CKV_SCAN_WARPS;
     float m = -CUDART_INF_F;
-    for (int i = lane; i < s_ccount; i += 32) m = fmaxf(m, cp[i * step]);
+    for (int i = lane; i < n_part; i += 32) m = fmaxf(m, cp[i * step]);
     m = warp_max(m);
     float l = 0.f;
-    for (int i = lane; i < s_ccount; i += 32) l = fmaf(cp[i * step + 2], exp2_diff(cp[i * step], m), l);
+    for (int i = lane; i < n_part; i += 32) l = fmaf(cp[i * step + 2], exp2_diff(cp[i * step], m), l);
     l = warp_sum(l);
     if (lane == 0) { s_M[warp] = m; s_invL[warp] = 1.0f / l; }
   }

@@ -12,8 +12,8 @@ namespace {
 template <typename T, bool NC>
 __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__restrict__ k_pool,
                                                  const T *__restrict__ v_pool, const int *__restrict__ pt_row,
-                                                 int h, int b, int cnt, float *sq_smem, float *kmean_row,
-                                                 float *dbar_row, float *vmean_row, int lane) {
+                                                 int h, int b, int cnt, float *sq_smem, __nv_bfloat16 *kmean_row,
+                                                 float *dbar_row, __nv_bfloat16 *vmean_row, int lane) {
   const int hw = lane >> 4, li = lane & 15;
   float ks[8], vs[8];
 #pragma unroll
@@ -65,15 +65,14 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
 #pragma unroll
   for (int i = 0; i < 8; ++i) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], 16);
   if (hw == 0) {
-    float4 *dst = reinterpret_cast<float4 *>(kmean_row + 8 * li);
-    dst[0] = make_float4(km[0], km[1], km[2], km[3]);
-    dst[1] = make_float4(km[4], km[5], km[6], km[7]);
+    store_split8(kmean_row, li, b, km);
 #pragma unroll
     for (int i = 0; i < 8; ++i) sq_smem[8 * li + i] = sq[i];
   } else {
-    float4 *dst = reinterpret_cast<float4 *>(vmean_row + 8 * li);
-    dst[0] = make_float4(vs[0] / fc, vs[1] / fc, vs[2] / fc, vs[3] / fc);
-    dst[1] = make_float4(vs[4] / fc, vs[5] / fc, vs[6] / fc, vs[7] / fc);
+    float vm[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) vm[i] = vs[i] / fc;
+    store_split8(vmean_row, li, b, vm);
   }
   __syncwarp();
   // grouped variance: average of the per-coordinate population variances of each group (Eq. 8)
@@ -110,7 +109,8 @@ __global__ void __launch_bounds__(256) ckv_stats_build_kernel(CkvDev P, const T 
   const int cnt = min(P.bs, N - b * P.bs);
   const size_t row = (size_t)unit * P.max_blocks + b;
   block_stats_warp<T, true>(P, k_pool, v_pool, page_table + (size_t)s * P.max_pages_per_seq, h, b, cnt,
-                            sq_smem[warp], P.kmean + row * CKV_D, P.dbar + row * P.r, P.vmean + row * CKV_D, lane);
+                            sq_smem[warp], P.kmean + row * CKV_ROW_ELEMS, P.dbar + row * P.r,
+                            P.vmean + row * CKV_ROW_ELEMS, lane);
 }
 
 // One CTA per sequence, one warp per KV head (looping when there are more heads than warps).
@@ -143,14 +143,36 @@ __global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T 
     }
     __syncwarp();
     const size_t row = ((size_t)s * P.Hkv + h) * P.max_blocks + b;
-    block_stats_warp<T, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * CKV_D,
-                               P.dbar + row * P.r, P.vmean + row * CKV_D, lane);
+    block_stats_warp<T, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * CKV_ROW_ELEMS,
+                               P.dbar + row * P.r, P.vmean + row * CKV_ROW_ELEMS, lane);
   }
   __syncthreads();
   if (threadIdx.x == 0) seq_lens[s] = N + 1;
 }
 
+// Summaries as plain fp32 arrays (hi + lo, chunks back in coordinate order): one warp per block row.
+__global__ void __launch_bounds__(256) ckv_stats_export_kernel(CkvDev P, int rows, float *__restrict__ kmean,
+                                                               float *__restrict__ dbar, float *__restrict__ vmean) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const int b = row % P.max_blocks, hw = lane >> 4, li = lane & 15;
+  float x[8];
+  load_split8((hw == 0 ? P.kmean : P.vmean) + (size_t)row * CKV_ROW_ELEMS, li, b, x);
+  float *dst = (hw == 0 ? kmean : vmean) + (size_t)row * CKV_D + 8 * li;
+  reinterpret_cast<float4 *>(dst)[0] = make_float4(x[0], x[1], x[2], x[3]);
+  reinterpret_cast<float4 *>(dst)[1] = make_float4(x[4], x[5], x[6], x[7]);
+  for (int t = lane; t < P.r; t += 32) dbar[(size_t)row * P.r + t] = P.dbar[(size_t)row * P.r + t];
+}
+
 }  // namespace
+
+cudaError_t ckv_launch_stats_export(ckv_ctx *c, int batch, float *kmean, float *dbar, float *vmean, cudaStream_t st) {
+  const CkvDev &P = c->dev;
+  const int rows = batch * P.Hkv * P.max_blocks;
+  ckv_stats_export_kernel<<<(rows + 7) / 8, 256, 0, st>>>(P, rows, kmean, dbar, vmean);
+  c->launches++;
+  return cudaGetLastError();
+}
 
 cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int *page_table,
                                    const int *seq_lens, int batch, int max_len, cudaStream_t st) {

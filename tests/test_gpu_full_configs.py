@@ -24,7 +24,7 @@ def test_config2_llama_32k():
     torch.cuda.synchronize()
     assert d.ckv.read_status() == 0
     assert cnt.cpu().tolist() == [[64] * 8]
-    km, db, vm = d.ckv.stats_views()
+    km, db, vm = d.ckv.export_stats()
     G = w.group
     for h in (0, 3, 7):
         check_unit_decode(d, 0, h, w.ctx, 0, w.budget_tokens, out, lse, ids, cnt, scores)
@@ -57,7 +57,7 @@ def test_config3_llama_128k_batch4_64_decode_steps():
     assert d.ckv.read_status() == 0
     assert d.lens.cpu().tolist() == [n0 + 64] * 4
     # summaries after 64 appends equal the oracle's over the longer cache
-    km, db, vm = d.ckv.stats_views()
+    km, db, vm = d.ckv.export_stats()
     for s, h in sample:
         _, K, V = unit_inputs(w, s, h, n0 + 64)
         check_stats(O.stats(K, V, 16), km[s, h], db[s, h], vm[s, h], K, V)
@@ -90,7 +90,7 @@ def test_config5_sweep_128k(bs):
     torch.cuda.synchronize()
     h = 2
     q, K, V = unit_inputs(w, 0, h, w.ctx)
-    km, db, vm = d.ckv.stats_views()
+    km, db, vm = d.ckv.export_stats()
     check_stats(O.stats(K, V, bs), km[0, h], db[0, h], vm[0, h], K, V)
     for budget in synth.SWEEP_BUDGETS:
         out, lse, ids, cnt = d.ckv.decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len, budget)

@@ -45,7 +45,7 @@ def test_stats_build(bs, r, layout, dtype):
     d = setup(w, dtype, var_groups=r, group_layout=layout)
     d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
     torch.cuda.synchronize()
-    km, db, vm = d.ckv.stats_views()
+    km, db, vm = d.ckv.export_stats()
     lens = d.lens.cpu().numpy()
     for s, h in all_units(w):
         _, K, V = unit_inputs(w, s, h, int(lens[s]))
@@ -67,11 +67,11 @@ def test_append_equals_rebuild_bit_for_bit(bs):
                      torch.from_numpy(k_new).to(d.dtype).cuda(), torch.from_numpy(v_new).to(d.dtype).cuda())
     torch.cuda.synchronize()
     assert d.lens.cpu().tolist() == [n0 + steps] * w.batch
-    km, db, vm = (t.clone() for t in d.ckv.stats_views())
+    km, db, vm = (t.clone() for t in d.ckv.export_stats())
     # the appended rows are now in the cache: a fresh build over the longer cache must agree exactly
     d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, n0 + steps)
     torch.cuda.synchronize()
-    km2, db2, vm2 = d.ckv.stats_views()
+    km2, db2, vm2 = d.ckv.export_stats()
     x = -(-(n0 + steps) // bs)
     assert torch.equal(km[:, :, :x], km2[:, :, :x]) and torch.equal(db[:, :, :x], db2[:, :, :x])
     assert torch.equal(vm[:, :, :x], vm2[:, :, :x])
