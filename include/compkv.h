@@ -66,7 +66,8 @@ enum ckv_device_status {
   CKV_DEV_BAD_PAGE = 1,     /* page table entry outside [0, num_pages): the page was skipped */
   CKV_DEV_SEQ_FULL = 2,     /* append past max_blocks_per_seq * block_size: the token was dropped */
   CKV_DEV_NONFINITE = 4,    /* a block score was NaN/Inf: it was ranked as 0 */
-  CKV_DEV_TIMEOUT = 8       /* a bounded wait inside a kernel ran out: the step's results are invalid */
+  CKV_DEV_TIMEOUT = 8,      /* a bounded wait inside a kernel ran out: the step's results are invalid */
+  CKV_DEV_BAD_COPY = 16     /* a kernel refused to issue a bulk copy whose arguments failed its checks */
 };
 
 typedef struct ckv_layout {

@@ -19,7 +19,7 @@ CKV_BF16, CKV_F32 = 0, 1
 CKV_OK = 0
 CKV_ERR_INVALID_ARG, CKV_ERR_BAD_LAYOUT, CKV_ERR_BUDGET_TOO_SMALL = -1, -2, -3
 CKV_ERR_CAPACITY, CKV_ERR_CUDA, CKV_ERR_TIMEOUT = -4, -5, -6
-CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE = 1, 2, 4
+CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_BAD_COPY = 1, 2, 4, 8, 16
 
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
            "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_decode_profile", "ckv_dense_decode",

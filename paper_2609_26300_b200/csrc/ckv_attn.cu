@@ -98,8 +98,10 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
       const size_t src = ((size_t)phys * P.Hkv + h) * kPageElems;
       T *dst = wbuf + (size_t)b * 2 * kPageElems;
       mbar_arrive_expect_tx(&wbar[b], 2 * bytes);
-      bulk_g2s(dst, k_pool + src, bytes, &wbar[b]);
-      bulk_g2s(dst + kPageElems, v_pool + src, bytes, &wbar[b]);
+      const uint32_t lo = smem_u32(pg_mem), hi = lo + (uint32_t)(8 * nbuf * 2 * kPageElems * sizeof(T));
+      bool ok = bulk_g2s_checked(dst, k_pool + src, bytes, &wbar[b], lo, hi);
+      ok = ok && bulk_g2s_checked(dst + kPageElems, v_pool + src, bytes, &wbar[b], lo, hi);
+      if (!ok) atomicOr(P.status, CKV_DEV_BAD_COPY);
     }
   };
   int issued = 0;

@@ -13,7 +13,7 @@
 #define CKV_ROW_ELEMS 256     // bf16 elements of one mean-key / mean-value summary row (128 hi halves + 128 lo halves)
 #define CKV_PART_STRIDE 132   // floats per split partial: m, l, pad, pad, acc[128]
 #define CKV_SCAN_TILE 32      // blocks per scan tile
-#define CKV_SCAN_WARPS 8       // consumer warps of a scan CTA, each with a partial of its own
+#define CKV_SCAN_WARPS 7       // consumer warps of a scan CTA (plus one producer warp: 256 threads), each with a partial of its own
 #define CKV_MAX_SCAN_CTAS 160 // persistent scan grid is capped at this many CTAs
 #define CKV_MAX_SPLITS 64     // attention partials per unit
 #define CKV_RESCALE_SLACK 16.0f  // log2 units: running maxima are only raised when exceeded by this much

@@ -51,6 +51,17 @@ __device__ __forceinline__ void bulk_g2s(void *dst_smem, const void *src_gmem, u
                "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
+// bulk_g2s with its arguments checked first: a copy that is misaligned, empty or would leave the window
+// [smem_lo, smem_hi) is not issued and the function returns false (the caller records the fault; the
+// barrier then never completes and the bounded waits on it run out).
+__device__ __forceinline__ bool bulk_g2s_checked(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar,
+                                                 uint32_t smem_lo, uint32_t smem_hi) {
+  const uint32_t d = smem_u32(dst_smem);
+  const bool ok = bytes != 0 && (bytes & 15u) == 0 && (d & 15u) == 0 && ((unsigned long long)src_gmem & 15ull) == 0 &&
+                  d >= smem_lo && d + bytes <= smem_hi;
+  if (ok) bulk_g2s(dst_smem, src_gmem, bytes, bar);
+  return ok;
+}
 // Orders this thread's earlier generic-proxy accesses to shared memory before later async-proxy
 // (bulk copy) accesses to it.
 __device__ __forceinline__ void fence_proxy_async() {

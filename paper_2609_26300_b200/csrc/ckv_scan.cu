@@ -21,10 +21,10 @@
 // (unit, position) order, are split into one contiguous range per CTA and the grid is one CTA per
 // SM.  A producer thread streams the CTA's tiles into a ring of shared-memory stages with
 // cp.async.bulk (two 16 KB copies and the variances per tile), completion on mbarriers.  Each of the
-// eight consumer warps takes every eighth half tile (16 blocks) on its own -- there is no CTA-wide
+// seven consumer warps takes every seventh half tile (16 blocks) on its own -- there is no CTA-wide
 // barrier in the loop -- with a per-warp running maximum that is only raised when exceeded by a
 // slack.  A warp writes one partial per unit its CTA touched; partial (CTA c, warp w, unit u) lives
-// in entry (c + u) * 8 + w, unique because the (c, u) pairs that occur form a monotone staircase.
+// in entry (c + u) * 7 + w, unique because the (c, u) pairs that occur form a monotone staircase.
 #include "ckv_internal.cuh"
 #include "ckv_pipe.cuh"
 
@@ -135,7 +135,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
       }
     }
     s_u0 = u0; s_tl0 = tl0; s_ulast = ulast; s_count = (int)cnt; s_abort = 0; s_issued = 0;
-    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], 2); }
+    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], kConsumerWarps); }
     fence_barrier_init();
   }
   __syncthreads();
@@ -162,9 +162,12 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         const uint32_t kbytes = (uint32_t)nb * kRowBytes;
         const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
         mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
-        bulk_g2s(sk, P.kmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st]);
-        bulk_g2s(sv, P.vmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st]);
-        if (dbar_bulk) bulk_g2s(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, &full_bar[st]);
+        const uint32_t lo = smem_u32(stage_mem), hi = lo + (uint32_t)stages * stage_bytes;
+        bool ok = nb >= 1 && u < units && row + nb <= (size_t)units * P.max_blocks;
+        ok = ok && bulk_g2s_checked(sk, P.kmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st], lo, hi);
+        ok = ok && bulk_g2s_checked(sv, P.vmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st], lo, hi);
+        if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, &full_bar[st], lo, hi);
+        if (!ok) atomicOr(P.status, CKV_DEV_BAD_COPY);
         *(volatile int *)&s_issued = it + 1;
         if (++st == stages) { st = 0; if (it >= stages) phase ^= 1; }
         if (++tl == ui.tiles) {
@@ -219,16 +222,30 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         if (unit_info(P, seq_lens, next_empty).tiles > 0) write_partial(next_empty, false);
     };
 
-    // advance the walk to this warp's first tile
-    int it = warp >> 1;
-    const int half = warp & 1;
-    for (int k = 0; k < it && k < count; ++k) {
-      if (++tl == ui.tiles) {
+    // Half tile j = 2 * tile + half belongs to warp j % W.  A parity wait can only tell a fill of a stage from
+    // the one before it, so every warp passes over ALL tiles in order -- waits for the tile's data, works on it
+    // if one of its halves is this warp's, then releases it -- and a stage is refilled only after all W warps
+    // have released it: no warp is ever more than one fill away from a barrier it waits on.
+    int st = 0;
+    uint32_t phase = 0;              // parity of the full-barrier phase of stage `st` this pass over the ring
+    for (int it = 0; it < count; ++it) {
+      if (it > 0 && ++tl == ui.tiles) {
         tl = 0;
         do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
       }
-    }
-    for (; it < count; it += kConsumerWarps / 2) {
+      const int j0 = (2 * it) % kConsumerWarps;
+      const int half = j0 == warp ? 0 : ((j0 + 1) % kConsumerWarps == warp ? 1 : -1);
+      // a wait that runs out marks the step invalid (`aborted`); the walk still runs to the end
+      if (!aborted) {
+        bool fail = *(volatile int *)&s_abort != 0;
+        if (!fail && !mbar_wait(&full_bar[st], phase)) {
+          atomicOr(P.status, CKV_DEV_TIMEOUT);
+          *(volatile int *)&s_abort = 1;
+          fail = true;
+        }
+        aborted = __any_sync(0xffffffffu, fail);
+      }
+      if (half >= 0) {
       if (u != cur) {
         if (cur >= 0) { write_partial(cur, true); next_empty = cur + 1; }
         fill_empty_upto(u);
@@ -284,18 +301,6 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         db = P.dbar + row0 * P.r;
         cur = u;
       }
-      const int st = it % stages;
-      const uint32_t phase = (uint32_t)(it / stages) & 1u;
-      // a wait that runs out marks the step invalid; the walk still runs to the end
-      if (!aborted) {
-        bool fail = *(volatile int *)&s_abort != 0;
-        if (!fail && !mbar_wait(&full_bar[st], phase)) {
-          atomicOr(P.status, CKV_DEV_TIMEOUT);
-          *(volatile int *)&s_abort = 1;
-          fail = true;
-        }
-        aborted = __any_sync(0xffffffffu, fail);
-      }
       const int b0 = tl * TB;
       const int nb = min(TB, ui.X - b0);
       const int rb = half * 16;          // first row of this warp's half tile
@@ -305,7 +310,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         const float *sd = reinterpret_cast<const float *>(stage_mem + (size_t)st * stage_bytes + 2 * TB * kRowBytes);
 
         // ---- Z^T = Q Kbar^T: heads x 16 blocks (two n-tiles of 8 blocks), hi and lo planes into one accumulator ----
-        float z[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        float z[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, zlo[2][2] = {{0.f, 0.f}, {0.f, 0.f}};   // two chains per n-tile
         {
           // ldmatrix lane roles: matrix lane / 8 -> 8-coordinate chunk, row lane % 8
           const int lrow = lane & 7, lmat = lane >> 3;
@@ -321,13 +326,14 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
               ldmatrix_x4(bl, rowaddr + 256 + coff);
               mma_rows8(z[nt][0], z[nt][1], qa[2 * j][0], qa[2 * j][1], bh[0], bh[1]);
               mma_rows8(z[nt][0], z[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bh[2], bh[3]);
-              mma_rows8(z[nt][0], z[nt][1], qa[2 * j][0], qa[2 * j][1], bl[0], bl[1]);
-              mma_rows8(z[nt][0], z[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bl[2], bl[3]);
+              mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j][0], qa[2 * j][1], bl[0], bl[1]);
+              mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bl[2], bl[3]);
               if (QS) {
-                mma_rows8(z[nt][0], z[nt][1], qb[QS ? 2 * j : 0][0], qb[QS ? 2 * j : 0][1], bh[0], bh[1]);
-                mma_rows8(z[nt][0], z[nt][1], qb[QS ? 2 * j + 1 : 0][0], qb[QS ? 2 * j + 1 : 0][1], bh[2], bh[3]);
+                mma_rows8(zlo[nt][0], zlo[nt][1], qb[QS ? 2 * j : 0][0], qb[QS ? 2 * j : 0][1], bh[0], bh[1]);
+                mma_rows8(zlo[nt][0], zlo[nt][1], qb[QS ? 2 * j + 1 : 0][0], qb[QS ? 2 * j + 1 : 0][1], bh[2], bh[3]);
               }
             }
+            z[nt][0] += zlo[nt][0]; z[nt][1] += zlo[nt][1];
           }
         }
 
@@ -410,14 +416,10 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
           }
         }
       }
+      }   // own half tile
       __syncwarp();
       if (lane == 0 && !aborted) mbar_arrive(&empty_bar[st]);
-      for (int k = 0; k < kConsumerWarps / 2 && u < units; ++k) {
-        if (++tl == ui.tiles) {
-          tl = 0;
-          do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
-        }
-      }
+      if (++st == stages) { st = 0; phase ^= 1; }
     }
     if (cur >= 0) { write_partial(cur, true); next_empty = cur + 1; }
     fill_empty_upto(ulast + 1);
