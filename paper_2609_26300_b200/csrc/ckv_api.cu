@@ -153,6 +153,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   cudaError_t e = ckv_configure_kernels();
   if (e == cudaSuccess) e = ckv_configure_scan(c);
   if (e == cudaSuccess) e = ckv_configure_attn(c);
+  if (e == cudaSuccess) e = ckv_configure_attn_mma(c);
   int dev_id = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev_id);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev_id);

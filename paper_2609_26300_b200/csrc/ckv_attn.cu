@@ -311,25 +311,29 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
 // c in [c_first, c_last], recomputed here from the same tile arithmetic the scan uses).
 constexpr int kMergeMax = CKV_MAX_SPLITS + CKV_MAX_SCAN_CTAS * CKV_SCAN_WARPS;
 
+constexpr int kMergeGroups = 4;   // thread groups of CKV_D threads, each summing every fourth partial
+
 template <typename T>
-__global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *__restrict__ seq_lens,
-                                                          const int *__restrict__ sel_cnt, int n_splits,
-                                                          int scan_grid, int units, bool dense, T *__restrict__ out,
-                                                          float *__restrict__ lse) {
+__global__ void __launch_bounds__(CKV_D *kMergeGroups) ckv_merge_kernel(CkvDev P, const int *__restrict__ seq_lens,
+                                                                        const int *__restrict__ sel_cnt, int n_splits,
+                                                                        int scan_grid, int units, bool dense,
+                                                                        T *__restrict__ out, float *__restrict__ lse) {
+  constexpr int NT = CKV_D * kMergeGroups;
   __shared__ float s_scale[kMergeMax];
   __shared__ float s_l[kMergeMax];
   __shared__ const float *s_ptr[kMergeMax];
-  __shared__ float s_wmax[CKV_D / 32];
+  __shared__ float s_wmax[NT / 32];
+  __shared__ float s_num[kMergeGroups][CKV_D], s_den[kMergeGroups];
   __shared__ int s_cfirst, s_ccount;
-  const int hq = blockIdx.x, s = blockIdx.y, c = threadIdx.x;
+  const int hq = blockIdx.x, s = blockIdx.y, tid = threadIdx.x, c = tid % CKV_D, grp = tid / CKV_D;
   const int G = P.G, unit = s * P.Hkv + hq / G, g = hq % G;
   const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
   const int X = (N + P.bs - 1) / P.bs;
   const bool comp = !dense && sel_cnt[unit] < X;
-  if (c < 32) {
+  if (tid < 32) {
     int cfirst = 0, ccount = 0;
-    if (comp) unit_scan_slots(P, seq_lens, units, unit, scan_grid, c, cfirst, ccount);
-    if (c == 0) { s_cfirst = cfirst; s_ccount = ccount; }
+    if (comp) unit_scan_slots(P, seq_lens, units, unit, scan_grid, tid, cfirst, ccount);
+    if (tid == 0) { s_cfirst = cfirst; s_ccount = ccount; }
   }
   __syncthreads();
   const int n_comp = s_ccount * CKV_SCAN_WARPS;
@@ -338,36 +342,47 @@ __global__ void __launch_bounds__(CKV_D) ckv_merge_kernel(CkvDev P, const int *_
   const float *ap = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS * G + g) * CKV_PART_STRIDE;
   const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * CKV_SCAN_WARPS * G + g) * CKV_PART_STRIDE;
   float mloc = -CUDART_INF_F;
-  for (int i = c; i < n; i += CKV_D) {
+  for (int i = tid; i < n; i += NT) {
     const float *p = i < n_splits ? ap + (size_t)i * step : cp + (size_t)(i - n_splits) * step;
     const float m = p[0];
     s_ptr[i] = p; s_scale[i] = m; s_l[i] = p[1];
     mloc = fmaxf(mloc, m);
   }
   mloc = warp_max(mloc);
-  if ((c & 31) == 0) s_wmax[c >> 5] = mloc;
+  if ((tid & 31) == 0) s_wmax[tid >> 5] = mloc;
   __syncthreads();
   float M = s_wmax[0];
 #pragma unroll
-  for (int w = 1; w < CKV_D / 32; ++w) M = fmaxf(M, s_wmax[w]);
-  for (int i = c; i < n; i += CKV_D) s_scale[i] = exp2_diff(s_scale[i], M);
+  for (int w = 1; w < NT / 32; ++w) M = fmaxf(M, s_wmax[w]);
+  for (int i = tid; i < n; i += NT) s_scale[i] = exp2_diff(s_scale[i], M);
   __syncthreads();
+  // group grp sums partials grp, grp + 4, ...; four loads in flight per thread; empty partials are skipped
   float num = 0.f, den = 0.f;
-  int i = 0;
-  for (; i + 4 <= n; i += 4) {   // four independent loads in flight
-    const float a0 = s_ptr[i][4 + c], a1 = s_ptr[i + 1][4 + c], a2 = s_ptr[i + 2][4 + c], a3 = s_ptr[i + 3][4 + c];
-    num = fmaf(a0, s_scale[i], num); num = fmaf(a1, s_scale[i + 1], num);
-    num = fmaf(a2, s_scale[i + 2], num); num = fmaf(a3, s_scale[i + 3], num);
-    den = fmaf(s_l[i], s_scale[i], den); den = fmaf(s_l[i + 1], s_scale[i + 1], den);
-    den = fmaf(s_l[i + 2], s_scale[i + 2], den); den = fmaf(s_l[i + 3], s_scale[i + 3], den);
+  for (int i = grp; i < n; i += 4 * kMergeGroups) {
+    float a[4], sc[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int ii = i + k * kMergeGroups;
+      sc[k] = ii < n ? s_scale[ii] : 0.f;
+      a[k] = sc[k] != 0.f ? s_ptr[ii][4 + c] : 0.f;
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int ii = i + k * kMergeGroups;
+      num = fmaf(a[k], sc[k], num);
+      if (ii < n) den = fmaf(s_l[ii], sc[k], den);
+    }
   }
-  for (; i < n; ++i) {
-    if (s_scale[i] != 0.f) num = fmaf(s_ptr[i][4 + c], s_scale[i], num);
-    den = fmaf(s_l[i], s_scale[i], den);
+  s_num[grp][c] = num;
+  if (c == 0) s_den[grp] = den;
+  __syncthreads();
+  if (grp == 0) {
+#pragma unroll
+    for (int k = 1; k < kMergeGroups; ++k) { num += s_num[k][c]; den += s_den[k]; }
+    const size_t o = ((size_t)s * P.Hq + hq) * CKV_D + c;
+    store_out(out + o, N > 0 ? num / den : 0.f);
+    if (lse != nullptr && c == 0) lse[(size_t)s * P.Hq + hq] = N > 0 ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
   }
-  const size_t o = ((size_t)s * P.Hq + hq) * CKV_D + c;
-  store_out(out + o, N > 0 ? num / den : 0.f);
-  if (lse != nullptr && c == 0) lse[(size_t)s * P.Hq + hq] = N > 0 ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
 }
 
 // Static shared memory of the attention kernel (query tile, probability tile, warp partials, barriers).
@@ -455,6 +470,8 @@ cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k
   *n_splits_out = n_splits;
   dim3 grid(n_splits, units);
   c->launches++;
+  if (c->layout.kv_dtype == CKV_BF16)   // bf16 pages go through the tensor-core kernel
+    return ckv_launch_attn_mma(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
   switch (P.G) {
     case 1: return launch_g<1>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
     case 2: return launch_g<2>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
@@ -470,10 +487,10 @@ cudaError_t ckv_launch_merge(ckv_ctx *c, bool dense, const int *seq_lens, const 
   dim3 grid(P.Hq, batch);
   const int units = batch * P.Hkv;
   if (c->layout.kv_dtype == CKV_BF16)
-    ckv_merge_kernel<__nv_bfloat16><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, n_splits, scan_grid, units, dense,
+    ckv_merge_kernel<__nv_bfloat16><<<grid, CKV_D * kMergeGroups, 0, st>>>(P, seq_lens, sel_cnt, n_splits, scan_grid, units, dense,
                                                            (__nv_bfloat16 *)out, lse);
   else
-    ckv_merge_kernel<float><<<grid, CKV_D, 0, st>>>(P, seq_lens, sel_cnt, n_splits, scan_grid, units, dense,
+    ckv_merge_kernel<float><<<grid, CKV_D * kMergeGroups, 0, st>>>(P, seq_lens, sel_cnt, n_splits, scan_grid, units, dense,
                                                     (float *)out, lse);
   c->launches++;
   return cudaGetLastError();

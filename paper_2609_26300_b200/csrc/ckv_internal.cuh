@@ -51,6 +51,10 @@ struct ckv_ctx {
 cudaError_t ckv_configure_kernels();   // selection kernel attributes
 cudaError_t ckv_configure_scan(const ckv_ctx *c);   // scan kernel attributes
 cudaError_t ckv_configure_attn(const ckv_ctx *c);   // attention kernel attributes
+cudaError_t ckv_configure_attn_mma(const ckv_ctx *c);
+cudaError_t ckv_launch_attn_mma(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
+                                const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
+                                int kcap, dim3 grid, int pps, cudaStream_t st);
 int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len);
 
 // ---- launchers (one per translation unit) ---------------------------------------------------------
