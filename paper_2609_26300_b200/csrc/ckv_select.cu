@@ -54,7 +54,8 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   __shared__ int s_hist[kBins];
   __shared__ float s_M[G], s_invL[G];
   __shared__ int s_wtot[32];
-  __shared__ int s_total, s_digit, s_remaining, s_cfirst, s_ccount;
+  __shared__ int s_total, s_digit, s_remaining, s_cfirst, s_ccount, s_ncand;
+  __shared__ int s_cand[kThreads];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = blockIdx.x, s = unit / P.Hkv;
@@ -69,48 +70,63 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
     // scores are still produced below for callers that read them
   }
 
-  // ---- normalisers of Eq. 9 from the scan partials of this unit (entries c + unit, c in [cfirst, cfirst + ccount)) ----
+  // ---- where the scan partials of this unit live (entries (c + unit) * W + w, c in [cfirst, cfirst + ccount)) ----
   if (warp == 0) {
     int cfirst, ccount;
     unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
-    if (lane == 0) { s_cfirst = cfirst; s_ccount = ccount; }
+    if (lane == 0) { s_cfirst = cfirst; s_ccount = ccount; s_ncand = 0; }
   }
-  __syncthreads();
-  if (warp < G) {
-    const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * CKV_SCAN_WARPS * G + warp) * CKV_PART_STRIDE;
-    const size_t step = (size_t)G * CKV_PART_STRIDE;
-    const int n_part = s_ccount * CKV_SCAN_WARPS;
-    float m = -CUDART_INF_F;
-    for (int i = lane; i < n_part; i += 32) m = fmaxf(m, cp[i * step]);
-    m = warp_max(m);
-    float l = 0.f;
-    for (int i = lane; i < n_part; i += 32) l = fmaf(cp[i * step + 2], exp2_diff(cp[i * step], m), l);
-    l = warp_sum(l);
-    if (lane == 0) { s_M[warp] = m; s_invL[warp] = 1.0f / l; }
-  }
-  __syncthreads();
-
-  // ---- S_b ----
+  // the first batch of (l, sigma^2) loads does not depend on the normalisers: start it before waiting for them
+  constexpr int NB = G >= 8 ? 2 : 4;   // blocks per thread and batch (their loads are in flight together)
   const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
   float *scores = P.scores + (size_t)unit * P.max_blocks;
-  float Mg[G], iL[G];
+  float2 v[NB][G];
+  auto load_batch = [&](int base) {
 #pragma unroll
-  for (int g = 0; g < G; ++g) { Mg[g] = s_M[g]; iL[g] = s_invL[g]; }
-  const bool cached = X <= kSmemKeys;
-  bool nonfinite = false;
-  // four blocks per thread at a time, so that their loads are in flight together
-  for (int base = 0; base < X; base += 4 * kThreads) {
-    float2 v[4][G];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < NB; ++j) {
       const int b = base + j * kThreads + tid;
       if (b < X) {
 #pragma unroll
         for (int g = 0; g < G; ++g) v[j][g] = ls[(size_t)g * P.max_blocks + b];   // head-major: coalesced per head
       }
     }
+  };
+  load_batch(0);
+  __syncthreads();
+  // ---- normalisers of Eq. 9: M_g, L_g from the partials (one round of loads for up to 128 partials) ----
+  if (warp < G) {
+    const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * CKV_SCAN_WARPS * G + warp) * CKV_PART_STRIDE;
+    const size_t step = (size_t)G * CKV_PART_STRIDE;
+    const int n_part = s_ccount * CKV_SCAN_WARPS;
+    float pm[4], pl[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int k = 0; k < 4; ++k) {
+      const int i = lane + 32 * k;
+      pm[k] = i < n_part ? cp[i * step] : -CUDART_INF_F;
+      pl[k] = i < n_part ? cp[i * step + 2] : 0.f;
+    }
+    float m = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
+    for (int i = lane + 128; i < n_part; i += 32) m = fmaxf(m, cp[i * step]);
+    m = warp_max(m);
+    float l = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) l = fmaf(pl[k], exp2_diff(pm[k], m), l);
+    for (int i = lane + 128; i < n_part; i += 32) l = fmaf(cp[i * step + 2], exp2_diff(cp[i * step], m), l);
+    l = warp_sum(l);
+    if (lane == 0) { s_M[warp] = m; s_invL[warp] = 1.0f / l; }
+  }
+  __syncthreads();
+
+  // ---- S_b ----
+  float Mg[G], iL[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) { Mg[g] = s_M[g]; iL[g] = s_invL[g]; }
+  const bool cached = X <= kSmemKeys;
+  bool nonfinite = false;
+  for (int base = 0; base < X; base += NB * kThreads) {
+    if (base > 0) load_batch(base);
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
       const int b = base + j * kThreads + tid;
       if (b < X) {
         float sc = 0.f;
@@ -133,11 +149,13 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   if (P.sink + n_tail > X) nF = X;
   const int Kr = K - nF;   // blocks to rank in (the host guarantees K >= sink + recent when K < X)
 
-  // ---- radix select of the Kr-th largest ranked score ----
+  // ---- the Kr-th largest ranked score: one 12-bit radix pass, then either a direct ranking of the blocks in the
+  //      digit bin that holds it (the usual case: a few dozen blocks) or the remaining radix passes ----
   uint32_t prefix = 0, pmask = 0;
   if (tid == 0) { s_remaining = Kr; s_total = 0; }
   __syncthreads();
-  int eq_total = 0;   // blocks scoring exactly the threshold
+  int eq_total = 0;   // blocks scoring exactly the threshold (radix path)
+  bool ranked = false;   // direct-ranking path taken: chosen blocks carry the sign bit in skeys
   if (Kr > 0) {
 #pragma unroll 1
     for (int pass = 0; pass < 3; ++pass) {
@@ -178,58 +196,74 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
       prefix |= (uint32_t)s_digit << shift;
       pmask |= (uint32_t)(bins - 1) << shift;
       eq_total = s_total;
+      const int take = s_remaining;
       __syncthreads();
+      if (pass == 0 && cached && eq_total <= kThreads) {
+        // rank the bin's blocks by (score descending, id ascending) and mark the first `take`
+        for (int b = tid; b < X; b += kThreads) {
+          if (mandatory(b)) continue;
+          if ((keys[b] & pmask) == prefix) s_cand[atomicAdd(&s_ncand, 1)] = b;
+        }
+        __syncthreads();
+        const int nc = s_ncand;
+        bool chosen = false;
+        int myb = -1;
+        if (tid < nc) {
+          myb = s_cand[tid];
+          const uint32_t mk = keys[myb];
+          int rank = 0;
+          for (int j = 0; j < nc; ++j) {
+            const int ob = s_cand[j];
+            const uint32_t ok = keys[ob];
+            rank += (ok > mk || (ok == mk && ob < myb)) ? 1 : 0;
+          }
+          chosen = rank < take;
+        }
+        __syncthreads();   // every rank is computed before any key is marked
+        if (chosen) skeys[myb] |= 0x80000000u;
+        __syncthreads();
+        ranked = true;
+        break;
+      }
     }
   }
-  const uint32_t thr = prefix;          // bit pattern of the Kr-th largest ranked score
-  const int need_eq = s_remaining;      // how many blocks scoring exactly thr are taken (lowest ids first)
+  const uint32_t thr = prefix;          // radix path: bit pattern of the Kr-th largest ranked score
+  const int need_eq = s_remaining;      // ... and how many blocks scoring exactly thr are taken (lowest ids first)
+  const uint32_t digit0 = prefix >> 20; // ranking path: the 12-bit digit of the bin that was ranked
 
   // ---- ordered emission: thread t owns a contiguous range of blocks (odd length: conflict-free smem reads) ----
   const int per = ((X + kThreads - 1) / kThreads) | 1;
   const int b0 = min(tid * per, X), b1 = min(b0 + per, X);
   int eq_rank = 0;
   const bool all_eq = need_eq >= eq_total;   // every block at the threshold is taken: no rank among ties needed
-  if (Kr > 0 && !all_eq) {
+  if (Kr > 0 && !ranked && !all_eq) {
     int c_eq = 0;
     for (int b = b0; b < b1; ++b) c_eq += (!mandatory(b) && keys[b] == thr) ? 1 : 0;
     eq_rank = block_exclusive_scan(c_eq, s_wtot, &s_total);
   }
-  int c_sel = 0;
-  uint32_t flags = 0;   // per <= 31 when X <= 31 * 1024; larger ranges recompute in the second walk
-  {
+  auto walk = [&](auto &&emit) {   // calls emit(b) for every selected block of this thread's range, in order
     int e = eq_rank;
     for (int b = b0; b < b1; ++b) {
       bool sel = mandatory(b);
       if (!sel && Kr > 0) {
         const uint32_t k = keys[b];
-        if (k > thr) sel = true;
-        else if (k == thr) { sel = all_eq || e < need_eq; ++e; }
+        if (ranked) {
+          sel = (k & 0x80000000u) != 0 || (k >> 20) > digit0;
+        } else if (k > thr) {
+          sel = true;
+        } else if (k == thr) {
+          sel = all_eq || e < need_eq;
+          ++e;
+        }
       }
-      c_sel += sel ? 1 : 0;
-      if (sel && b - b0 < 32) flags |= 1u << (b - b0);
+      if (sel) emit(b);
     }
-  }
+  };
+  int c_sel = 0;
+  walk([&](int) { ++c_sel; });
   int pos = block_exclusive_scan(c_sel, s_wtot, &s_total);
   const int total = s_total;
-  if (per <= 32) {
-    while (flags) {
-      const int j = __ffs(flags) - 1;
-      flags &= flags - 1;
-      if (pos < kcap) ids[pos] = b0 + j;
-      ++pos;
-    }
-  } else {
-    int e = eq_rank;
-    for (int b = b0; b < b1; ++b) {
-      bool sel = mandatory(b);
-      if (!sel && Kr > 0) {
-        const uint32_t k = keys[b];
-        if (k > thr) sel = true;
-        else if (k == thr) { sel = all_eq || e < need_eq; ++e; }
-      }
-      if (sel) { if (pos < kcap) ids[pos] = b; ++pos; }
-    }
-  }
+  walk([&](int b) { if (pos < kcap) ids[pos] = b; ++pos; });
   for (int i = total + tid; i < kcap; i += kThreads) ids[i] = -1;
   if (tid == 0) sel_cnt[unit] = min(total, kcap);
 }
