@@ -170,6 +170,20 @@ int ckv_dense_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void
                      const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
                      void *out, float *lse, ckv_stream stream);
 
+/* Dense decode attention without a context and without any caller-provided scratch.  (The paper has no
+ * counterpart: this entry point exists for hosts that cannot give the library device memory to work in -- a
+ * plugin handed only the operation's own tensors, code under a memory pool or a capture that forbids
+ * cudaMalloc, a process whose device memory is already committed to the KV cache.)
+ * Same inputs, outputs and result as ckv_dense_decode(), with `layout` passed directly.  The split partials
+ * live in a fixed device array inside the library image (4 MiB + 256 B, held by every GPU that loads the
+ * library until the process exits); the call allocates nothing.  It returns CKV_ERR_CAPACITY, before launching
+ * anything, when batch * num_q_heads * 528 B * 64 exceeds 4 MiB.  All calls share that array: calls that overlap
+ * on the GPU (other streams, other host threads) race on it, so serialise them.  The first call on a device
+ * looks up the array's device address and sets kernel attributes: make it outside any stream capture. */
+int ckv_dense_decode_static(const ckv_layout *layout, const void *q, const void *k_pool, const void *v_pool,
+                            const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
+                            void *out, float *lse, ckv_stream stream);
+
 /* Copy the block scores S_b of the last ckv_decode (Eq. 10) into dst (device),
  * fp32 [batch][num_kv_heads][max_blocks_per_seq]; entries at or past X_s are unspecified.
  * Mandatory blocks carry their score too (they are excluded from the ranking, not from Eq. 9). */

@@ -23,6 +23,7 @@ CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_
 
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
            "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_decode_profile", "ckv_dense_decode",
+           "ckv_dense_decode_static",
            "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
 
 
@@ -74,6 +75,8 @@ def load() -> ctypes.CDLL:
     lib.ckv_decode_profile.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp,
                                        ctypes.POINTER(ctypes.c_float)]
     lib.ckv_dense_decode.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+    lib.ckv_dense_decode_static.argtypes = [lp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+    lib.ckv_dense_decode_static.restype = i32
     lib.ckv_copy_scores.argtypes = [vp, vp, i32, vp]
     lib.ckv_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.ckv_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
@@ -117,6 +120,23 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+def dense_decode_static(layout: ckv_layout, q, k_pool, v_pool, page_table, seq_lens, max_seq_len: int, out=None,
+                        lse=None):
+    """ckv_dense_decode_static: dense decode attention that needs no context and no workspace.
+
+    For callers that cannot allocate device memory for the library.  The scratch is a fixed array inside the
+    library, shared by all calls: do not let two calls overlap on the GPU.  Returns (out, lse)."""
+    batch = q.shape[0]
+    if out is None:
+        out = torch.empty(batch, layout.num_q_heads, layout.head_dim, dtype=q.dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty(batch, layout.num_q_heads, dtype=torch.float32, device=q.device)
+    _check(load().ckv_dense_decode_static(ctypes.byref(layout), _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(page_table),
+                                          _ptr(seq_lens), batch, int(max_seq_len), _ptr(out), _ptr(lse), _stream()),
+           "ckv_dense_decode_static")
+    return out, lse
 
 
 class CompKV:

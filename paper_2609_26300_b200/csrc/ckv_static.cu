@@ -1,0 +1,94 @@
+// Dense decode attention for callers that cannot allocate device memory.
+//
+// Some hosts of this library have no way to hand it a workspace: a plugin that is given only the tensors
+// of the operation it implements, code running inside a stream capture or under a memory pool that forbids
+// cudaMalloc, a process whose device memory is fully committed to the KV cache.  ckv_dense_decode_static()
+// serves them: it needs no context and no caller-provided scratch.  The split partials the attention kernel
+// produces (and the merge kernel consumes) live in a fixed device array that is part of this library's
+// image, so every GPU that loads the library holds CKV_STATIC_SCRATCH_BYTES of it until the process exits.
+//
+// Consequences the caller has to know:
+//   * the array is shared by every call: two calls that overlap on the GPU (different streams, or the same
+//     call from two host threads) race on it and produce garbage.  Serialise them;
+//   * a problem whose partials do not fit returns CKV_ERR_CAPACITY before anything is launched;
+//   * the first call on a device looks the array's device address up and sets kernel attributes; make that
+//     first call outside any stream capture.
+#include <mutex>
+
+#include "ckv_internal.cuh"
+
+#define CKV_STATIC_SCRATCH_BYTES (4u << 20)   // 4 MiB of split partials + 256 B for the status word
+
+namespace {
+
+// In host code these names are host-side stand-ins for the device arrays, not device addresses: the address a
+// kernel may use comes from cudaGetSymbolAddress(), once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[CKV_STATIC_SCRATCH_BYTES + 256];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_mutex;
+void *g_scratch_ptr[kMaxDevices];   // device address of g_static_scratch on each device, null until looked up
+int g_sm_count[kMaxDevices];
+
+}  // namespace
+
+extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, const void *k_pool, const void *v_pool,
+                                       const int32_t *page_table, const int32_t *seq_lens, int batch,
+                                       int max_seq_len_host, void *out, float *lse, ckv_stream stream) {
+  if (layout == nullptr || !q || !k_pool || !v_pool || !page_table || !seq_lens || !out) return CKV_ERR_INVALID_ARG;
+  size_t stats_bytes = 0, work_bytes = 0;
+  const int lst = ckv_query_sizes(layout, &stats_bytes, &work_bytes);   // host-only: validates the layout
+  if (lst != CKV_OK) return lst;
+  if (batch <= 0 || batch > layout->max_batch) return CKV_ERR_INVALID_ARG;
+  if (max_seq_len_host <= 0 || (long long)max_seq_len_host > (long long)layout->max_blocks_per_seq * layout->block_size)
+    return CKV_ERR_INVALID_ARG;
+
+  // a context on the host stack: only the fields the dense path reads are filled in
+  ckv_ctx c{};
+  c.layout = *layout;
+  if (c.layout.sm_scale == 0.f) c.layout.sm_scale = 1.0f / sqrtf((float)layout->head_dim);
+  CkvDev &P = c.dev;
+  P.Hq = layout->num_q_heads; P.Hkv = layout->num_kv_heads; P.G = P.Hq / P.Hkv;
+  P.bs = layout->block_size; P.ppb = layout->block_size / layout->page_size;
+  P.r = layout->var_groups; P.glayout = layout->group_layout;
+  P.max_blocks = layout->max_blocks_per_seq; P.max_pages_per_seq = P.max_blocks * P.ppb;
+  P.num_pages = layout->num_pages; P.sink = layout->sink_blocks; P.recent = layout->recent_blocks;
+  P.scale = c.layout.sm_scale;
+
+  // the partials of the largest split count the launch heuristic may pick must fit the fixed array
+  const size_t per_split = (size_t)batch * P.Hkv * P.G * CKV_PART_STRIDE * sizeof(float);
+  if (per_split * CKV_MAX_SPLITS > CKV_STATIC_SCRATCH_BYTES) return CKV_ERR_CAPACITY;
+
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CKV_ERR_CUDA;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_scratch_ptr[dev] == nullptr) {   // once per device, with that device current
+      void *ptr = nullptr;
+      e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+      if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+      if (e == cudaSuccess) e = ckv_configure_attn(&c);
+      if (e == cudaSuccess) e = ckv_configure_attn_mma(&c);
+      if (e != cudaSuccess || ptr == nullptr) return CKV_ERR_CUDA;
+      g_scratch_ptr[dev] = ptr;
+    }
+  }
+  unsigned char *scratch = (unsigned char *)g_scratch_ptr[dev];
+  P.attn_part = (float *)scratch;
+  P.status = (int *)(scratch + CKV_STATIC_SCRATCH_BYTES);
+  c.sm_count = g_sm_count[dev];
+
+  cudaStream_t s = (cudaStream_t)stream;
+  // the array keeps whatever the previous call left: the status word must start at zero; every partial the merge
+  // reads is rewritten by this call's attention kernel
+  e = cudaMemsetAsync(P.status, 0, sizeof(int), s);
+  if (e != cudaSuccess) return CKV_ERR_CUDA;
+  int n_splits = 0;
+  e = ckv_launch_attn(&c, true, q, k_pool, v_pool, page_table, seq_lens, nullptr, nullptr, 0, batch, max_seq_len_host,
+                      &n_splits, s);
+  if (e != cudaSuccess) return CKV_ERR_CUDA;
+  e = ckv_launch_merge(&c, true, seq_lens, nullptr, n_splits, 0, batch, out, lse, s);
+  if (e != cudaSuccess) return CKV_ERR_CUDA;
+  return CKV_OK;
+}
