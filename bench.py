@@ -209,10 +209,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2609_26300_b200.replicas import Replicas
+    rep = Replicas(device=torch.device("cuda", local))
+    dist = rep.dist
 
     W, K, KP, KE = max(args.warmup, 3), args.steps, args.profile_steps, args.e2e_steps
     total = W + K + KP + KE + W
@@ -354,15 +353,11 @@ def main():
     assert ckv.read_status() == 0
 
     # ---- max over ranks ----
-    vals = torch.tensor([ms_per_step, e2e_us, scan_us, dense_us], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms_per_step, e2e_us, scan_us, dense_us = (float(x) for x in vals.tolist())
+    ms_per_step, e2e_us, scan_us, dense_us = rep.max_over_ranks([ms_per_step, e2e_us, scan_us, dense_us])
     us_per_step = ms_per_step * 1e3
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+        rep.close()
         return 0
 
     peak, peak_kind = measured_peak()
@@ -379,7 +374,7 @@ def main():
                    "l2": "flushed between steps (256 MiB memset then 256 MiB read, outside the events); per-step inputs exceed L2",
                    "replicas": "every rank runs the whole workload (the path does not shard)",
                    "kv_storage": "bf16", "seed": w.seed},
-        "tokens_per_s": world * w.batch / (us_per_step * 1e-6),
+        "tokens_per_s": rep.aggregate_tokens_per_s(w.batch, us_per_step),
         "required_bytes_per_step": req, "hbm_gbs": step_gbs,
         "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS, "frac_of_%s_peak" % peak_kind: step_gbs / peak,
         "dense_us": dense_us, "dense_gbs": dense_bytes / (dense_us * 1e-6) / 1e9,
@@ -410,8 +405,7 @@ def main():
                                           "on the %d KV heads of sequence 0, %d steps, wall time x %d sequences"
                                           % (w.num_kv_heads, reps, w.batch)}
     print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    rep.close()
     return 0
 
 
