@@ -32,7 +32,7 @@ int check_layout(const ckv_layout *L) {
 
 struct Regions {
   size_t kmean, dbar, vmean, stats_total;
-  size_t ls, scores, comp, attn, status, stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt, work_total;
+  size_t ls, scores, comp, attn, status, done, stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt, work_total;
 };
 
 Regions regions(const ckv_layout *L) {
@@ -48,6 +48,7 @@ Regions regions(const ckv_layout *L) {
   R.stats_total = o;
   o = 0;
   R.status = o; o = align_up(o + 256, 256);
+  R.done = o;   o = align_up(o + units * 4, 256);
   R.ls = o;     o = align_up(o + rows * G * sizeof(float2), 256);
   R.scores = o; o = align_up(o + rows * 4, 256);
   R.comp = o;   o = align_up(o + (units + CKV_MAX_SCAN_CTAS) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE * 4, 256);
@@ -143,7 +144,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.num_pages = layout->num_pages; P.sink = layout->sink_blocks; P.recent = layout->recent_blocks;
   P.scale = c->layout.sm_scale;
   P.kmean = (__nv_bfloat16 *)(sb + R.kmean); P.dbar = (float *)(sb + R.dbar); P.vmean = (__nv_bfloat16 *)(sb + R.vmean);
-  P.status = (int *)(wb + R.status);
+  P.status = (int *)(wb + R.status); P.unit_done = (int *)(wb + R.done);
   P.ls = (float2 *)(wb + R.ls); P.scores = (float *)(wb + R.scores);
   P.comp_part = (float *)(wb + R.comp); P.attn_part = (float *)(wb + R.attn);
   c->work = wb; c->work_bytes = work_bytes;
@@ -157,7 +158,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   int dev_id = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev_id);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev_id);
-  if (e == cudaSuccess) e = cudaMemsetAsync(P.status, 0, 256, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(P.status, 0, R.ls - R.status, (cudaStream_t)stream);   // status word, split counters
   if (e != cudaSuccess) { delete c; return cuda_fail(e); }
   *out = c;
   return CKV_OK;
@@ -210,10 +211,11 @@ int decode_impl(ckv_ctx *c, const void *q, const void *k_pool, const void *v_poo
   if (ev) CKV_CUDA(cudaEventRecord(ev[1], s));
   CKV_CUDA(ckv_launch_select(c, seq_lens, batch, kcap, scan_grid, sel_ids, sel_cnt, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[2], s));
+  bool merged = false;
   CKV_CUDA(ckv_launch_attn(c, false, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, batch,
-                           max_seq_len_host, &n_splits, s));
+                           max_seq_len_host, scan_grid, out, lse, &n_splits, &merged, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[3], s));
-  CKV_CUDA(ckv_launch_merge(c, false, seq_lens, sel_cnt, n_splits, scan_grid, batch, out, lse, s));
+  if (!merged) CKV_CUDA(ckv_launch_merge(c, false, seq_lens, sel_cnt, n_splits, scan_grid, batch, out, lse, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[4], s));
   return CKV_OK;
 }
@@ -254,9 +256,10 @@ int ckv_dense_decode(ckv_ctx *c, const void *q, const void *k_pool, const void *
   if (!q || !k_pool || !v_pool || !page_table || !seq_lens || !out) return CKV_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   int n_splits = 0;
+  bool merged = false;
   CKV_CUDA(ckv_launch_attn(c, true, q, k_pool, v_pool, page_table, seq_lens, nullptr, nullptr, 0, batch,
-                           max_seq_len_host, &n_splits, s));
-  CKV_CUDA(ckv_launch_merge(c, true, seq_lens, nullptr, n_splits, 0, batch, out, lse, s));
+                           max_seq_len_host, 0, out, lse, &n_splits, &merged, s));
+  if (!merged) CKV_CUDA(ckv_launch_merge(c, true, seq_lens, nullptr, n_splits, 0, batch, out, lse, s));
   return CKV_OK;
 }
 

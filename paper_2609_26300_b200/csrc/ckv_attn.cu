@@ -456,22 +456,29 @@ cudaError_t ckv_configure_attn(const ckv_ctx *c) {
 
 cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                             const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
-                            int kcap, int batch, int max_len, int *n_splits_out, cudaStream_t st) {
+                            int kcap, int batch, int max_len, int scan_grid, void *out, float *lse,
+                            int *n_splits_out, bool *merged_out, cudaStream_t st) {
   const CkvDev &P = c->dev;
   const int units = batch * P.Hkv;
   const int xmax = (max_len + P.bs - 1) / P.bs;
   const int total = dense ? (max_len + CKV_PAGE - 1) / CKV_PAGE : min(kcap, xmax) * P.ppb;
-  // about four CTAs per SM overall, at least one page per warp, at most CKV_MAX_SPLITS splits
-  int n_splits = (148 * 4 + units - 1) / units;
+  const bool mma = c->layout.kv_dtype == CKV_BF16;
+  const int sms = c->sm_count > 0 ? c->sm_count : 148;
+  // Splits per unit: the selected list is short, so the tensor-core kernel gets one wave of three CTAs per SM; the
+  // dense pass (and the fp32 kernel) about four CTAs per SM overall.  At least eight pages per split, at most
+  // CKV_MAX_SPLITS splits.
+  int n_splits = (mma && !dense) ? max(1, 3 * sms / units) : (sms * 4 + units - 1) / units;
   n_splits = max(1, min(n_splits, min(CKV_MAX_SPLITS, (total + 7) / 8)));
   int pps = (total + n_splits - 1) / n_splits;
-  pps = (pps + 7) / 8 * 8;
+  if (!(mma && !dense)) pps = (pps + 7) / 8 * 8;   // the tensor-core kernel deals pages to its warps one by one
   n_splits = max(1, (total + pps - 1) / pps);
   *n_splits_out = n_splits;
+  *merged_out = mma && P.unit_done != nullptr;
   dim3 grid(n_splits, units);
   c->launches++;
   if (c->layout.kv_dtype == CKV_BF16)   // bf16 pages go through the tensor-core kernel
-    return ckv_launch_attn_mma(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
+    return ckv_launch_attn_mma(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps,
+                               scan_grid, out, lse, st);
   switch (P.G) {
     case 1: return launch_g<1>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
     case 2: return launch_g<2>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);

@@ -1,32 +1,44 @@
-// Exact attention over a list of cache pages on tensor cores (bf16 layout), split along the list, plus the
-// removal of the selected blocks' mean-compensation terms (Eq. 12).  Same contract as the fp32-capable
-// kernel in ckv_attn.cu: one partial (m, l, acc[128]) per (unit, split, head) for the merge kernel.
+// Exact attention over a list of cache pages on tensor cores (bf16 layout), split along the list, with the
+// removal of the selected blocks' mean-compensation terms and the final merge (Eq. 12) in the same launch.
 //
 // Sparse mode: the page list of a unit is the pages of its selected blocks, in position order.
 // Dense mode: every page of the sequence (Eq. 12 with S = all blocks; Sec. 3.1).
 //
-// A CTA takes a contiguous slice of the list; each of its 8 warps takes every 8th page.  A warp copies its
-// page (16 tokens: a 4 KB K tile and a 4 KB V tile, each contiguous in the paged pool) into shared memory
-// with 16-byte cp.async pieces whose destinations are XOR-swizzled by the token row, so that the matrix
-// loads below are conflict-free; rows past the sequence end are zero-filled.  Then, with the G heads as the
-// M dimension (rows 0..7 of 16) of mma.sync.m16n8k16:
+// A CTA takes a contiguous slice of the list; each of its W warps takes every W-th page.  A warp copies its
+// page (16 tokens: a 4 KB K tile and a 4 KB V tile, each contiguous in the paged pool) into one of its two
+// shared-memory buffers with 16-byte cp.async pieces whose destinations are XOR-swizzled by the token row, so
+// that the matrix loads below are conflict-free; rows past the sequence end are zero-filled; the next page is
+// in flight while the current one is multiplied.  Then, with the G heads as the M dimension (rows 0..7 of 16)
+// of mma.sync.m16n8k16:
 //   S^T = Q K^T      heads x 16 tokens, Q fragments held in registers for the whole kernel
 //   P   = 2^(S^T - m) per warp, running maximum raised only when exceeded by a slack; split into bf16 hi + lo
 //   O  += P V        heads x 128 coordinates; the accumulator layout of S^T is the A-operand layout of P V
 // For every selected block the scan kernel has already added the block's mean term |b| e^{zbar} vbar_b to
-// the all-block compensation sum; here the same term is subtracted with one more P V-shaped product whose
-// only non-zero row is the block's mean value (read as its stored hi + lo halves), so that
+// the all-block compensation sum; here the same terms are subtracted, three blocks at a time, with one more
+// P V-shaped product whose non-zero rows are the blocks' mean values (read as their stored hi + lo halves):
 //   merge = exact(S) + mean(all) - mean(S) = exact(S) + mean(not S).
+//
+// Merge.  The scan's partials of the unit (one per scan CTA and consumer warp) exist before this kernel
+// starts, so the unit's active CTAs share them out, fetch their share while their last page is in flight and
+// fold it into their own partial.  Each CTA then publishes one partial (m, l, acc[128]) per head and bumps
+// the unit's counter; the CTA that finds the counter complete reads the unit's partials back (they are few)
+// and writes the output row and the log-sum-exp.  The counter is left at zero for the next step.
 #include "ckv_internal.cuh"
 #include "ckv_mma.cuh"
 
 namespace {
 
-constexpr int kWarps = 8;
 constexpr int kTileBytes = CKV_PAGE * CKV_D * 2;      // one head's K (or V) page in bf16: 4 KB
+constexpr int kPageBytes = 2 * kTileBytes;            // K tile | V tile
 constexpr int kRowBytes = CKV_D * 2;                  // 256
-constexpr int kAuxBytes = 1536;                       // per warp: a mean-value row (512 B) per page buffer and a row of zeros
-constexpr int kZeroRow = 1024;                        // offset of the row of zeros inside the aux area
+constexpr int kMeanSlots = 4;                         // mean-value rows (512 B each) a warp can hold
+constexpr int kMeanFlush = 3;                         // ... of which at most 3 wait for removal while one is in flight
+constexpr int kZeroRow = kMeanSlots * 512;            // offset of the row of zeros inside the aux area
+constexpr int kAuxBytes = kZeroRow + 256;
+constexpr int kMaxEntries = 32;                       // partials a CTA folds per round: one per lane
+constexpr int kPartBytes = CKV_PART_STRIDE * 4;       // one head's partial
+
+template <int W> constexpr size_t dyn_smem() { return (size_t)W * (2 * kPageBytes + kAuxBytes); }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
   // valid == false copies nothing and zero-fills the 16 bytes
@@ -35,38 +47,34 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool v
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int G, bool DENSE>
-__global__ void __launch_bounds__(kWarps * 32, DENSE ? 1 : 2)
+template <int G, bool DENSE, int W>
+__global__ void __launch_bounds__(W * 32, DENSE ? 1 : 3)
 ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_pool,
                     const __nv_bfloat16 *__restrict__ v_pool, const int *__restrict__ page_table,
                     const int *__restrict__ seq_lens, const int *__restrict__ sel_ids,
-                    const int *__restrict__ sel_cnt, int kcap, int pages_per_split, int nbuf) {
-  extern __shared__ __align__(128) unsigned char smem[];   // [8 warps][nbuf][K tile | V tile], then [8 warps][aux]
-  __shared__ __align__(16) float red[kWarps][G][CKV_PART_STRIDE];
+                    const int *__restrict__ sel_cnt, int kcap, int pages_per_split, int scan_grid, int units,
+                    __nv_bfloat16 *__restrict__ out, float *__restrict__ lse) {
+  extern __shared__ __align__(128) unsigned char smem[];   // [W warps][2 buffers][K tile | V tile], then [W warps][aux]
+  __shared__ float s_scale[kMaxEntries][G];
+  __shared__ float s_M[G], s_den[G];
+  __shared__ int s_ent[kMaxEntries];   // float offset of each entry inside smem
+  __shared__ int s_last;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int head = lane >> 2, qd = lane & 3;
   const bool hv = head < G;
   const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
-  const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
-  const int X = (N + P.bs - 1) / P.bs;
-  const int nsel = DENSE ? X : min(sel_cnt[unit], kcap);
-  const int total = DENSE ? (N + CKV_PAGE - 1) / CKV_PAGE : nsel * P.ppb;
-  const bool comp = !DENSE && nsel < X;
+  const int pshift = P.ppb == 1 ? 0 : (P.ppb == 2 ? 1 : 2);
   const int p0 = blockIdx.x * pages_per_split;
-  const int p1 = min(p0 + pages_per_split, total);
-  float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
-  if (p0 >= total) {
-    if (tid < G) { part[tid * CKV_PART_STRIDE] = -CUDART_INF_F; part[tid * CKV_PART_STRIDE + 1] = 0.f; }
-    return;
+
+  // ---- first round trip: everything that depends on nothing else is requested together ----
+  const int n_raw = seq_lens[s];
+  const int cnt_raw = DENSE ? 0 : sel_cnt[unit];
+  int blk0 = -1;   // block of the page this lane will look up first (read before the list length is known)
+  if (!DENSE) {
+    const int i = p0 + warp + W * lane;
+    if (i < kcap * P.ppb) blk0 = sel_ids[(size_t)unit * kcap + (i >> pshift)];
   }
-
-  unsigned char *wtiles = smem + (size_t)warp * nbuf * 2 * kTileBytes;
-  unsigned char *waux = smem + (size_t)kWarps * nbuf * 2 * kTileBytes + (size_t)warp * kAuxBytes;
-  const uint32_t aux_u32 = (uint32_t)__cvta_generic_to_shared(waux);
-  // the row of zeros every unused row of the mean-value product points at
-  if (lane < 16) reinterpret_cast<uint4 *>(waux + kZeroRow)[lane] = make_uint4(0u, 0u, 0u, 0u);
-
   // Q fragments: A operand rows 0..7 = heads, scaled logits come out of the products in log2 units
   uint32_t qa[8][2];
   {
@@ -79,29 +87,73 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         qa[ks][hh] = hv ? v : 0u;
       }
   }
-  const float sl2 = P.scale * kLog2e;
+  int cfirst = 0, ccount = 0;   // where the unit's scan partials sit
+  if (!DENSE) unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
 
+  const int N = max(min(n_raw, P.max_blocks * P.bs), 0);
+  const int X = (N + P.bs - 1) / P.bs;
+  const int nsel = DENSE ? X : min(cnt_raw, kcap);
+  const int total = DENSE ? (N + CKV_PAGE - 1) / CKV_PAGE : nsel * P.ppb;
+  const bool comp = !DENSE && nsel < X;
+  const int p1 = min(p0 + pages_per_split, total);
+  float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
+  if (p0 >= total) {   // no pages for this split: it takes no part in the unit's merge
+    if (total == 0 && blockIdx.x == 0) {   // an empty unit: its output is defined as zero
+      for (int idx = tid; idx < G * CKV_D; idx += W * 32)
+        out[((size_t)s * P.Hq + h * G) * CKV_D + idx] = __float2bfloat16_rn(0.f);
+      if (lse != nullptr && tid < G) lse[(size_t)s * P.Hq + h * G + tid] = -CUDART_INF_F;
+    }
+    return;
+  }
+  const int n_active = (total + pages_per_split - 1) / pages_per_split;   // splits of this unit that have pages
+
+  unsigned char *wtiles = smem + (size_t)warp * 2 * kPageBytes;
+  const uint32_t wtiles_u32 = (uint32_t)__cvta_generic_to_shared(wtiles);
+  unsigned char *waux = smem + (size_t)W * 2 * kPageBytes + (size_t)warp * kAuxBytes;
+  const uint32_t aux_u32 = (uint32_t)__cvta_generic_to_shared(waux);
+  // the row of zeros every unused row of the mean-value product points at
+  if (lane < 16) reinterpret_cast<uint4 *>(waux + kZeroRow)[lane] = make_uint4(0u, 0u, 0u, 0u);
+
+  const float sl2 = P.scale * kLog2e;
   float acc[16][2];
 #pragma unroll
   for (int t = 0; t < 16; ++t) { acc[t][0] = 0.f; acc[t][1] = 0.f; }
   float m_ref = -CUDART_INF_F, l_acc = 0.f;
   const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
-  const int pshift = P.ppb == 1 ? 0 : (P.ppb == 2 ? 1 : 2);
-  const int n_mine = (p1 - p0 - warp + kWarps - 1) / kWarps;   // this warp's pages: list index p0 + warp + 8 n
+  const int n_mine = max((p1 - p0 - warp + W - 1) / W, 0);   // this warp's pages: list index p0 + warp + W n
   const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
   const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * CKV_ROW_ELEMS;
   bool bad = false;
 
+  // the scan partials this CTA folds in: partial j of the unit goes to split j % n_active
+  constexpr int kSlotsPerWarp = (kPageBytes / (G * kPartBytes)) < ((kMaxEntries - W) / W) ? (kPageBytes / (G * kPartBytes))
+                                                                                       : ((kMaxEntries - W) / W);
+  constexpr int kSlots = W * kSlotsPerWarp;
+  const int n_comp = comp ? ccount * CKV_SCAN_WARPS : 0;
+  const int my_cnt = n_comp > (int)blockIdx.x ? (n_comp - (int)blockIdx.x + n_active - 1) / n_active : 0;
+  const size_t step = (size_t)G * CKV_PART_STRIDE;
+  const float *cp0 = P.comp_part + (size_t)(cfirst + unit) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE;
+  // start the copies of this warp's share of the round that begins at `base` into its buffer `bufsel`
+  auto issue_comp = [&](int bufsel, int base) {
+#pragma unroll
+    for (int k = 0; k < kSlotsPerWarp; ++k) {
+      const int idx = base + warp * kSlotsPerWarp + k;
+      if (idx < my_cnt) {
+        const float *src = cp0 + (size_t)(blockIdx.x + (size_t)idx * n_active) * step;
+        const uint32_t dst = wtiles_u32 + bufsel * kPageBytes + k * (G * kPartBytes);
+        for (int c = lane; c < G * (kPartBytes / 16); c += 32) cp_async16(dst + 16 * c, src + 4 * c, true);
+      }
+    }
+  };
+
   struct PageRef { int phys, ntok, blk; bool first; };
-  auto resolve = [&](int n) {
+  auto resolve = [&](int i, int blk) {   // list index -> physical page; blk is the selected block (sparse mode)
     PageRef r{-1, 0, -1, false};
-    const int i = p0 + warp + kWarps * n;
     int page = i;
     bool ok = true;
     if (!DENSE) {
-      r.blk = sel_ids[(size_t)unit * kcap + (i >> pshift)];
-      ok = r.blk >= 0 && r.blk < X;
-      if (!ok) r.blk = -1;
+      ok = blk >= 0 && blk < X;
+      r.blk = ok ? blk : -1;
       page = (r.blk << pshift) + (i & (P.ppb - 1));
       r.first = ok && (i & (P.ppb - 1)) == 0;
     }
@@ -116,12 +168,32 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     }
     return r;
   };
+  // Page lookups are dependent loads; lane l does the lookup of page (chunk base + l) so that a chunk of 32 pages
+  // costs one round trip, and fetch(n), called once per page in increasing order, hands the result to all lanes.
+  PageRef mine{-1, 0, -1, false};
+  auto fetch = [&](int n) {
+    if ((n & 31) == 0) {
+      mine = PageRef{-1, 0, -1, false};
+      if (n + lane < n_mine) {
+        const int i = p0 + warp + W * (n + lane);
+        int blk = -1;
+        if (!DENSE) blk = n == 0 ? blk0 : sel_ids[(size_t)unit * kcap + (i >> pshift)];
+        mine = resolve(i, blk);
+      }
+    }
+    PageRef r;
+    r.phys = __shfl_sync(0xffffffffu, mine.phys, n & 31);
+    r.ntok = __shfl_sync(0xffffffffu, mine.ntok, n & 31);
+    r.blk = __shfl_sync(0xffffffffu, mine.blk, n & 31);
+    r.first = __shfl_sync(0xffffffffu, (int)mine.first, n & 31) != 0;
+    return r;
+  };
   // start the copies of one page into buffer `buf`: 256 16-byte pieces per tile, 8 per lane; piece c of row r
-  // lands at chunk c ^ (r & 7) of the row
-  auto issue = [&](const PageRef &r, int buf) {
+  // lands at chunk c ^ (r & 7) of the row; the block's mean-value row goes to aux slot `slot`
+  auto issue = [&](const PageRef &r, int buf, int slot) {
     if (r.phys >= 0) {
       const size_t src = ((size_t)r.phys * P.Hkv + h) * (CKV_PAGE * CKV_D);
-      const uint32_t kb = (uint32_t)__cvta_generic_to_shared(wtiles + (size_t)buf * 2 * kTileBytes);
+      const uint32_t kb = wtiles_u32 + buf * kPageBytes;
       const uint32_t vb = kb + kTileBytes;
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
@@ -132,27 +204,101 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         cp_async16(kb + off, k_pool + so, valid);
         cp_async16(vb + off, v_pool + so, valid);
       }
-      if (comp && r.first)   // the block's mean-value row, verbatim (hi halves then lo halves, swizzled by block index)
-        cp_async16(aux_u32 + 512 * buf + 16 * lane, vmean + (size_t)r.blk * CKV_ROW_ELEMS + 8 * lane, true);
+      if (comp && r.first)   // verbatim: hi halves then lo halves, swizzled by block index
+        cp_async16(aux_u32 + 512 * slot + 16 * lane, vmean + (size_t)r.blk * CKV_ROW_ELEMS + 8 * lane, true);
     }
-    cp_async_commit();
   };
 
-  PageRef cur = n_mine > 0 ? resolve(0) : PageRef{-1, 0, -1, false};
-  if (n_mine > 0) issue(cur, 0);
-  for (int n = 0, buf = 0; n < n_mine; ++n) {
-    PageRef nxt{-1, 0, -1, false};
-    const bool prefetch = nbuf > 1 && n + 1 < n_mine;
-    if (prefetch) {
-      nxt = resolve(n + 1);
-      issue(nxt, buf ^ 1);
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
+  // Blocks whose mean term |b| e^{zbar} vbar_b is still to be taken back out (it is part of the all-block sum the
+  // scan produced): up to kMeanFlush of them are removed by one product, weights x mean-value rows.
+  int bb[kMeanFlush], bsl[kMeanFlush], nb = 0;
+#pragma unroll
+  for (int j = 0; j < kMeanFlush; ++j) { bb[j] = 0; bsl[j] = 0; }
+  auto remove_means = [&]() {
+    float zl[2] = {-CUDART_INF_F, -CUDART_INF_F};
+    if (hv && qd < 2) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int j = 2 * qd + e;
+        if (j < nb) {
+          const int blk = j == 0 ? bb[0] : (j == 1 ? bb[1] : bb[2]);
+          const float2 v = __ldg(ls + (size_t)head * P.max_blocks + blk);
+          zl[e] = (v.x - 0.5f * v.y) * kLog2e;
+        }
+      }
     }
+    float zmax = fmaxf(zl[0], zl[1]);
+    zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, 1));
+    zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, 2));
+    if (zmax > m_ref + CKV_RESCALE_SLACK) {
+      const float sc = exp2_diff(m_ref, zmax);
+      m_ref = zmax;
+      l_acc *= sc;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) { acc[t][0] *= sc; acc[t][1] *= sc; }
+    }
+    const float w0 = zl[0] == -CUDART_INF_F ? 0.f : fast_exp2(zl[0] - m_ref);
+    const float w1 = zl[1] == -CUDART_INF_F ? 0.f : fast_exp2(zl[1] - m_ref);
+    l_acc -= w0 + w1;
+    // A operand: columns 0..nb-1 (the real rows of the B operand) hold the negated weights
+    const uint32_t wh = pack_bf16(-w0, -w1);
+    const uint32_t wl = pack_bf16(-(w0 - bf16_round(w0)), -(w1 - bf16_round(w1)));
+    // B operand: row j < nb is the mean-value row of batch entry j, every other row the row of zeros
+    const int r = ((lane >> 3) & 1) * 8 + (lane & 7);
+    const bool real = r < nb;
+    const int rblk = r == 0 ? bb[0] : (r == 1 ? bb[1] : bb[2]);
+    const int rslot = r == 0 ? bsl[0] : (r == 1 ? bsl[1] : bsl[2]);
+    const uint32_t rowaddr = aux_u32 + 512 * (real ? rslot : 0);
+    const int cpar = lane >> 4;
+#pragma unroll
+    for (int t2 = 0; t2 < 8; ++t2) {
+      const uint32_t coff = (uint32_t)(swz_chunk(2 * t2 + cpar, rblk) << 4);
+      uint32_t vh[4], vl[4];
+      ldmatrix_x4_trans(vh, real ? rowaddr + coff : aux_u32 + kZeroRow);
+      ldmatrix_x4_trans(vl, real ? rowaddr + 256 + coff : aux_u32 + kZeroRow);
+      mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh, 0u, vh[0], vh[1]);
+      mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wl, 0u, vh[0], vh[1]);
+      mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh, 0u, vl[0], vl[1]);
+      mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh, 0u, vh[2], vh[3]);
+      mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wl, 0u, vh[2], vh[3]);
+      mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh, 0u, vl[2], vl[3]);
+    }
+    nb = 0;
+  };
+
+  // Mean-value slots are handed out in ring order when a block's first page is issued.  At most kMeanFlush
+  // recorded blocks, the page being multiplied and the page in flight hold a slot at any time: <= kMeanSlots.
+  int si = 0;
+  auto take_slot = [&](const PageRef &r) {
+    const int slot = si;
+    if (comp && r.first && r.phys >= 0) si = (si + 1) & (kMeanSlots - 1);
+    return slot;
+  };
+  PageRef cur{-1, 0, -1, false};
+  int cur_slot = 0;
+  if (n_mine > 0) {
+    cur = fetch(0);
+    cur_slot = take_slot(cur);
+    issue(cur, 0, cur_slot);
+  } else {
+    issue_comp(1, 0);   // a warp without pages only brings in its share of the scan partials
+  }
+  cp_async_commit();
+  for (int n = 0, buf = 0; n < n_mine; ++n, buf ^= 1) {
+    PageRef nxt{-1, 0, -1, false};
+    int nxt_slot = 0;
+    if (n + 1 < n_mine) {
+      nxt = fetch(n + 1);
+      nxt_slot = take_slot(nxt);
+      issue(nxt, buf ^ 1, nxt_slot);
+    } else {
+      issue_comp(buf ^ 1, 0);   // the other buffer is idle during the last page
+    }
+    cp_async_commit();
+    cp_async_wait<1>();
     __syncwarp();
     if (cur.phys >= 0) {
-      const uint32_t kb = (uint32_t)__cvta_generic_to_shared(wtiles + (size_t)buf * 2 * kTileBytes);
+      const uint32_t kb = wtiles_u32 + buf * kPageBytes;
       const uint32_t vb = kb + kTileBytes;
       // ---- S^T = Q K^T: heads x 16 tokens (two n-tiles of 8 tokens) ----
       float sv[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, sv2[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
@@ -218,107 +364,176 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
           mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], pl[0], pl[1], v[2], v[3]);
         }
       }
-      if (comp && cur.first) {
-        // take this block's mean term |b| e^{zbar} vbar_b back out (it is part of the all-block sum)
-        float zl2 = -CUDART_INF_F;
-        if (hv) {
-          const float2 v = __ldg(ls + (size_t)head * P.max_blocks + cur.blk);
-          zl2 = (v.x - 0.5f * v.y) * kLog2e;
-        }
-        if (zl2 > m_ref + CKV_RESCALE_SLACK) {
-          const float sc = exp2_diff(m_ref, zl2);
-          m_ref = zl2;
-          l_acc *= sc;
+      if (comp && cur.first) {   // its mean-value row sits in aux slot cur_slot
 #pragma unroll
-          for (int t = 0; t < 16; ++t) { acc[t][0] *= sc; acc[t][1] *= sc; }
-        }
-        const float wbar = hv ? fast_exp2(zl2 - m_ref) : 0.f;
-        if (qd == 0) l_acc -= wbar;
-        // A operand: column 0 (the only real row of the B operand) holds -wbar for this thread's head
-        const uint32_t wh = qd == 0 ? pack_bf16(-wbar, 0.f) : 0u;
-        const uint32_t wl = qd == 0 ? pack_bf16(-(wbar - bf16_round(wbar)), 0.f) : 0u;
-        // B operand rows: row 0 is the mean-value row, every other row the row of zeros
-        const bool row0 = (lane & 15) == 0;   // lanes 0 and 16 address row 0 of their 8x8 matrices (chunks c, c + 1)
-        const int cpar = lane >> 4;
-#pragma unroll
-        for (int t2 = 0; t2 < 8; ++t2) {
-          const uint32_t coff = (uint32_t)(swz_chunk(2 * t2 + cpar, cur.blk) << 4);
-          uint32_t vh[4], vl[4];
-          ldmatrix_x4_trans(vh, row0 ? aux_u32 + 512 * buf + coff : aux_u32 + kZeroRow);
-          ldmatrix_x4_trans(vl, row0 ? aux_u32 + 512 * buf + 256 + coff : aux_u32 + kZeroRow);
-          mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh, 0u, vh[0], vh[1]);
-          mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wl, 0u, vh[0], vh[1]);
-          mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh, 0u, vl[0], vl[1]);
-          mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh, 0u, vh[2], vh[3]);
-          mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wl, 0u, vh[2], vh[3]);
-          mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh, 0u, vl[2], vl[3]);
-        }
+        for (int j = 0; j < kMeanFlush; ++j)
+          if (j == nb) { bb[j] = cur.blk; bsl[j] = cur_slot; }
+        ++nb;
       }
     }
-    __syncwarp();   // the buffer (and the mean-value row) may be overwritten from here on
-    if (nbuf > 1) {
-      cur = nxt;
-      buf ^= 1;
-    } else if (n + 1 < n_mine) {
-      cur = resolve(n + 1);
-      issue(cur, 0);
-    }
+    if (nb == kMeanFlush || (nb > 0 && n + 1 == n_mine)) remove_means();
+    __syncwarp();   // the page buffer (and, after a removal, the mean-value slots) may be overwritten from here on
+    cur = nxt;
+    cur_slot = nxt_slot;
   }
   cp_async_wait<0>();
-  if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
+  __syncwarp();
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
 
-  // ---- CTA partial: fold the warps (each with its own running maximum) ----
+  // ---- CTA partial: fold the warps (each with its own running maximum) and this CTA's scan partials ----
+  // A warp's partial [G][CKV_PART_STRIDE] goes into the buffer of its last page; the other buffer holds its
+  // share of the scan partials.  Entry e < W is warp e's partial, entry W + c is scan-partial slot c.
+  auto red_buf = [&](int e) {
+    const int nm = max((p1 - p0 - e + W - 1) / W, 0);
+    return nm > 0 ? (nm - 1) & 1 : 0;
+  };
+  auto region = [&](int e, int b) { return (int)(((size_t)e * 2 * kPageBytes + (size_t)b * kPageBytes) / 4); };   // in floats
+  float *sf = reinterpret_cast<float *>(smem);
   l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 1);
   l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 2);
   if (hv) {
-    float *r = red[warp][head];
+    float *r = sf + region(warp, red_buf(warp)) + head * CKV_PART_STRIDE;
 #pragma unroll
     for (int t = 0; t < 16; ++t) *reinterpret_cast<float2 *>(r + 4 + 8 * t + 2 * qd) = make_float2(acc[t][0], acc[t][1]);
     if (qd == 0) { r[0] = m_ref; r[1] = l_acc; }
   }
-  __syncthreads();
-  for (int idx = tid; idx < G * CKV_D; idx += kWarps * 32) {
-    const int g = idx / CKV_D, c = idx % CKV_D;
-    float M = -CUDART_INF_F;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, red[w][g][0]);
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-      const float sc = exp2_diff(red[w][g][0], M);
-      num = fmaf(red[w][g][4 + c], sc, num);
-      den = fmaf(red[w][g][1], sc, den);
+  if (tid < W + kSlots) {
+    int off;
+    if (tid < W) {
+      off = region(tid, red_buf(tid));
+    } else {
+      const int c = tid - W, we = c / kSlotsPerWarp, k = c % kSlotsPerWarp;
+      off = region(we, red_buf(we) ^ 1) + k * G * CKV_PART_STRIDE;
     }
-    part[g * CKV_PART_STRIDE + 4 + c] = num;
-    if (c == 0) { part[g * CKV_PART_STRIDE] = M; part[g * CKV_PART_STRIDE + 1] = den; }
+    s_ent[tid] = off;
+  }
+  constexpr int NI = (G * CKV_D + W * 32 - 1) / (W * 32);
+  float num[NI];
+  for (int base = 0;; base += kSlots) {
+    __syncthreads();   // the entries of this round are in place
+    for (int g = warp; g < G; g += W) {   // per head: maximum, scale factor of every entry, normaliser
+      const bool valid = lane < W ? (base == 0 || lane == 0) : (lane < W + kSlots && base + lane - W < my_cnt);
+      const float *p = sf + s_ent[lane < W + kSlots ? lane : 0] + g * CKV_PART_STRIDE;
+      const float m = valid ? p[0] : -CUDART_INF_F, l = valid ? p[1] : 0.f;
+      const float M = warp_max(m);
+      const float sc = exp2_diff(m, M);
+      const float den = warp_sum(l * sc);
+      s_scale[lane][g] = sc;
+      if (lane == 0) { s_M[g] = M; s_den[g] = den; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < NI; ++it) {
+      const int idx = tid + it * W * 32;
+      float a = 0.f;
+      if (idx < G * CKV_D) {
+        const int g = idx / CKV_D, c = idx % CKV_D;
+#pragma unroll 4
+        for (int e = 0; e < W + kSlots; ++e) {
+          const float sc = s_scale[e][g];
+          if (sc != 0.f) a = fmaf(sf[s_ent[e] + g * CKV_PART_STRIDE + 4 + c], sc, a);   // scale 0: empty or absent
+        }
+      }
+      num[it] = a;
+    }
+    if (base + kSlots >= my_cnt) break;
+    // more scan partials than slots (few splits, many scan CTAs): keep the result as entry 0 and go round again
+    __syncthreads();
+    {
+      float *carry = sf + s_ent[0];
+#pragma unroll
+      for (int it = 0; it < NI; ++it) {
+        const int idx = tid + it * W * 32;
+        if (idx < G * CKV_D) carry[(idx / CKV_D) * CKV_PART_STRIDE + 4 + idx % CKV_D] = num[it];
+      }
+      if (tid < G) { carry[tid * CKV_PART_STRIDE] = s_M[tid]; carry[tid * CKV_PART_STRIDE + 1] = s_den[tid]; }
+    }
+    issue_comp(red_buf(warp) ^ 1, base + kSlots);
+    cp_async_commit();
+    cp_async_wait<0>();
+  }
+#pragma unroll
+  for (int it = 0; it < NI; ++it) {
+    const int idx = tid + it * W * 32;
+    if (idx < G * CKV_D) part[(idx / CKV_D) * CKV_PART_STRIDE + 4 + idx % CKV_D] = num[it];
+  }
+  if (tid < G) { part[tid * CKV_PART_STRIDE] = s_M[tid]; part[tid * CKV_PART_STRIDE + 1] = s_den[tid]; }
+
+  // ---- the last split of the unit to finish merges the unit's partials into the output (Eq. 12) ----
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int done = atomicAdd(P.unit_done + unit, 1);
+    s_last = done == n_active - 1;
+    if (s_last) P.unit_done[unit] = 0;   // leave the counter ready for the next step
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float *ap0 = P.attn_part + (size_t)unit * CKV_MAX_SPLITS * G * CKV_PART_STRIDE;
+  const int c4 = 4 * lane;
+  for (int g = warp; g < G; g += W) {   // a warp per head; lane i holds (m, l) of partials i and i + 32, and four coordinates
+    const float *ag = ap0 + (size_t)g * CKV_PART_STRIDE;
+    float2 ml0 = make_float2(-CUDART_INF_F, 0.f), ml1 = make_float2(-CUDART_INF_F, 0.f);
+    if (lane < n_active) ml0 = __ldcg(reinterpret_cast<const float2 *>(ag + (size_t)lane * step));
+    if (lane + 32 < n_active) ml1 = __ldcg(reinterpret_cast<const float2 *>(ag + (size_t)(lane + 32) * step));
+    float4 a[8];   // the first eight partials are requested before the scale factors are known
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      a[k] = k < n_active ? __ldcg(reinterpret_cast<const float4 *>(ag + (size_t)k * step + 4 + c4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    const float M = warp_max(fmaxf(ml0.x, ml1.x));
+    const float sc0 = exp2_diff(ml0.x, M), sc1 = exp2_diff(ml1.x, M);
+    const float den = warp_sum(ml0.y * sc0 + ml1.y * sc1);
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < n_active; i += 8) {
+      if (i > 0) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          a[k] = i + k < n_active ? __ldcg(reinterpret_cast<const float4 *>(ag + (size_t)(i + k) * step + 4 + c4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int ii = i + k;
+        const float sc = __shfl_sync(0xffffffffu, ii < 32 ? sc0 : sc1, ii & 31);
+        if (ii < n_active && sc != 0.f) {
+          o.x = fmaf(a[k].x, sc, o.x); o.y = fmaf(a[k].y, sc, o.y);
+          o.z = fmaf(a[k].z, sc, o.z); o.w = fmaf(a[k].w, sc, o.w);
+        }
+      }
+    }
+    const float inv = 1.0f / den;
+    uint2 o2;
+    o2.x = pack_bf16(o.x * inv, o.y * inv);
+    o2.y = pack_bf16(o.z * inv, o.w * inv);
+    *reinterpret_cast<uint2 *>(out + ((size_t)s * P.Hq + h * G + g) * CKV_D + c4) = o2;
+    if (lse != nullptr && lane == 0) lse[(size_t)s * P.Hq + h * G + g] = (M + log2f(den)) * kLn2;
   }
 }
 
-inline size_t static_smem(int G) { return (size_t)kWarps * G * CKV_PART_STRIDE * 4 + 256; }
-inline size_t dyn_smem(int nbuf) { return (size_t)kWarps * (nbuf * 2 * kTileBytes + kAuxBytes); }
+constexpr int kSparseWarps = 4, kDenseWarps = 8;
 
 template <int G>
 cudaError_t launch_g(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                      const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt, int kcap,
-                     dim3 grid, int pps, cudaStream_t st) {
-  const int nbuf = (dense || pps > kWarps) ? 2 : 1;
-  const size_t smem = dyn_smem(nbuf);
+                     dim3 grid, int pps, int scan_grid, void *out, float *lse, cudaStream_t st) {
+  const int units = (int)grid.y;
   const __nv_bfloat16 *qp = (const __nv_bfloat16 *)q, *kp = (const __nv_bfloat16 *)k_pool, *vp = (const __nv_bfloat16 *)v_pool;
   if (dense)
-    ckv_attn_mma_kernel<G, true><<<grid, kWarps * 32, smem, st>>>(c->dev, qp, kp, vp, page_table, seq_lens, sel_ids,
-                                                                  sel_cnt, kcap, pps, nbuf);
+    ckv_attn_mma_kernel<G, true, kDenseWarps><<<grid, kDenseWarps * 32, dyn_smem<kDenseWarps>(), st>>>(
+        c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
   else
-    ckv_attn_mma_kernel<G, false><<<grid, kWarps * 32, smem, st>>>(c->dev, qp, kp, vp, page_table, seq_lens, sel_ids,
-                                                                   sel_cnt, kcap, pps, nbuf);
+    ckv_attn_mma_kernel<G, false, kSparseWarps><<<grid, kSparseWarps * 32, dyn_smem<kSparseWarps>(), st>>>(
+        c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
   return cudaGetLastError();
 }
 
 template <int G>
 cudaError_t configure_g() {
-  const int smem = (int)dyn_smem(2);
-  cudaError_t e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaError_t e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, true, kDenseWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)dyn_smem<kDenseWarps>());
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)dyn_smem<kSparseWarps>());
   return e;
 }
 
@@ -336,12 +551,12 @@ cudaError_t ckv_configure_attn_mma(const ckv_ctx *c) {
 
 cudaError_t ckv_launch_attn_mma(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                                 const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
-                                int kcap, dim3 grid, int pps, cudaStream_t st) {
+                                int kcap, dim3 grid, int pps, int scan_grid, void *out, float *lse, cudaStream_t st) {
   switch (c->dev.G) {
-    case 1: return launch_g<1>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
-    case 2: return launch_g<2>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
-    case 4: return launch_g<4>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
-    case 8: return launch_g<8>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, st);
+    case 1: return launch_g<1>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, scan_grid, out, lse, st);
+    case 2: return launch_g<2>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, scan_grid, out, lse, st);
+    case 4: return launch_g<4>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, scan_grid, out, lse, st);
+    case 8: return launch_g<8>(c, dense, q, k_pool, v_pool, page_table, seq_lens, sel_ids, sel_cnt, kcap, grid, pps, scan_grid, out, lse, st);
   }
   return cudaErrorInvalidValue;
 }

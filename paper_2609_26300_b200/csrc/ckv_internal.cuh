@@ -34,6 +34,7 @@ struct CkvDev {
   float *scores;     // [unit][max_blocks]     S_b
   float *comp_part;  // [(scan CTA + unit) * CKV_SCAN_WARPS + warp][G][CKV_PART_STRIDE]  all-block mean-compensation partials
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials
+  int *unit_done;    // [unit] attention splits finished this step (zero between steps); null = merge is a separate launch
   int *status;       // device status word
 };
 
@@ -54,7 +55,7 @@ cudaError_t ckv_configure_attn(const ckv_ctx *c);   // attention kernel attribut
 cudaError_t ckv_configure_attn_mma(const ckv_ctx *c);
 cudaError_t ckv_launch_attn_mma(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                                 const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
-                                int kcap, dim3 grid, int pps, cudaStream_t st);
+                                int kcap, dim3 grid, int pps, int scan_grid, void *out, float *lse, cudaStream_t st);
 int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len);
 
 // ---- launchers (one per translation unit) ---------------------------------------------------------
@@ -69,7 +70,8 @@ cudaError_t ckv_launch_select(ckv_ctx *c, const int *seq_lens, int batch, int kc
                               int *sel_cnt, cudaStream_t st);
 cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
                             const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
-                            int kcap, int batch, int max_len, int *n_splits_out, cudaStream_t st);
+                            int kcap, int batch, int max_len, int scan_grid, void *out, float *lse,
+                            int *n_splits_out, bool *merged_out, cudaStream_t st);
 cudaError_t ckv_launch_merge(ckv_ctx *c, bool dense, const int *seq_lens, const int *sel_cnt, int n_splits,
                              int scan_grid, int batch, void *out, float *lse, cudaStream_t st);
 

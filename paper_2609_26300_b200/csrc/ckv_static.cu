@@ -4,7 +4,7 @@
 // of the operation it implements, code running inside a stream capture or under a memory pool that forbids
 // cudaMalloc, a process whose device memory is fully committed to the KV cache.  ckv_dense_decode_static()
 // serves them: it needs no context and no caller-provided scratch.  The split partials the attention kernel
-// produces (and the merge kernel consumes) live in a fixed device array that is part of this library's
+// produces (and its last split merges) live in a fixed device array that is part of this library's
 // image, so every GPU that loads the library holds CKV_STATIC_SCRATCH_BYTES of it until the process exits.
 //
 // Consequences the caller has to know:
@@ -17,13 +17,14 @@
 
 #include "ckv_internal.cuh"
 
-#define CKV_STATIC_SCRATCH_BYTES (4u << 20)   // 4 MiB of split partials + 256 B for the status word
+#define CKV_STATIC_SCRATCH_BYTES (4u << 20)   // 4 MiB of split partials, followed by the words below
+#define CKV_STATIC_TAIL_BYTES 1024            // status word at +0, per-unit split counters at +256 (192 of them)
 
 namespace {
 
 // In host code these names are host-side stand-ins for the device arrays, not device addresses: the address a
 // kernel may use comes from cudaGetSymbolAddress(), once per device.
-static __device__ __align__(256) unsigned char g_static_scratch[CKV_STATIC_SCRATCH_BYTES + 256];
+static __device__ __align__(256) unsigned char g_static_scratch[CKV_STATIC_SCRATCH_BYTES + CKV_STATIC_TAIL_BYTES];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
@@ -58,6 +59,7 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
   // the partials of the largest split count the launch heuristic may pick must fit the fixed array
   const size_t per_split = (size_t)batch * P.Hkv * P.G * CKV_PART_STRIDE * sizeof(float);
   if (per_split * CKV_MAX_SPLITS > CKV_STATIC_SCRATCH_BYTES) return CKV_ERR_CAPACITY;
+  if ((size_t)batch * P.Hkv * sizeof(int) > CKV_STATIC_TAIL_BYTES - 256) return CKV_ERR_CAPACITY;
 
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -77,18 +79,22 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
   unsigned char *scratch = (unsigned char *)g_scratch_ptr[dev];
   P.attn_part = (float *)scratch;
   P.status = (int *)(scratch + CKV_STATIC_SCRATCH_BYTES);
+  P.unit_done = (int *)(scratch + CKV_STATIC_SCRATCH_BYTES + 256);
   c.sm_count = g_sm_count[dev];
 
   cudaStream_t s = (cudaStream_t)stream;
-  // the array keeps whatever the previous call left: the status word must start at zero; every partial the merge
-  // reads is rewritten by this call's attention kernel
-  e = cudaMemsetAsync(P.status, 0, sizeof(int), s);
+  // the array keeps whatever the previous call left: the status word and the split counters must start at zero
+  // (an interrupted call may have left counters behind); every partial that is read is rewritten by this call
+  e = cudaMemsetAsync(P.status, 0, CKV_STATIC_TAIL_BYTES, s);
   if (e != cudaSuccess) return CKV_ERR_CUDA;
   int n_splits = 0;
+  bool merged = false;
   e = ckv_launch_attn(&c, true, q, k_pool, v_pool, page_table, seq_lens, nullptr, nullptr, 0, batch, max_seq_len_host,
-                      &n_splits, s);
+                      0, out, lse, &n_splits, &merged, s);
   if (e != cudaSuccess) return CKV_ERR_CUDA;
-  e = ckv_launch_merge(&c, true, seq_lens, nullptr, n_splits, 0, batch, out, lse, s);
-  if (e != cudaSuccess) return CKV_ERR_CUDA;
+  if (!merged) {   // fp32 pages: the merge is a launch of its own
+    e = ckv_launch_merge(&c, true, seq_lens, nullptr, n_splits, 0, batch, out, lse, s);
+    if (e != cudaSuccess) return CKV_ERR_CUDA;
+  }
   return CKV_OK;
 }
