@@ -42,17 +42,18 @@ constexpr int kRowBytes = CKV_ROW_ELEMS * 2;
 
 struct UnitInfo { int N, X, tiles; };
 
-__device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *__restrict__ seq_lens, int u) {
+// s_len holds the clamped lengths of the first kMaxSeqs sequences (staged once per CTA)
+__device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *s_len, const int *__restrict__ seq_lens, int u) {
   UnitInfo ui;
-  ui.N = max(min(seq_lens[u / P.Hkv], P.max_blocks * P.bs), 0);
+  const int s = u / P.Hkv;
+  ui.N = s < kMaxSeqs ? s_len[s] : max(min(seq_lens[s], P.max_blocks * P.bs), 0);
   ui.X = (ui.N + P.bs - 1) / P.bs;
   ui.tiles = (ui.X + TB - 1) / TB;
   return ui;
 }
 
-__device__ __forceinline__ int seq_tiles(const int *s_tiles, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
-  if (i < kMaxSeqs) return s_tiles[i];
-  const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
+__device__ __forceinline__ int seq_tiles(const int *s_len, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
+  const int n = i < kMaxSeqs ? s_len[i] : max(min(seq_lens[i], P.max_blocks * P.bs), 0);
   return ((n + P.bs - 1) / P.bs + TB - 1) / TB;
 }
 
@@ -66,7 +67,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
   __shared__ int s_u0, s_tl0, s_count, s_ulast, s_abort, s_issued;
-  __shared__ int s_tiles[kMaxSeqs];
+  __shared__ int s_len[kMaxSeqs];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool dbar_bulk = P.r >= 4;   // smaller rows cannot keep the 16-byte alignment bulk copies need
@@ -75,19 +76,19 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
   // per-warp w_{g,t} table for r != 4, behind the ring
   float *sw_all = reinterpret_cast<float *>(stage_mem + (size_t)stages * stage_bytes);
 
+  // the sequence lengths are requested first; the ring is cleared while they are on their way
+  const int batch = units / P.Hkv;
+  const int len_mine = tid < batch ? seq_lens[tid] : 0;
   // rows past a unit's last block are never copied: clear the ring once so that they hold zeros or old summaries,
   // never arbitrary bit patterns (a NaN times a zero weight would poison the accumulators)
   for (int i = tid; i < stages * stage_bytes / 16; i += kThreads) reinterpret_cast<uint4 *>(stage_mem)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async();
-  const int batch = units / P.Hkv;
-  for (int i = tid; i < batch && i < kMaxSeqs; i += kThreads) {
-    const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
-    s_tiles[i] = ((n + P.bs - 1) / P.bs + TB - 1) / TB;
-  }
+  if (tid < batch) s_len[tid] = max(min(len_mine, P.max_blocks * P.bs), 0);
+  for (int i = tid + kThreads; i < batch && i < kMaxSeqs; i += kThreads) s_len[i] = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
   __syncthreads();
   if (tid == 0) {
     long long T = 0;
-    for (int i = 0; i < batch; ++i) T += (long long)seq_tiles(s_tiles, seq_lens, P, i) * P.Hkv;
+    for (int i = 0; i < batch; ++i) T += (long long)seq_tiles(s_len, seq_lens, P, i) * P.Hkv;
     const long long tpc = (T + gridDim.x - 1) / gridDim.x;
     const long long first = (long long)blockIdx.x * tpc;
     long long cnt = T - first;
@@ -98,7 +99,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
       long long accum = 0;
       bool have_first = false;
       for (int i = 0; i < batch; ++i) {
-        const long long t = seq_tiles(s_tiles, seq_lens, P, i);
+        const long long t = seq_tiles(s_len, seq_lens, P, i);
         if (t > 0) {
           if (!have_first && first < accum + t * P.Hkv) {
             const long long off = first - accum;
@@ -126,7 +127,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     if (lane == 0) {
       int u = s_u0, tl = s_tl0, st = 0;
       uint32_t phase = 0;            // parity of the empty-barrier phase the next refill of stage `st` waits for
-      UnitInfo ui = unit_info(P, seq_lens, u);
+      UnitInfo ui = unit_info(P, s_len, seq_lens, u);
       for (int it = 0; it < count; ++it) {
         if (it >= stages && !mbar_wait(&empty_bar[st], phase)) {
           atomicOr(P.status, CKV_DEV_TIMEOUT);
@@ -151,7 +152,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         if (++st == stages) { st = 0; if (it >= stages) phase ^= 1; }
         if (++tl == ui.tiles) {
           tl = 0;
-          do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+          do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
         }
       }
     }
@@ -168,7 +169,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     float log_last = 0.f;
     const int ulast = s_ulast;
     int u = s_u0, tl = s_tl0, cur = -1, next_empty = s_u0;
-    UnitInfo ui = unit_info(P, seq_lens, u);
+    UnitInfo ui = unit_info(P, s_len, seq_lens, u);
     float2 *ls = nullptr;
     const float *db = nullptr;
     bool aborted = false;
@@ -198,7 +199,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     // units of this CTA's range that this warp never worked on still need an (empty) partial
     auto fill_empty_upto = [&](int upto) {
       for (; next_empty < upto; ++next_empty)
-        if (unit_info(P, seq_lens, next_empty).tiles > 0) write_partial(next_empty, false);
+        if (unit_info(P, s_len, seq_lens, next_empty).tiles > 0) write_partial(next_empty, false);
     };
 
     // Half tile j = 2 * tile + half belongs to warp j % W.  A parity wait can only tell a fill of a stage from
@@ -210,7 +211,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     for (int it = 0; it < count; ++it) {
       if (it > 0 && ++tl == ui.tiles) {
         tl = 0;
-        do { ++u; } while (u < units && (ui = unit_info(P, seq_lens, u)).tiles == 0);
+        do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
       }
       const int j0 = (2 * it) % kConsumerWarps;
       const int half = j0 == warp ? 0 : ((j0 + 1) % kConsumerWarps == warp ? 1 : -1);
