@@ -33,9 +33,9 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 PAPER_CONTEXT = {"speedup_vs_full": 6.85, "hardware": "NVIDIA H100 80GB HBM3, CPU-offload pipeline, batch 1",
                  "setting": "128K endpoint, budget 512, r=4 (1.456 ms vs 9.966 ms)", "note": "context only"}
-# DRAM traffic per algorithmic byte of the summary-scan kernel, from the committed ncu capture
-# (profiles/): None until a capture has been summarised.
-SCAN_TRAFFIC_RATIO = None
+# DRAM traffic (reads + writes) per algorithmic byte of the summary-scan kernel, from the committed ncu capture
+# (profiles/ckv_scan_kernel_llama8b_128k_b4.md): 272.84 MB read + 10.04 MB written for 272.9 MB of summaries.
+SCAN_TRAFFIC_RATIO = 1.037
 
 
 def measured_peak():
