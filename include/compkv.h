@@ -157,12 +157,21 @@ int ckv_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_po
                ckv_stream stream);
 
 /* ckv_decode with CUDA events recorded on `stream` between its four kernels (summary scan, score +
- * top-k selection, exact attention on the selected blocks, merge).  Waits for the step to finish and
- * writes the four durations in milliseconds to stage_ms_host[0..3] (host).  For measurement only. */
+ * top-k selection, exact attention on the selected blocks, merge; the bf16 layout merges inside the attention
+ * kernel, its fourth duration is then an empty interval).  Waits for the step to finish and writes the four
+ * durations in milliseconds to stage_ms_host[0..3] (host).  For measurement only. */
 int ckv_decode_profile(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_pool,
                        const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
                        int budget_tokens, void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt,
                        ckv_stream stream, float *stage_ms_host);
+
+/* The summary scan of ckv_decode (Eq. 8-10 logits and the all-block compensation sums of Eq. 12) launched
+ * `reps` times back to back between two CUDA events on `stream`; waits, and writes the average duration of
+ * one launch in milliseconds to *avg_ms_host (host).  The scan only rewrites its own workspace rows, so the
+ * repetitions are idempotent; the summaries of the bench workloads exceed L2, so every launch streams them
+ * from HBM.  For measurement only (the roofline figure of the dominant kernel). */
+int ckv_scan_profile(ckv_ctx *ctx, const void *q, const int32_t *seq_lens, int batch, int max_seq_len_host,
+                     int reps, ckv_stream stream, float *avg_ms_host);
 
 /* Dense decode attention over the whole paged cache (Sec. 3.1; Eq. 12 with S = all blocks),
  * split along the sequence with a log-sum-exp merge.  Same tile code as the sparse path. */

@@ -22,7 +22,7 @@ CKV_ERR_CAPACITY, CKV_ERR_CUDA, CKV_ERR_TIMEOUT = -4, -5, -6
 CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_BAD_COPY = 1, 2, 4, 8, 16
 
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
-           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_decode_profile", "ckv_dense_decode",
+           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
            "ckv_dense_decode_static",
            "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
 
@@ -74,6 +74,7 @@ def load() -> ctypes.CDLL:
     lib.ckv_decode.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.ckv_decode_profile.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp,
                                        ctypes.POINTER(ctypes.c_float)]
+    lib.ckv_scan_profile.argtypes = [vp, vp, vp, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_float)]
     lib.ckv_dense_decode.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     lib.ckv_dense_decode_static.argtypes = [lp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     lib.ckv_dense_decode_static.restype = i32
@@ -83,7 +84,7 @@ def load() -> ctypes.CDLL:
     lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_launch_count.restype = ctypes.c_int64
     for name in ("ckv_query_sizes", "ckv_stats_offsets", "ckv_create", "ckv_stats_build", "ckv_stats_export", "ckv_append",
-                 "ckv_decode", "ckv_decode_profile", "ckv_dense_decode", "ckv_copy_scores", "ckv_step_host", "ckv_read_status"):
+                 "ckv_decode", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode", "ckv_copy_scores", "ckv_step_host", "ckv_read_status"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -221,6 +222,13 @@ class CompKV:
                                            _ptr(seq_lens), batch, int(max_seq_len), int(budget_tokens), _ptr(out),
                                            _ptr(lse), _ptr(ids), _ptr(cnt), _stream(), ms), "ckv_decode_profile")
         return (out, lse, ids, cnt), [float(x) for x in ms]
+
+    def scan_profile(self, q, seq_lens, max_seq_len: int, reps: int) -> float:
+        """ckv_scan_profile: average milliseconds of one summary-scan launch over `reps` back-to-back launches."""
+        ms = ctypes.c_float(0.0)
+        _check(self.lib.ckv_scan_profile(self._ctx, _ptr(q), _ptr(seq_lens), q.shape[0], int(max_seq_len), int(reps),
+                                         _stream(), ctypes.byref(ms)), "ckv_scan_profile")
+        return float(ms.value)
 
     def dense_decode(self, q, k_pool, v_pool, page_table, seq_lens, max_seq_len: int, out=None, lse=None):
         batch = q.shape[0]

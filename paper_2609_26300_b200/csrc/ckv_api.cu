@@ -248,6 +248,32 @@ int ckv_decode_profile(ckv_ctx *c, const void *q, const void *k_pool, const void
   return rc;
 }
 
+int ckv_scan_profile(ckv_ctx *c, const void *q, const int32_t *seq_lens, int batch, int max_seq_len_host, int reps,
+                     ckv_stream stream, float *avg_ms_host) {
+  const int st = check_step_args(c, batch, max_seq_len_host);
+  if (st != CKV_OK) return st;
+  if (!q || !seq_lens || !avg_ms_host || reps <= 0) return CKV_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaEvent_t ev[2] = {nullptr, nullptr};
+  int rc = CKV_OK;
+  for (int i = 0; i < 2 && rc == CKV_OK; ++i)
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  int scan_grid = 0;
+  if (rc == CKV_OK && cudaEventRecord(ev[0], s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  for (int i = 0; i < reps && rc == CKV_OK; ++i) {
+    const cudaError_t e = ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, &scan_grid, s);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+  }
+  if (rc == CKV_OK && cudaEventRecord(ev[1], s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  if (rc == CKV_OK && cudaEventSynchronize(ev[1]) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  float ms = 0.f;
+  if (rc == CKV_OK && cudaEventElapsedTime(&ms, ev[0], ev[1]) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+  if (rc == CKV_OK) *avg_ms_host = ms / (float)reps;
+  for (int i = 0; i < 2; ++i)
+    if (ev[i]) cudaEventDestroy(ev[i]);
+  return rc;
+}
+
 int ckv_dense_decode(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
                      const int32_t *seq_lens, int batch, int max_seq_len_host, void *out, float *lse,
                      ckv_stream stream) {
