@@ -96,9 +96,29 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def workload(total_steps: int):
+def workload(total_steps: int, args=None):
+    """The bench workload: configs[2] of the baseline file (synth.CONFIGS[3]) unless overridden for a sweep point."""
     from paper_2609_26300_b200 import synth
-    return synth.CONFIGS[3].with_(decode_steps=total_steps)
+    w = synth.CONFIGS[getattr(args, "config", 3) if args is not None else 3].with_(decode_steps=total_steps)
+    if args is not None:
+        over = {}
+        if args.block_size:
+            over["block_size"] = args.block_size
+        if args.budget:
+            over["budget_tokens"] = args.budget
+        if args.var_groups:
+            over["var_groups"] = args.var_groups
+        if over:
+            w = w.with_(**over)
+    return w
+
+
+def describe(w, default: bool) -> str:
+    head = "configs[2] " if default else "sweep point of "
+    ctx = "ctx %d" % w.ctx if w.ctx_min is None else "ctx %d..%d (ragged)" % (w.ctx_min, w.ctx)
+    return ("%s%s: batch %d, %dq/%dkv heads, d%d, %s (+ appended tokens), block %d, budget %d, r=%d, "
+            "fp32 summaries, bf16 paged KV" % (head, w.name, w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, ctx,
+                                               w.block_size, w.budget_tokens, w.var_groups))
 
 
 def step_inputs(w, n_steps: int):
@@ -196,6 +216,11 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=48)
     ap.add_argument("--e2e-steps", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    # sweep points (the default line is configs[2]; these leave the metric's workload)
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5], help="synth.CONFIGS index")
+    ap.add_argument("--block-size", type=int, default=0)
+    ap.add_argument("--budget", type=int, default=0)
+    ap.add_argument("--var-groups", type=int, default=0)
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -215,7 +240,8 @@ def main():
 
     W, K, KP, KE = max(args.warmup, 3), args.steps, args.profile_steps, args.e2e_steps
     total = W + K + KP + KE + W + 2 * min(K, 64)
-    w = workload(total)
+    w = workload(total, args)
+    is_default = args.config == 3 and not (args.block_size or args.budget or args.var_groups)
     dev = torch.device("cuda", local)
 
     # ---- inputs: every rank holds a full replica of the workload (the path does not shard) ----
@@ -396,11 +422,10 @@ def main():
     step_gbs = req / (us_per_step * 1e-6) / 1e9
     scan_gbs = stats_b / (scan_us * 1e-6) / 1e9
     line = {
-        "metric": METRIC, "value": us_per_step, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "metric": METRIC if is_default else "sparse decode-attn us/step (append + decode)", "value": us_per_step, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "configs[2] llama8b_128k_b4: batch 4, 32q/8kv heads, d128, ctx 131072 (+ appended "
-                               "tokens), block 16, budget 2048, r=4, fp32 summaries, bf16 paged KV",
+        "config": {"workload": describe(w, is_default),
                    "step": "ckv_append + ckv_decode replayed as one CUDA graph; CUDA events around each replay",
                    "l2": "flushed between steps (256 MiB memset then 256 MiB read, outside the events); per-step inputs exceed L2",
                    "replicas": "every rank runs the whole workload (the path does not shard)",
