@@ -34,7 +34,8 @@ constexpr int kRowBytes = CKV_D * 2;                  // 256
 constexpr int kMeanSlots = 4;                         // mean-value rows (512 B each) a warp can hold
 constexpr int kMeanFlush = 3;                         // ... of which at most 3 wait for removal while one is in flight
 constexpr int kZeroRow = kMeanSlots * 512;            // offset of the row of zeros inside the aux area
-constexpr int kAuxBytes = kZeroRow + 256;
+constexpr int kLsOff = kZeroRow + 256;                // then the blocks' (logit, variance) pairs: [slot][G] float2
+constexpr int kAuxBytes = kLsOff + 256;
 constexpr int kMaxEntries = 32;                       // partials a CTA folds per round: one per lane
 constexpr int kPartBytes = CKV_PART_STRIDE * 4;       // one head's partial
 
@@ -43,6 +44,9 @@ template <int W> constexpr size_t dyn_smem() { return (size_t)W * (2 * kPageByte
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
   // valid == false copies nothing and zero-fills the 16 bytes
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -55,9 +59,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
                     const int *__restrict__ sel_cnt, int kcap, int pages_per_split, int scan_grid, int units,
                     __nv_bfloat16 *__restrict__ out, float *__restrict__ lse) {
   extern __shared__ __align__(128) unsigned char smem[];   // [W warps][2 buffers][K tile | V tile], then [W warps][aux]
-  __shared__ float s_scale[kMaxEntries][G];
   __shared__ float s_M[G], s_den[G];
-  __shared__ int s_ent[kMaxEntries];   // float offset of each entry inside smem
   __shared__ int s_last;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -204,8 +206,11 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         cp_async16(kb + off, k_pool + so, valid);
         cp_async16(vb + off, v_pool + so, valid);
       }
-      if (comp && r.first)   // verbatim: hi halves then lo halves, swizzled by block index
+      if (comp && r.first) {   // verbatim: hi halves then lo halves, swizzled by block index
         cp_async16(aux_u32 + 512 * slot + 16 * lane, vmean + (size_t)r.blk * CKV_ROW_ELEMS + 8 * lane, true);
+        if (lane < G)          // and the block's (logit, variance) of every head, for the weight of its mean term
+          cp_async8(aux_u32 + kLsOff + (slot * G + lane) * 8, ls + (size_t)lane * P.max_blocks + r.blk);
+      }
     }
   };
 
@@ -221,8 +226,8 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
       for (int e = 0; e < 2; ++e) {
         const int j = 2 * qd + e;
         if (j < nb) {
-          const int blk = j == 0 ? bb[0] : (j == 1 ? bb[1] : bb[2]);
-          const float2 v = __ldg(ls + (size_t)head * P.max_blocks + blk);
+          const int slot = j == 0 ? bsl[0] : (j == 1 ? bsl[1] : bsl[2]);
+          const float2 v = *reinterpret_cast<const float2 *>(waux + kLsOff + (slot * G + head) * 8);
           zl[e] = (v.x - 0.5f * v.y) * kLog2e;
         }
       }
@@ -389,6 +394,10 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   };
   auto region = [&](int e, int b) { return (int)(((size_t)e * 2 * kPageBytes + (size_t)b * kPageBytes) / 4); };   // in floats
   float *sf = reinterpret_cast<float *>(smem);
+  // scale factors [entry][G] and entry offsets live in the aux area, which the page loop no longer needs
+  float(*s_scale)[G] = reinterpret_cast<float(*)[G]>(smem + (size_t)W * 2 * kPageBytes);
+  int *s_ent = reinterpret_cast<int *>(smem + (size_t)W * 2 * kPageBytes + kMaxEntries * G * 4);
+  __syncthreads();   // every warp is done with its aux rows
   l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 1);
   l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 2);
   if (hv) {
@@ -423,18 +432,20 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     }
     __syncthreads();
 #pragma unroll
-    for (int it = 0; it < NI; ++it) {
-      const int idx = tid + it * W * 32;
-      float a = 0.f;
-      if (idx < G * CKV_D) {
-        const int g = idx / CKV_D, c = idx % CKV_D;
+    for (int it = 0; it < NI; ++it) num[it] = 0.f;
+    // every entry is read (a slot that holds nothing is multiplied by a zero that replaces its value, not by
+    // its bits), so the loads of all entries are independent and in flight together
 #pragma unroll 4
-        for (int e = 0; e < W + kSlots; ++e) {
-          const float sc = s_scale[e][g];
-          if (sc != 0.f) a = fmaf(sf[s_ent[e] + g * CKV_PART_STRIDE + 4 + c], sc, a);   // scale 0: empty or absent
-        }
+    for (int e = 0; e < W + kSlots; ++e) {
+      const float *ep = sf + s_ent[e] + 4;
+#pragma unroll
+      for (int it = 0; it < NI; ++it) {
+        const int idx = min(tid + it * W * 32, G * CKV_D - 1);
+        const int g = idx / CKV_D, c = idx % CKV_D;
+        const float sc = s_scale[e][g];
+        const float x = ep[g * CKV_PART_STRIDE + c];
+        num[it] = fmaf(sc != 0.f ? x : 0.f, sc, num[it]);
       }
-      num[it] = a;
     }
     if (base + kSlots >= my_cnt) break;
     // more scan partials than slots (few splits, many scan CTAs): keep the result as entry 0 and go round again
