@@ -56,6 +56,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   __shared__ int s_wtot[32];
   __shared__ int s_total, s_digit, s_remaining, s_cfirst, s_ccount, s_ncand;
   __shared__ int s_cand[kThreads];
+  __shared__ uint32_t s_candk[kThreads];   // the candidates' keys, so that the ranking loop reads no key through an id
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = blockIdx.x, s = unit / P.Hkv;
@@ -202,7 +203,12 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
         // rank the bin's blocks by (score descending, id ascending) and mark the first `take`
         for (int b = tid; b < X; b += kThreads) {
           if (mandatory(b)) continue;
-          if ((keys[b] & pmask) == prefix) s_cand[atomicAdd(&s_ncand, 1)] = b;
+          const uint32_t k = keys[b];
+          if ((k & pmask) == prefix) {
+            const int slot = atomicAdd(&s_ncand, 1);
+            s_cand[slot] = b;
+            s_candk[slot] = k;
+          }
         }
         __syncthreads();
         const int nc = s_ncand;
@@ -210,11 +216,12 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
         int myb = -1;
         if (tid < nc) {
           myb = s_cand[tid];
-          const uint32_t mk = keys[myb];
+          const uint32_t mk = s_candk[tid];
           int rank = 0;
+#pragma unroll 8
           for (int j = 0; j < nc; ++j) {
             const int ob = s_cand[j];
-            const uint32_t ok = keys[ob];
+            const uint32_t ok = s_candk[j];
             rank += (ok > mk || (ok == mk && ob < myb)) ? 1 : 0;
           }
           chosen = rank < take;
