@@ -60,7 +60,9 @@ __device__ __forceinline__ int seq_tiles(const int *s_len, const int *__restrict
 template <typename QT> struct QSplit { static constexpr bool value = false; };
 template <> struct QSplit<float> { static constexpr bool value = true; };
 
-template <int G, typename QT>
+// RD: one variance group per coordinate (r = d).  The variance rows then have the mean rows' layout and
+// sigma^2 = sum_i (scale q_i)^2 Dbar_i is a third tensor-core product, with the squared queries as the A operand.
+template <int G, typename QT, bool RD>
 __global__ void __launch_bounds__(kThreads, 1)
 ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_lens, int units, int stages) {
   constexpr bool QS = QSplit<QT>::value;   // fp32 queries are split into hi + lo like the summaries
@@ -161,6 +163,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     const int head = lane >> 2, qd = lane & 3;   // this thread's accumulator row (head) and column pair
     const bool hv = head < G;
     uint32_t qa[8][2], qb[QS ? 8 : 1][2];        // A fragments of the unit's queries (rows 0..7), per 16-coordinate step
+    uint32_t qsh[RD ? 8 : 1][2], qsl[RD ? 8 : 1][2];   // (scale q)^2 as hi and lo halves, same fragment positions
     float acc[16][2];                            // W Vbar accumulator: head `head`, coordinates 8 t + 2 qd + {0, 1}
     float m_ref = -CUDART_INF_F, l_acc = 0.f, lp_acc = 0.f;
     float wown[4] = {0.f, 0.f, 0.f, 0.f};
@@ -240,9 +243,16 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
             const float x0 = hv ? to_float(qrow[c0]) : 0.f, x1 = hv ? to_float(qrow[c0 + 1]) : 0.f;
             qa[ks][hh] = pack_bf16(x0, x1);
             if (QS) qb[QS ? ks : 0][hh] = pack_bf16(x0 - bf16_round(x0), x1 - bf16_round(x1));
+            if (RD) {
+              const float s0 = (x0 * P.scale) * (x0 * P.scale), s1 = (x1 * P.scale) * (x1 * P.scale);
+              qsh[RD ? ks : 0][hh] = pack_bf16(s0, s1);
+              qsl[RD ? ks : 0][hh] = pack_bf16(s0 - bf16_round(s0), s1 - bf16_round(s1));
+            }
           }
         }
-        if (r4) {
+        if (RD) {
+          // nothing to tabulate: the weights are the squared queries held above
+        } else if (r4) {
           // w_{g,t} for this thread's head: every lane of the quad sums all 128 coordinates (once per unit)
           float wsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -316,6 +326,31 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
             z[nt][0] += zlo[nt][0]; z[nt][1] += zlo[nt][1];
           }
         }
+        float sgm[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        if (RD) {   // sigma^2 for the same heads x blocks tile: (qs_hi + qs_lo) (D_hi + D_lo) without the lo lo term
+          float sg2[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+          const uint32_t sdr = sv + TB * kRowBytes;
+          const int lrow = lane & 7, lmat = lane >> 3;
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt) {
+            const int r = rb + nt * 8 + lrow;
+            const uint32_t rowaddr = sdr + r * kRowBytes;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t coff = (uint32_t)swz_chunk(4 * j + lmat, r) * 16;
+              uint32_t dh[4], dl[4];
+              ldmatrix_x4(dh, rowaddr + coff);
+              ldmatrix_x4(dl, rowaddr + 256 + coff);
+              mma_rows8(sgm[nt][0], sgm[nt][1], qsh[RD ? 2 * j : 0][0], qsh[RD ? 2 * j : 0][1], dh[0], dh[1]);
+              mma_rows8(sgm[nt][0], sgm[nt][1], qsh[RD ? 2 * j + 1 : 0][0], qsh[RD ? 2 * j + 1 : 0][1], dh[2], dh[3]);
+              mma_rows8(sg2[nt][0], sg2[nt][1], qsl[RD ? 2 * j : 0][0], qsl[RD ? 2 * j : 0][1], dh[0], dh[1]);
+              mma_rows8(sg2[nt][0], sg2[nt][1], qsl[RD ? 2 * j + 1 : 0][0], qsl[RD ? 2 * j + 1 : 0][1], dh[2], dh[3]);
+              mma_rows8(sg2[nt][0], sg2[nt][1], qsh[RD ? 2 * j : 0][0], qsh[RD ? 2 * j : 0][1], dl[0], dl[1]);
+              mma_rows8(sg2[nt][0], sg2[nt][1], qsh[RD ? 2 * j + 1 : 0][0], qsh[RD ? 2 * j + 1 : 0][1], dl[2], dl[3]);
+            }
+            sgm[nt][0] += sg2[nt][0]; sgm[nt][1] += sg2[nt][1];
+          }
+        }
 
         // ---- per (head, block): variance projection, l, running maximum, compensation weight ----
         float zl2[2][2], sig[2][2], wt[2][2];
@@ -331,7 +366,9 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
             val[nt][e] = hv && r < nb;
             float sg = 0.f;
             if (val[nt][e]) {
-              if (r4) {
+              if (RD) {
+                sg = fmaxf(sgm[nt][e], 0.f);
+              } else if (r4) {
                 const float4 dv = *reinterpret_cast<const float4 *>(sd + r * 4);
                 sg = fmaf(wown[0], dv.x, fmaf(wown[1], dv.y, fmaf(wown[2], dv.z, wown[3] * dv.w)));
               } else {
@@ -417,7 +454,7 @@ struct ScanCfg { int stages; size_t smem; };
 
 ScanCfg scan_cfg(const CkvDev &P, int G) {
   const size_t stage_bytes = (size_t)TB * 2 * kRowBytes + (P.r >= 4 ? (size_t)TB * P.r * 4 : 0);
-  const size_t sw_bytes = P.r == 4 ? 0 : (size_t)kConsumerWarps * P.r * G * 4;
+  const size_t sw_bytes = (P.r == 4 || P.r == CKV_D) ? 0 : (size_t)kConsumerWarps * P.r * G * 4;   // weight table of the generic path
   const size_t budget = 220 * 1024 - 8 * 1024 - sw_bytes;   // static shared memory stays below 8 KB
   int stages = (int)(budget / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
@@ -428,7 +465,10 @@ ScanCfg scan_cfg(const CkvDev &P, int G) {
 template <int G, typename QT>
 cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, cudaStream_t st) {
   const ScanCfg cfg = scan_cfg(c->dev, G);
-  ckv_scan_kernel<G, QT><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+  if (c->dev.r == CKV_D)
+    ckv_scan_kernel<G, QT, true><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+  else
+    ckv_scan_kernel<G, QT, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
   return cudaGetLastError();
 }
 
@@ -440,7 +480,10 @@ cudaError_t launch_g(ckv_ctx *c, const void *q, const int *seq_lens, int units, 
 
 template <int G, typename QT>
 cudaError_t configure_gt(const ckv_ctx *c) {
-  return cudaFuncSetAttribute(ckv_scan_kernel<G, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (c->dev.r == CKV_D)
+    return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)scan_cfg(c->dev, G).smem);
+  return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)scan_cfg(c->dev, G).smem);
 }
 

@@ -66,8 +66,17 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
   for (int i = 0; i < 8; ++i) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], 16);
   if (hw == 0) {
     store_split8(kmean_row, li, b, km);
+    if (P.r == CKV_D) {
+      // one group per coordinate: the variance row has the mean rows' layout (split bf16 pairs, swizzled chunks),
+      // so that the scan can project it with the same tensor-core product as the mean keys
+      float dv[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) sq_smem[8 * li + i] = sq[i];
+      for (int i = 0; i < 8; ++i) dv[i] = sq[i] / fc;
+      store_split8(reinterpret_cast<__nv_bfloat16 *>(dbar_row), li, b, dv);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sq_smem[8 * li + i] = sq[i];
+    }
   } else {
     float vm[8];
 #pragma unroll
@@ -77,11 +86,9 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
   __syncwarp();
   // grouped variance: average of the per-coordinate population variances of each group (Eq. 8)
   const int gs = CKV_D / P.r;
-  for (int t = lane; t < P.r; t += 32) {
+  for (int t = lane; t < P.r && P.r != CKV_D; t += 32) {
     float s = 0.f;
-    if (P.r == CKV_D) {
-      s = sq_smem[t];
-    } else if (P.glayout == 0) {
+    if (P.glayout == 0) {
       for (int i = 0; i < gs; ++i) s += sq_smem[t * gs + i];
     } else {
       const int hg = gs / 2;
@@ -161,7 +168,16 @@ __global__ void __launch_bounds__(256) ckv_stats_export_kernel(CkvDev P, int row
   float *dst = (hw == 0 ? kmean : vmean) + (size_t)row * CKV_D + 8 * li;
   reinterpret_cast<float4 *>(dst)[0] = make_float4(x[0], x[1], x[2], x[3]);
   reinterpret_cast<float4 *>(dst)[1] = make_float4(x[4], x[5], x[6], x[7]);
-  for (int t = lane; t < P.r; t += 32) dbar[(size_t)row * P.r + t] = P.dbar[(size_t)row * P.r + t];
+  if (P.r == CKV_D) {
+    if (hw == 0) {
+      load_split8(reinterpret_cast<const __nv_bfloat16 *>(P.dbar + (size_t)row * CKV_D), li, b, x);
+      float *dd = dbar + (size_t)row * CKV_D + 8 * li;
+      reinterpret_cast<float4 *>(dd)[0] = make_float4(x[0], x[1], x[2], x[3]);
+      reinterpret_cast<float4 *>(dd)[1] = make_float4(x[4], x[5], x[6], x[7]);
+    }
+  } else {
+    for (int t = lane; t < P.r; t += 32) dbar[(size_t)row * P.r + t] = P.dbar[(size_t)row * P.r + t];
+  }
 }
 
 }  // namespace
