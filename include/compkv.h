@@ -70,6 +70,13 @@ enum ckv_device_status {
   CKV_DEV_BAD_COPY = 16     /* a kernel refused to issue a bulk copy whose arguments failed its checks */
 };
 
+/* Bits of ckv_layout.variant: the scorer / merge ablations of Sec. 5.3 and App. A.6.  0 is the method as printed. */
+enum ckv_variant {
+  CKV_VARIANT_FIRST_ORDER_MASS = 1,  /* estimated mass without the sigma^2/2 term of Eq. 9 */
+  CKV_VARIANT_RANK_BY_MASS = 2,      /* S_b = sum_g p_hat (no outer variance factor in Eq. 10) */
+  CKV_VARIANT_DROP = 4               /* unselected blocks are dropped: no mean compensation in Eq. 12 */
+};
+
 typedef struct ckv_layout {
   int32_t num_q_heads;        /* multiple of num_kv_heads; G = ratio in {1, 2, 4, 8} */
   int32_t num_kv_heads;
@@ -86,6 +93,7 @@ typedef struct ckv_layout {
   int32_t sink_blocks;        /* mandatory leading blocks (Sec. 4.2: 1) */
   int32_t recent_blocks;      /* mandatory trailing blocks (Sec. 4.2: 2) */
   float   sm_scale;           /* logit scale; 0 means 1/sqrt(head_dim) (Sec. 3.1) */
+  int32_t variant;            /* OR of ckv_variant bits; 0 = the method as printed */
 } ckv_layout;
 
 /* Library version (major * 100 + minor). */

@@ -15,6 +15,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libcompkv.so")
 
+VARIANT_FIRST_ORDER_MASS, VARIANT_RANK_BY_MASS, VARIANT_DROP = 1, 2, 4
 CKV_BF16, CKV_F32 = 0, 1
 CKV_OK = 0
 CKV_ERR_INVALID_ARG, CKV_ERR_BAD_LAYOUT, CKV_ERR_BUDGET_TOO_SMALL = -1, -2, -3
@@ -32,7 +33,8 @@ class ckv_layout(ctypes.Structure):
                 ("block_size", ctypes.c_int32), ("page_size", ctypes.c_int32), ("var_groups", ctypes.c_int32),
                 ("group_layout", ctypes.c_int32), ("kv_dtype", ctypes.c_int32), ("max_batch", ctypes.c_int32),
                 ("max_blocks_per_seq", ctypes.c_int32), ("num_pages", ctypes.c_int32),
-                ("sink_blocks", ctypes.c_int32), ("recent_blocks", ctypes.c_int32), ("sm_scale", ctypes.c_float)]
+                ("sink_blocks", ctypes.c_int32), ("recent_blocks", ctypes.c_int32), ("sm_scale", ctypes.c_float),
+                ("variant", ctypes.c_int32)]
 
 
 class CompKVError(RuntimeError):
@@ -146,11 +148,11 @@ class CompKV:
     def __init__(self, num_q_heads: int, num_kv_heads: int, max_batch: int, max_blocks_per_seq: int, num_pages: int,
                  block_size: int = 16, var_groups: int = 4, group_layout: int = 1, kv_dtype: int = CKV_BF16,
                  sink_blocks: int = 1, recent_blocks: int = 2, sm_scale: float = 0.0, head_dim: int = 128,
-                 page_size: int = 16, device: str = "cuda"):
+                 page_size: int = 16, device: str = "cuda", variant: int = 0):
         self.lib = load()
         self.layout = ckv_layout(num_q_heads, num_kv_heads, head_dim, block_size, page_size, var_groups,
                                  group_layout, kv_dtype, max_batch, max_blocks_per_seq, num_pages, sink_blocks,
-                                 recent_blocks, sm_scale)
+                                 recent_blocks, sm_scale, variant)
         self.stats_bytes, self.work_bytes = query_sizes(self.layout)
         self.device = torch.device(device)
         self.stats = torch.zeros(self.stats_bytes, dtype=torch.uint8, device=self.device)

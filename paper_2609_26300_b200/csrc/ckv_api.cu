@@ -27,6 +27,7 @@ int check_layout(const ckv_layout *L) {
   if ((long long)L->max_batch * L->num_kv_heads > 65535) return CKV_ERR_BAD_LAYOUT;   // grid.y
   if (L->sink_blocks < 0 || L->recent_blocks < 0) return CKV_ERR_BAD_LAYOUT;
   if (!(L->sm_scale >= 0.f) || !isfinite(L->sm_scale)) return CKV_ERR_BAD_LAYOUT;
+  if (L->variant & ~(CKV_VARIANT_FIRST_ORDER_MASS | CKV_VARIANT_RANK_BY_MASS | CKV_VARIANT_DROP)) return CKV_ERR_BAD_LAYOUT;
   return CKV_OK;
 }
 
@@ -143,6 +144,8 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.max_blocks = layout->max_blocks_per_seq; P.max_pages_per_seq = P.max_blocks * P.ppb;
   P.num_pages = layout->num_pages; P.sink = layout->sink_blocks; P.recent = layout->recent_blocks;
   P.scale = c->layout.sm_scale;
+  P.variant = layout->variant;
+  P.half_var = (layout->variant & CKV_VARIANT_FIRST_ORDER_MASS) ? 0.f : 0.5f;
   P.kmean = (__nv_bfloat16 *)(sb + R.kmean); P.dbar = (float *)(sb + R.dbar); P.vmean = (__nv_bfloat16 *)(sb + R.vmean);
   P.status = (int *)(wb + R.status); P.unit_done = (int *)(wb + R.done);
   P.ls = (float2 *)(wb + R.ls); P.scores = (float *)(wb + R.scores);

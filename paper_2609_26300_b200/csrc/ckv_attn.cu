@@ -48,7 +48,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
   const int X = (N + P.bs - 1) / P.bs;
   const int nsel = DENSE ? X : min(sel_cnt[unit], kcap);
   const int total = DENSE ? (N + CKV_PAGE - 1) / CKV_PAGE : nsel * P.ppb;
-  const bool comp = !DENSE && nsel < X;
+  const bool comp = !DENSE && nsel < X && !(P.variant & CKV_VARIANT_DROP);
   const int p0 = blockIdx.x * pages_per_split;
   const int p1 = min(p0 + pages_per_split, total);
   float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
@@ -222,7 +222,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           const float2 v = __ldg(ls + (size_t)g * P.max_blocks + blk);
-          zl2[g] = (v.x - 0.5f * v.y) * kLog2e;
+          zl2[g] = (v.x - P.half_var * v.y) * kLog2e;
           raise |= zl2[g] > m_ref[g] + CKV_RESCALE_SLACK;
         }
         if (raise) {   // warp-uniform: every lane evaluates the same values
@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(CKV_D *kMergeGroups) ckv_merge_kernel(CkvDev P
   const int G = P.G, unit = s * P.Hkv + hq / G, g = hq % G;
   const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
   const int X = (N + P.bs - 1) / P.bs;
-  const bool comp = !dense && sel_cnt[unit] < X;
+  const bool comp = !dense && sel_cnt[unit] < X && !(P.variant & CKV_VARIANT_DROP);
   if (tid < 32) {
     int cfirst = 0, ccount = 0;
     if (comp) unit_scan_slots(P, seq_lens, units, unit, scan_grid, tid, cfirst, ccount);

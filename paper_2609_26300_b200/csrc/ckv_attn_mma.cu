@@ -96,7 +96,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   const int X = (N + P.bs - 1) / P.bs;
   const int nsel = DENSE ? X : min(cnt_raw, kcap);
   const int total = DENSE ? (N + CKV_PAGE - 1) / CKV_PAGE : nsel * P.ppb;
-  const bool comp = !DENSE && nsel < X;
+  const bool comp = !DENSE && nsel < X && !(P.variant & CKV_VARIANT_DROP);
   const int p1 = min(p0 + pages_per_split, total);
   float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
   if (p0 >= total) {   // no pages for this split: it takes no part in the unit's merge
@@ -228,7 +228,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         if (j < nb) {
           const int slot = j == 0 ? bsl[0] : (j == 1 ? bsl[1] : bsl[2]);
           const float2 v = *reinterpret_cast<const float2 *>(waux + kLsOff + (slot * G + head) * 8);
-          zl[e] = (v.x - 0.5f * v.y) * kLog2e;
+          zl[e] = (v.x - P.half_var * v.y) * kLog2e;
         }
       }
     }

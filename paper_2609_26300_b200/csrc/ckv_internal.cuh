@@ -34,6 +34,8 @@ struct CkvDev {
   float *scores;     // [unit][max_blocks]     S_b
   float *comp_part;  // [(scan CTA + unit) * CKV_SCAN_WARPS + warp][G][CKV_PART_STRIDE]  all-block mean-compensation partials
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials
+  int variant;       // ckv_variant bits
+  float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
   int *unit_done;    // [unit] attention splits finished this step (zero between steps); null = merge is a separate launch
   int *status;       // device status word
 };

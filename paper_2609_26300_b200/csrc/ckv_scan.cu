@@ -381,7 +381,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
             sig[nt][e] = sg;
             const float zbar = z[nt][e] * P.scale;
             const float logc = (b == ui.X - 1) ? log_last : log_bs;
-            ell[e] = logc + zbar + 0.5f * sg;
+            ell[e] = logc + zbar + P.half_var * sg;
             zl2[nt][e] = val[nt][e] ? (zbar + logc) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
             tmax = fmaxf(tmax, zl2[nt][e]);
           }
@@ -406,7 +406,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
           for (int e = 0; e < 2; ++e) {
             wt[nt][e] = val[nt][e] ? fast_exp2(zl2[nt][e] - m_ref) : 0.f;
             l_acc += wt[nt][e];
-            lp_acc = fmaf(wt[nt][e], fast_exp2(0.5f * kLog2e * sig[nt][e]), lp_acc);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
+            lp_acc = fmaf(wt[nt][e], fast_exp2(P.half_var * kLog2e * sig[nt][e]), lp_acc);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
           }
           wh[nt] = pack_bf16(wt[nt][0], wt[nt][1]);
           wl[nt] = pack_bf16(wt[nt][0] - bf16_round(wt[nt][0]), wt[nt][1] - bf16_round(wt[nt][1]));

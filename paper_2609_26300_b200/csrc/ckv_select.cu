@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
 #pragma unroll
   for (int g = 0; g < G; ++g) { Mg[g] = s_M[g]; iL[g] = s_invL[g]; }
   const bool cached = X <= kSmemKeys;
+  const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;   // ablation: rank by estimated mass alone
   bool nonfinite = false;
   for (int base = 0; base < X; base += NB * kThreads) {
     if (base > 0) load_batch(base);
@@ -132,7 +133,8 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
       if (b < X) {
         float sc = 0.f;
 #pragma unroll
-        for (int g = 0; g < G; ++g) sc = fmaf(fast_exp2(fmaf(v[j][g].x, kLog2e, -Mg[g])) * iL[g], v[j][g].y, sc);
+        for (int g = 0; g < G; ++g)
+          sc = fmaf(fast_exp2(fmaf(v[j][g].x, kLog2e, -Mg[g])) * iL[g], by_mass ? 1.0f : v[j][g].y, sc);
         if (!(sc >= 0.f) || sc > 3.0e38f) { nonfinite = true; sc = 0.f; }
         scores[b] = sc;
         if (cached) skeys[b] = __float_as_uint(sc);

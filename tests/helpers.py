@@ -33,7 +33,7 @@ class Device:
 
 def setup(w: synth.Workload, kv_dtype: torch.dtype = torch.bfloat16, poison_tail: bool = True,
           var_groups: Optional[int] = None, group_layout: int = 1, sink: int = 1, recent: int = 2,
-          sm_scale: float = 0.0) -> Device:
+          sm_scale: float = 0.0, variant: int = 0) -> Device:
     from paper_2609_26300_b200 import binding
     k_pool, v_pool, table, lens = synth.make_pools(w, dtype=kv_dtype)
     if poison_tail and w.decode_steps > 0:
@@ -51,7 +51,7 @@ def setup(w: synth.Workload, kv_dtype: torch.dtype = torch.bfloat16, poison_tail
                          num_pages=k_pool.shape[0], block_size=w.block_size,
                          var_groups=var_groups or w.var_groups, group_layout=group_layout,
                          kv_dtype=binding.CKV_BF16 if kv_dtype == torch.bfloat16 else binding.CKV_F32,
-                         sink_blocks=sink, recent_blocks=recent, sm_scale=sm_scale)
+                         sink_blocks=sink, recent_blocks=recent, sm_scale=sm_scale, variant=variant)
     return Device(w, ckv, k_pool.to(dev), v_pool.to(dev), table.to(dev), lens.to(dev),
                   int(lens.max()), kv_dtype)
 
@@ -117,13 +117,16 @@ def check_ids(gpu_ids: Sequence[int], ref_ids: Sequence[int], S: np.ndarray, K: 
 
 def check_unit_decode(d: Device, s: int, h: int, n: int, step: int, budget: int, out, lse, ids, cnt,
                       scores=None, var_groups: Optional[int] = None, group_layout: int = 1, sink: int = 1,
-                      recent: int = 2, scale: Optional[float] = None) -> Dict[str, float]:
-    """Compare one unit of a finished ckv_decode with the oracle on the same inputs."""
+                      recent: int = 2, scale: Optional[float] = None, variant: int = 0) -> Dict[str, float]:
+    """Compare one unit of a finished ckv_decode with the oracle on the same inputs.
+
+    variant: the ablation bits the context was created with (1: first-order mass, 2: rank by mass, 4: drop);
+    the oracle is run with the matching switches."""
     w = d.w
     G = w.group
     q, K, V = unit_inputs(w, s, h, n, step)
     st = O.stats(K, V, w.block_size, var_groups or w.var_groups, group_layout)
-    sc = O.scores(q, st, scale)
+    sc = O.scores(q, st, scale, mass_order=1 if variant & 1 else 2, outer_var=0 if variant & 2 else 1)
     kblocks = budget // w.block_size
     ref_ids = O.select(sc.S, kblocks, sink, recent)
     nsel = int(cnt[s, h])
@@ -134,7 +137,7 @@ def check_unit_decode(d: Device, s: int, h: int, n: int, step: int, budget: int,
         check_scores(scores[s, h].double().cpu().numpy(), sc)
     same = check_ids(gpu_ids, ref_ids, sc.S, kblocks, sink, recent)
     # when the sets differ only by near ties, the output is checked against the oracle on the GPU's ids
-    ref_out, ref_lse = O.sparse(q, K, V, st, ref_ids if same else gpu_ids, scale)
+    ref_out, ref_lse = O.sparse(q, K, V, st, ref_ids if same else gpu_ids, scale, drop=bool(variant & 4))
     got = out[s, h * G:(h + 1) * G].double().cpu().numpy()
     err = rel_inf(got, ref_out)
     assert err <= OUT_TOL[d.dtype], "output error %.3g" % err

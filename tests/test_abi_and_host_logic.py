@@ -62,7 +62,8 @@ def test_sizes_follow_the_summary_layout():
 @pytest.mark.parametrize("bad", [dict(num_q_heads=24), dict(head_dim=64), dict(block_size=48), dict(page_size=32),
                                  dict(var_groups=3), dict(var_groups=96), dict(group_layout=2), dict(kv_dtype=5),
                                  dict(max_batch=0), dict(num_pages=0), dict(sink_blocks=-1),
-                                 dict(sm_scale=float("nan")), dict(max_blocks_per_seq=0)])
+                                 dict(sm_scale=float("nan")), dict(max_blocks_per_seq=0), dict(variant=8),
+                                 dict(variant=-1)])
 def test_bad_layouts_are_rejected(bad):
     with pytest.raises(binding.CompKVError) as e:
         binding.query_sizes(layout(**bad))
@@ -70,7 +71,8 @@ def test_bad_layouts_are_rejected(bad):
 
 
 @pytest.mark.parametrize("ok", [dict(var_groups=1), dict(var_groups=64), dict(var_groups=128), dict(block_size=64),
-                                dict(num_q_heads=64), dict(num_q_heads=8), dict(kv_dtype=binding.CKV_F32)])
+                                dict(num_q_heads=64), dict(num_q_heads=8), dict(kv_dtype=binding.CKV_F32),
+                                dict(variant=7), dict(variant=binding.VARIANT_DROP)])
 def test_good_layouts_are_accepted(ok):
     stats, work = binding.query_sizes(layout(**ok))
     assert stats > 0 and work > 0

@@ -107,6 +107,18 @@ def test_decode_small_block_sizes_and_groups(bs, budget, r, layout):
                           group_layout=layout)
 
 
+@pytest.mark.parametrize("variant", [1, 2, 4, 3, 7])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_decode_scorer_and_merge_ablations(variant, dtype):
+    """The ablations of Sec. 5.3 / App. A.6 as layout flags: first-order mass, ranking by mass alone, Drop."""
+    w = small(block_size=16, budget_tokens=16 * 12, ctx=16 * 70 + 5)
+    d = setup(w, dtype, variant=variant)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, int(d.lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores, variant=variant)
+
+
 def test_decode_toy_config_fp32_and_bf16():
     for dtype in (torch.float32, torch.bfloat16):
         d = setup(TOY, dtype)
