@@ -77,21 +77,6 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     const int i = p0 + warp + W * lane;
     if (i < kcap * P.ppb) blk0 = sel_ids[(size_t)unit * kcap + (i >> pshift)];
   }
-  // Q fragments: A operand rows 0..7 = heads, scaled logits come out of the products in log2 units
-  uint32_t qa[8][2];
-  {
-    const __nv_bfloat16 *qrow = q + ((size_t)s * P.Hq + h * G + (hv ? head : 0)) * CKV_D;
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks)
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const uint32_t v = __ldg(reinterpret_cast<const uint32_t *>(qrow + 16 * ks + 8 * hh + 2 * qd));
-        qa[ks][hh] = hv ? v : 0u;
-      }
-  }
-  int cfirst = 0, ccount = 0;   // where the unit's scan partials sit
-  if (!DENSE) unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
-
   const int N = max(min(n_raw, P.max_blocks * P.bs), 0);
   const int X = (N + P.bs - 1) / P.bs;
   const int nsel = DENSE ? X : min(cnt_raw, kcap);
@@ -131,10 +116,9 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   constexpr int kSlotsPerWarp = (kPageBytes / (G * kPartBytes)) < ((kMaxEntries - W) / W) ? (kPageBytes / (G * kPartBytes))
                                                                                        : ((kMaxEntries - W) / W);
   constexpr int kSlots = W * kSlotsPerWarp;
-  const int n_comp = comp ? ccount * CKV_SCAN_WARPS : 0;
-  const int my_cnt = n_comp > (int)blockIdx.x ? (n_comp - (int)blockIdx.x + n_active - 1) / n_active : 0;
+  int my_cnt = 0;               // scan partials this CTA folds in; known once the scan slots are (below)
+  const float *cp0 = nullptr;
   const size_t step = (size_t)G * CKV_PART_STRIDE;
-  const float *cp0 = P.comp_part + (size_t)(cfirst + unit) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE;
   // start the copies of this warp's share of the round that begins at `base` into its buffer `bufsel`
   auto issue_comp = [&](int bufsel, int base) {
 #pragma unroll
@@ -285,9 +269,31 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     cur = fetch(0);
     cur_slot = take_slot(cur);
     issue(cur, 0, cur_slot);
-  } else {
-    issue_comp(1, 0);   // a warp without pages only brings in its share of the scan partials
   }
+  // Everything the first page copy does not need is requested behind it: the queries (first used by the first
+  // product) and the place of the unit's scan partials (first used with the last page).
+  // Q fragments: A operand rows 0..7 = heads, scaled logits come out of the products in log2 units
+  uint32_t qa[8][2];
+  {
+    const __nv_bfloat16 *qrow = q + ((size_t)s * P.Hq + h * G + (hv ? head : 0)) * CKV_D;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        // rows G..7 repeat head 0: finite values whose products are never used (their weights are zero), and a
+        // load that nothing has to look at before the first product
+        qa[ks][hh] = __ldg(reinterpret_cast<const uint32_t *>(qrow + 16 * ks + 8 * hh + 2 * qd));
+      }
+  }
+  if (comp) {
+    int cfirst = 0, ccount = 0;   // where the unit's scan partials sit
+    unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
+    const int n_comp = ccount * CKV_SCAN_WARPS;
+    my_cnt = n_comp > (int)blockIdx.x ? (n_comp - (int)blockIdx.x + n_active - 1) / n_active : 0;
+    cp0 = P.comp_part + (size_t)(cfirst + unit) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE;
+  }
+
+  if (n_mine == 0) issue_comp(1, 0);   // a warp without pages only brings in its share of the scan partials
   cp_async_commit();
   for (int n = 0, buf = 0; n < n_mine; ++n, buf ^= 1) {
     PageRef nxt{-1, 0, -1, false};
