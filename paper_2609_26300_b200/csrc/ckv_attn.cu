@@ -467,7 +467,7 @@ cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k
   // Splits per unit: the selected list is short, so the tensor-core kernel gets one wave of three CTAs per SM; the
   // dense pass (and the fp32 kernel) about four CTAs per SM overall.  At least eight pages per split, at most
   // CKV_MAX_SPLITS splits.
-  int n_splits = (mma && !dense) ? max(1, 3 * sms / units) : (sms * 4 + units - 1) / units;
+  int n_splits = (mma && !dense) ? max(1, min(3 * sms / units, 8)) : (sms * 4 + units - 1) / units;   // 16: one cluster
   n_splits = max(1, min(n_splits, min(CKV_MAX_SPLITS, (total + 7) / 8)));
   int pps = (total + n_splits - 1) / n_splits;
   if (!(mma && !dense)) pps = (pps + 7) / 8 * 8;   // the tensor-core kernel deals pages to its warps one by one

@@ -51,8 +51,32 @@ __device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int G, bool DENSE, int W>
-__global__ void __launch_bounds__(W * 32, DENSE ? 1 : 3)
+// Thread-block cluster helpers: the splits of a unit are launched as one cluster (CL) when the device can place
+// it, and then exchange their partials through distributed shared memory instead of global memory.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_map(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+
+template <int G, bool DENSE, int W, bool CL>
+__global__ void __launch_bounds__(W * 32, DENSE ? 1 : (W <= 4 ? 3 : 2))
 ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_pool,
                     const __nv_bfloat16 *__restrict__ v_pool, const int *__restrict__ page_table,
                     const int *__restrict__ seq_lens, const int *__restrict__ sel_ids,
@@ -84,11 +108,53 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   const bool comp = !DENSE && nsel < X && !(P.variant & CKV_VARIANT_DROP);
   const int p1 = min(p0 + pages_per_split, total);
   float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
-  if (p0 >= total) {   // no pages for this split: it takes no part in the unit's merge
-    if (total == 0 && blockIdx.x == 0) {   // an empty unit: its output is defined as zero
-      for (int idx = tid; idx < G * CKV_D; idx += W * 32)
-        out[((size_t)s * P.Hq + h * G) * CKV_D + idx] = __float2bfloat16_rn(0.f);
-      if (lse != nullptr && tid < G) lse[(size_t)s * P.Hq + h * G + tid] = -CUDART_INF_F;
+  // Cluster merge: every CTA of the cluster (= every split of the unit) has put its partial [G][CKV_PART_STRIDE] at the
+  // start of its dynamic shared memory; CTA r reduces head r, r + cluster size, ... over all of them and writes the
+  // output rows.  Both cluster barriers are reached by every CTA of the cluster, with or without pages.
+  auto cluster_merge = [&]() {
+    cluster_sync_all();   // all partials are in place
+    const uint32_t rank = cluster_rank(), csize = cluster_size();
+    const uint32_t res0 = (uint32_t)__cvta_generic_to_shared(smem);
+    for (int g = (int)rank; g < G; g += (int)csize) {
+      float2 ml = make_float2(-CUDART_INF_F, 0.f);
+      if (lane < (int)csize) ml = ld_cluster_f32x2(cluster_map(res0 + g * kPartBytes, lane));
+      const float M = warp_max(ml.x);
+      const float sc = exp2_diff(ml.x, M);
+      const float den = warp_sum(ml.y * sc);
+      for (int c = tid; c < CKV_D; c += W * 32) {
+        float o = 0.f;
+        const uint32_t mine = res0 + g * kPartBytes + (4 + c) * 4;
+        for (uint32_t e0 = 0; e0 < csize; e0 += 8) {   // eight remote loads in flight
+          float x[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) x[k] = e0 + k < csize ? ld_cluster_f32(cluster_map(mine, e0 + k)) : 0.f;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float sce = __shfl_sync(0xffffffffu, sc, (e0 + k) & 31);
+            if (e0 + k < csize && sce != 0.f) o = fmaf(x[k], sce, o);
+          }
+        }
+        out[((size_t)s * P.Hq + h * G + g) * CKV_D + c] = __float2bfloat16_rn(o / den);
+      }
+      if (lse != nullptr && tid == 0) lse[(size_t)s * P.Hq + h * G + g] = (M + log2f(den)) * kLn2;
+    }
+    cluster_sync_all();   // no CTA leaves while its shared memory may still be read
+  };
+  if (p0 >= total) {   // no pages for this split
+    if (total == 0) {    // an empty unit (the same for every split of it): its output is defined as zero
+      if (blockIdx.x == 0) {
+        for (int idx = tid; idx < G * CKV_D; idx += W * 32)
+          out[((size_t)s * P.Hq + h * G) * CKV_D + idx] = __float2bfloat16_rn(0.f);
+        if (lse != nullptr && tid < G) lse[(size_t)s * P.Hq + h * G + tid] = -CUDART_INF_F;
+      }
+      return;
+    }
+    if (CL) {   // it still takes part in the cluster's merge, with an empty partial
+      if (tid < G) {
+        reinterpret_cast<float *>(smem)[tid * CKV_PART_STRIDE] = -CUDART_INF_F;
+        reinterpret_cast<float *>(smem)[tid * CKV_PART_STRIDE + 1] = 0.f;
+      }
+      cluster_merge();
     }
     return;
   }
@@ -469,6 +535,17 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     cp_async_commit();
     cp_async_wait<0>();
   }
+  if (CL) {
+    __syncthreads();   // every entry has been read: the CTA's partial takes the start of the shared memory
+#pragma unroll
+    for (int it = 0; it < NI; ++it) {
+      const int idx = tid + it * W * 32;
+      if (idx < G * CKV_D) sf[(idx / CKV_D) * CKV_PART_STRIDE + 4 + idx % CKV_D] = num[it];
+    }
+    if (tid < G) { sf[tid * CKV_PART_STRIDE] = s_M[tid]; sf[tid * CKV_PART_STRIDE + 1] = s_den[tid]; }
+    cluster_merge();
+    return;
+  }
 #pragma unroll
   for (int it = 0; it < NI; ++it) {
     const int idx = tid + it * W * 32;
@@ -528,6 +605,29 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
 }
 
 constexpr int kSparseWarps = 4, kDenseWarps = 8;
+constexpr int kMaxCluster = 16;   // splits of a unit that can be one cluster (8 is portable, 16 needs an opt-in)
+
+// Whether `n_splits` sparse CTAs of this instantiation can be placed as one cluster on the current device.
+template <int G>
+bool cluster_fits(int n_splits, cudaStream_t st) {
+  if (n_splits > kMaxCluster) return false;
+  static int cache[kMaxCluster + 1];   // 0 unknown, 1 fits, 2 does not (per G: the template instantiates one array each)
+  if (cache[n_splits] != 0) return cache[n_splits] == 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_splits, 1, 1);
+  cfg.blockDim = dim3(kSparseWarps * 32);
+  cfg.dynamicSmemBytes = dyn_smem<kSparseWarps>();
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = n_splits; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int n = 0;
+  const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, ckv_attn_mma_kernel<G, false, kSparseWarps, true>, &cfg);
+  if (e != cudaSuccess) (void)cudaGetLastError();
+  cache[n_splits] = (e == cudaSuccess && n > 0) ? 1 : 2;
+  return cache[n_splits] == 1;
+}
 
 template <int G>
 cudaError_t launch_g(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
@@ -535,22 +635,42 @@ cudaError_t launch_g(ckv_ctx *c, bool dense, const void *q, const void *k_pool, 
                      dim3 grid, int pps, int scan_grid, void *out, float *lse, cudaStream_t st) {
   const int units = (int)grid.y;
   const __nv_bfloat16 *qp = (const __nv_bfloat16 *)q, *kp = (const __nv_bfloat16 *)k_pool, *vp = (const __nv_bfloat16 *)v_pool;
-  if (dense)
-    ckv_attn_mma_kernel<G, true, kDenseWarps><<<grid, kDenseWarps * 32, dyn_smem<kDenseWarps>(), st>>>(
+  if (dense) {
+    ckv_attn_mma_kernel<G, true, kDenseWarps, false><<<grid, kDenseWarps * 32, dyn_smem<kDenseWarps>(), st>>>(
         c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
-  else
-    ckv_attn_mma_kernel<G, false, kSparseWarps><<<grid, kSparseWarps * 32, dyn_smem<kSparseWarps>(), st>>>(
-        c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
+    return cudaGetLastError();
+  }
+  if (cluster_fits<G>((int)grid.x, st)) {   // the unit's splits as one cluster: partials never leave the SMs
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kSparseWarps * 32);
+    cfg.dynamicSmemBytes = dyn_smem<kSparseWarps>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = grid.x; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, ckv_attn_mma_kernel<G, false, kSparseWarps, true>, c->dev, qp, kp, vp, page_table,
+                              seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
+  }
+  ckv_attn_mma_kernel<G, false, kSparseWarps, false><<<grid, kSparseWarps * 32, dyn_smem<kSparseWarps>(), st>>>(
+      c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
   return cudaGetLastError();
 }
 
 template <int G>
 cudaError_t configure_g() {
-  cudaError_t e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, true, kDenseWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)dyn_smem<kDenseWarps>());
+  cudaError_t e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, true, kDenseWarps, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem<kDenseWarps>());
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)dyn_smem<kSparseWarps>());
+    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, false>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem<kSparseWarps>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, true>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem<kSparseWarps>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, true>,
+                             cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   return e;
 }
 
