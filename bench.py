@@ -289,8 +289,7 @@ def main():
     step = 0
 
     def eager_step(t):
-        ckv.append(k_pool, v_pool, table, lens, kn_all[t], vn_all[t])
-        ckv.decode(q_all[t], k_pool, v_pool, table, lens, max_len, w.budget_tokens, outputs)
+        ckv.step(q_all[t], kn_all[t], vn_all[t], k_pool, v_pool, table, lens, max_len, w.budget_tokens, outputs)
 
     for _ in range(W):           # untimed eager warm-up (also pages in the kernels before capture)
         eager_step(step); step += 1
@@ -299,8 +298,7 @@ def main():
     graph = torch.cuda.CUDAGraph()
     sq.copy_(q_all[step]); sk.copy_(kn_all[step]); sv.copy_(vn_all[step])
     with torch.cuda.graph(graph):
-        ckv.append(k_pool, v_pool, table, lens, sk, sv)
-        ckv.decode(sq, k_pool, v_pool, table, lens, max_len, w.budget_tokens, outputs)
+        ckv.step(sq, sk, sv, k_pool, v_pool, table, lens, max_len, w.budget_tokens, outputs)
     launches_per_step = ckv.launch_count() - launches0
     # capture does not execute: seq_lens is unchanged, the captured step runs on replay
 
@@ -426,7 +424,7 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": describe(w, is_default),
-                   "step": "ckv_append + ckv_decode replayed as one CUDA graph; CUDA events around each replay",
+                   "step": "ckv_step (append, summary scan, select, attention + merge: four launches) replayed as one CUDA graph; CUDA events around each replay",
                    "l2": "flushed between steps (256 MiB memset then 256 MiB read, outside the events); per-step inputs exceed L2",
                    "replicas": "every rank runs the whole workload (the path does not shard)",
                    "kv_storage": "bf16", "seed": w.seed},

@@ -164,6 +164,14 @@ int ckv_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_po
                int budget_tokens, void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt,
                ckv_stream stream);
 
+/* One decode step in one call: ckv_append(k_new, v_new) followed by ckv_decode(q, ...), with the same arguments,
+ * results and errors as the two calls in that order (Sec. 4.3: the new token enters the cache and the summaries
+ * before blocks are selected; seq_lens holds N on entry and N + 1 once the step has run; max_seq_len_host bounds the
+ * lengths after the append).  The decode arguments are validated before anything is appended. */
+int ckv_step(ckv_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k_pool, void *v_pool,
+             const int32_t *page_table, int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens,
+             void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt, ckv_stream stream);
+
 /* ckv_decode with CUDA events recorded on `stream` between its four kernels (summary scan, score +
  * top-k selection, exact attention on the selected blocks, merge; the bf16 layout merges inside the attention
  * kernel, its fourth duration is then an empty interval).  Waits for the step to finish and writes the four

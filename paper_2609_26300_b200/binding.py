@@ -23,7 +23,7 @@ CKV_ERR_CAPACITY, CKV_ERR_CUDA, CKV_ERR_TIMEOUT = -4, -5, -6
 CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_BAD_COPY = 1, 2, 4, 8, 16
 
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
-           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
+           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
            "ckv_dense_decode_static",
            "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
 
@@ -74,6 +74,7 @@ def load() -> ctypes.CDLL:
     lib.ckv_stats_export.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.ckv_decode.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.ckv_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.ckv_decode_profile.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp,
                                        ctypes.POINTER(ctypes.c_float)]
     lib.ckv_scan_profile.argtypes = [vp, vp, vp, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_float)]
@@ -86,7 +87,7 @@ def load() -> ctypes.CDLL:
     lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_launch_count.restype = ctypes.c_int64
     for name in ("ckv_query_sizes", "ckv_stats_offsets", "ckv_create", "ckv_stats_build", "ckv_stats_export", "ckv_append",
-                 "ckv_decode", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode", "ckv_copy_scores", "ckv_step_host", "ckv_read_status"):
+                 "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode", "ckv_copy_scores", "ckv_step_host", "ckv_read_status"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -212,6 +213,16 @@ class CompKV:
         _check(self.lib.ckv_decode(self._ctx, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(page_table), _ptr(seq_lens),
                                    batch, int(max_seq_len), int(budget_tokens), _ptr(out), _ptr(lse), _ptr(ids),
                                    _ptr(cnt), _stream()), "ckv_decode")
+        return out, lse, ids, cnt
+
+    def step(self, q, k_new, v_new, k_pool, v_pool, page_table, seq_lens, max_seq_len: int, budget_tokens: int,
+             outputs=None):
+        """ckv_step: append (k_new, v_new), then decode q; returns (out, lse, sel_ids, sel_cnt)."""
+        batch = q.shape[0]
+        out, lse, ids, cnt = outputs if outputs is not None else self.alloc_outputs(batch, budget_tokens)
+        _check(self.lib.ckv_step(self._ctx, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool),
+                                 _ptr(page_table), _ptr(seq_lens), batch, int(max_seq_len), int(budget_tokens),
+                                 _ptr(out), _ptr(lse), _ptr(ids), _ptr(cnt), _stream()), "ckv_step")
         return out, lse, ids, cnt
 
     def decode_profile(self, q, k_pool, v_pool, page_table, seq_lens, max_seq_len: int, budget_tokens: int,

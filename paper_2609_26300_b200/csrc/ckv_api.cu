@@ -232,6 +232,24 @@ int ckv_decode(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool
                      sel_ids, sel_cnt, (cudaStream_t)stream, nullptr);
 }
 
+int ckv_step(ckv_ctx *c, const void *q, const void *k_new, const void *v_new, void *k_pool, void *v_pool,
+             const int32_t *page_table, int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens, void *out,
+             float *lse, int32_t *sel_ids, int32_t *sel_cnt, ckv_stream stream) {
+  // validate the decode half before anything is appended, so that a refused step leaves the cache untouched
+  const int st = check_step_args(c, batch, max_seq_len_host);
+  if (st != CKV_OK) return st;
+  if (!q || !out || !sel_ids || !sel_cnt) return CKV_ERR_INVALID_ARG;
+  const ckv_layout &L = c->layout;
+  const int kcap = budget_tokens / L.block_size;
+  if (budget_tokens <= 0 || kcap <= 0) return CKV_ERR_BUDGET_TOO_SMALL;
+  if (kcap < L.sink_blocks + L.recent_blocks && (long long)kcap * L.block_size < max_seq_len_host)
+    return CKV_ERR_BUDGET_TOO_SMALL;
+  const int r = ckv_append(c, k_pool, v_pool, page_table, seq_lens, k_new, v_new, batch, stream);
+  if (r != CKV_OK) return r;
+  return ckv_decode(c, q, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, out, lse, sel_ids,
+                    sel_cnt, stream);
+}
+
 int ckv_decode_profile(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
                        const int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens, void *out,
                        float *lse, int32_t *sel_ids, int32_t *sel_cnt, ckv_stream stream, float *stage_ms_host) {
@@ -322,10 +340,8 @@ int ckv_step_host(ckv_ctx *c, const void *q_host, const void *k_new_host, const 
   CKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
   CKV_CUDA(cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
   CKV_CUDA(cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
-  int r = ckv_append(c, k_pool, v_pool, page_table, seq_lens, dk, dv, batch, stream);
-  if (r != CKV_OK) return r;
-  r = ckv_decode(c, dq, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, dout, nullptr,
-                 dids, dcnt, stream);
+  const int r = ckv_step(c, dq, dk, dv, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, dout,
+                         nullptr, dids, dcnt, stream);
   if (r != CKV_OK) return r;
   CKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s));
   CKV_CUDA(cudaMemcpyAsync(sel_ids_host, dids, ids_bytes, cudaMemcpyDeviceToHost, s));

@@ -1,4 +1,4 @@
-"""One decode step (ckv_append + ckv_decode) captured as a CUDA graph over static input buffers.
+"""One decode step (ckv_step: append + decode) captured as a CUDA graph over static input buffers.
 
 Launch plumbing only: the graph holds the library's own kernel launches; per-step inputs are copied
 into the static buffers before each replay.  bench.py and the full-size parity tests share it so
@@ -22,8 +22,7 @@ class GraphStep:
         self.graph = torch.cuda.CUDAGraph()
         torch.cuda.synchronize()
         with torch.cuda.graph(self.graph):   # capture only records the launches; nothing runs here
-            ckv.append(k_pool, v_pool, table, lens, self.k_new, self.v_new)
-            ckv.decode(self.q, k_pool, v_pool, table, lens, max_len, budget_tokens, self.outputs)
+            ckv.step(self.q, self.k_new, self.v_new, k_pool, v_pool, table, lens, max_len, budget_tokens, self.outputs)
         self.launches_per_step = ckv.launch_count() - before
 
     def set_inputs(self, q, k_new, v_new) -> None:

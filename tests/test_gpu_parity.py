@@ -294,7 +294,7 @@ def test_append_past_capacity_sets_status():
 
 # ---- decode steps with appends ----------------------------------------------------------------------------------------
 
-def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False):
+def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False, fused=False, **ck):
     w = d.w
     n0 = d.lens.cpu().numpy().copy()
     d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
@@ -312,6 +312,11 @@ def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False
             d.ckv.step_host(hq, hk, hv, d.k_pool, d.v_pool, d.table, d.lens, max_len, budget, ho, hi, hc)
             out, ids, cnt = ho, hi, hc
             lse = None
+        elif fused:   # ckv_step: the same step in one call
+            out, lse, ids, cnt = d.ckv.step(torch.from_numpy(q).to(d.dtype).cuda(),
+                                            torch.from_numpy(k_new).to(d.dtype).cuda(),
+                                            torch.from_numpy(v_new).to(d.dtype).cuda(), d.k_pool, d.v_pool, d.table,
+                                            d.lens, max_len, budget)
         else:
             d.ckv.append(d.k_pool, d.v_pool, d.table, d.lens, torch.from_numpy(k_new).to(d.dtype).cuda(),
                          torch.from_numpy(v_new).to(d.dtype).cuda())
@@ -332,7 +337,7 @@ def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False
                     ref, _ = O.sparse(qq, K, V, st, ref_ids if same else got)
                     assert rel_inf(out[s, h * G:(h + 1) * G].double().numpy(), ref) <= OUT_TOL[d.dtype]
                 else:
-                    check_unit_decode(d, s, h, int(n0[s]) + t + 1, t, budget, out, lse, ids, cnt, scores)
+                    check_unit_decode(d, s, h, int(n0[s]) + t + 1, t, budget, out, lse, ids, cnt, scores, **ck)
     torch.cuda.synchronize()
     assert d.ckv.read_status() == 0
     assert np.array_equal(d.lens.cpu().numpy(), n0 + steps)
@@ -342,6 +347,45 @@ def test_decode_loop_small_with_appends():
     w = small(ctx_min=16 * 30 + 1, ctx=16 * 60, decode_steps=36)
     d = setup(w)
     decode_loop(d, 36, w.budget_tokens, set(range(36)), all_units(w))
+
+
+@pytest.mark.parametrize("bs,r", [(16, 4), (32, 4), (64, 4), (16, 128), (16, 8)])
+def test_fused_step_loop(bs, r):
+    """ckv_step over block roll-overs, one-token blocks and ragged lengths: every unit, every step."""
+    w = small(ctx_min=16 * 30 + 1, ctx=16 * 60, decode_steps=36, block_size=bs, budget_tokens=bs * 7)
+    d = setup(w, var_groups=r)
+    decode_loop(d, 36, w.budget_tokens, set(range(36)), all_units(w), fused=True, var_groups=r)
+
+
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (16, 2)])   # G = 1 and 8
+def test_fused_step_group_sizes(hq, hkv):
+    w = small(ctx=16 * 40 + 9, decode_steps=20, num_q_heads=hq, num_kv_heads=hkv)
+    d = setup(w)
+    decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), fused=True)
+
+
+@pytest.mark.parametrize("variant", [1, 2, 4])
+def test_fused_step_ablations(variant):
+    w = small(ctx=16 * 40 + 15, decode_steps=6)
+    d = setup(w, variant=variant)
+    decode_loop(d, 6, w.budget_tokens, set(range(6)), all_units(w), fused=True, variant=variant)
+
+
+def test_fused_step_from_short_and_single_block_sequences():
+    """Sequences that start with one token / exactly one block: the scan has nothing or one block to cover."""
+    for n in (1, 15, 16, 17):
+        w = small(ctx=n, decode_steps=20, budget_tokens=16 * 4, needles=0)
+        d = setup(w)
+        decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), fused=True)
+
+
+def test_fused_step_select_all_and_recent_zero_fallback():
+    w = small(ctx=16 * 12 + 3, decode_steps=8, budget_tokens=16 * 64)     # K >= X: dense
+    d = setup(w)
+    decode_loop(d, 8, w.budget_tokens, set(range(8)), all_units(w), fused=True)
+    w = small(ctx=16 * 40 + 3, decode_steps=8)
+    d = setup(w, sink=1, recent=0)                                         # no mandatory tail block
+    decode_loop(d, 8, w.budget_tokens, set(range(8)), all_units(w), fused=True, sink=1, recent=0)
 
 
 def test_decode_loop_through_host_buffer_call():
