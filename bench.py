@@ -170,12 +170,12 @@ def oracle_step(w, kv, stats, n0, cores, step: int):
     return time.perf_counter() - t0
 
 
-def required_bytes(w, lens, sel_tokens_per_unit):
+def required_bytes(w, lens, sel_tokens_per_unit, mean_bytes: int = 4):
     """Bytes one decode step must read: every block summary once, plus K and V of the selected tokens."""
     stats = 0
     for n in lens:
         x = -(-int(n) // w.block_size)
-        stats += w.num_kv_heads * x * (2 * w.head_dim * 4 + 4 * w.var_groups)
+        stats += w.num_kv_heads * x * (2 * w.head_dim * mean_bytes + 4 * w.var_groups)
     sel = int(np.sum(sel_tokens_per_unit)) * 2 * w.head_dim * 2
     return stats, sel
 
@@ -221,6 +221,7 @@ def main():
     ap.add_argument("--block-size", type=int, default=0)
     ap.add_argument("--budget", type=int, default=0)
     ap.add_argument("--var-groups", type=int, default=0)
+    ap.add_argument("--stat-bf16", action="store_true", help="bf16 mean keys / mean values (half the summary bytes)")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -241,7 +242,7 @@ def main():
     W, K, KP, KE = max(args.warmup, 3), args.steps, args.profile_steps, args.e2e_steps
     total = W + K + KP + KE + W + 2 * min(K, 64)
     w = workload(total, args)
-    is_default = args.config == 3 and not (args.block_size or args.budget or args.var_groups)
+    is_default = args.config == 3 and not (args.block_size or args.budget or args.var_groups or args.stat_bf16)
     dev = torch.device("cuda", local)
 
     # ---- inputs: every rank holds a full replica of the workload (the path does not shard) ----
@@ -249,7 +250,8 @@ def main():
     q_np, kn_np, vn_np = step_inputs(w, total)
     max_blocks = synth.pages_per_seq(w)
     ckv = binding.CompKV(w.num_q_heads, w.num_kv_heads, w.batch, max_blocks, k_pool.shape[0],
-                         block_size=w.block_size, var_groups=w.var_groups, device=str(dev))
+                         block_size=w.block_size, var_groups=w.var_groups, device=str(dev),
+                         stat_bf16=int(args.stat_bf16))
     k_pool, v_pool, table, lens = (t.to(dev) for t in (k_pool, v_pool, table, lens))
     q_all = torch.from_numpy(q_np).to(torch.bfloat16).to(dev)
     kn_all = torch.from_numpy(kn_np).to(torch.bfloat16).to(dev)
@@ -282,7 +284,7 @@ def main():
         build_ms.append(e0.elapsed_time(e1))
     build_us = float(np.median(build_ms[2:])) * 1e3
     build_bytes = sum(int(n) for n in lens.tolist()) * w.num_kv_heads * 2 * w.head_dim * 2 + \
-        required_bytes(w, lens.tolist(), 0)[0]
+        required_bytes(w, lens.tolist(), 0, 2 if args.stat_bf16 else 4)[0]
 
     # ---- one step as a CUDA graph over static input buffers ----
     sq, sk, sv = q_all[0].clone(), kn_all[0].clone(), vn_all[0].clone()
@@ -327,7 +329,7 @@ def main():
     ms_per_step = float(step_ms.mean())
     sel_cnt = outputs[3].cpu().numpy()
     lens_now = lens.cpu().numpy()
-    stats_b, sel_b = required_bytes(w, lens_now, sel_cnt * w.block_size)
+    stats_b, sel_b = required_bytes(w, lens_now, sel_cnt * w.block_size, 2 if args.stat_bf16 else 4)
     assert ckv.read_status() == 0
 
     # ---- per-kernel durations (events between the launches), L2 flushed before each step ----
@@ -423,7 +425,8 @@ def main():
         "metric": METRIC if is_default else "sparse decode-attn us/step (append + decode)", "value": us_per_step, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": describe(w, is_default),
+        "config": {"workload": describe(w, is_default).replace("fp32 summaries", "bf16 summaries") if args.stat_bf16
+                   else describe(w, is_default),
                    "step": "ckv_step (append, summary scan, select, attention + merge: four launches) replayed as one CUDA graph; CUDA events around each replay",
                    "l2": "flushed between steps (256 MiB memset then 256 MiB read, outside the events); per-step inputs exceed L2",
                    "replicas": "every rank runs the whole workload (the path does not shard)",

@@ -34,7 +34,7 @@ class ckv_layout(ctypes.Structure):
                 ("group_layout", ctypes.c_int32), ("kv_dtype", ctypes.c_int32), ("max_batch", ctypes.c_int32),
                 ("max_blocks_per_seq", ctypes.c_int32), ("num_pages", ctypes.c_int32),
                 ("sink_blocks", ctypes.c_int32), ("recent_blocks", ctypes.c_int32), ("sm_scale", ctypes.c_float),
-                ("variant", ctypes.c_int32)]
+                ("variant", ctypes.c_int32), ("stat_bf16", ctypes.c_int32)]
 
 
 class CompKVError(RuntimeError):
@@ -149,11 +149,11 @@ class CompKV:
     def __init__(self, num_q_heads: int, num_kv_heads: int, max_batch: int, max_blocks_per_seq: int, num_pages: int,
                  block_size: int = 16, var_groups: int = 4, group_layout: int = 1, kv_dtype: int = CKV_BF16,
                  sink_blocks: int = 1, recent_blocks: int = 2, sm_scale: float = 0.0, head_dim: int = 128,
-                 page_size: int = 16, device: str = "cuda", variant: int = 0):
+                 page_size: int = 16, device: str = "cuda", variant: int = 0, stat_bf16: int = 0):
         self.lib = load()
         self.layout = ckv_layout(num_q_heads, num_kv_heads, head_dim, block_size, page_size, var_groups,
                                  group_layout, kv_dtype, max_batch, max_blocks_per_seq, num_pages, sink_blocks,
-                                 recent_blocks, sm_scale, variant)
+                                 recent_blocks, sm_scale, variant, stat_bf16)
         self.stats_bytes, self.work_bytes = query_sizes(self.layout)
         self.device = torch.device(device)
         self.stats = torch.zeros(self.stats_bytes, dtype=torch.uint8, device=self.device)

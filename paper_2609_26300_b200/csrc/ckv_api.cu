@@ -28,6 +28,8 @@ int check_layout(const ckv_layout *L) {
   if (L->sink_blocks < 0 || L->recent_blocks < 0) return CKV_ERR_BAD_LAYOUT;
   if (!(L->sm_scale >= 0.f) || !isfinite(L->sm_scale)) return CKV_ERR_BAD_LAYOUT;
   if (L->variant & ~(CKV_VARIANT_FIRST_ORDER_MASS | CKV_VARIANT_RANK_BY_MASS | CKV_VARIANT_DROP)) return CKV_ERR_BAD_LAYOUT;
+  if (L->stat_bf16 != 0 && L->stat_bf16 != 1) return CKV_ERR_BAD_LAYOUT;
+  if (L->stat_bf16 == 1 && (L->kv_dtype != CKV_BF16 || L->var_groups == CKV_D)) return CKV_ERR_BAD_LAYOUT;
   return CKV_OK;
 }
 
@@ -43,9 +45,10 @@ Regions regions(const ckv_layout *L) {
   const int G = L->num_q_heads / L->num_kv_heads;
   const size_t esz = L->kv_dtype == CKV_BF16 ? 2 : 4;
   size_t o = 0;
-  R.kmean = o; o = align_up(o + rows * CKV_D * 4, 256);
+  const size_t mean_row = L->stat_bf16 ? CKV_D * 2 : CKV_D * 4;   // bf16 values, or split pairs with fp32 precision
+  R.kmean = o; o = align_up(o + rows * mean_row, 256);
   R.dbar = o;  o = align_up(o + rows * L->var_groups * 4, 256);
-  R.vmean = o; o = align_up(o + rows * CKV_D * 4, 256);
+  R.vmean = o; o = align_up(o + rows * mean_row, 256);
   R.stats_total = o;
   o = 0;
   R.status = o; o = align_up(o + 256, 256);
@@ -144,6 +147,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.max_blocks = layout->max_blocks_per_seq; P.max_pages_per_seq = P.max_blocks * P.ppb;
   P.num_pages = layout->num_pages; P.sink = layout->sink_blocks; P.recent = layout->recent_blocks;
   P.scale = c->layout.sm_scale;
+  P.row_elems = layout->stat_bf16 ? CKV_D : CKV_ROW_ELEMS;
   P.variant = layout->variant;
   P.half_var = (layout->variant & CKV_VARIANT_FIRST_ORDER_MASS) ? 0.f : 0.5f;
   P.kmean = (__nv_bfloat16 *)(sb + R.kmean); P.dbar = (float *)(sb + R.dbar); P.vmean = (__nv_bfloat16 *)(sb + R.vmean);

@@ -128,7 +128,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
   const int g_own0 = (G >= 2) ? (li & 1) * KEEP : 0;
   const int t_own = hw + 2 * (li >> 1);
   const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
-  const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * CKV_ROW_ELEMS;
+  const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * P.row_elems;
   uint32_t phase_bits = 0;   // bit b: parity of the next completion of buffer b
   bool aborted = false;
   int n_abort = 0;
@@ -241,7 +241,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
         }
         if (hw == 0) {
           float vb[8];
-          load_split8(vmean + (size_t)blk * CKV_ROW_ELEMS, li, blk, vb);
+          load_split8(vmean + (size_t)blk * P.row_elems, li, blk, vb, P.row_elems == CKV_ROW_ELEMS);
 #pragma unroll
           for (int g = 0; g < G; ++g) {
             const float wbar_g = exp2f(zl2[g] - m_ref[g]);

@@ -175,7 +175,8 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
   const int n_mine = max((p1 - p0 - warp + W - 1) / W, 0);   // this warp's pages: list index p0 + warp + W n
   const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
-  const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * CKV_ROW_ELEMS;
+  const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * P.row_elems;
+  const bool mean_lo = P.row_elems == CKV_ROW_ELEMS;   // the mean-value rows carry lo halves (fp32-precision summaries)
   bool bad = false;
 
   // the scan partials this CTA folds in: partial j of the unit goes to split j % n_active
@@ -257,7 +258,8 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         cp_async16(vb + off, v_pool + so, valid);
       }
       if (comp && r.first) {   // verbatim: hi halves then lo halves, swizzled by block index
-        cp_async16(aux_u32 + 512 * slot + 16 * lane, vmean + (size_t)r.blk * CKV_ROW_ELEMS + 8 * lane, true);
+        if (mean_lo || lane < 16)
+          cp_async16(aux_u32 + 512 * slot + 16 * lane, vmean + (size_t)r.blk * P.row_elems + 8 * lane, true);
         if (lane < G)          // and the block's (logit, variance) of every head, for the weight of its mean term
           cp_async8(aux_u32 + kLsOff + (slot * G + lane) * 8, ls + (size_t)lane * P.max_blocks + r.blk);
       }
@@ -310,7 +312,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
       const uint32_t coff = (uint32_t)(swz_chunk(2 * t2 + cpar, rblk) << 4);
       uint32_t vh[4], vl[4];
       ldmatrix_x4_trans(vh, real ? rowaddr + coff : aux_u32 + kZeroRow);
-      ldmatrix_x4_trans(vl, real ? rowaddr + 256 + coff : aux_u32 + kZeroRow);
+      ldmatrix_x4_trans(vl, real && mean_lo ? rowaddr + 256 + coff : aux_u32 + kZeroRow);   // no lo halves: zeros
       mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh, 0u, vh[0], vh[1]);
       mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wl, 0u, vh[0], vh[1]);
       mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh, 0u, vl[0], vl[1]);

@@ -34,6 +34,7 @@ struct CkvDev {
   float *scores;     // [unit][max_blocks]     S_b
   float *comp_part;  // [(scan CTA + unit) * CKV_SCAN_WARPS + warp][G][CKV_PART_STRIDE]  all-block mean-compensation partials
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials
+  int row_elems;     // bf16 elements of one mean-key / mean-value row: CKV_ROW_ELEMS, or CKV_D when only hi halves are kept
   int variant;       // ckv_variant bits
   float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
   int *unit_done;    // [unit] attention splits finished this step (zero between steps); null = merge is a separate launch
@@ -116,7 +117,8 @@ __device__ __forceinline__ void store_out(__nv_bfloat16 *p, float x) { *p = __fl
 // so that a matrix load touching one chunk column of 8 consecutive rows hits 8 different bank groups.
 __device__ __forceinline__ int swz_chunk(int chunk, int block) { return chunk ^ (block & 7); }
 
-__device__ __forceinline__ void store_split8(__nv_bfloat16 *row, int chunk, int block, const float (&x)[8]) {
+// lo_half false: only the hi halves are kept (the bf16 summary layout, rows of 256 bytes).
+__device__ __forceinline__ void store_split8(__nv_bfloat16 *row, int chunk, int block, const float (&x)[8], bool lo_half = true) {
   uint32_t hi[4], lo[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -128,14 +130,14 @@ __device__ __forceinline__ void store_split8(__nv_bfloat16 *row, int chunk, int 
   }
   const int p = swz_chunk(chunk, block) * 8;
   *reinterpret_cast<uint4 *>(row + p) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-  *reinterpret_cast<uint4 *>(row + CKV_D + p) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  if (lo_half) *reinterpret_cast<uint4 *>(row + CKV_D + p) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
 }
 
-// The eight entries of one chunk, hi + lo, as floats.
-__device__ __forceinline__ void load_split8(const __nv_bfloat16 *row, int chunk, int block, float (&x)[8]) {
+// The eight entries of one chunk, hi + lo (hi alone when the row has no lo halves), as floats.
+__device__ __forceinline__ void load_split8(const __nv_bfloat16 *row, int chunk, int block, float (&x)[8], bool lo_half = true) {
   const int p = swz_chunk(chunk, block) * 8;
   const uint4 h = __ldg(reinterpret_cast<const uint4 *>(row + p));
-  const uint4 l = __ldg(reinterpret_cast<const uint4 *>(row + CKV_D + p));
+  const uint4 l = lo_half ? __ldg(reinterpret_cast<const uint4 *>(row + CKV_D + p)) : make_uint4(0u, 0u, 0u, 0u);
   float a[8], b[8];
   bf16x8_to_float(h, a);
   bf16x8_to_float(l, b);

@@ -38,7 +38,6 @@ constexpr int kMaxStages = 8;
 constexpr int kConsumerWarps = CKV_SCAN_WARPS;
 constexpr int kThreads = kConsumerWarps * 32 + 32;   // plus the producer warp
 constexpr int kMaxSeqs = 1024;      // sequence lengths are staged in shared memory up to this many sequences
-constexpr int kRowBytes = CKV_ROW_ELEMS * 2;
 
 struct UnitInfo { int N, X, tiles; };
 
@@ -62,10 +61,12 @@ template <> struct QSplit<float> { static constexpr bool value = true; };
 
 // RD: one variance group per coordinate (r = d).  The variance rows then have the mean rows' layout and
 // sigma^2 = sum_i (scale q_i)^2 Dbar_i is a third tensor-core product, with the squared queries as the A operand.
-template <int G, typename QT, bool RD>
+// HS: the mean rows hold hi halves only (bf16 summaries, 256-byte rows); every product with a lo plane drops out.
+template <int G, typename QT, bool RD, bool HS>
 __global__ void __launch_bounds__(kThreads, 1)
 ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_lens, int units, int stages) {
   constexpr bool QS = QSplit<QT>::value;   // fp32 queries are split into hi + lo like the summaries
+  constexpr int kRowBytes = HS ? CKV_D * 2 : CKV_ROW_ELEMS * 2;   // bytes of one mean-key / mean-value row
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
   __shared__ int s_u0, s_tl0, s_count, s_ulast, s_abort, s_issued;
@@ -146,8 +147,8 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
         const uint32_t lo = smem_u32(stage_mem), hi = lo + (uint32_t)stages * stage_bytes;
         bool ok = nb >= 1 && u < units && row + nb <= (size_t)units * P.max_blocks;
-        ok = ok && bulk_g2s_checked(sk, P.kmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st], lo, hi);
-        ok = ok && bulk_g2s_checked(sv, P.vmean + row * CKV_ROW_ELEMS, kbytes, &full_bar[st], lo, hi);
+        ok = ok && bulk_g2s_checked(sk, P.kmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
+        ok = ok && bulk_g2s_checked(sv, P.vmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
         if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, &full_bar[st], lo, hi);
         if (!ok) atomicOr(P.status, CKV_DEV_BAD_COPY);
         *(volatile int *)&s_issued = it + 1;
@@ -313,11 +314,13 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
               const uint32_t coff = (uint32_t)swz_chunk(4 * j + lmat, r) * 16;
               uint32_t bh[4], bl[4];
               ldmatrix_x4(bh, rowaddr + coff);
-              ldmatrix_x4(bl, rowaddr + 256 + coff);
               mma_rows8(z[nt][0], z[nt][1], qa[2 * j][0], qa[2 * j][1], bh[0], bh[1]);
               mma_rows8(z[nt][0], z[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bh[2], bh[3]);
-              mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j][0], qa[2 * j][1], bl[0], bl[1]);
-              mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bl[2], bl[3]);
+              if (!HS) {
+                ldmatrix_x4(bl, rowaddr + 256 + coff);
+                mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j][0], qa[2 * j][1], bl[0], bl[1]);
+                mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bl[2], bl[3]);
+              }
               if (QS) {
                 mma_rows8(zlo[nt][0], zlo[nt][1], qb[QS ? 2 * j : 0][0], qb[QS ? 2 * j : 0][1], bh[0], bh[1]);
                 mma_rows8(zlo[nt][0], zlo[nt][1], qb[QS ? 2 * j + 1 : 0][0], qb[QS ? 2 * j + 1 : 0][1], bh[2], bh[3]);
@@ -423,13 +426,15 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
             const uint32_t coff = (uint32_t)swz_chunk(2 * t2 + cpar, r) * 16;
             uint32_t vh[4], vl[4];
             ldmatrix_x4_trans(vh, rowaddr + coff);
-            ldmatrix_x4_trans(vl, rowaddr + 256 + coff);
             mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vh[0], vh[1]);
             mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wl[0], wl[1], vh[0], vh[1]);
-            mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vl[0], vl[1]);
             mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vh[2], vh[3]);
             mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wl[0], wl[1], vh[2], vh[3]);
-            mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vl[2], vl[3]);
+            if (!HS) {
+              ldmatrix_x4_trans(vl, rowaddr + 256 + coff);
+              mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vl[0], vl[1]);
+              mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vl[2], vl[3]);
+            }
           }
         }
       }
@@ -453,7 +458,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
 struct ScanCfg { int stages; size_t smem; };
 
 ScanCfg scan_cfg(const CkvDev &P, int G) {
-  const size_t stage_bytes = (size_t)TB * 2 * kRowBytes + (P.r >= 4 ? (size_t)TB * P.r * 4 : 0);
+  const size_t stage_bytes = (size_t)TB * 2 * (P.row_elems * 2) + (P.r >= 4 ? (size_t)TB * P.r * 4 : 0);
   const size_t sw_bytes = (P.r == 4 || P.r == CKV_D) ? 0 : (size_t)kConsumerWarps * P.r * G * 4;   // weight table of the generic path
   const size_t budget = 220 * 1024 - 8 * 1024 - sw_bytes;   // static shared memory stays below 8 KB
   int stages = (int)(budget / stage_bytes);
@@ -466,9 +471,14 @@ template <int G, typename QT>
 cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, cudaStream_t st) {
   const ScanCfg cfg = scan_cfg(c->dev, G);
   if (c->dev.r == CKV_D)
-    ckv_scan_kernel<G, QT, true><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
-  else
-    ckv_scan_kernel<G, QT, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+    ckv_scan_kernel<G, QT, true, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+  else if (c->dev.row_elems == CKV_D) {
+    if constexpr (!QSplit<QT>::value)   // bf16 summaries come with bf16 pages and queries only
+      ckv_scan_kernel<G, QT, false, true><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+    else
+      return cudaErrorInvalidValue;
+  } else
+    ckv_scan_kernel<G, QT, false, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
   return cudaGetLastError();
 }
 
@@ -480,11 +490,15 @@ cudaError_t launch_g(ckv_ctx *c, const void *q, const int *seq_lens, int units, 
 
 template <int G, typename QT>
 cudaError_t configure_gt(const ckv_ctx *c) {
+  const int smem = (int)scan_cfg(c->dev, G).smem;
   if (c->dev.r == CKV_D)
-    return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)scan_cfg(c->dev, G).smem);
-  return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)scan_cfg(c->dev, G).smem);
+    return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (c->dev.row_elems == CKV_D) {
+    if constexpr (!QSplit<QT>::value)
+      return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    return cudaErrorInvalidValue;
+  }
+  return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
 template <int G>

@@ -55,6 +55,7 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
   P.max_blocks = layout->max_blocks_per_seq; P.max_pages_per_seq = P.max_blocks * P.ppb;
   P.num_pages = layout->num_pages; P.sink = layout->sink_blocks; P.recent = layout->recent_blocks;
   P.scale = c.layout.sm_scale;
+  P.row_elems = layout->stat_bf16 ? CKV_D : CKV_ROW_ELEMS;
   P.variant = layout->variant; P.half_var = 0.5f;   // the dense pass reads neither
 
   // the partials of the largest split count the launch heuristic may pick must fit the fixed array

@@ -65,7 +65,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
 #pragma unroll
   for (int i = 0; i < 8; ++i) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], 16);
   if (hw == 0) {
-    store_split8(kmean_row, li, b, km);
+    store_split8(kmean_row, li, b, km, P.row_elems == CKV_ROW_ELEMS);
     if (P.r == CKV_D) {
       // one group per coordinate: the variance row has the mean rows' layout (split bf16 pairs, swizzled chunks),
       // so that the scan can project it with the same tensor-core product as the mean keys
@@ -81,7 +81,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
     float vm[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) vm[i] = vs[i] / fc;
-    store_split8(vmean_row, li, b, vm);
+    store_split8(vmean_row, li, b, vm, P.row_elems == CKV_ROW_ELEMS);
   }
   __syncwarp();
   // grouped variance: average of the per-coordinate population variances of each group (Eq. 8)
@@ -116,8 +116,8 @@ __global__ void __launch_bounds__(256) ckv_stats_build_kernel(CkvDev P, const T 
   const int cnt = min(P.bs, N - b * P.bs);
   const size_t row = (size_t)unit * P.max_blocks + b;
   block_stats_warp<T, true>(P, k_pool, v_pool, page_table + (size_t)s * P.max_pages_per_seq, h, b, cnt,
-                            sq_smem[warp], P.kmean + row * CKV_ROW_ELEMS, P.dbar + row * P.r,
-                            P.vmean + row * CKV_ROW_ELEMS, lane);
+                            sq_smem[warp], P.kmean + row * P.row_elems, P.dbar + row * P.r,
+                            P.vmean + row * P.row_elems, lane);
 }
 
 // One CTA per sequence, one warp per KV head (looping when there are more heads than warps).
@@ -150,8 +150,8 @@ __global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T 
     }
     __syncwarp();
     const size_t row = ((size_t)s * P.Hkv + h) * P.max_blocks + b;
-    block_stats_warp<T, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * CKV_ROW_ELEMS,
-                               P.dbar + row * P.r, P.vmean + row * CKV_ROW_ELEMS, lane);
+    block_stats_warp<T, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * P.row_elems,
+                               P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
   }
   __syncthreads();
   if (threadIdx.x == 0) seq_lens[s] = N + 1;
@@ -164,7 +164,7 @@ __global__ void __launch_bounds__(256) ckv_stats_export_kernel(CkvDev P, int row
   if (row >= rows) return;
   const int b = row % P.max_blocks, hw = lane >> 4, li = lane & 15;
   float x[8];
-  load_split8((hw == 0 ? P.kmean : P.vmean) + (size_t)row * CKV_ROW_ELEMS, li, b, x);
+  load_split8((hw == 0 ? P.kmean : P.vmean) + (size_t)row * P.row_elems, li, b, x, P.row_elems == CKV_ROW_ELEMS);
   float *dst = (hw == 0 ? kmean : vmean) + (size_t)row * CKV_D + 8 * li;
   reinterpret_cast<float4 *>(dst)[0] = make_float4(x[0], x[1], x[2], x[3]);
   reinterpret_cast<float4 *>(dst)[1] = make_float4(x[4], x[5], x[6], x[7]);

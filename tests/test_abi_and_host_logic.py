@@ -55,6 +55,8 @@ def test_sizes_follow_the_summary_layout():
     assert ko == 0 and do >= rows * 128 * 4 and vo >= do + rows * 4 * 4
     assert ko % 256 == do % 256 == vo % 256 == 0
     assert work > rows * 4 * 8      # at least the per-(block, head) pairs
+    half, _ = binding.query_sizes(layout(stat_bf16=1))
+    assert rows * (128 + 4) * 4 <= half <= rows * (128 + 4) * 4 + 3 * 256   # bf16 means: half the mean bytes
     s128, _ = binding.query_sizes(layout(var_groups=128))
     assert s128 - stats >= rows * (128 - 4) * 4 - 256
 
@@ -63,7 +65,8 @@ def test_sizes_follow_the_summary_layout():
                                  dict(var_groups=3), dict(var_groups=96), dict(group_layout=2), dict(kv_dtype=5),
                                  dict(max_batch=0), dict(num_pages=0), dict(sink_blocks=-1),
                                  dict(sm_scale=float("nan")), dict(max_blocks_per_seq=0), dict(variant=8),
-                                 dict(variant=-1)])
+                                 dict(variant=-1), dict(stat_bf16=2), dict(stat_bf16=1, kv_dtype=binding.CKV_F32),
+                                 dict(stat_bf16=1, var_groups=128)])
 def test_bad_layouts_are_rejected(bad):
     with pytest.raises(binding.CompKVError) as e:
         binding.query_sizes(layout(**bad))
@@ -72,7 +75,7 @@ def test_bad_layouts_are_rejected(bad):
 
 @pytest.mark.parametrize("ok", [dict(var_groups=1), dict(var_groups=64), dict(var_groups=128), dict(block_size=64),
                                 dict(num_q_heads=64), dict(num_q_heads=8), dict(kv_dtype=binding.CKV_F32),
-                                dict(variant=7), dict(variant=binding.VARIANT_DROP)])
+                                dict(variant=7), dict(variant=binding.VARIANT_DROP), dict(stat_bf16=1)])
 def test_good_layouts_are_accepted(ok):
     stats, work = binding.query_sizes(layout(**ok))
     assert stats > 0 and work > 0

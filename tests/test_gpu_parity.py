@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from oracle import compkv_oracle as O
+import helpers
 from paper_2609_26300_b200 import synth
 
 from helpers import (OUT_TOL, check_ids, check_stats, check_unit_decode, dev_q, rel_inf, setup, unit_inputs)
@@ -117,6 +118,27 @@ def test_decode_scorer_and_merge_ablations(variant, dtype):
     out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
     for s, h in all_units(w):
         check_unit_decode(d, s, h, int(d.lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores, variant=variant)
+
+
+@pytest.mark.parametrize("bs,hq", [(16, 8), (32, 8), (64, 8), (16, 16), (16, 2)])
+def test_bf16_summaries_layout(bs, hq):
+    """ckv_layout.stat_bf16: mean keys / mean values stored as bf16 (half the summary bytes).  The oracle runs on
+    its own summaries rounded to bf16; stats must match to a bf16 ulp, the step within the layout's tolerances."""
+    w = small(block_size=bs, budget_tokens=bs * 9, ctx=16 * 90 + 7, num_q_heads=hq, decode_steps=20)
+    d = setup(w, stat_bf16=1)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    km, db, vm = d.ckv.export_stats(w.batch)
+    for s, h in all_units(w):
+        n = int(d.lens[s])
+        _, K, V = unit_inputs(w, s, h, n)
+        st = helpers.round_stats_bf16(O.stats(K, V, bs))
+        x = len(st.cnt)
+        for got, ref in ((km[s, h, :x], st.kmean), (vm[s, h, :x], st.vmean)):
+            err = np.abs(got.double().cpu().numpy() - ref)
+            assert np.all(err <= 2.0 ** -7 * np.abs(ref) + 1e-30)          # at most one bf16 ulp (a rounding flip)
+            assert np.mean(err == 0.0) > 0.99                                # and almost always none
+        assert np.allclose(db[s, h, :x].double().cpu().numpy(), st.Dbar, rtol=1e-5, atol=1e-12)
+    decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), fused=True, stat_bf16=True)
 
 
 def test_decode_toy_config_fp32_and_bf16():
