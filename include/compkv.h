@@ -213,6 +213,17 @@ int ckv_dense_decode_static(const ckv_layout *layout, const void *q, const void 
                             const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
                             void *out, float *lse, ckv_stream stream);
 
+/* Diagnostic, not part of the decode step: exact per-block logit statistics of every query head over the whole
+ * cache (Eq. 3; App. B.1).  For sequence s, query head g and block b < ceil(N_s / block_size) the kernel writes, at
+ * [s][g][b] of three device fp32 arrays shaped [batch][num_q_heads][max_blocks_per_seq],
+ *   logZ  = log sum_{j in b} exp(z_j),  zmean = mean_{j in b} z_j,  zvar = population variance of z_j,
+ * with z_j = sm_scale * q_g . k_j.  Entries of blocks past a sequence's end are left untouched.  Exact block masses,
+ * compensation residuals and the KL divergences of a selection follow from these by block-level arithmetic
+ * (paper_2609_26300_b200/diagnostics.py).  Reads every key once: as expensive as a dense decode. */
+int ckv_exact_blocks(ckv_ctx *ctx, const void *q, const void *k_pool, const int32_t *page_table,
+                     const int32_t *seq_lens, int batch, int max_seq_len_host, float *logZ, float *zmean,
+                     float *zvar, ckv_stream stream);
+
 /* Copy the block scores S_b of the last ckv_decode (Eq. 10) into dst (device),
  * fp32 [batch][num_kv_heads][max_blocks_per_seq]; entries at or past X_s are unspecified.
  * Mandatory blocks carry their score too (they are excluded from the ranking, not from Eq. 9). */

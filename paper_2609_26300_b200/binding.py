@@ -25,7 +25,7 @@ CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
            "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
            "ckv_dense_decode_static",
-           "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
+           "ckv_exact_blocks", "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
 
 
 class ckv_layout(ctypes.Structure):
@@ -81,6 +81,8 @@ def load() -> ctypes.CDLL:
     lib.ckv_dense_decode.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     lib.ckv_dense_decode_static.argtypes = [lp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     lib.ckv_dense_decode_static.restype = i32
+    lib.ckv_exact_blocks.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
+    lib.ckv_exact_blocks.restype = i32
     lib.ckv_copy_scores.argtypes = [vp, vp, i32, vp]
     lib.ckv_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.ckv_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
@@ -254,6 +256,17 @@ class CompKV:
                                          _ptr(seq_lens), batch, int(max_seq_len), _ptr(out), _ptr(lse), _stream()),
                "ckv_dense_decode")
         return out, lse
+
+    def exact_blocks(self, q, k_pool, page_table, seq_lens, max_seq_len: int):
+        """ckv_exact_blocks: (logZ, zmean, zvar), each fp32 [batch][q_heads][max_blocks] (blocks past the end: NaN)."""
+        L = self.layout
+        batch = q.shape[0]
+        outs = [torch.full((batch, L.num_q_heads, L.max_blocks_per_seq), float("nan"), dtype=torch.float32,
+                           device=self.device) for _ in range(3)]
+        _check(self.lib.ckv_exact_blocks(self._ctx, _ptr(q), _ptr(k_pool), _ptr(page_table), _ptr(seq_lens), batch,
+                                         int(max_seq_len), _ptr(outs[0]), _ptr(outs[1]), _ptr(outs[2]), _stream()),
+               "ckv_exact_blocks")
+        return tuple(outs)
 
     def copy_scores(self, batch: int) -> torch.Tensor:
         L = self.layout

@@ -314,6 +314,16 @@ int ckv_dense_decode(ckv_ctx *c, const void *q, const void *k_pool, const void *
   return CKV_OK;
 }
 
+int ckv_exact_blocks(ckv_ctx *c, const void *q, const void *k_pool, const int32_t *page_table, const int32_t *seq_lens,
+                     int batch, int max_seq_len_host, float *logZ, float *zmean, float *zvar, ckv_stream stream) {
+  const int st = check_step_args(c, batch, max_seq_len_host);
+  if (st != CKV_OK) return st;
+  if (!q || !k_pool || !page_table || !seq_lens || !logZ || !zmean || !zvar) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(ckv_launch_exact_blocks(c, q, k_pool, page_table, seq_lens, batch, max_seq_len_host, logZ, zmean, zvar,
+                                   (cudaStream_t)stream));
+  return CKV_OK;
+}
+
 int ckv_copy_scores(ckv_ctx *c, float *dst, int batch, ckv_stream stream) {
   if (c == nullptr || dst == nullptr || batch <= 0 || batch > c->layout.max_batch) return CKV_ERR_INVALID_ARG;
   const size_t bytes = (size_t)batch * c->layout.num_kv_heads * c->layout.max_blocks_per_seq * sizeof(float);

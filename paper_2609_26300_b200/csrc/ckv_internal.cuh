@@ -75,6 +75,9 @@ cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k
                             const int *page_table, const int *seq_lens, const int *sel_ids, const int *sel_cnt,
                             int kcap, int batch, int max_len, int scan_grid, void *out, float *lse,
                             int *n_splits_out, bool *merged_out, cudaStream_t st);
+cudaError_t ckv_launch_exact_blocks(ckv_ctx *c, const void *q, const void *k_pool, const int *page_table,
+                                    const int *seq_lens, int batch, int max_len, float *logZ, float *zmean, float *zvar,
+                                    cudaStream_t st);
 cudaError_t ckv_launch_merge(ckv_ctx *c, bool dense, const int *seq_lens, const int *sel_cnt, int n_splits,
                              int scan_grid, int batch, void *out, float *lse, cudaStream_t st);
 
