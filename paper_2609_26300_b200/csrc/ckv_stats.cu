@@ -20,45 +20,97 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
   for (int i = 0; i < 8; ++i) { ks[i] = 0.f; vs[i] = 0.f; }
   const int npages = (cnt + CKV_PAGE - 1) / CKV_PAGE;
   bool bad = false;
-  for (int pg = 0; pg < npages; ++pg) {
-    const int phys = pt_row[b * P.ppb + pg];
-    if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
-    const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
-    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+  const float fc = (float)cnt;
+  float km[8], sq[8];
+  bool done = false;
+  if constexpr (sizeof(T) == 2) {
+    if (npages == 1) {
+      // One page of bf16 rows (every block of the default 16-token layout): the key rows stay in registers between
+      // the two passes, so the cache is read exactly once.  Same operations in the same order as the general path
+      // below (rows that do not exist contribute exact zeros), hence the same bits.
+      done = true;
+      const int phys = pt_row[b * P.ppb];
+      const bool ok = phys >= 0 && phys < P.num_pages;
+      bad = !ok;
+      const size_t base = ok ? ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li : 0;
+      uint4 kraw[8], vraw[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int t = hw + 2 * j;
-      if (t < ntok) {
-        float a[8], c[8];
-        load8<NC>(k_pool + base + (size_t)t * CKV_D, a);
-        load8<NC>(v_pool + base + (size_t)t * CKV_D, c);
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        const bool valid = ok && t < cnt;
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        const uint4 *kp = reinterpret_cast<const uint4 *>(k_pool + base + (size_t)t * CKV_D);
+        const uint4 *vp = reinterpret_cast<const uint4 *>(v_pool + base + (size_t)t * CKV_D);
+        kraw[j] = valid ? (NC ? __ldg(kp) : *kp) : zero;
+        vraw[j] = valid ? (NC ? __ldg(vp) : *vp) : zero;
+      }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+      for (int j = 0; j < 8; ++j) {
+        if (ok && hw + 2 * j < cnt) {
+          float a[8], c[8];
+          bf16x8_to_float(kraw[j], a);
+          bf16x8_to_float(vraw[j], c);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
+        vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
+        km[i] = ks[i] / fc;
+        sq[i] = 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (ok && hw + 2 * j < cnt) {
+          float a[8];
+          bf16x8_to_float(kraw[j], a);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+        }
       }
     }
   }
-  const float fc = (float)cnt;
-  float km[8], sq[8];
+  if (!done) {
+    for (int pg = 0; pg < npages; ++pg) {
+      const int phys = pt_row[b * P.ppb + pg];
+      if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
+      const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+      const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
-    vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
-    km[i] = ks[i] / fc;
-    sq[i] = 0.f;
-  }
-  for (int pg = 0; pg < npages; ++pg) {
-    const int phys = pt_row[b * P.ppb + pg];
-    if (phys < 0 || phys >= P.num_pages) continue;
-    const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
-    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          float a[8], c[8];
+          load8<NC>(k_pool + base + (size_t)t * CKV_D, a);
+          load8<NC>(v_pool + base + (size_t)t * CKV_D, c);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int t = hw + 2 * j;
-      if (t < ntok) {
-        float a[8];
-        load8<NC>(k_pool + base + (size_t)t * CKV_D, a);
+          for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+        }
+      }
+    }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+    for (int i = 0; i < 8; ++i) {
+      ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
+      vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
+      km[i] = ks[i] / fc;
+      sq[i] = 0.f;
+    }
+    for (int pg = 0; pg < npages; ++pg) {
+      const int phys = pt_row[b * P.ppb + pg];
+      if (phys < 0 || phys >= P.num_pages) continue;
+      const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+      const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          float a[8];
+          load8<NC>(k_pool + base + (size_t)t * CKV_D, a);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+        }
       }
     }
   }
@@ -102,7 +154,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) ckv_stats_build_kernel(CkvDev P, const T *__restrict__ k_pool,
+__global__ void __launch_bounds__(256, 3) ckv_stats_build_kernel(CkvDev P, const T *__restrict__ k_pool,
                                                               const T *__restrict__ v_pool,
                                                               const int *__restrict__ page_table,
                                                               const int *__restrict__ seq_lens) {
