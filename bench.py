@@ -221,6 +221,7 @@ def main():
     ap.add_argument("--block-size", type=int, default=0)
     ap.add_argument("--budget", type=int, default=0)
     ap.add_argument("--var-groups", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=8, help="layers of the stacked-cache measurement (0 or 1: skip)")
     ap.add_argument("--stat-bf16", action="store_true", help="bf16 mean keys / mean values (half the summary bytes)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -240,7 +241,7 @@ def main():
     dist = rep.dist
 
     W, K, KP, KE = max(args.warmup, 3), args.steps, args.profile_steps, args.e2e_steps
-    total = W + K + KP + KE + W + 2 * min(K, 64)
+    total = W + K + KP + KE + W + 2 * min(K, 64) + 16   # + the stacked-layers measurement
     w = workload(total, args)
     is_default = args.config == 3 and not (args.block_size or args.budget or args.var_groups or args.stat_bf16)
     dev = torch.device("cuda", local)
@@ -375,6 +376,47 @@ def main():
     pipe_us = e0.elapsed_time(e1) * 1e3 / n_pipe
     step += n_pipe
 
+    # ---- a stack of layers: L independent caches (device copies of the same values in different memory), one step
+    # of each per token, back to back with no flush -- every layer's summaries and pages are cold because the other
+    # layers' 2.7 GB each went through L2 since they were last touched ----
+    multi = None
+    if args.layers > 1:
+        try:
+            layers = []
+            for li in range(args.layers):
+                kp, vp, ln = k_pool.clone(), v_pool.clone(), lens.clone()
+                ck = binding.CompKV(w.num_q_heads, w.num_kv_heads, w.batch, max_blocks, k_pool.shape[0],
+                                    block_size=w.block_size, var_groups=w.var_groups, device=str(dev),
+                                    stat_bf16=int(args.stat_bf16))
+                ck.stats_build(kp, vp, table, ln, int(ln.max()))
+                outs = ck.alloc_outputs(w.batch, w.budget_tokens)
+                ck.step(sq, sk, sv, kp, vp, table, ln, max_len, w.budget_tokens, outs)   # eager warm-up
+                layers.append((ck, kp, vp, ln, outs))
+            torch.cuda.synchronize()
+            g_all = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_all):
+                for ck, kp, vp, ln, outs in layers:
+                    ck.step(sq, sk, sv, kp, vp, table, ln, max_len, w.budget_tokens, outs)
+            n_tok = 8
+            for _ in range(3):
+                g_all.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(n_tok):
+                g_all.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            assert all(ck.read_status() == 0 for ck, *_ in layers)
+            multi = {"layers": args.layers, "tokens": n_tok,
+                     "us_per_layer_step": e0.elapsed_time(e1) * 1e3 / (n_tok * args.layers),
+                     "note": "one CUDA graph holding one ckv_step per layer, replayed per token; no flush: each "
+                             "layer owns its own cache, summaries and workspace"}
+            del layers, g_all
+            torch.cuda.empty_cache()
+        except RuntimeError as e:   # not enough device memory for the stack
+            multi = {"layers": args.layers, "error": str(e)[:120]}
+
     # ---- dense decode attention over the same cache ----
     dense_ms = []
     dout = torch.empty_like(outputs[0])
@@ -434,6 +476,7 @@ def main():
         "us_per_step_median": float(np.median(step_ms)) * 1e3, "us_per_step_min": float(step_ms.min()) * 1e3,
         "us_per_step_warm_l2": warm_us,
         "us_per_step_back_to_back": pipe_us,
+        "multi_layer": multi,
         "us_per_step_note": "value: one graph replay per event pair, L2 flushed before it (includes the launch latency "
                             "of the graph); warm_l2: same without the flush; back_to_back: 64 replays queued inside "
                             "one event pair, no flush (every step still streams 273 MB of summaries through a "
