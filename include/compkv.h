@@ -168,6 +168,21 @@ int ckv_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_po
                int budget_tokens, void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt,
                ckv_stream stream);
 
+/* Chunked prefill: append new_lens[s] tokens to sequence s from contiguous rows and bring the summaries of every
+ * block they touch up to date, in one pass (Sec. 4.2: summaries are built as the cache is filled; the new keys and
+ * values are read once, not written first and read back by ckv_stats_build).
+ *   k_src, v_src: [batch][src_stride_tokens][num_kv_heads][head_dim], device, kv_dtype; row t of sequence s is the
+ *                 token at position seq_lens[s] + t.
+ *   new_lens:     int32 [batch] (device), 0 .. src_stride_tokens; max_new_host >= every new_lens[s] (host, sizes the grid).
+ *   seq_lens:     holds N on entry and N + new_lens once the call has run.  Tokens past the capacity
+ *                 max_blocks_per_seq * block_size are dropped and CKV_DEV_SEQ_FULL is set.
+ * The page table must already map the pages of the new positions.  A chunk may start and end anywhere inside a
+ * block; the result equals ckv_append called once per token, and ckv_stats_build over the filled cache, bit for bit.
+ * Uses the context's split counters: not to be overlapped with a decode call on another stream. */
+int ckv_prefill(ckv_ctx *ctx, void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens,
+                const void *k_src, const void *v_src, const int32_t *new_lens, int src_stride_tokens, int batch,
+                int max_new_host, ckv_stream stream);
+
 /* One decode step in one call: ckv_append(k_new, v_new) followed by ckv_decode(q, ...), with the same arguments,
  * results and errors as the two calls in that order (Sec. 4.3: the new token enters the cache and the summaries
  * before blocks are selected; seq_lens holds N on entry and N + 1 once the step has run; max_seq_len_host bounds the

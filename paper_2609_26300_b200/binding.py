@@ -23,7 +23,7 @@ CKV_ERR_CAPACITY, CKV_ERR_CUDA, CKV_ERR_TIMEOUT = -4, -5, -6
 CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_BAD_COPY = 1, 2, 4, 8, 16
 
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
-           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
+           "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_prefill", "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
            "ckv_dense_decode_static",
            "ckv_exact_blocks", "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
 
@@ -73,6 +73,8 @@ def load() -> ctypes.CDLL:
     lib.ckv_stats_build.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp]
     lib.ckv_stats_export.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.ckv_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
+    lib.ckv_prefill.restype = i32
     lib.ckv_decode.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.ckv_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.ckv_decode_profile.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp,
@@ -216,6 +218,12 @@ class CompKV:
                                    batch, int(max_seq_len), int(budget_tokens), _ptr(out), _ptr(lse), _ptr(ids),
                                    _ptr(cnt), _stream()), "ckv_decode")
         return out, lse, ids, cnt
+
+    def prefill(self, k_pool, v_pool, page_table, seq_lens, k_src, v_src, new_lens, max_new: int) -> None:
+        """ckv_prefill: k_src / v_src [batch][tokens][kv_heads][128]; new_lens int32 [batch] on the device."""
+        _check(self.lib.ckv_prefill(self._ctx, _ptr(k_pool), _ptr(v_pool), _ptr(page_table), _ptr(seq_lens),
+                                    _ptr(k_src), _ptr(v_src), _ptr(new_lens), int(k_src.shape[1]), int(k_src.shape[0]),
+                                    int(max_new), _stream()), "ckv_prefill")
 
     def step(self, q, k_new, v_new, k_pool, v_pool, page_table, seq_lens, max_seq_len: int, budget_tokens: int,
              outputs=None):

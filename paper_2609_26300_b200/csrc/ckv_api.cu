@@ -198,6 +198,17 @@ int ckv_append(ckv_ctx *c, void *k_pool, void *v_pool, const int32_t *page_table
   return CKV_OK;
 }
 
+int ckv_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens, const void *k_src,
+                const void *v_src, const int32_t *new_lens, int src_stride_tokens, int batch, int max_new_host,
+                ckv_stream stream) {
+  if (c == nullptr || batch <= 0 || batch > c->layout.max_batch) return CKV_ERR_INVALID_ARG;
+  if (!k_pool || !v_pool || !page_table || !seq_lens || !k_src || !v_src || !new_lens) return CKV_ERR_INVALID_ARG;
+  if (src_stride_tokens <= 0 || max_new_host < 0 || max_new_host > src_stride_tokens) return CKV_ERR_INVALID_ARG;
+  CKV_CUDA(ckv_launch_prefill(c, k_pool, v_pool, page_table, seq_lens, k_src, v_src, new_lens, src_stride_tokens, batch,
+                              max_new_host, (cudaStream_t)stream));
+  return CKV_OK;
+}
+
 namespace {
 
 // The four launches of a sparse decode step; ev (may be null) receives 5 events bracketing them.

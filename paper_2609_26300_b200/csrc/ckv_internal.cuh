@@ -65,6 +65,9 @@ int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len);
 cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int *page_table,
                                    const int *seq_lens, int batch, int max_len, cudaStream_t st);
 cudaError_t ckv_launch_stats_export(ckv_ctx *c, int batch, float *kmean, float *dbar, float *vmean, cudaStream_t st);
+cudaError_t ckv_launch_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
+                               const void *k_src, const void *v_src, const int *new_lens, int src_stride, int batch,
+                               int max_new, cudaStream_t st);
 cudaError_t ckv_launch_append(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
                               const void *k_new, const void *v_new, int batch, cudaStream_t st);
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,

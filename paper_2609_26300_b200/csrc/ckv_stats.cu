@@ -209,6 +209,75 @@ __global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T 
   if (threadIdx.x == 0) seq_lens[s] = N + 1;
 }
 
+// Chunked prefill: new_lens[s] tokens per sequence arrive as contiguous rows; one warp per touched block copies the
+// block's new rows into their pages and then runs the block routine over the block (rows that were already in the
+// cache included), so the new keys and values cross DRAM once on the way in and the summaries come out of the same
+// pass.  The CTA that finishes last stores the new sequence lengths (every warp read the old ones when it started).
+template <typename T>
+__global__ void __launch_bounds__(256) ckv_prefill_kernel(CkvDev P, T *k_pool, T *v_pool,
+                                                          const int *__restrict__ page_table, int *seq_lens,
+                                                          const T *__restrict__ k_src, const T *__restrict__ v_src,
+                                                          const int *__restrict__ new_lens, int src_stride, int batch) {
+  __shared__ float sq_smem[8][CKV_D];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
+  const int cap = P.max_blocks * P.bs;
+  const int N = seq_lens[s], M = new_lens[s];
+  const int m_eff = N < 0 ? 0 : max(min(min(M, src_stride), cap - N), 0);   // tokens that fit
+  if (M > m_eff && blockIdx.x == 0 && threadIdx.x == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
+  const int b = (N >= 0 ? N / P.bs : 0) + blockIdx.x * 8 + warp;
+  if (m_eff > 0 && b <= (N + m_eff - 1) / P.bs) {
+    const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
+    const int p_lo = max(b * P.bs, N), p_hi = min((b + 1) * P.bs, N + m_eff);
+    constexpr int PIECES = (int)(CKV_D * sizeof(T) / 16);   // 16-byte pieces of a row: 16 (bf16) or 32 (fp32)
+    constexpr int PP = PIECES / 16;                          // pieces per lane and row
+    bool bad = false;
+    const T *src_base = (lane < 16 ? k_src : v_src);         // lanes 0-15 copy K, lanes 16-31 copy V
+    T *dst_base = (lane < 16 ? k_pool : v_pool);
+    for (int pg = p_lo / CKV_PAGE; pg * CKV_PAGE < p_hi; ++pg) {
+      const int phys = pt_row[pg];
+      if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
+      // all rows of the page are requested before any is stored
+      uint4 r[CKV_PAGE][PP];
+#pragma unroll
+      for (int t = 0; t < CKV_PAGE; ++t) {
+        const int p = pg * CKV_PAGE + t;
+        if (p >= p_lo && p < p_hi) {
+          const uint4 *src = reinterpret_cast<const uint4 *>(src_base + (((size_t)s * src_stride + (p - N)) * P.Hkv + h) * CKV_D);
+#pragma unroll
+          for (int k = 0; k < PP; ++k) r[t][k] = __ldg(src + (lane & 15) + 16 * k);
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < CKV_PAGE; ++t) {
+        const int p = pg * CKV_PAGE + t;
+        if (p >= p_lo && p < p_hi) {
+          uint4 *dst = reinterpret_cast<uint4 *>(dst_base + (((size_t)phys * P.Hkv + h) * CKV_PAGE + t) * CKV_D);
+#pragma unroll
+          for (int k = 0; k < PP; ++k) dst[(lane & 15) + 16 * k] = r[t][k];
+        }
+      }
+    }
+    if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
+    __syncwarp();
+    const int cnt = min(P.bs, N + m_eff - b * P.bs);
+    const size_t row = (size_t)unit * P.max_blocks + b;
+    block_stats_warp<T, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * P.row_elems,
+                               P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(P.unit_done, 1) == (int)(gridDim.x * gridDim.y) - 1) {
+      P.unit_done[0] = 0;
+      for (int i = 0; i < batch; ++i) {
+        const int n = seq_lens[i];
+        if (n >= 0) seq_lens[i] = n + max(min(min(new_lens[i], src_stride), cap - n), 0);
+      }
+    }
+  }
+}
+
 // Summaries as plain fp32 arrays (hi + lo, chunks back in coordinate order): one warp per block row.
 __global__ void __launch_bounds__(256) ckv_stats_export_kernel(CkvDev P, int rows, float *__restrict__ kmean,
                                                                float *__restrict__ dbar, float *__restrict__ vmean) {
@@ -254,6 +323,24 @@ cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v
   else
     ckv_stats_build_kernel<float><<<grid, 256, 0, st>>>(P, (const float *)k_pool, (const float *)v_pool, page_table,
                                                         seq_lens);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+cudaError_t ckv_launch_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
+                               const void *k_src, const void *v_src, const int *new_lens, int src_stride, int batch,
+                               int max_new, cudaStream_t st) {
+  const CkvDev &P = c->dev;
+  if (batch <= 0 || max_new <= 0) return cudaSuccess;
+  const int touched = (max_new + P.bs - 1) / P.bs + 1;   // a chunk that starts inside a block touches one more
+  dim3 grid((touched + 7) / 8, batch * P.Hkv);
+  if (c->layout.kv_dtype == CKV_BF16)
+    ckv_prefill_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool, page_table,
+                                                            seq_lens, (const __nv_bfloat16 *)k_src,
+                                                            (const __nv_bfloat16 *)v_src, new_lens, src_stride, batch);
+  else
+    ckv_prefill_kernel<float><<<grid, 256, 0, st>>>(P, (float *)k_pool, (float *)v_pool, page_table, seq_lens,
+                                                    (const float *)k_src, (const float *)v_src, new_lens, src_stride, batch);
   c->launches++;
   return cudaGetLastError();
 }
