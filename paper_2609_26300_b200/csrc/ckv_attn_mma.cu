@@ -20,9 +20,13 @@
 //
 // Merge.  The scan's partials of the unit (one per scan CTA and consumer warp) exist before this kernel
 // starts, so the unit's active CTAs share them out, fetch their share while their last page is in flight and
-// fold it into their own partial.  Each CTA then publishes one partial (m, l, acc[128]) per head and bumps
-// the unit's counter; the CTA that finds the counter complete reads the unit's partials back (they are few)
-// and writes the output row and the log-sum-exp.  The counter is left at zero for the next step.
+// fold it into their own partial.  What is left is one partial (m, l, acc[128]) per head and CTA:
+//   * sparse mode launches the unit's splits (at most 8) as one thread-block cluster: the partials stay in shared
+//     memory, and after a cluster barrier CTA r reduces head r over all of them with distributed-shared-memory
+//     loads and writes the output row and the log-sum-exp;
+//   * dense mode (more splits than a cluster holds), and sparse mode when a cluster cannot be placed, publish the
+//     partials in global memory and bump the unit's counter; the CTA that finds the counter complete reads them
+//     back and writes the output.  The counter is left at zero for the next step.
 #include "ckv_internal.cuh"
 #include "ckv_mma.cuh"
 

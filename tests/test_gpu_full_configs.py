@@ -99,3 +99,22 @@ def test_config5_sweep_128k(bs):
         assert cnt.cpu().tolist() == [[budget // bs] * 8]
         check_unit_decode(d, 0, h, w.ctx, 0, budget, out, lse, ids, cnt, scores)
     assert d.ckv.read_status() == 0
+
+
+@pytest.mark.parametrize("kw,ck", [(dict(var_groups=128), dict(var_groups=128)),
+                                   (dict(stat_bf16=1), dict(stat_bf16=True))])
+def test_config2_other_layouts(kw, ck):
+    """The 32K configuration at the r = d operating point and with bf16 summaries, a few decode steps each."""
+    w = synth.CONFIGS[2].with_(decode_steps=3)
+    d = setup(w, **kw)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    for t in range(3):
+        k_new, v_new = synth.appended_rows(w, t)
+        out, lse, ids, cnt = d.ckv.step(torch.from_numpy(synth.queries(w, t)).bfloat16().cuda(),
+                                        torch.from_numpy(k_new).bfloat16().cuda(), torch.from_numpy(v_new).bfloat16().cuda(),
+                                        d.k_pool, d.v_pool, d.table, d.lens, w.ctx + t + 1, w.budget_tokens)
+        scores = d.ckv.copy_scores(w.batch)
+        torch.cuda.synchronize()
+        assert d.ckv.read_status() == 0
+        for h in (1, 6):
+            check_unit_decode(d, 0, h, w.ctx + t + 1, t, w.budget_tokens, out, lse, ids, cnt, scores, **ck)
