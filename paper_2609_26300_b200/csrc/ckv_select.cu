@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   __shared__ int s_hist[kBins];
   __shared__ float s_M[G], s_invL[G];
   __shared__ int s_wtot[32];
-  __shared__ int s_total, s_digit, s_remaining, s_cfirst, s_ccount, s_ncand;
+  __shared__ int s_total, s_digit, s_remaining, s_ncand;
   __shared__ int s_cand[kThreads];
   __shared__ uint32_t s_candk[kThreads];   // the candidates' keys, so that the ranking loop reads no key through an id
 
@@ -71,13 +71,28 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
     // scores are still produced below for callers that read them
   }
 
-  // ---- where the scan partials of this unit live (entries (c + unit) * W + w, c in [cfirst, cfirst + ccount)) ----
-  if (warp == 0) {
+  // ---- normalisers of Eq. 9: M_g, L_g from the scan partials of this unit (entries (c + unit) * W + w, c in
+  // [cfirst, cfirst + ccount)).  Warp g works them out for head g; its loads are issued before the much larger
+  // batch of score-term loads below, which would otherwise sit in front of them in the memory pipeline. ----
+  if (tid == 0) s_ncand = 0;
+  for (int i = tid; i < kBins; i += kThreads) s_hist[i] = 0;   // the first radix pass fills it while scoring
+  float pm[4], pl[4];
+  const float *cp = nullptr;
+  int n_part = 0;
+  const size_t pstep = (size_t)G * CKV_PART_STRIDE;
+  if (warp < G) {
     int cfirst, ccount;
     unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
-    if (lane == 0) { s_cfirst = cfirst; s_ccount = ccount; s_ncand = 0; }
+    cp = P.comp_part + ((size_t)(cfirst + unit) * CKV_SCAN_WARPS * G + warp) * CKV_PART_STRIDE;
+    n_part = ccount * CKV_SCAN_WARPS;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = lane + 32 * k;
+      pm[k] = i < n_part ? cp[i * pstep] : -CUDART_INF_F;
+      pl[k] = i < n_part ? cp[i * pstep + 2] : 0.f;
+    }
   }
-  // the first batch of (l, sigma^2) loads does not depend on the normalisers: start it before waiting for them
+  // the first batch of (l, sigma^2) loads does not depend on the normalisers: it is in flight while they are reduced
   constexpr int NB = G >= 8 ? 2 : 4;   // blocks per thread and batch (their loads are in flight together)
   const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
   float *scores = P.scores + (size_t)unit * P.max_blocks;
@@ -93,26 +108,14 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
     }
   };
   load_batch(0);
-  __syncthreads();
-  // ---- normalisers of Eq. 9: M_g, L_g from the partials (one round of loads for up to 128 partials) ----
   if (warp < G) {
-    const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * CKV_SCAN_WARPS * G + warp) * CKV_PART_STRIDE;
-    const size_t step = (size_t)G * CKV_PART_STRIDE;
-    const int n_part = s_ccount * CKV_SCAN_WARPS;
-    float pm[4], pl[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int i = lane + 32 * k;
-      pm[k] = i < n_part ? cp[i * step] : -CUDART_INF_F;
-      pl[k] = i < n_part ? cp[i * step + 2] : 0.f;
-    }
     float m = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
-    for (int i = lane + 128; i < n_part; i += 32) m = fmaxf(m, cp[i * step]);
+    for (int i = lane + 128; i < n_part; i += 32) m = fmaxf(m, cp[i * pstep]);
     m = warp_max(m);
     float l = 0.f;
 #pragma unroll
     for (int k = 0; k < 4; ++k) l = fmaf(pl[k], exp2_diff(pm[k], m), l);
-    for (int i = lane + 128; i < n_part; i += 32) l = fmaf(cp[i * step + 2], exp2_diff(cp[i * step], m), l);
+    for (int i = lane + 128; i < n_part; i += 32) l = fmaf(cp[i * pstep + 2], exp2_diff(cp[i * pstep], m), l);
     l = warp_sum(l);
     if (lane == 0) { s_M[warp] = m; s_invL[warp] = 1.0f / l; }
   }
@@ -122,6 +125,12 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   float Mg[G], iL[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) { Mg[g] = s_M[g]; iL[g] = s_invL[g]; }
+  const int n_tail = min(P.recent, X);
+  auto mandatory = [&](int b) { return b < P.sink || b >= X - n_tail; };
+  int nF = min(P.sink, X) + n_tail;
+  if (P.sink + n_tail > X) nF = X;
+  const int Kr = K - nF;   // blocks to rank in (the host guarantees K >= sink + recent when K < X)
+  const bool hist0 = X > kcap && Kr > 0;   // the first radix pass (top 12 bits of every ranked key) is built on the fly
   const bool cached = X <= kSmemKeys;
   const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;   // ablation: rank by estimated mass alone
   bool nonfinite = false;
@@ -138,6 +147,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
         if (!(sc >= 0.f) || sc > 3.0e38f) { nonfinite = true; sc = 0.f; }
         scores[b] = sc;
         if (cached) skeys[b] = __float_as_uint(sc);
+        if (hist0 && !mandatory(b)) atomicAdd(&s_hist[__float_as_uint(sc) >> 20], 1);
       }
     }
   }
@@ -146,11 +156,6 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   if (X <= kcap) return;
 
   const uint32_t *keys = cached ? skeys : reinterpret_cast<const uint32_t *>(scores);
-  const int n_tail = min(P.recent, X);
-  auto mandatory = [&](int b) { return b < P.sink || b >= X - n_tail; };
-  int nF = min(P.sink, X) + n_tail;
-  if (P.sink + n_tail > X) nF = X;
-  const int Kr = K - nF;   // blocks to rank in (the host guarantees K >= sink + recent when K < X)
 
   // ---- the Kr-th largest ranked score: one 12-bit radix pass, then either a direct ranking of the blocks in the
   //      digit bin that holds it (the usual case: a few dozen blocks) or the remaining radix passes ----
@@ -164,14 +169,16 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
     for (int pass = 0; pass < 3; ++pass) {
       const int shift = pass == 0 ? 20 : (pass == 1 ? 8 : 0);
       const int bins = pass == 2 ? 256 : kBins;
-      for (int i = tid; i < bins; i += kThreads) s_hist[i] = 0;
-      __syncthreads();
-      for (int b = tid; b < X; b += kThreads) {
-        if (mandatory(b)) continue;
-        const uint32_t k = keys[b];
-        if ((k & pmask) == prefix) atomicAdd(&s_hist[(k >> shift) & (bins - 1)], 1);
+      if (pass > 0) {   // pass 0's histogram was built while the scores were computed
+        for (int i = tid; i < bins; i += kThreads) s_hist[i] = 0;
+        __syncthreads();
+        for (int b = tid; b < X; b += kThreads) {
+          if (mandatory(b)) continue;
+          const uint32_t k = keys[b];
+          if ((k & pmask) == prefix) atomicAdd(&s_hist[(k >> shift) & (bins - 1)], 1);
+        }
+        __syncthreads();
       }
-      __syncthreads();
       // thread t owns the four bins bins-1-4t ... bins-4-4t (highest digits first)
       int c[4], c4 = 0;
 #pragma unroll
@@ -268,11 +275,23 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
       if (sel) emit(b);
     }
   };
+  // one pass decides; the thread's selected blocks are remembered as a bit mask (ranges longer than 32 walk twice)
   int c_sel = 0;
-  walk([&](int) { ++c_sel; });
+  uint32_t picked = 0;
+  const bool masked = per <= 32;
+  walk([&](int b) { ++c_sel; if (masked) picked |= 1u << (b - b0); });
   int pos = block_exclusive_scan(c_sel, s_wtot, &s_total);
   const int total = s_total;
-  walk([&](int b) { if (pos < kcap) ids[pos] = b; ++pos; });
+  if (masked) {
+    while (picked != 0) {
+      const int j = __ffs(picked) - 1;
+      picked &= picked - 1;
+      if (pos < kcap) ids[pos] = b0 + j;
+      ++pos;
+    }
+  } else {
+    walk([&](int b) { if (pos < kcap) ids[pos] = b; ++pos; });
+  }
   for (int i = total + tid; i < kcap; i += kThreads) ids[i] = -1;
   if (tid == 0) sel_cnt[unit] = min(total, kcap);
 }
