@@ -35,7 +35,7 @@ int check_layout(const ckv_layout *L) {
 
 struct Regions {
   size_t kmean, dbar, vmean, stats_total;
-  size_t ls, scores, comp, attn, status, done, stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt, work_total;
+  size_t ls, lz, scores, comp, attn, status, done, stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt, work_total;
 };
 
 Regions regions(const ckv_layout *L) {
@@ -53,7 +53,8 @@ Regions regions(const ckv_layout *L) {
   o = 0;
   R.status = o; o = align_up(o + 256, 256);
   R.done = o;   o = align_up(o + units * 4, 256);
-  R.ls = o;     o = align_up(o + rows * G * sizeof(float2), 256);
+  R.ls = o;     o = align_up(o + rows * G * sizeof(float), 256);
+  R.lz = o;     o = align_up(o + rows * G * sizeof(float), 256);
   R.scores = o; o = align_up(o + rows * 4, 256);
   R.comp = o;   o = align_up(o + (units + CKV_MAX_SCAN_CTAS) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE * 4, 256);
   R.attn = o;   o = align_up(o + units * CKV_MAX_SPLITS * G * CKV_PART_STRIDE * 4, 256);
@@ -152,7 +153,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.half_var = (layout->variant & CKV_VARIANT_FIRST_ORDER_MASS) ? 0.f : 0.5f;
   P.kmean = (__nv_bfloat16 *)(sb + R.kmean); P.dbar = (float *)(sb + R.dbar); P.vmean = (__nv_bfloat16 *)(sb + R.vmean);
   P.status = (int *)(wb + R.status); P.unit_done = (int *)(wb + R.done);
-  P.ls = (float2 *)(wb + R.ls); P.scores = (float *)(wb + R.scores);
+  P.lu = (float *)(wb + R.ls); P.lz = (float *)(wb + R.lz); P.scores = (float *)(wb + R.scores);
   P.comp_part = (float *)(wb + R.comp); P.attn_part = (float *)(wb + R.attn);
   c->work = wb; c->work_bytes = work_bytes;
   c->stage_q = R.stage_q; c->stage_knew = R.stage_knew; c->stage_vnew = R.stage_vnew;

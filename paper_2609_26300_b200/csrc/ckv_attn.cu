@@ -127,7 +127,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
   // after the reduction this lane owns row (li / 2) of its half warp and heads [g_own0, g_own0 + KEEP)
   const int g_own0 = (G >= 2) ? (li & 1) * KEEP : 0;
   const int t_own = hw + 2 * (li >> 1);
-  const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
+  const float *lz = P.lz + (size_t)unit * P.max_blocks * G;
   const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * P.row_elems;
   uint32_t phase_bits = 0;   // bit b: parity of the next completion of buffer b
   bool aborted = false;
@@ -221,8 +221,7 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
         bool raise = false;
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-          const float2 v = __ldg(ls + (size_t)g * P.max_blocks + blk);
-          zl2[g] = (v.x - P.half_var * v.y) * kLog2e;
+          zl2[g] = __ldg(lz + (size_t)g * P.max_blocks + blk);
           raise |= zl2[g] > m_ref[g] + CKV_RESCALE_SLACK;
         }
         if (raise) {   // warp-uniform: every lane evaluates the same values

@@ -38,7 +38,7 @@ constexpr int kRowBytes = CKV_D * 2;                  // 256
 constexpr int kMeanSlots = 4;                         // mean-value rows (512 B each) a warp can hold
 constexpr int kMeanFlush = 3;                         // ... of which at most 3 wait for removal while one is in flight
 constexpr int kZeroRow = kMeanSlots * 512;            // offset of the row of zeros inside the aux area
-constexpr int kLsOff = kZeroRow + 256;                // then the blocks' (logit, variance) pairs: [slot][G] float2
+constexpr int kLsOff = kZeroRow + 256;                // then log2 of the blocks' mean-compensation weights: [slot][G] float
 constexpr int kAuxBytes = kLsOff + 256;
 constexpr int kMaxEntries = 32;                       // partials a CTA folds per round: one per lane
 constexpr int kPartBytes = CKV_PART_STRIDE * 4;       // one head's partial
@@ -49,8 +49,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool v
   // valid == false copies nothing and zero-fills the 16 bytes
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
 }
-__device__ __forceinline__ void cp_async8(uint32_t dst, const void *src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -178,7 +178,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   float m_ref = -CUDART_INF_F, l_acc = 0.f;
   const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
   const int n_mine = max((p1 - p0 - warp + W - 1) / W, 0);   // this warp's pages: list index p0 + warp + W n
-  const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
+  const float *lz = P.lz + (size_t)unit * P.max_blocks * G;
   const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * P.row_elems;
   const bool mean_lo = P.row_elems == CKV_ROW_ELEMS;   // the mean-value rows carry lo halves (fp32-precision summaries)
   bool bad = false;
@@ -264,8 +264,8 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
       if (comp && r.first) {   // verbatim: hi halves then lo halves, swizzled by block index
         if (mean_lo || lane < 16)
           cp_async16(aux_u32 + 512 * slot + 16 * lane, vmean + (size_t)r.blk * P.row_elems + 8 * lane, true);
-        if (lane < G)          // and the block's (logit, variance) of every head, for the weight of its mean term
-          cp_async8(aux_u32 + kLsOff + (slot * G + lane) * 8, ls + (size_t)lane * P.max_blocks + r.blk);
+        if (lane < G)          // and log2 of the weight of its mean term, for every head
+          cp_async4(aux_u32 + kLsOff + (slot * G + lane) * 4, lz + (size_t)lane * P.max_blocks + r.blk);
       }
     }
   };
@@ -283,8 +283,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         const int j = 2 * qd + e;
         if (j < nb) {
           const int slot = j == 0 ? bsl[0] : (j == 1 ? bsl[1] : bsl[2]);
-          const float2 v = *reinterpret_cast<const float2 *>(waux + kLsOff + (slot * G + head) * 8);
-          zl[e] = (v.x - P.half_var * v.y) * kLog2e;
+          zl[e] = *reinterpret_cast<const float *>(waux + kLsOff + (slot * G + head) * 4);
         }
       }
     }

@@ -30,7 +30,8 @@ struct CkvDev {
   __nv_bfloat16 *kmean, *vmean;   // [unit][max_blocks][CKV_ROW_ELEMS]
   float *dbar;                    // [unit][max_blocks][r]
   // workspace
-  float2 *ls;        // [unit][G][max_blocks]  (log block weight estimate l_{g,b}, sigma_hat^2_{g,b})
+  float *lu;         // [unit][G][max_blocks]  log2 of the head's score term e^{l_{g,b}} sigma_hat^2_{g,b} (selection reads it)
+  float *lz;         // [unit][G][max_blocks]  log2 of the block's mean-compensation weight |b| e^{zbar_{g,b}} (attention)
   float *scores;     // [unit][max_blocks]     S_b
   float *comp_part;  // [(scan CTA + unit) * CKV_SCAN_WARPS + warp][G][CKV_PART_STRIDE]  all-block mean-compensation partials
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials

@@ -170,11 +170,13 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     float wown[4] = {0.f, 0.f, 0.f, 0.f};
     float *sw = sw_all + (size_t)warp * P.r * G;   // [t][g], r != 4 only
     const float log_bs = logf((float)P.bs);
+    const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;
+    const bool pair_ok = (P.max_blocks & 1) == 0;   // rows of the per-block outputs start on 8-byte boundaries
     float log_last = 0.f;
     const int ulast = s_ulast;
     int u = s_u0, tl = s_tl0, cur = -1, next_empty = s_u0;
     UnitInfo ui = unit_info(P, s_len, seq_lens, u);
-    float2 *ls = nullptr;
+    float *lu = nullptr, *lz = nullptr;
     const float *db = nullptr;
     bool aborted = false;
 
@@ -288,7 +290,8 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
         m_ref = -CUDART_INF_F; l_acc = 0.f; lp_acc = 0.f;
         log_last = logf((float)(ui.N - (ui.X - 1) * P.bs));
         const size_t row0 = (size_t)u * P.max_blocks;
-        ls = P.ls + row0 * G;   // [head][block] within the unit
+        lu = P.lu + row0 * G;   // [head][block] within the unit
+        lz = P.lz + row0 * G;
         db = P.dbar + row0 * P.r;
         cur = u;
       }
@@ -388,10 +391,19 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
             zl2[nt][e] = val[nt][e] ? (zbar + logc) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
             tmax = fmaxf(tmax, zl2[nt][e]);
           }
-          // 8-byte stores: a head's row of (l, sigma^2) pairs starts at head * max_blocks, which may be odd
-          float2 *lrow = ls + (size_t)head * P.max_blocks + b0 + r0;
-          if (val[nt][0]) lrow[0] = make_float2(ell[0], sig[nt][0]);
-          if (val[nt][1]) lrow[1] = make_float2(ell[1], sig[nt][1]);
+          // what the later kernels read, both in log2 units: the head's term of the block score, e^l sigma^2 (e^l
+          // alone when blocks are ranked by mass), and the block's mean-compensation weight |b| e^{zbar}.  The
+          // thread's two blocks are neighbours: one 8-byte store each when the rows are 8-byte aligned.
+          const size_t o = (size_t)head * P.max_blocks + b0 + r0;
+          const float u0 = fmaf(ell[0], kLog2e, by_mass ? 0.f : __log2f(sig[nt][0]));
+          const float u1 = fmaf(ell[1], kLog2e, by_mass ? 0.f : __log2f(sig[nt][1]));
+          if (pair_ok && val[nt][1]) {
+            *reinterpret_cast<float2 *>(lu + o) = make_float2(u0, u1);
+            *reinterpret_cast<float2 *>(lz + o) = make_float2(zl2[nt][0], zl2[nt][1]);
+          } else {
+            if (val[nt][0]) { lu[o] = u0; lz[o] = zl2[nt][0]; }
+            if (val[nt][1]) { lu[o + 1] = u1; lz[o + 1] = zl2[nt][1]; }
+          }
         }
         tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
         tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));

@@ -93,17 +93,17 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
     }
   }
   // the first batch of (l, sigma^2) loads does not depend on the normalisers: it is in flight while they are reduced
-  constexpr int NB = G >= 8 ? 2 : 4;   // blocks per thread and batch (their loads are in flight together)
-  const float2 *ls = P.ls + (size_t)unit * P.max_blocks * G;
+  constexpr int NB = G >= 8 ? 4 : 8;   // blocks per thread and batch (their loads are in flight together)
+  const float *lu = P.lu + (size_t)unit * P.max_blocks * G;   // log2(e^l sigma^2) per head and block, from the scan
   float *scores = P.scores + (size_t)unit * P.max_blocks;
-  float2 v[NB][G];
+  float v[NB][G];
   auto load_batch = [&](int base) {
 #pragma unroll
     for (int j = 0; j < NB; ++j) {
       const int b = base + j * kThreads + tid;
       if (b < X) {
 #pragma unroll
-        for (int g = 0; g < G; ++g) v[j][g] = ls[(size_t)g * P.max_blocks + b];   // head-major: coalesced per head
+        for (int g = 0; g < G; ++g) v[j][g] = lu[(size_t)g * P.max_blocks + b];   // head-major: coalesced per head
       }
     }
   };
@@ -132,7 +132,6 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   const int Kr = K - nF;   // blocks to rank in (the host guarantees K >= sink + recent when K < X)
   const bool hist0 = X > kcap && Kr > 0;   // the first radix pass (top 12 bits of every ranked key) is built on the fly
   const bool cached = X <= kSmemKeys;
-  const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;   // ablation: rank by estimated mass alone
   bool nonfinite = false;
   for (int base = 0; base < X; base += NB * kThreads) {
     if (base > 0) load_batch(base);
@@ -142,8 +141,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
       if (b < X) {
         float sc = 0.f;
 #pragma unroll
-        for (int g = 0; g < G; ++g)
-          sc = fmaf(fast_exp2(fmaf(v[j][g].x, kLog2e, -Mg[g])) * iL[g], by_mass ? 1.0f : v[j][g].y, sc);
+        for (int g = 0; g < G; ++g) sc = fmaf(fast_exp2(v[j][g] - Mg[g]), iL[g], sc);
         if (!(sc >= 0.f) || sc > 3.0e38f) { nonfinite = true; sc = 0.f; }
         scores[b] = sc;
         if (cached) skeys[b] = __float_as_uint(sc);
@@ -279,7 +277,19 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   int c_sel = 0;
   uint32_t picked = 0;
   const bool masked = per <= 32;
-  walk([&](int b) { ++c_sel; if (masked) picked |= 1u << (b - b0); });
+  if (ranked && cached && masked) {
+    // the usual case in one comparison per key: marked keys carry the sign bit and every key of a higher bin is at
+    // least (digit + 1) << 20, so "selected" is an unsigned >= ; mandatory blocks only matter at the two ends
+    const uint32_t floor_key = (digit0 + 1u) << 20;
+    const bool ends = b0 < P.sink || b1 > X - n_tail;
+    for (int b = b0; b < b1; ++b) {
+      const bool sel = skeys[b] >= floor_key || (ends && mandatory(b));
+      c_sel += sel ? 1 : 0;
+      picked |= (sel ? 1u : 0u) << (b - b0);
+    }
+  } else {
+    walk([&](int b) { ++c_sel; if (masked) picked |= 1u << (b - b0); });
+  }
   int pos = block_exclusive_scan(c_sel, s_wtot, &s_total);
   const int total = s_total;
   if (masked) {
