@@ -91,6 +91,15 @@ def test_null_arguments_are_rejected_before_any_cuda_call():
         == binding.CKV_ERR_INVALID_ARG
     assert lib.ckv_append(None, None, None, None, None, None, None, 1, None) == binding.CKV_ERR_INVALID_ARG
     assert lib.ckv_launch_count(None) == 0
+    # the entry points added after the first ones: a null context is refused before anything else is looked at
+    bad = binding.CKV_ERR_INVALID_ARG
+    assert lib.ckv_step(None, None, None, None, None, None, None, None, 1, 16, 64, None, None, None, None, None) == bad
+    assert lib.ckv_prefill(None, None, None, None, None, None, None, None, 16, 1, 16, None) == bad
+    assert lib.ckv_exact_blocks(None, None, None, None, None, 1, 16, None, None, None, None) == bad
+    assert lib.ckv_scan_profile(None, None, None, 1, 16, 1, None, None) == bad
+    assert lib.ckv_dense_decode(None, None, None, None, None, None, 1, 16, None, None, None) == bad
+    assert lib.ckv_stats_build(None, None, None, None, None, 1, 16, None) == bad
+    assert lib.ckv_dense_decode_static(None, None, None, None, None, None, 1, 16, None, None, None) == bad
     lib.ckv_destroy(None)
 
 
