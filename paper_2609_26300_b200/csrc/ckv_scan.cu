@@ -5,8 +5,8 @@
 //   zbar_{g,b}        = q_g . kbar_b * scale                      (block-mean logit, Sec. 4.1)
 //   sigma_hat^2_{g,b} = scale^2 sum_t w_{g,t} Dbar_{b,t}         (Eq. 8 with 1/d = scale^2, w_{g,t} = sum_{i in G_t} q_{g,i}^2)
 //   l_{g,b}           = log|b| + zbar + sigma_hat^2 / 2           (log of the numerator of Eq. 9)
-// and stores (l, sigma_hat^2) for the selection kernel, together with partials of the normaliser of
-// Eq. 9.  In the same pass it accumulates the mean-compensation terms of Eq. 12 over ALL blocks,
+// and stores, in log2 units, e^l sigma_hat^2 for the selection kernel and |b| e^{zbar} for the attention kernel
+// (4 bytes each per head and block), together with partials of the normaliser of Eq. 9.  In the same pass it accumulates the mean-compensation terms of Eq. 12 over ALL blocks,
 // sum_b |b| e^{zbar} vbar_b  and  sum_b |b| e^{zbar},  as online-softmax partials; the terms of the
 // blocks that end up selected are taken out again by the attention kernel.  That way kbar, Dbar and
 // vbar are each read from HBM exactly once per decode step.

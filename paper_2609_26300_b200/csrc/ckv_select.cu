@@ -5,11 +5,14 @@
 //   S          = F  u  TopK_{K-|F|} { S_b : b not in F },  ids ascending        (Eq. 11)
 // F = first `sink` and last `recent` blocks.  Equal scores go to the lower block id.
 //
-// The normalisers (M_g, L_g) arrive as per-CTA partials from the scan kernel, so the (l, sigma^2)
-// pairs are read once.  The K-th largest score is found exactly with a most-significant-digit-first
-// radix select on the fp32 bit patterns (scores are >= 0, so unsigned order is numeric order), 12 +
-// 12 + 8 bits with a 4096-bin shared-memory histogram; ids come out in position order from a
-// prefix sum over selection flags.
+// The scan kernel leaves, per head and block, u_{g,b} = log2(e^{l_{g,b}} sigma_hat^2_{g,b}) (4 bytes) and the
+// normalisers (M_g, L_g) as per-CTA partials, so S_b = sum_g 2^{u_{g,b} - M_g} / L_g and every term is read
+// once.  The normaliser loads are issued before the (much larger) batch of u loads, which would otherwise sit in
+// front of them in the memory pipeline.  The K-th largest score is found exactly with a most-significant-
+// digit-first radix select on the fp32 bit patterns (scores are >= 0, so unsigned order is numeric order): a
+// 4096-bin histogram of the top 12 bits, built while the scores are computed, then a direct ranking of the blocks
+// in the bin that holds the threshold (falling back to 12 + 8 more bits on heavy ties); ids come out in position
+// order from a prefix sum over selection flags.
 #include "ckv_internal.cuh"
 
 namespace {
