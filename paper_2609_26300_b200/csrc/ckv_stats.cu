@@ -181,6 +181,16 @@ __global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   const int s = blockIdx.x;
   const int N = seq_lens[s];
+  // the new row of this warp's first head does not depend on N: it is requested together with it, so that the
+  // chain length -> page -> row has no fourth link (16-byte pieces: lanes 0-15 hold K, lanes 16-31 hold V)
+  constexpr int PIECES = (int)(CKV_D * sizeof(T) / 16);
+  constexpr int PP = PIECES / 16;
+  uint4 fresh[PP];
+  if (warp < P.Hkv) {
+    const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + ((size_t)s * P.Hkv + warp) * CKV_D);
+#pragma unroll
+    for (int k = 0; k < PP; ++k) fresh[k] = __ldg(src + (lane & 15) + 16 * k);
+  }
   __syncthreads();   // every warp has read N before thread 0 may change it
   if (N < 0 || N >= P.max_blocks * P.bs) {
     if (threadIdx.x == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
@@ -193,12 +203,15 @@ __global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T 
   const int b = N / P.bs, cnt = N + 1 - b * P.bs;
   for (int h = warp; h < P.Hkv; h += nwarps) {
     if (ok) {
-      // 16-byte pieces of the new row: lanes 0-15 copy K, lanes 16-31 copy V
-      constexpr int PIECES = (int)(CKV_D * sizeof(T) / 16);
-      const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + ((size_t)s * P.Hkv + h) * CKV_D);
+      if (h != warp) {   // further heads of this warp (more KV heads than warps)
+        const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + ((size_t)s * P.Hkv + h) * CKV_D);
+#pragma unroll
+        for (int k = 0; k < PP; ++k) fresh[k] = __ldg(src + (lane & 15) + 16 * k);
+      }
       uint4 *dst = reinterpret_cast<uint4 *>((lane < 16 ? k_pool : v_pool) +
                                              (((size_t)phys * P.Hkv + h) * CKV_PAGE + slot) * CKV_D);
-      for (int i = lane & 15; i < PIECES; i += 16) dst[i] = src[i];
+#pragma unroll
+      for (int k = 0; k < PP; ++k) dst[(lane & 15) + 16 * k] = fresh[k];
     }
     __syncwarp();
     const size_t row = ((size_t)s * P.Hkv + h) * P.max_blocks + b;
