@@ -141,6 +141,19 @@ def test_bf16_summaries_layout(bs, hq):
     decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), fused=True, stat_bf16=True)
 
 
+@pytest.mark.parametrize("blocks", [70, 71, 72, 73])
+def test_decode_with_odd_and_even_row_strides(blocks):
+    """max_blocks_per_seq = 70 .. 73: the per-block outputs of the scan are stored in pairs only when their rows start
+    on 8-byte boundaries; both forms must give the same step."""
+    w = small(ctx=16 * blocks - 3, decode_steps=0)
+    d = setup(w)
+    assert d.ckv.layout.max_blocks_per_seq == blocks
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, int(d.lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores)
+
+
 def test_decode_toy_config_fp32_and_bf16():
     for dtype in (torch.float32, torch.bfloat16):
         d = setup(TOY, dtype)
