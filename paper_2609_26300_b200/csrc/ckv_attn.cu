@@ -463,11 +463,19 @@ cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k
   const int total = dense ? (max_len + CKV_PAGE - 1) / CKV_PAGE : min(kcap, xmax) * P.ppb;
   const bool mma = c->layout.kv_dtype == CKV_BF16;
   const int sms = c->sm_count > 0 ? c->sm_count : 148;
-  // Splits per unit: the selected list is short, so the tensor-core kernel gets one wave of three CTAs per SM; the
-  // dense pass (and the fp32 kernel) about four CTAs per SM overall.  At least eight pages per split, at most
-  // CKV_MAX_SPLITS splits.
-  int n_splits = (mma && !dense) ? max(1, min(3 * sms / units, 8)) : (sms * 4 + units - 1) / units;   // 16: one cluster
-  n_splits = max(1, min(n_splits, min(CKV_MAX_SPLITS, (total + 7) / 8)));
+  // Splits per unit: the dense pass (and the fp32 kernel) get about four CTAs per SM overall; the tensor-core
+  // kernel's sparse mode is sized below.  At most CKV_MAX_SPLITS splits.
+  int n_splits = (sms * 4 + units - 1) / units;
+  if (mma && !dense) {
+    // Up to 8 splits of a unit run as one cluster and merge in shared memory.  With so few units that 8 splits each
+    // would leave most SMs idle, many short splits (merged through global memory) finish sooner.
+    // (measured: about 1.75 CTAs per SM is the best grid there; more, shorter splits cost more in the merge)
+    const int by_sm = max(1, 3 * sms / units);
+    n_splits = (by_sm > 8 && units * 16 <= sms) ? (7 * sms / 4 + units - 1) / units : min(by_sm, 8);
+  }
+  // at least one page per warp of a split: 8-warp CTAs everywhere except the tensor-core kernel's sparse mode (4 warps)
+  const int min_pages = (mma && !dense) ? 4 : 8;
+  n_splits = max(1, min(n_splits, min(CKV_MAX_SPLITS, (total + min_pages - 1) / min_pages)));
   int pps = (total + n_splits - 1) / n_splits;
   if (!(mma && !dense)) pps = (pps + 7) / 8 * 8;   // the tensor-core kernel deals pages to its warps one by one
   n_splits = max(1, (total + pps - 1) / pps);

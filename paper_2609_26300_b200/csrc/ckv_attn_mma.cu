@@ -610,7 +610,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
 }
 
 constexpr int kSparseWarps = 4, kDenseWarps = 8;
-constexpr int kMaxCluster = 16;   // splits of a unit that can be one cluster (8 is portable, 16 needs an opt-in)
+constexpr int kMaxCluster = 8;    // splits of a unit that can be one cluster (the portable size; 13 measured far slower)
 
 // Whether `n_splits` sparse CTAs of this instantiation can be placed as one cluster on the current device.
 template <int G>
@@ -673,9 +673,6 @@ cudaError_t configure_g() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, true>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem<kSparseWarps>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, true>,
-                             cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   return e;
 }
 
