@@ -133,6 +133,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   int nF = min(P.sink, X) + n_tail;
   if (P.sink + n_tail > X) nF = X;
   const int Kr = K - nF;   // blocks to rank in (the host guarantees K >= sink + recent when K < X)
+  if (tid == 0) { s_remaining = Kr; s_total = 0; }   // read after the barrier that follows the scoring loop
   const bool hist0 = X > kcap && Kr > 0;   // the first radix pass (top 12 bits of every ranked key) is built on the fly
   const bool cached = X <= kSmemKeys;
   bool nonfinite = false;
@@ -161,8 +162,6 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   // ---- the Kr-th largest ranked score: one 12-bit radix pass, then either a direct ranking of the blocks in the
   //      digit bin that holds it (the usual case: a few dozen blocks) or the remaining radix passes ----
   uint32_t prefix = 0, pmask = 0;
-  if (tid == 0) { s_remaining = Kr; s_total = 0; }
-  __syncthreads();
   int eq_total = 0;   // blocks scoring exactly the threshold (radix path)
   bool ranked = false;   // direct-ranking path taken: chosen blocks carry the sign bit in skeys
   if (Kr > 0) {
