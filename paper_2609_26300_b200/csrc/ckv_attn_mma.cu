@@ -540,7 +540,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     cp_async_commit();
     cp_async_wait<0>();
   }
-  if (CL) {
+  if constexpr (CL) {
     __syncthreads();   // every entry has been read: the CTA's partial takes the start of the shared memory
 #pragma unroll
     for (int it = 0; it < NI; ++it) {
@@ -550,7 +550,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     if (tid < G) { sf[tid * CKV_PART_STRIDE] = s_M[tid]; sf[tid * CKV_PART_STRIDE + 1] = s_den[tid]; }
     cluster_merge();
     return;
-  }
+  } else {
 #pragma unroll
   for (int it = 0; it < NI; ++it) {
     const int idx = tid + it * W * 32;
@@ -607,6 +607,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     *reinterpret_cast<uint2 *>(out + ((size_t)s * P.Hq + h * G + g) * CKV_D + c4) = o2;
     if (lse != nullptr && lane == 0) lse[(size_t)s * P.Hq + h * G + g] = (M + log2f(den)) * kLn2;
   }
+  }   // !CL
 }
 
 constexpr int kSparseWarps = 4, kDenseWarps = 8;

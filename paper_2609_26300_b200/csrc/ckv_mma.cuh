@@ -21,6 +21,7 @@ __device__ __forceinline__ void mma_rows8(float &d0, float &d1, uint32_t a0, uin
                "{%0, %1, %9, %9};"
                : "+f"(d0), "+f"(d1), "=f"(x), "=f"(y)
                : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
+  (void)x; (void)y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
