@@ -21,9 +21,11 @@
 // Merge.  The scan's partials of the unit (one per scan CTA and consumer warp) exist before this kernel
 // starts, so the unit's active CTAs share them out, fetch their share while their last page is in flight and
 // fold it into their own partial.  What is left is one partial (m, l, acc[128]) per head and CTA:
-//   * sparse mode launches the unit's splits (at most 8) as one thread-block cluster: the partials stay in shared
-//     memory, and after a cluster barrier CTA r reduces head r over all of them with distributed-shared-memory
-//     loads and writes the output row and the log-sum-exp;
+//   * sparse mode launches the unit's splits (at most 8) as one thread-block cluster: every CTA stores its
+//     partial of head g into the shared memory of CTA g mod cluster size (distributed-shared-memory stores), and
+//     after one cluster barrier that CTA reduces the head from its own shared memory and writes the output row
+//     and the log-sum-exp.  Nobody's shared memory is read remotely, so no CTA waits for another before it
+//     leaves (the pull version, remote loads between two barriers, was 3 us slower per step);
 //   * dense mode (more splits than a cluster holds), and sparse mode when a cluster cannot be placed, publish the
 //     partials in global memory and bump the unit's counter; the CTA that finds the counter complete reads them
 //     back and writes the output.  The counter is left at zero for the next step.
@@ -68,16 +70,16 @@ __device__ __forceinline__ uint32_t cluster_map(uint32_t local, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
   return r;
 }
-__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-  return v;
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
-__device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t addr) {
-  float2 v;
-  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
-  return v;
+__device__ __forceinline__ void st_cluster_f32x2(uint32_t addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
+
+constexpr int kMaxCluster = 8;    // splits of a unit that can be one cluster (the portable size; 13 measured far slower)
 
 template <int G, bool DENSE, int W, bool CL>
 __global__ void __launch_bounds__(W * 32, DENSE ? 1 : (W <= 4 ? 3 : 2))
@@ -89,6 +91,10 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   extern __shared__ __align__(128) unsigned char smem[];   // [W warps][2 buffers][K tile | V tile], then [W warps][aux]
   __shared__ float s_M[G], s_den[G];
   __shared__ int s_last;
+  // Cluster merge: where the other splits of the unit deposit their partials of the heads this CTA reduces.
+  // Entry (j * cluster size + source rank) belongs to head (this rank + j * cluster size).
+  __shared__ __align__(16) float s_recv[CL ? (G + kMaxCluster) * CKV_PART_STRIDE : 4];
+  if (CL) cluster_arrive_relaxed();   // first phase of the cluster barrier: "this CTA runs, its shared memory exists"
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int head = lane >> 2, qd = lane & 3;
@@ -112,37 +118,51 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   const bool comp = !DENSE && nsel < X && !(P.variant & CKV_VARIANT_DROP);
   const int p1 = min(p0 + pages_per_split, total);
   float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
-  // Cluster merge: every CTA of the cluster (= every split of the unit) has put its partial [G][CKV_PART_STRIDE] at the
-  // start of its dynamic shared memory; CTA r reduces head r, r + cluster size, ... over all of them and writes the
-  // output rows.  Both cluster barriers are reached by every CTA of the cluster, with or without pages.
-  auto cluster_merge = [&]() {
-    cluster_sync_all();   // all partials are in place
+  // Cluster merge: CTA r of the cluster (= split r of the unit) reduces heads r, r + cluster size, ...  Every CTA
+  // stores its partial of a head into the shared memory of the CTA that reduces it; one cluster barrier later the
+  // data is local there.  No CTA's shared memory is read remotely, so nobody has to wait before leaving.
+  // `num` holds this CTA's numerators (thread t: element t, t + W * 32, ... of [G][CKV_D]); `have` is false for a
+  // split without pages, which only announces an empty partial.
+  auto cluster_merge = [&](const float *num, bool have) {
+    cluster_wait();   // every CTA of the cluster has started
     const uint32_t rank = cluster_rank(), csize = cluster_size();
-    const uint32_t res0 = (uint32_t)__cvta_generic_to_shared(smem);
-    for (int g = (int)rank; g < G; g += (int)csize) {
+    const uint32_t recv0 = (uint32_t)__cvta_generic_to_shared(s_recv);
+    constexpr int NP = (G * CKV_D + W * 32 - 1) / (W * 32);
+    if (have) {
+#pragma unroll
+      for (int it = 0; it < NP; ++it) {
+        const int idx = tid + it * W * 32;
+        if (idx < G * CKV_D) {
+          const uint32_t g = idx / CKV_D, c = idx % CKV_D;
+          const uint32_t ent = (g / csize) * csize + rank;
+          st_cluster_f32(cluster_map(recv0 + (ent * CKV_PART_STRIDE + 4 + c) * 4, g % csize), num[it]);
+        }
+      }
+    }
+    if (tid < G) {
+      const uint32_t ent = ((uint32_t)tid / csize) * csize + rank;
+      st_cluster_f32x2(cluster_map(recv0 + ent * kPartBytes, (uint32_t)tid % csize),
+                       have ? s_M[tid] : -CUDART_INF_F, have ? s_den[tid] : 0.f);
+    }
+    cluster_sync_all();   // release the stores, acquire everybody else's
+    for (int g = (int)rank, j = 0; g < G; g += (int)csize, ++j) {
+      const float *e0 = s_recv + (size_t)j * csize * CKV_PART_STRIDE;
       float2 ml = make_float2(-CUDART_INF_F, 0.f);
-      if (lane < (int)csize) ml = ld_cluster_f32x2(cluster_map(res0 + g * kPartBytes, lane));
+      if (lane < (int)csize) ml = *reinterpret_cast<const float2 *>(e0 + lane * CKV_PART_STRIDE);
       const float M = warp_max(ml.x);
       const float sc = exp2_diff(ml.x, M);
       const float den = warp_sum(ml.y * sc);
       for (int c = tid; c < CKV_D; c += W * 32) {
         float o = 0.f;
-        const uint32_t mine = res0 + g * kPartBytes + (4 + c) * 4;
-        for (uint32_t e0 = 0; e0 < csize; e0 += 8) {   // eight remote loads in flight
-          float x[8];
 #pragma unroll
-          for (int k = 0; k < 8; ++k) x[k] = e0 + k < csize ? ld_cluster_f32(cluster_map(mine, e0 + k)) : 0.f;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const float sce = __shfl_sync(0xffffffffu, sc, (e0 + k) & 31);
-            if (e0 + k < csize && sce != 0.f) o = fmaf(x[k], sce, o);
-          }
+        for (int e = 0; e < kMaxCluster; ++e) {
+          const float sce = __shfl_sync(0xffffffffu, sc, e);
+          if (e < (int)csize && sce != 0.f) o = fmaf(e0[e * CKV_PART_STRIDE + 4 + c], sce, o);
         }
         out[((size_t)s * P.Hq + h * G + g) * CKV_D + c] = __float2bfloat16_rn(o / den);
       }
       if (lse != nullptr && tid == 0) lse[(size_t)s * P.Hq + h * G + g] = (M + log2f(den)) * kLn2;
     }
-    cluster_sync_all();   // no CTA leaves while its shared memory may still be read
   };
   if (p0 >= total) {   // no pages for this split
     if (total == 0) {    // an empty unit (the same for every split of it): its output is defined as zero
@@ -153,13 +173,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
       }
       return;
     }
-    if (CL) {   // it still takes part in the cluster's merge, with an empty partial
-      if (tid < G) {
-        reinterpret_cast<float *>(smem)[tid * CKV_PART_STRIDE] = -CUDART_INF_F;
-        reinterpret_cast<float *>(smem)[tid * CKV_PART_STRIDE + 1] = 0.f;
-      }
-      cluster_merge();
-    }
+    if (CL) cluster_merge(nullptr, false);   // it still takes part in the cluster's merge, with an empty partial
     return;
   }
   const int n_active = (total + pages_per_split - 1) / pages_per_split;   // splits of this unit that have pages
@@ -541,14 +555,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     cp_async_wait<0>();
   }
   if constexpr (CL) {
-    __syncthreads();   // every entry has been read: the CTA's partial takes the start of the shared memory
-#pragma unroll
-    for (int it = 0; it < NI; ++it) {
-      const int idx = tid + it * W * 32;
-      if (idx < G * CKV_D) sf[(idx / CKV_D) * CKV_PART_STRIDE + 4 + idx % CKV_D] = num[it];
-    }
-    if (tid < G) { sf[tid * CKV_PART_STRIDE] = s_M[tid]; sf[tid * CKV_PART_STRIDE + 1] = s_den[tid]; }
-    cluster_merge();
+    cluster_merge(num, true);
     return;
   } else {
 #pragma unroll
@@ -611,7 +618,6 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
 }
 
 constexpr int kSparseWarps = 4, kDenseWarps = 8;
-constexpr int kMaxCluster = 8;    // splits of a unit that can be one cluster (the portable size; 13 measured far slower)
 
 // Whether `n_splits` sparse CTAs of this instantiation can be placed as one cluster on the current device.
 template <int G>
