@@ -56,7 +56,7 @@ Regions regions(const ckv_layout *L) {
   R.ls = o;     o = align_up(o + rows * G * sizeof(float), 256);
   R.lz = o;     o = align_up(o + rows * G * sizeof(float), 256);
   R.scores = o; o = align_up(o + rows * 4, 256);
-  R.comp = o;   o = align_up(o + (units + CKV_MAX_SCAN_CTAS) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE * 4, 256);
+  R.comp = o;   o = align_up(o + (2 * units + CKV_MAX_SCAN_CTAS + 1) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE * 4, 256);
   R.attn = o;   o = align_up(o + units * CKV_MAX_SPLITS * G * CKV_PART_STRIDE * 4, 256);
   R.stage_q = o;    o = align_up(o + (size_t)L->max_batch * L->num_q_heads * CKV_D * esz, 256);
   R.stage_knew = o; o = align_up(o + units * CKV_D * esz, 256);
@@ -212,10 +212,11 @@ int ckv_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int32_t *page_tabl
 
 namespace {
 
-// The four launches of a sparse decode step; ev (may be null) receives 5 events bracketing them.
+// The launches of a sparse decode step; ev (may be null) receives 5 events bracketing them.  With `fresh` the
+// scan launch also appends the step's new token (its tail CTAs do, beside the scan CTAs).
 int decode_impl(ckv_ctx *c, const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
                 const int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens, void *out, float *lse,
-                int32_t *sel_ids, int32_t *sel_cnt, cudaStream_t s, cudaEvent_t *ev) {
+                int32_t *sel_ids, int32_t *sel_cnt, cudaStream_t s, cudaEvent_t *ev, const CkvNewToken *fresh = nullptr) {
   const int st = check_step_args(c, batch, max_seq_len_host);
   if (st != CKV_OK) return st;
   if (!q || !k_pool || !v_pool || !page_table || !seq_lens || !out || !sel_ids || !sel_cnt) return CKV_ERR_INVALID_ARG;
@@ -226,7 +227,7 @@ int decode_impl(ckv_ctx *c, const void *q, const void *k_pool, const void *v_poo
     return CKV_ERR_BUDGET_TOO_SMALL;
   int scan_grid = 0, n_splits = 0;
   if (ev) CKV_CUDA(cudaEventRecord(ev[0], s));
-  CKV_CUDA(ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, &scan_grid, s));
+  CKV_CUDA(ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, fresh, &scan_grid, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[1], s));
   CKV_CUDA(ckv_launch_select(c, seq_lens, batch, kcap, scan_grid, sel_ids, sel_cnt, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[2], s));
@@ -260,6 +261,12 @@ int ckv_step(ckv_ctx *c, const void *q, const void *k_new, const void *v_new, vo
   if (budget_tokens <= 0 || kcap <= 0) return CKV_ERR_BUDGET_TOO_SMALL;
   if (kcap < L.sink_blocks + L.recent_blocks && (long long)kcap * L.block_size < max_seq_len_host)
     return CKV_ERR_BUDGET_TOO_SMALL;
+  if (!k_pool || !v_pool || !page_table || !seq_lens || !k_new || !v_new) return CKV_ERR_INVALID_ARG;
+  if (ckv_scan_can_append(c, batch)) {   // the append rides in the scan launch: three launches per step
+    const CkvNewToken fresh = {k_pool, v_pool, page_table, seq_lens, k_new, v_new};
+    return decode_impl(c, q, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, out, lse,
+                       sel_ids, sel_cnt, (cudaStream_t)stream, nullptr, &fresh);
+  }
   const int r = ckv_append(c, k_pool, v_pool, page_table, seq_lens, k_new, v_new, batch, stream);
   if (r != CKV_OK) return r;
   return ckv_decode(c, q, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, out, lse, sel_ids,
@@ -298,7 +305,7 @@ int ckv_scan_profile(ckv_ctx *c, const void *q, const int32_t *seq_lens, int bat
   int scan_grid = 0;
   if (rc == CKV_OK && cudaEventRecord(ev[0], s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
   for (int i = 0; i < reps && rc == CKV_OK; ++i) {
-    const cudaError_t e = ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, &scan_grid, s);
+    const cudaError_t e = ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, nullptr, &scan_grid, s);
     if (e != cudaSuccess) rc = cuda_fail(e);
   }
   if (rc == CKV_OK && cudaEventRecord(ev[1], s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());

@@ -306,9 +306,9 @@ ckv_attn_kernel(CkvDev P, const T *__restrict__ q, const T *__restrict__ k_pool,
 
 // out_{g} = sum of all partials under one normaliser (Eq. 12).  One CTA per (sequence, query head),
 // one thread per output coordinate.  Partials: the unit's attention splits and, unless every block
-// was selected, the scan partials of the CTAs whose tile range touched the unit (entries c + unit for
-// c in [c_first, c_last], recomputed here from the same tile arithmetic the scan uses).
-constexpr int kMergeMax = CKV_MAX_SPLITS + CKV_MAX_SCAN_CTAS * CKV_SCAN_WARPS;
+// was selected, the unit's scan partials (a contiguous run of entries, recomputed here from the same tile
+// arithmetic the scan uses).
+constexpr int kMergeMax = CKV_MAX_SPLITS + CKV_MAX_SCAN_CTAS * CKV_SCAN_WARPS + 1;
 
 constexpr int kMergeGroups = 4;   // thread groups of CKV_D threads, each summing every fourth partial
 
@@ -330,16 +330,16 @@ __global__ void __launch_bounds__(CKV_D *kMergeGroups) ckv_merge_kernel(CkvDev P
   const int X = (N + P.bs - 1) / P.bs;
   const bool comp = !dense && sel_cnt[unit] < X && !(P.variant & CKV_VARIANT_DROP);
   if (tid < 32) {
-    int cfirst = 0, ccount = 0;
-    if (comp) unit_scan_slots(P, seq_lens, units, unit, scan_grid, tid, cfirst, ccount);
+    int cfirst = 0, ccount = 0;   // first entry, number of entries
+    if (comp) unit_scan_entries(P, CkvClampedLens{seq_lens, P.max_blocks * P.bs}, units, unit, scan_grid, tid, cfirst, ccount);
     if (tid == 0) { s_cfirst = cfirst; s_ccount = ccount; }
   }
   __syncthreads();
-  const int n_comp = s_ccount * CKV_SCAN_WARPS;
+  const int n_comp = s_ccount;
   const int n = n_splits + n_comp;
   const size_t step = (size_t)G * CKV_PART_STRIDE;
   const float *ap = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS * G + g) * CKV_PART_STRIDE;
-  const float *cp = P.comp_part + ((size_t)(s_cfirst + unit) * CKV_SCAN_WARPS * G + g) * CKV_PART_STRIDE;
+  const float *cp = P.comp_part + ((size_t)s_cfirst * G + g) * CKV_PART_STRIDE;
   float mloc = -CUDART_INF_F;
   for (int i = tid; i < n; i += NT) {
     const float *p = i < n_splits ? ap + (size_t)i * step : cp + (size_t)(i - n_splits) * step;

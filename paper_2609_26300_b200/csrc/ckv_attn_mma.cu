@@ -371,11 +371,10 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
       }
   }
   if (comp) {
-    int cfirst = 0, ccount = 0;   // where the unit's scan partials sit
-    unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
-    const int n_comp = ccount * CKV_SCAN_WARPS;
+    int efirst = 0, n_comp = 0;   // where the unit's scan partials sit
+    unit_scan_entries(P, CkvClampedLens{seq_lens, P.max_blocks * P.bs}, units, unit, scan_grid, lane, efirst, n_comp);
     my_cnt = n_comp > (int)blockIdx.x ? (n_comp - (int)blockIdx.x + n_active - 1) / n_active : 0;
-    cp0 = P.comp_part + (size_t)(cfirst + unit) * CKV_SCAN_WARPS * G * CKV_PART_STRIDE;
+    cp0 = P.comp_part + (size_t)efirst * G * CKV_PART_STRIDE;
   }
 
   if (n_mine == 0) issue_comp(1, 0);   // a warp without pages only brings in its share of the scan partials

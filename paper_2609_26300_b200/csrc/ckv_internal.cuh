@@ -33,7 +33,7 @@ struct CkvDev {
   float *lu;         // [unit][G][max_blocks]  log2 of the head's score term e^{l_{g,b}} sigma_hat^2_{g,b} (selection reads it)
   float *lz;         // [unit][G][max_blocks]  log2 of the block's mean-compensation weight |b| e^{zbar_{g,b}} (attention)
   float *scores;     // [unit][max_blocks]     S_b
-  float *comp_part;  // [(scan CTA + unit) * CKV_SCAN_WARPS + warp][G][CKV_PART_STRIDE]  all-block mean-compensation partials
+  float *comp_part;  // [(scan CTA + 2 unit) * CKV_SCAN_WARPS + warp][G][CKV_PART_STRIDE]  all-block mean-compensation partials (see unit_scan_entries)
   float *attn_part;  // [unit][CKV_MAX_SPLITS][G][CKV_PART_STRIDE]  exact-attention partials
   int row_elems;     // bf16 elements of one mean-key / mean-value row: CKV_ROW_ELEMS, or CKV_D when only hi halves are kept
   int variant;       // ckv_variant bits
@@ -71,8 +71,17 @@ cudaError_t ckv_launch_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int
                                int max_new, cudaStream_t st);
 cudaError_t ckv_launch_append(ckv_ctx *c, void *k_pool, void *v_pool, const int *page_table, int *seq_lens,
                               const void *k_new, const void *v_new, int batch, cudaStream_t st);
+// The new token of a fused step (append inside the scan launch); all null for a plain decode.
+struct CkvNewToken {
+  void *k_pool, *v_pool;      // paged pools, written at position seq_lens[s]
+  const int *page_table;
+  int *seq_lens;              // read as the lengths before the append; holds the new lengths when the launch is over
+  const void *k_new, *v_new;  // [batch][Hkv][128]
+};
+// max_len is an upper bound of the lengths the step works on (after the append, if there is one).
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
-                            int *grid_out, cudaStream_t st);
+                            const CkvNewToken *fresh, int *grid_out, cudaStream_t st);
+bool ckv_scan_can_append(const ckv_ctx *c, int batch);   // whether ckv_launch_scan accepts a new token at this batch size
 cudaError_t ckv_launch_select(ckv_ctx *c, const int *seq_lens, int batch, int kcap, int scan_grid, int *sel_ids,
                               int *sel_cnt, cudaStream_t st);
 cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
@@ -141,10 +150,13 @@ __device__ __forceinline__ void store_split8(__nv_bfloat16 *row, int chunk, int 
 }
 
 // The eight entries of one chunk, hi + lo (hi alone when the row has no lo halves), as floats.
+// NC = false for rows the same kernel has just written.
+template <bool NC = true>
 __device__ __forceinline__ void load_split8(const __nv_bfloat16 *row, int chunk, int block, float (&x)[8], bool lo_half = true) {
   const int p = swz_chunk(chunk, block) * 8;
-  const uint4 h = __ldg(reinterpret_cast<const uint4 *>(row + p));
-  const uint4 l = lo_half ? __ldg(reinterpret_cast<const uint4 *>(row + CKV_D + p)) : make_uint4(0u, 0u, 0u, 0u);
+  const uint4 *ph = reinterpret_cast<const uint4 *>(row + p), *pl = reinterpret_cast<const uint4 *>(row + CKV_D + p);
+  const uint4 h = NC ? __ldg(ph) : *ph;
+  const uint4 l = lo_half ? (NC ? __ldg(pl) : *pl) : make_uint4(0u, 0u, 0u, 0u);
   float a[8], b[8];
   bf16x8_to_float(h, a);
   bf16x8_to_float(l, b);
@@ -235,28 +247,43 @@ __device__ __forceinline__ float exp2_diff(float a, float b) {
   return (a == -CUDART_INF_F) ? 0.0f : exp2f(a - b);
 }
 
-// Which scan partials belong to `unit`: the scan cuts all units' summaries into tiles of CKV_SCAN_TILE
-// blocks, gives CTA c the tiles [c * tpc, (c + 1) * tpc) and stores its partial for unit u in entry
-// c + u.  Must be called by all 32 lanes of a warp; every lane gets the result.
-__device__ __forceinline__ void unit_scan_slots(const CkvDev &P, const int *__restrict__ seq_lens, int units, int unit,
-                                                int scan_grid, int lane, int &cfirst, int &ccount) {
+// Which scan partials belong to `unit`.  The scan leaves the LAST block of every sequence (the one a new token
+// lands in) to its tail CTAs and cuts the other X - 1 blocks of all units into tiles of CKV_SCAN_TILE blocks; scan
+// CTA c gets the tiles [c * tpc, (c + 1) * tpc) and consumer warp w stores its partial for unit u in entry
+// (c + 2 u) * CKV_SCAN_WARPS + w.  The (c, u) pairs that occur form a monotone staircase, so with the factor 2 the
+// group behind a unit's last CTA is free: its first entry holds the last block's partial.  A unit's entries are
+// therefore contiguous: `first`, and `count` of them (zero for an empty sequence).
+// len_of(i) is the clamped length of sequence i.  Must be called by all 32 lanes of a warp; every lane gets the result.
+__device__ __forceinline__ int ckv_scan_blocks(int n, int bs) { return max((n + bs - 1) / bs - 1, 0); }
+template <class LenFn>
+__device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of, int units, int unit, int scan_grid,
+                                                  int lane, int &first, int &count) {
   const int batch = units / P.Hkv, s = unit / P.Hkv, h = unit % P.Hkv;
-  unsigned tot = 0, before = 0, mine = 0;
+  unsigned tot = 0, before = 0, mine = 0, n_mine = 0;
   for (int i = lane; i < batch; i += 32) {
-    const int n = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
-    const unsigned t = (unsigned)(((n + P.bs - 1) / P.bs + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE);
+    const int n = len_of(i);
+    const unsigned t = (unsigned)((ckv_scan_blocks(n, P.bs) + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE);
     tot += t;
     if (i < s) before += t;
-    if (i == s) mine = t;
+    if (i == s) { mine = t; n_mine = (unsigned)n; }
   }
   tot = __reduce_add_sync(0xffffffffu, tot);
   before = __reduce_add_sync(0xffffffffu, before);
   mine = __reduce_add_sync(0xffffffffu, mine);
+  n_mine = __reduce_add_sync(0xffffffffu, n_mine);
   const long long T = (long long)tot * P.Hkv;
   const long long T0 = (long long)before * P.Hkv + (long long)h * mine;
   const long long tpc = max((T + scan_grid - 1) / scan_grid, 1ll);
-  cfirst = (int)(T0 / tpc);
-  ccount = mine == 0 ? 0 : (int)((T0 + mine - 1) / tpc) - cfirst + 1;
+  const int cfirst = (int)(T0 / tpc);
+  const int ccount = mine == 0 ? 0 : (int)((T0 + mine - 1) / tpc) - cfirst + 1;
+  first = (cfirst + 2 * unit) * CKV_SCAN_WARPS;
+  count = n_mine == 0 ? 0 : ccount * CKV_SCAN_WARPS + 1;
 }
+// The usual length source: the device array, clamped to the cache's capacity.
+struct CkvClampedLens {
+  const int *seq_lens;
+  int cap;
+  __device__ __forceinline__ int operator()(int i) const { return max(min(seq_lens[i], cap), 0); }
+};
 
 #endif  // __CUDACC__

@@ -17,17 +17,27 @@
 // split bf16 pairs (hi + lo), so x * y is hi * y + lo * y with no conversion instructions; the weights
 // w = |b| e^{zbar - m} are split the same way (three products per tile: hi hi, lo hi, hi lo).
 //
-// Schedule: the summaries of all units are cut into tiles of 32 consecutive blocks; the tiles, in
-// (unit, position) order, are split into one contiguous range per CTA and the grid is one CTA per
-// SM.  A producer thread streams the CTA's tiles into a ring of shared-memory stages with
-// cp.async.bulk (two 16 KB copies and the variances per tile), completion on mbarriers.  Each of the
-// seven consumer warps takes every seventh half tile (16 blocks) on its own -- there is no CTA-wide
-// barrier in the loop -- with a per-warp running maximum that is only raised when exceeded by a
-// slack.  A warp writes one partial per unit its CTA touched; partial (CTA c, warp w, unit u) lives
-// in entry (c + u) * 7 + w, unique because the (c, u) pairs that occur form a monotone staircase.
+// Schedule: the launch has two kinds of CTAs.  The first few ("tail" CTAs, one warp per unit) take the LAST block
+// of every sequence -- the only block a decode step can change -- and, in a fused step, first append the step's new
+// token to it (page write + block summary); see scan_tail.  All other blocks of all units are cut into tiles of
+// 32 consecutive blocks; the tiles, in (unit, position) order, are split into one contiguous range per scan CTA,
+// one scan CTA per remaining SM.  A producer thread streams the CTA's tiles into a ring of shared-memory stages
+// with cp.async.bulk (two 16 KB copies and the variances per tile), completion on mbarriers.  Each of the seven
+// consumer warps takes every seventh half tile (16 blocks) on its own -- there is no CTA-wide barrier in the
+// loop -- with a per-warp running maximum that is only raised when exceeded by a slack.  A warp writes one
+// partial per unit its CTA touched; partial (scan CTA c, warp w, unit u) lives in entry (c + 2 u) * 7 + w, unique
+// because the (c, u) pairs that occur form a monotone staircase; the entry behind a unit's last one is free and
+// takes the last block's partial, so a unit's partials are one contiguous run (unit_scan_entries).
+//
+// Lengths in a fused step: every CTA reads the lengths as they were before the append and works with them plus
+// one; a counter of CTAs that are done reading decides who stores the new lengths (lens_arrive), so the kernels
+// that follow in the stream see them in place and nobody waits on anybody inside the launch.
+#include <algorithm>
+
 #include "ckv_internal.cuh"
 #include "ckv_pipe.cuh"
 #include "ckv_mma.cuh"
+#include "ckv_blockstats.cuh"
 
 namespace {
 
@@ -39,21 +49,184 @@ constexpr int kConsumerWarps = CKV_SCAN_WARPS;
 constexpr int kThreads = kConsumerWarps * 32 + 32;   // plus the producer warp
 constexpr int kMaxSeqs = 1024;      // sequence lengths are staged in shared memory up to this many sequences
 
-struct UnitInfo { int N, X, tiles; };
+struct UnitInfo { int N, X, tiles; };   // X: the blocks the scan CTAs cover, all but the sequence's last one
 
-// s_len holds the clamped lengths of the first kMaxSeqs sequences (staged once per CTA)
+// s_len holds the clamped lengths (after this step's append, if any) of the first kMaxSeqs sequences, staged once
+// per CTA; longer batches never come with an append and read the device array
+__device__ __forceinline__ int seq_len_of(const CkvDev &P, const int *s_len, const int *__restrict__ seq_lens, int s) {
+  return s < kMaxSeqs ? s_len[s] : max(min(seq_lens[s], P.max_blocks * P.bs), 0);
+}
 __device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *s_len, const int *__restrict__ seq_lens, int u) {
   UnitInfo ui;
-  const int s = u / P.Hkv;
-  ui.N = s < kMaxSeqs ? s_len[s] : max(min(seq_lens[s], P.max_blocks * P.bs), 0);
-  ui.X = (ui.N + P.bs - 1) / P.bs;
+  ui.N = seq_len_of(P, s_len, seq_lens, u / P.Hkv);
+  ui.X = ckv_scan_blocks(ui.N, P.bs);
   ui.tiles = (ui.X + TB - 1) / TB;
   return ui;
 }
 
 __device__ __forceinline__ int seq_tiles(const int *s_len, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
-  const int n = i < kMaxSeqs ? s_len[i] : max(min(seq_lens[i], P.max_blocks * P.bs), 0);
-  return ((n + P.bs - 1) / P.bs + TB - 1) / TB;
+  return (ckv_scan_blocks(seq_len_of(P, s_len, seq_lens, i), P.bs) + TB - 1) / TB;
+}
+
+constexpr int kLenCounter = 16;   // word of the status region that counts the CTAs which have read the lengths
+
+// Length hand-over of a fused step.  Every CTA of the launch works with the lengths as they were before the
+// append (plus one); a CTA calls this once it will not read the length array again, and the last one to call
+// stores the new lengths, so that the kernels that follow find them in place.  Nobody waits: it is a counter.
+// whole_cta: called by all threads of the CTA (which then share the stores), else by one thread.
+__device__ __noinline__ void lens_arrive(int *counter, const int *seq_lens, int *seq_lens_out, int batch, int cap,
+                                         int n_ctas, bool whole_cta) {
+  if (whole_cta) {
+    __shared__ int s_is_last;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      s_is_last = atomicAdd(counter, 1) == n_ctas - 1;
+      if (s_is_last) *counter = 0;   // ready for the next launch
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    for (int i = threadIdx.x; i < batch; i += blockDim.x) {
+      const int raw = seq_lens[i];
+      if (raw >= 0 && raw < cap) seq_lens_out[i] = raw + 1;
+    }
+  } else {
+    if (atomicAdd(counter, 1) != n_ctas - 1) return;
+    *counter = 0;
+    for (int i0 = 0; i0 < batch; i0 += 8) {   // loads of a group first: the arrays are one and the same
+      int raw[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) raw[k] = i0 + k < batch ? seq_lens[i0 + k] : -1;
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (raw[k] >= 0 && raw[k] < cap) seq_lens_out[i0 + k] = raw[k] + 1;
+    }
+  }
+}
+
+// Tail CTAs of the scan launch: one warp per unit.  With a new token (fused step) the warp first stores the
+// token's key and value rows into their page and recomputes the summary of the block they land in, with the
+// routine the stand-alone append uses.  Then, new token or not, it does for the unit's LAST block what the scan
+// CTAs do for all the others -- the block's two per-head terms and its mean-compensation partial -- reading the
+// summary as stored.  The last block is the only one a step can change, so the scan CTAs depend on nothing this
+// warp writes and the append costs the step no time of its own.
+//
+// Deliberately not inlined, and with the kernel's parameter block passed BY VALUE: inlined, its code doubled the
+// kernel's size and the scan CTAs stalled on instruction fetch (the launch went from 55 to 68 us); handed a
+// reference, the compiler moves the parameter block to local memory for every CTA, scan loop included.
+template <int G, typename QT>
+__device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q, const int *seq_lens, int *s_len,
+                                       int len_mine, int units, int nscan, const CkvNewToken fresh, int n_tail,
+                                       float *smem_f) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, hw = lane >> 4, li = lane & 15;
+  const int batch = units / P.Hkv, cap = P.max_blocks * P.bs;
+  const bool append = fresh.k_new != nullptr;
+  const bool lo_half = P.row_elems == CKV_ROW_ELEMS;
+  const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;
+  QT *k_pool = reinterpret_cast<QT *>(fresh.k_pool), *v_pool = reinterpret_cast<QT *>(fresh.v_pool);
+  const QT *k_new = reinterpret_cast<const QT *>(fresh.k_new), *v_new = reinterpret_cast<const QT *>(fresh.v_new);
+  float *sq = smem_f + warp * CKV_D;
+  constexpr int PIECES = (int)(CKV_D * sizeof(QT) / 16);   // 16-byte pieces of a row: lanes 0-15 hold K, 16-31 hold V
+  constexpr int PP = PIECES / 16;
+  const int u_first = (int)blockIdx.x * 8 + warp;
+  // the new row of the warp's first unit does not depend on the lengths: it is requested together with them
+  uint4 piece[PP];
+  float qx[G][8];   // this lane's 8 coordinates of the unit's G query rows (rows u G .. u G + G - 1): also independent of the lengths
+  if (u_first < units) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) load8<true>(q + ((size_t)u_first * G + g) * CKV_D + 8 * li, qx[g]);
+  }
+  if (append && u_first < units) {
+    const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + (size_t)u_first * CKV_D);
+#pragma unroll
+    for (int k = 0; k < PP; ++k) piece[k] = __ldg(src + li + 16 * k);
+  }
+  auto eff_len = [&](int raw) { return max(min(raw + ((append && raw >= 0 && raw < cap) ? 1 : 0), cap), 0); };
+  if (tid < batch) s_len[tid] = eff_len(len_mine);
+  for (int i = tid + kThreads; i < batch && i < kMaxSeqs; i += kThreads) s_len[i] = eff_len(seq_lens[i]);
+  __syncthreads();
+  auto len_of = [&](int i) { return seq_len_of(P, s_len, seq_lens, i); };
+
+  for (int u = u_first; u < units; u += n_tail * 8) {
+    const int s = u / P.Hkv, h = u % P.Hkv;
+    if (u != u_first) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) load8<true>(q + ((size_t)u * G + g) * CKV_D + 8 * li, qx[g]);
+    }
+    if (append) {
+      const int raw = seq_lens[s];
+      if (raw < 0 || raw >= cap) {
+        if (lane == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
+      } else {
+        const int *pt_row = fresh.page_table + (size_t)s * P.max_pages_per_seq;
+        const int phys = pt_row[raw / CKV_PAGE], slot = raw % CKV_PAGE;
+        const int b = raw / P.bs, cnt = raw + 1 - b * P.bs;
+        if (phys >= 0 && phys < P.num_pages) {
+          if (u != u_first) {
+            const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + (size_t)u * CKV_D);
+#pragma unroll
+            for (int k = 0; k < PP; ++k) piece[k] = __ldg(src + li + 16 * k);
+          }
+          uint4 *dst = reinterpret_cast<uint4 *>((lane < 16 ? k_pool : v_pool) +
+                                                 (((size_t)phys * P.Hkv + h) * CKV_PAGE + slot) * CKV_D);
+#pragma unroll
+          for (int k = 0; k < PP; ++k) dst[li + 16 * k] = piece[k];
+        }
+        __syncwarp();
+        const size_t row = (size_t)u * P.max_blocks + b;
+        block_stats_warp<QT, false, true>(P, k_pool, v_pool, pt_row, h, b, cnt, sq, P.kmean + row * P.row_elems,
+                                    P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
+      }
+    }
+    const int N = len_of(s);
+    if (N == 0) continue;   // warp-uniform
+    const int b = (N + P.bs - 1) / P.bs - 1, cnt = N - b * P.bs;
+    const size_t row = (size_t)u * P.max_blocks + b;
+    __syncwarp();
+    float kx[8], vx[8], dx[8];   // this lane's 8 coordinates of kbar, vbar and of the variance of their group
+    load_split8<false>(P.kmean + row * P.row_elems, li, b, kx, lo_half);
+    load_split8<false>(P.vmean + row * P.row_elems, li, b, vx, lo_half);
+    if (P.r == CKV_D) {
+      load_split8<false>(reinterpret_cast<const __nv_bfloat16 *>(P.dbar + row * CKV_D), li, b, dx);
+    } else {
+      const float *drow = P.dbar + row * P.r;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) dx[i] = drow[group_of(8 * li + i, P.r, P.glayout)];
+    }
+    int first = 0, count = 0;
+    unit_scan_entries(P, len_of, units, u, nscan, lane, first, count);
+    float *part = P.comp_part + (size_t)(first + count - 1) * G * CKV_PART_STRIDE;
+    const float logc = logf((float)cnt);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float d = 0.f, sg = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        d = fmaf(qx[g][i], kx[i], d);
+        const float qs = qx[g][i] * P.scale;
+        sg = fmaf(qs * qs, dx[i], sg);   // Eq. 8: the squared logit scale is its 1/d
+      }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) {
+        d += __shfl_xor_sync(0xffffffffu, d, o);
+        sg += __shfl_xor_sync(0xffffffffu, sg, o);
+      }
+      sg = fmaxf(sg, 0.f);
+      const float zbar = d * P.scale;
+      const float ell = logc + zbar + P.half_var * sg;
+      const float zl2 = (zbar + logc) * kLog2e;
+      float *pg = part + g * CKV_PART_STRIDE;
+      if (lane == 0) {
+        const size_t o = ((size_t)u * G + g) * P.max_blocks + b;
+        P.lu[o] = fmaf(ell, kLog2e, by_mass ? 0.f : __log2f(sg));
+        P.lz[o] = zl2;
+        pg[0] = zl2; pg[1] = 1.f; pg[2] = fast_exp2(P.half_var * kLog2e * sg);   // maximum, weight 1, e^{l - m}
+      }
+      if (hw == 1) {   // weight 1 times the mean value
+        *reinterpret_cast<float4 *>(pg + 4 + 8 * li) = make_float4(vx[0], vx[1], vx[2], vx[3]);
+        *reinterpret_cast<float4 *>(pg + 8 + 8 * li) = make_float4(vx[4], vx[5], vx[6], vx[7]);
+      }
+    }
+  }
 }
 
 template <typename QT> struct QSplit { static constexpr bool value = false; };
@@ -64,7 +237,8 @@ template <> struct QSplit<float> { static constexpr bool value = true; };
 // HS: the mean rows hold hi halves only (bf16 summaries, 256-byte rows); every product with a lo plane drops out.
 template <int G, typename QT, bool RD, bool HS>
 __global__ void __launch_bounds__(kThreads, 1)
-ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_lens, int units, int stages) {
+ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int units, int stages, CkvNewToken fresh,
+                int n_tail) {
   constexpr bool QS = QSplit<QT>::value;   // fp32 queries are split into hi + lo like the summaries
   constexpr int kRowBytes = HS ? CKV_D * 2 : CKV_ROW_ELEMS * 2;   // bytes of one mean-key / mean-value row
   extern __shared__ __align__(128) unsigned char stage_mem[];
@@ -81,19 +255,31 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
 
   // the sequence lengths are requested first; the ring is cleared while they are on their way
   const int batch = units / P.Hkv;
+  const bool append = fresh.k_new != nullptr;
+  const int cap = P.max_blocks * P.bs;
+  // length the step works on: one more than stored when a token is being appended (a full sequence keeps its length)
+  auto eff_len = [&](int raw) { return max(min(raw + ((append && raw >= 0 && raw < cap) ? 1 : 0), cap), 0); };
   const int len_mine = tid < batch ? seq_lens[tid] : 0;
+  if ((int)blockIdx.x < n_tail) {
+    // ---------------- tail CTAs: the new token and the last block of every unit ----------------
+    scan_tail<G, QT>(P, q, seq_lens, s_len, len_mine, units, (int)gridDim.x - n_tail, fresh, n_tail,
+                     reinterpret_cast<float *>(stage_mem));
+    if (append) lens_arrive(P.status + kLenCounter, seq_lens, fresh.seq_lens, batch, cap, (int)gridDim.x, /*whole_cta=*/true);
+    return;
+  }
+  const int bid = (int)blockIdx.x - n_tail, nscan = (int)gridDim.x - n_tail;   // this CTA among the scan CTAs
   // rows past a unit's last block are never copied: clear the ring once so that they hold zeros or old summaries,
   // never arbitrary bit patterns (a NaN times a zero weight would poison the accumulators)
   for (int i = tid; i < stages * stage_bytes / 16; i += kThreads) reinterpret_cast<uint4 *>(stage_mem)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async();
-  if (tid < batch) s_len[tid] = max(min(len_mine, P.max_blocks * P.bs), 0);
-  for (int i = tid + kThreads; i < batch && i < kMaxSeqs; i += kThreads) s_len[i] = max(min(seq_lens[i], P.max_blocks * P.bs), 0);
+  if (tid < batch) s_len[tid] = eff_len(len_mine);
+  for (int i = tid + kThreads; i < batch && i < kMaxSeqs; i += kThreads) s_len[i] = eff_len(seq_lens[i]);
   __syncthreads();
   if (tid == 0) {
     long long T = 0;
     for (int i = 0; i < batch; ++i) T += (long long)seq_tiles(s_len, seq_lens, P, i) * P.Hkv;
-    const long long tpc = (T + gridDim.x - 1) / gridDim.x;
-    const long long first = (long long)blockIdx.x * tpc;
+    const long long tpc = (T + nscan - 1) / nscan;
+    const long long first = (long long)bid * tpc;
     long long cnt = T - first;
     if (cnt > tpc) cnt = tpc;
     if (cnt < 0) cnt = 0;
@@ -123,7 +309,13 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
   }
   __syncthreads();
   const int count = s_count;
-  if (count == 0) return;   // uniform: this CTA has no tiles
+  // Every length this CTA needs is in shared memory now: one thread says so (the last CTA of the grid to say it
+  // stores the new lengths).  It is a spare lane of the producer warp, in the same if/else as the producer, so
+  // that nobody waits for its round trip.
+  if (count == 0) {   // uniform: this CTA has no tiles
+    if (append && tid == kThreads - 1) lens_arrive(P.status + kLenCounter, seq_lens, fresh.seq_lens, batch, cap, (int)gridDim.x, false);
+    return;
+  }
 
   if (warp == kConsumerWarps) {
     // ---------------- producer: one thread streams the CTA's tiles into the ring ----------------
@@ -158,6 +350,8 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
           do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
         }
       }
+    } else if (append && lane == 31) {
+      lens_arrive(P.status + kLenCounter, seq_lens, fresh.seq_lens, batch, cap, (int)gridDim.x, false);
     }
   } else {
     // ---------------- consumer warps: half tile j = warp, warp + 8, ... of the CTA's range ----------------
@@ -172,7 +366,6 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     const float log_bs = logf((float)P.bs);
     const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;
     const bool pair_ok = (P.max_blocks & 1) == 0;   // rows of the per-block outputs start on 8-byte boundaries
-    float log_last = 0.f;
     const int ulast = s_ulast;
     int u = s_u0, tl = s_tl0, cur = -1, next_empty = s_u0;
     UnitInfo ui = unit_info(P, s_len, seq_lens, u);
@@ -181,7 +374,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
     bool aborted = false;
 
     auto write_partial = [&](int unit_id, bool real) {
-      float *part = P.comp_part + ((size_t)(blockIdx.x + unit_id) * kConsumerWarps + warp) * G * CKV_PART_STRIDE;
+      float *part = P.comp_part + ((size_t)(bid + 2 * unit_id) * kConsumerWarps + warp) * G * CKV_PART_STRIDE;
       if (!real) {
         if (lane < G) {
           part[lane * CKV_PART_STRIDE] = -CUDART_INF_F;
@@ -288,7 +481,6 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
 #pragma unroll
         for (int t = 0; t < 16; ++t) { acc[t][0] = 0.f; acc[t][1] = 0.f; }
         m_ref = -CUDART_INF_F; l_acc = 0.f; lp_acc = 0.f;
-        log_last = logf((float)(ui.N - (ui.X - 1) * P.bs));
         const size_t row0 = (size_t)u * P.max_blocks;
         lu = P.lu + row0 * G;   // [head][block] within the unit
         lz = P.lz + row0 * G;
@@ -386,9 +578,8 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *__restrict__ seq_
             }
             sig[nt][e] = sg;
             const float zbar = z[nt][e] * P.scale;
-            const float logc = (b == ui.X - 1) ? log_last : log_bs;
-            ell[e] = logc + zbar + P.half_var * sg;
-            zl2[nt][e] = val[nt][e] ? (zbar + logc) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
+            ell[e] = log_bs + zbar + P.half_var * sg;   // every block the scan CTAs see is full
+            zl2[nt][e] = val[nt][e] ? (zbar + log_bs) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
             tmax = fmaxf(tmax, zl2[nt][e]);
           }
           // what the later kernels read, both in log2 units: the head's term of the block score, e^l sigma^2 (e^l
@@ -480,24 +671,26 @@ ScanCfg scan_cfg(const CkvDev &P, int G) {
 }
 
 template <int G, typename QT>
-cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, cudaStream_t st) {
+cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, const CkvNewToken &fresh,
+                      int n_tail, cudaStream_t st) {
   const ScanCfg cfg = scan_cfg(c->dev, G);
   if (c->dev.r == CKV_D)
-    ckv_scan_kernel<G, QT, true, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+    ckv_scan_kernel<G, QT, true, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail);
   else if (c->dev.row_elems == CKV_D) {
     if constexpr (!QSplit<QT>::value)   // bf16 summaries come with bf16 pages and queries only
-      ckv_scan_kernel<G, QT, false, true><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+      ckv_scan_kernel<G, QT, false, true><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail);
     else
       return cudaErrorInvalidValue;
   } else
-    ckv_scan_kernel<G, QT, false, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages);
+    ckv_scan_kernel<G, QT, false, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail);
   return cudaGetLastError();
 }
 
 template <int G>
-cudaError_t launch_g(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, cudaStream_t st) {
-  if (c->layout.kv_dtype == CKV_BF16) return launch_gt<G, __nv_bfloat16>(c, q, seq_lens, units, grid, st);
-  return launch_gt<G, float>(c, q, seq_lens, units, grid, st);
+cudaError_t launch_g(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, const CkvNewToken &fresh,
+                     int n_tail, cudaStream_t st) {
+  if (c->layout.kv_dtype == CKV_BF16) return launch_gt<G, __nv_bfloat16>(c, q, seq_lens, units, grid, fresh, n_tail, st);
+  return launch_gt<G, float>(c, q, seq_lens, units, grid, fresh, n_tail, st);
 }
 
 template <int G, typename QT>
@@ -532,29 +725,45 @@ cudaError_t ckv_configure_scan(const ckv_ctx *c) {
   return cudaErrorInvalidValue;
 }
 
-// Grid size the scan uses for a step (one persistent CTA per SM, never more CTAs than tiles).
+namespace {
+constexpr int kMaxTailCtas = 8;   // tail CTAs of a launch: 8 warps each, one unit per warp and round
+int tail_ctas(const ckv_ctx *c, int batch) {
+  const int units = batch * c->dev.Hkv;
+  return std::max(1, std::min((units + 7) / 8, kMaxTailCtas));
+}
+}  // namespace
+
+// Scan CTAs of a step: one persistent CTA per SM the tail CTAs leave free, never more CTAs than tiles.
 int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
   const CkvDev &P = c->dev;
-  const int xmax = (max_len + P.bs - 1) / P.bs;
+  const int xmax = std::max((max_len + P.bs - 1) / P.bs - 1, 0);   // the last block of a sequence is the tail CTAs'
   const long long tiles = (long long)batch * P.Hkv * ((xmax + TB - 1) / TB);
-  long long grid = c->sm_count;
+  long long grid = c->sm_count - tail_ctas(c, batch);
   if (grid > CKV_MAX_SCAN_CTAS) grid = CKV_MAX_SCAN_CTAS;
   if (grid > tiles) grid = tiles;
   return (int)(grid < 1 ? 1 : grid);
 }
 
-cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len, int *grid_out,
-                            cudaStream_t st) {
+bool ckv_scan_can_append(const ckv_ctx *, int batch) { return batch <= kMaxSeqs; }
+
+cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
+                            const CkvNewToken *fresh_in, int *grid_out, cudaStream_t st) {
   const CkvDev &P = c->dev;
   const int units = batch * P.Hkv;
-  const int grid = ckv_scan_grid(c, batch, max_len);
-  *grid_out = grid;
+  const int n_scan = ckv_scan_grid(c, batch, max_len), n_tail = tail_ctas(c, batch);
+  const int grid = n_tail + n_scan;
+  CkvNewToken fresh = {};
+  if (fresh_in != nullptr) {
+    if (!ckv_scan_can_append(c, batch)) return cudaErrorInvalidValue;
+    fresh = *fresh_in;
+  }
+  *grid_out = n_scan;
   c->launches++;
   switch (P.G) {
-    case 1: return launch_g<1>(c, q, seq_lens, units, grid, st);
-    case 2: return launch_g<2>(c, q, seq_lens, units, grid, st);
-    case 4: return launch_g<4>(c, q, seq_lens, units, grid, st);
-    case 8: return launch_g<8>(c, q, seq_lens, units, grid, st);
+    case 1: return launch_g<1>(c, q, seq_lens, units, grid, fresh, n_tail, st);
+    case 2: return launch_g<2>(c, q, seq_lens, units, grid, fresh, n_tail, st);
+    case 4: return launch_g<4>(c, q, seq_lens, units, grid, fresh, n_tail, st);
+    case 8: return launch_g<8>(c, q, seq_lens, units, grid, fresh, n_tail, st);
   }
   return cudaErrorInvalidValue;
 }

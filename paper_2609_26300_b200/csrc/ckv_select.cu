@@ -84,10 +84,9 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   int n_part = 0;
   const size_t pstep = (size_t)G * CKV_PART_STRIDE;
   if (warp < G) {
-    int cfirst, ccount;
-    unit_scan_slots(P, seq_lens, units, unit, scan_grid, lane, cfirst, ccount);
-    cp = P.comp_part + ((size_t)(cfirst + unit) * CKV_SCAN_WARPS * G + warp) * CKV_PART_STRIDE;
-    n_part = ccount * CKV_SCAN_WARPS;
+    int efirst;
+    unit_scan_entries(P, CkvClampedLens{seq_lens, P.max_blocks * P.bs}, units, unit, scan_grid, lane, efirst, n_part);
+    cp = P.comp_part + ((size_t)efirst * G + warp) * CKV_PART_STRIDE;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const int i = lane + 32 * k;

@@ -1,0 +1,147 @@
+"""The fused step (ckv_step: the new token's append rides in the scan launch) against the two-call sequence
+ckv_append + ckv_decode on identical caches, and its corner cases: full sequences, more units than one round of
+tail warps, fp32 pages, bf16 summaries."""
+import pytest
+import torch
+
+from paper_2609_26300_b200 import binding, synth
+from helpers import setup
+
+pytestmark = pytest.mark.gpu
+
+TOY = synth.CONFIGS[1]
+
+
+def small(**kw):
+    base = dict(batch=2, num_q_heads=8, num_kv_heads=2, ctx=16 * 70 + 5, budget_tokens=16 * 12, needles=4,
+                outlier_dims=2, decode_steps=3, name="small")
+    base.update(kw)
+    return TOY.with_(**base)
+
+
+def rows(d, t):
+    k_new, v_new = synth.appended_rows(d.w, t)
+    q = synth.queries(d.w, t)
+    return (torch.from_numpy(q).to(d.dtype).cuda(), torch.from_numpy(k_new).to(d.dtype).cuda(),
+            torch.from_numpy(v_new).to(d.dtype).cuda())
+
+
+def run_both(w, steps, dtype=torch.bfloat16, **layout):
+    """Two identical caches: one stepped with ckv_step, one with ckv_append + ckv_decode.  The summaries, pages,
+    lengths and selected ids must be identical; the outputs agree bit for bit (same kernels, same order)."""
+    a, b = setup(w, dtype, **layout), setup(w, dtype, **layout)
+    for d in (a, b):
+        d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    for t in range(steps):
+        q, kn, vn = rows(a, t)
+        max_len = a.max_len + t + 1
+        oa, la, ia, ca = a.ckv.step(q, kn, vn, a.k_pool, a.v_pool, a.table, a.lens, max_len, w.budget_tokens)
+        b.ckv.append(b.k_pool, b.v_pool, b.table, b.lens, kn, vn)
+        ob, lb, ib, cb = b.ckv.decode(q, b.k_pool, b.v_pool, b.table, b.lens, max_len, w.budget_tokens)
+        torch.cuda.synchronize()
+        assert torch.equal(a.lens, b.lens), t
+        assert torch.equal(ca, cb) and torch.equal(ia, ib), t
+        assert torch.equal(oa, ob) and torch.equal(la, lb), t
+        sa, sb = a.ckv.copy_scores(w.batch), b.ckv.copy_scores(w.batch)
+        assert torch.equal(sa, sb), t
+    torch.cuda.synchronize()
+    assert torch.equal(a.k_pool, b.k_pool) and torch.equal(a.v_pool, b.v_pool)
+    for x, y in zip(a.ckv.export_stats(), b.ckv.export_stats()):
+        assert torch.equal(x, y)
+    assert a.ckv.read_status() == 0 and b.ckv.read_status() == 0
+    return a
+
+
+@pytest.mark.parametrize("bs", [16, 32, 64])
+def test_step_equals_append_then_decode(bs):
+    w = small(block_size=bs, ctx_min=16 * 20 + 1, ctx=16 * 70 + 5, budget_tokens=bs * 7, decode_steps=40)
+    run_both(w, 40)   # crosses block boundaries in every sequence: full block, roll-over, one-token block
+
+
+@pytest.mark.parametrize("r,layout", [(128, 1), (8, 0), (1, 1)])
+def test_step_equals_append_then_decode_variance_layouts(r, layout):
+    w = small(ctx=16 * 33 + 14, decode_steps=20)
+    run_both(w, 20, var_groups=r, group_layout=layout)
+
+
+def test_step_equals_append_then_decode_fp32_pages():
+    w = small(ctx=16 * 33 + 14, decode_steps=20)
+    run_both(w, 20, dtype=torch.float32)
+
+
+def test_step_equals_append_then_decode_bf16_summaries():
+    w = small(ctx=16 * 33 + 14, decode_steps=20)
+    run_both(w, 20, stat_bf16=1)
+
+
+def test_step_launch_count_is_three():
+    w = small(decode_steps=2)
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    n0 = d.ckv.launch_count()
+    q, kn, vn = rows(d, 0)
+    d.ckv.step(q, kn, vn, d.k_pool, d.v_pool, d.table, d.lens, d.max_len + 1, w.budget_tokens)
+    torch.cuda.synchronize()
+    assert d.ckv.launch_count() - n0 == 3   # scan (with the append in its tail CTAs), select, attention + merge
+
+
+def test_more_units_than_one_round_of_tail_warps():
+    """72 units: the eight tail CTAs (64 warps) go round twice."""
+    w = small(batch=9, num_q_heads=16, num_kv_heads=8, ctx_min=16 * 8 + 1, ctx=16 * 20 + 3, decode_steps=18,
+              budget_tokens=16 * 6, needles=1)
+    run_both(w, 18)
+
+
+def test_step_on_full_sequence_sets_status_and_keeps_length():
+    """One sequence of the batch is at capacity: its token is dropped (status bit), its length stays, the step is
+    still the decode step of the cache as it is; the other sequence advances."""
+    w = small(batch=2, ctx_min=16 * 10, ctx=16 * 12, decode_steps=0)
+    a, b = setup(w), setup(w)
+    cap = a.table.shape[1] * 16
+    for d in (a, b):
+        d.lens[0] = cap                                  # sequence 0 fills its page table completely
+        d.lens[1] = cap - 21
+        d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, cap)
+    q = torch.from_numpy(synth.queries(w, 0)).to(a.dtype).cuda()
+    gen = torch.Generator().manual_seed(7)
+    kn = torch.randn(w.batch, w.num_kv_heads, 128, generator=gen).to(a.dtype).cuda()
+    vn = torch.randn(w.batch, w.num_kv_heads, 128, generator=gen).to(a.dtype).cuda()
+    n1 = int(a.lens[1])
+    oa, la, ia, ca = a.ckv.step(q, kn, vn, a.k_pool, a.v_pool, a.table, a.lens, cap, w.budget_tokens)
+    b.ckv.append(b.k_pool, b.v_pool, b.table, b.lens, kn, vn)
+    ob, lb, ib, cb = b.ckv.decode(q, b.k_pool, b.v_pool, b.table, b.lens, cap, w.budget_tokens)
+    torch.cuda.synchronize()
+    assert a.ckv.read_status() & binding.CKV_DEV_SEQ_FULL
+    assert b.ckv.read_status() & binding.CKV_DEV_SEQ_FULL
+    assert a.lens.cpu().tolist() == [cap, n1 + 1] and torch.equal(a.lens, b.lens)
+    assert torch.equal(ia, ib) and torch.equal(ca, cb) and torch.equal(oa, ob) and torch.equal(la, lb)
+
+
+def test_step_replayed_in_a_cuda_graph_advances_lengths():
+    """The length hand-over inside the launch (a counter of CTAs that have read the old lengths) must leave the
+    counter ready for the next replay: 12 replays of one captured step advance every length by 12."""
+    w = small(ctx=16 * 30 + 7, decode_steps=12)
+    a, b = setup(w), setup(w)
+    for d in (a, b):
+        d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    q, kn, vn = rows(a, 0)
+    max_len = a.max_len + 12
+    outs = a.ckv.alloc_outputs(w.batch, w.budget_tokens)
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        a.ckv.step(q, kn, vn, a.k_pool, a.v_pool, a.table, a.lens, max_len, w.budget_tokens, outs)   # warm-up, step 1
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            a.ckv.step(q, kn, vn, a.k_pool, a.v_pool, a.table, a.lens, max_len, w.budget_tokens, outs)
+        for _ in range(11):
+            g.replay()
+    torch.cuda.synchronize()
+    for _ in range(12):
+        b.ckv.append(b.k_pool, b.v_pool, b.table, b.lens, kn, vn)
+    ob, lb, ib, cb = b.ckv.decode(q, b.k_pool, b.v_pool, b.table, b.lens, max_len, w.budget_tokens)
+    torch.cuda.synchronize()
+    assert torch.equal(a.lens, b.lens)
+    assert torch.equal(outs[0], ob) and torch.equal(outs[2], ib) and torch.equal(outs[3], cb)
+    assert a.ckv.read_status() == 0

@@ -240,7 +240,10 @@ def test_exact_ties_go_to_lower_block_ids():
     d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
     out, lse, ids, cnt, scores = run_decode(d, 16 * 20)
     sc = scores[0, 0, :64].cpu().numpy()
-    assert np.array_equal(sc[8:36], sc[36:64])
+    assert np.array_equal(sc[8:35], sc[36:63])
+    # the last block of a sequence is scored by the launch's tail CTAs (plain FMAs, not tensor-core tiles): its
+    # pair agrees to rounding, not bit for bit; it is a mandatory block, so no tie is decided by it
+    assert abs(sc[35] - sc[63]) <= 1e-6 * abs(sc[63])
     K = d.k_pool[:64, 0].float().reshape(-1, 128).cpu().numpy()
     V = d.v_pool[:64, 0].float().reshape(-1, 128).cpu().numpy()
     q = synth.queries(w)[0]
