@@ -183,10 +183,14 @@ int ckv_prefill(ckv_ctx *ctx, void *k_pool, void *v_pool, const int32_t *page_ta
                 const void *k_src, const void *v_src, const int32_t *new_lens, int src_stride_tokens, int batch,
                 int max_new_host, ckv_stream stream);
 
-/* One decode step in one call: ckv_append(k_new, v_new) followed by ckv_decode(q, ...), with the same arguments,
- * results and errors as the two calls in that order (Sec. 4.3: the new token enters the cache and the summaries
- * before blocks are selected; seq_lens holds N on entry and N + 1 once the step has run; max_seq_len_host bounds the
- * lengths after the append).  The decode arguments are validated before anything is appended. */
+/* One decode step in one call: the results, the cache, the summaries, the lengths and the errors are those of
+ * ckv_append(k_new, v_new) followed by ckv_decode(q, ...), bit for bit (Sec. 4.3: the new token enters the cache
+ * and the summaries before blocks are selected; seq_lens holds N on entry and N + 1 once the step has run;
+ * max_seq_len_host bounds the lengths after the append).  It is three launches, not four: a step can only change
+ * the last block of a sequence, so a few CTAs of the scan launch write the new rows and redo that block's summary
+ * while the other CTAs stream the summaries of all the other blocks; seq_lens is updated inside that launch, after
+ * every CTA has read it.  (Batches above 1024 sequences take the two-call route.)  The decode arguments are
+ * validated before anything is appended. */
 int ckv_step(ckv_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k_pool, void *v_pool,
              const int32_t *page_table, int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens,
              void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt, ckv_stream stream);
