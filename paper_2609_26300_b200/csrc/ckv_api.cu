@@ -262,7 +262,7 @@ int ckv_step(ckv_ctx *c, const void *q, const void *k_new, const void *v_new, vo
   if (kcap < L.sink_blocks + L.recent_blocks && (long long)kcap * L.block_size < max_seq_len_host)
     return CKV_ERR_BUDGET_TOO_SMALL;
   if (!k_pool || !v_pool || !page_table || !seq_lens || !k_new || !v_new) return CKV_ERR_INVALID_ARG;
-  if (ckv_scan_can_append(c, batch)) {   // the append rides in the scan launch: three launches per step
+  if (ckv_scan_can_append(c, batch, max_seq_len_host)) {   // the append rides in the scan launch: three launches per step
     const CkvNewToken fresh = {k_pool, v_pool, page_table, seq_lens, k_new, v_new};
     return decode_impl(c, q, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, out, lse,
                        sel_ids, sel_cnt, (cudaStream_t)stream, nullptr, &fresh);

@@ -81,7 +81,7 @@ struct CkvNewToken {
 // max_len is an upper bound of the lengths the step works on (after the append, if there is one).
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
                             const CkvNewToken *fresh, int *grid_out, cudaStream_t st);
-bool ckv_scan_can_append(const ckv_ctx *c, int batch);   // whether ckv_launch_scan accepts a new token at this batch size
+bool ckv_scan_can_append(const ckv_ctx *c, int batch, int max_len);   // whether ckv_launch_scan should take the new token
 cudaError_t ckv_launch_select(ckv_ctx *c, const int *seq_lens, int batch, int kcap, int scan_grid, int *sel_ids,
                               int *sel_cnt, cudaStream_t st);
 cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,

@@ -726,10 +726,18 @@ cudaError_t ckv_configure_scan(const ckv_ctx *c) {
 }
 
 namespace {
-constexpr int kMaxTailCtas = 8;   // tail CTAs of a launch: 8 warps each, one unit per warp and round
+// Tail CTAs of a launch: 8 warps each, one unit per warp and round.  One round is the goal: a warp's work is a chain
+// of three or four dependent cache misses, each of which costs several microseconds once the scan CTAs have
+// saturated DRAM (two rounds for 32 units made the whole step 7 us slower than one).
 int tail_ctas(const ckv_ctx *c, int batch) {
   const int units = batch * c->dev.Hkv;
-  return std::max(1, std::min((units + 7) / 8, kMaxTailCtas));
+  const int one_round = (units + 7) / 8;
+  if (one_round <= 16) return std::max(1, one_round);
+  return std::min((units + 15) / 16, std::max(16, c->sm_count / 4));   // many units: two rounds, at most a quarter of the SMs
+}
+int tail_rounds(const ckv_ctx *c, int batch) {
+  const int units = batch * c->dev.Hkv;
+  return (units + 8 * tail_ctas(c, batch) - 1) / (8 * tail_ctas(c, batch));
 }
 }  // namespace
 
@@ -744,7 +752,17 @@ int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
   return (int)(grid < 1 ? 1 : grid);
 }
 
-bool ckv_scan_can_append(const ckv_ctx *, int batch) { return batch <= kMaxSeqs; }
+// Whether the step's append should ride in the scan launch: the lengths must fit the staging array, and the tail
+// CTAs' rounds (about 20 us each under load) must hide behind the scan (about 5 MB per us), otherwise the
+// stand-alone append launch, whose warps all run at once, is the shorter way.
+bool ckv_scan_can_append(const ckv_ctx *c, int batch, int max_len) {
+  if (batch > kMaxSeqs) return false;
+  const CkvDev &P = c->dev;
+  const int rounds = tail_rounds(c, batch);
+  if (rounds == 1) return true;
+  const double bytes = (double)batch * P.Hkv * ((max_len + P.bs - 1) / P.bs) * (2.0 * P.row_elems * 2 + 4.0 * P.r);
+  return bytes / 5.0e6 >= 30.0 * rounds;   // scan microseconds against tail microseconds, with a margin
+}
 
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
                             const CkvNewToken *fresh_in, int *grid_out, cudaStream_t st) {
@@ -754,7 +772,7 @@ cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int 
   const int grid = n_tail + n_scan;
   CkvNewToken fresh = {};
   if (fresh_in != nullptr) {
-    if (!ckv_scan_can_append(c, batch)) return cudaErrorInvalidValue;
+    if (!ckv_scan_can_append(c, batch, max_len)) return cudaErrorInvalidValue;
     fresh = *fresh_in;
   }
   *grid_out = n_scan;

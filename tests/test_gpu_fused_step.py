@@ -26,7 +26,7 @@ def rows(d, t):
             torch.from_numpy(v_new).to(d.dtype).cuda())
 
 
-def run_both(w, steps, dtype=torch.bfloat16, **layout):
+def run_both(w, steps, dtype=torch.bfloat16, step_launches=3, **layout):
     """Two identical caches: one stepped with ckv_step, one with ckv_append + ckv_decode.  The summaries, pages,
     lengths and selected ids must be identical; the outputs agree bit for bit (same kernels, same order)."""
     a, b = setup(w, dtype, **layout), setup(w, dtype, **layout)
@@ -35,7 +35,9 @@ def run_both(w, steps, dtype=torch.bfloat16, **layout):
     for t in range(steps):
         q, kn, vn = rows(a, t)
         max_len = a.max_len + t + 1
+        n_before = a.ckv.launch_count()
         oa, la, ia, ca = a.ckv.step(q, kn, vn, a.k_pool, a.v_pool, a.table, a.lens, max_len, w.budget_tokens)
+        assert a.ckv.launch_count() - n_before == step_launches
         b.ckv.append(b.k_pool, b.v_pool, b.table, b.lens, kn, vn)
         ob, lb, ib, cb = b.ckv.decode(q, b.k_pool, b.v_pool, b.table, b.lens, max_len, w.budget_tokens)
         torch.cuda.synchronize()
@@ -66,7 +68,7 @@ def test_step_equals_append_then_decode_variance_layouts(r, layout):
 
 def test_step_equals_append_then_decode_fp32_pages():
     w = small(ctx=16 * 33 + 14, decode_steps=20)
-    run_both(w, 20, dtype=torch.float32)
+    run_both(w, 20, dtype=torch.float32, step_launches=4)   # fp32 pages merge in a launch of their own
 
 
 def test_step_equals_append_then_decode_bf16_summaries():
@@ -86,11 +88,25 @@ def test_step_launch_count_is_three():
     assert d.ckv.launch_count() - n0 == 3   # scan (with the append in its tail CTAs), select, attention + merge
 
 
-def test_more_units_than_one_round_of_tail_warps():
-    """72 units: the eight tail CTAs (64 warps) go round twice."""
+def test_many_units_one_round_of_tail_warps():
+    """72 units: nine tail CTAs, one unit per warp."""
     w = small(batch=9, num_q_heads=16, num_kv_heads=8, ctx_min=16 * 8 + 1, ctx=16 * 20 + 3, decode_steps=18,
               budget_tokens=16 * 6, needles=1)
     run_both(w, 18)
+
+
+def test_more_units_than_one_round_of_tail_warps():
+    """136 units: the tail warps go round twice, and the cache is long enough (35K tokens per sequence) for the
+    library to keep the append inside the scan launch (short caches with this many units take the two-call route,
+    which the second half checks)."""
+    w = small(batch=17, num_q_heads=8, num_kv_heads=8, ctx_min=16 * 2100, ctx=16 * 2200 + 5, decode_steps=3,
+              budget_tokens=16 * 8, needles=0, outlier_dims=0)
+    a = run_both(w, 3)   # three launches per step: scan (with the append), select, attention + merge
+    del a
+    torch.cuda.empty_cache()
+    w = small(batch=17, num_q_heads=8, num_kv_heads=8, ctx_min=16 * 8 + 1, ctx=16 * 20 + 3, decode_steps=6,
+              budget_tokens=16 * 6, needles=0)
+    run_both(w, 6, step_launches=4)   # append, scan, select, attention + merge
 
 
 def test_step_on_full_sequence_sets_status_and_keeps_length():
