@@ -264,6 +264,16 @@ int ckv_read_status(ckv_ctx *ctx, int32_t *host_status, ckv_stream stream);
 /* Number of kernel launches the library has enqueued through this context so far. */
 int64_t ckv_launch_count(const ckv_ctx *ctx);
 
+/* How the decode step treats the last block of every sequence (the only block a step can change).  In "tail
+ * mode" a few CTAs of the scan launch own that block -- and, in ckv_step, append the new token to it inside the
+ * same launch -- while the other CTAs stream the remaining summaries; otherwise the scan covers every block and
+ * ckv_step appends in a launch of its own.  The results agree to rounding (the last block's two per-head terms are
+ * computed by different code); tail mode is the faster one once the scan runs for tens of microseconds.
+ * mode: CKV_TAIL_AUTO (default: chosen per call from the batch and max_seq_len_host), CKV_TAIL_OFF, CKV_TAIL_ON
+ * (honoured up to 1024 sequences).  Returns CKV_ERR_INVALID_ARG for a null context or an unknown mode. */
+enum ckv_tail_mode { CKV_TAIL_AUTO = 0, CKV_TAIL_OFF = 1, CKV_TAIL_ON = 2 };
+int ckv_set_tail_mode(ckv_ctx *ctx, int mode);
+
 #ifdef __cplusplus
 }
 #endif

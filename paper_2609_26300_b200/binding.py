@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libcompkv.so")
 
 VARIANT_FIRST_ORDER_MASS, VARIANT_RANK_BY_MASS, VARIANT_DROP = 1, 2, 4
 CKV_BF16, CKV_F32 = 0, 1
+CKV_TAIL_AUTO, CKV_TAIL_OFF, CKV_TAIL_ON = 0, 1, 2
 CKV_OK = 0
 CKV_ERR_INVALID_ARG, CKV_ERR_BAD_LAYOUT, CKV_ERR_BUDGET_TOO_SMALL = -1, -2, -3
 CKV_ERR_CAPACITY, CKV_ERR_CUDA, CKV_ERR_TIMEOUT = -4, -5, -6
@@ -25,7 +26,8 @@ CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
            "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_prefill", "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
            "ckv_dense_decode_static",
-           "ckv_exact_blocks", "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count"]
+           "ckv_exact_blocks", "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count",
+           "ckv_set_tail_mode"]
 
 
 class ckv_layout(ctypes.Structure):
@@ -90,6 +92,8 @@ def load() -> ctypes.CDLL:
     lib.ckv_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
     lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_launch_count.restype = ctypes.c_int64
+    lib.ckv_set_tail_mode.argtypes = [vp, ctypes.c_int]
+    lib.ckv_set_tail_mode.restype = ctypes.c_int
     for name in ("ckv_query_sizes", "ckv_stats_offsets", "ckv_create", "ckv_stats_build", "ckv_stats_export", "ckv_append",
                  "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode", "ckv_copy_scores", "ckv_step_host", "ckv_read_status"):
         getattr(lib, name).restype = i32
@@ -299,3 +303,7 @@ class CompKV:
 
     def launch_count(self) -> int:
         return int(self.lib.ckv_launch_count(self._ctx))
+
+    def set_tail_mode(self, mode: int) -> None:
+        """ckv_set_tail_mode: CKV_TAIL_AUTO (default), CKV_TAIL_OFF, CKV_TAIL_ON."""
+        _check(self.lib.ckv_set_tail_mode(self._ctx, int(mode)), "ckv_set_tail_mode")

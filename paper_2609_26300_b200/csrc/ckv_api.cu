@@ -226,6 +226,7 @@ int decode_impl(ckv_ctx *c, const void *q, const void *k_pool, const void *v_poo
   if (kcap < L.sink_blocks + L.recent_blocks && (long long)kcap * L.block_size < max_seq_len_host)
     return CKV_ERR_BUDGET_TOO_SMALL;
   int scan_grid = 0, n_splits = 0;
+  c->dev.tail = (fresh != nullptr || ckv_scan_wants_tail(c, batch, max_seq_len_host)) ? 1 : 0;   // one mode for the step's launches
   if (ev) CKV_CUDA(cudaEventRecord(ev[0], s));
   CKV_CUDA(ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, fresh, &scan_grid, s));
   if (ev) CKV_CUDA(cudaEventRecord(ev[1], s));
@@ -262,7 +263,7 @@ int ckv_step(ckv_ctx *c, const void *q, const void *k_new, const void *v_new, vo
   if (kcap < L.sink_blocks + L.recent_blocks && (long long)kcap * L.block_size < max_seq_len_host)
     return CKV_ERR_BUDGET_TOO_SMALL;
   if (!k_pool || !v_pool || !page_table || !seq_lens || !k_new || !v_new) return CKV_ERR_INVALID_ARG;
-  if (ckv_scan_can_append(c, batch, max_seq_len_host)) {   // the append rides in the scan launch: three launches per step
+  if (ckv_scan_wants_tail(c, batch, max_seq_len_host)) {   // the append rides in the scan launch: three launches per step
     const CkvNewToken fresh = {k_pool, v_pool, page_table, seq_lens, k_new, v_new};
     return decode_impl(c, q, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, out, lse,
                        sel_ids, sel_cnt, (cudaStream_t)stream, nullptr, &fresh);
@@ -305,6 +306,7 @@ int ckv_scan_profile(ckv_ctx *c, const void *q, const int32_t *seq_lens, int bat
   int scan_grid = 0;
   if (rc == CKV_OK && cudaEventRecord(ev[0], s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
   for (int i = 0; i < reps && rc == CKV_OK; ++i) {
+    c->dev.tail = ckv_scan_wants_tail(c, batch, max_seq_len_host) ? 1 : 0;
     const cudaError_t e = ckv_launch_scan(c, q, seq_lens, batch, max_seq_len_host, nullptr, &scan_grid, s);
     if (e != cudaSuccess) rc = cuda_fail(e);
   }
@@ -393,5 +395,11 @@ int ckv_read_status(ckv_ctx *c, int32_t *host_status, ckv_stream stream) {
 }
 
 int64_t ckv_launch_count(const ckv_ctx *c) { return c == nullptr ? 0 : c->launches; }
+
+int ckv_set_tail_mode(ckv_ctx *c, int mode) {
+  if (c == nullptr || mode < CKV_TAIL_AUTO || mode > CKV_TAIL_ON) return CKV_ERR_INVALID_ARG;
+  c->tail_mode = mode;
+  return CKV_OK;
+}
 
 }  // extern "C"

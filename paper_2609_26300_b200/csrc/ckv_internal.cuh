@@ -38,6 +38,7 @@ struct CkvDev {
   int row_elems;     // bf16 elements of one mean-key / mean-value row: CKV_ROW_ELEMS, or CKV_D when only hi halves are kept
   int variant;       // ckv_variant bits
   float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
+  int tail;          // 1: the scan launch leaves the last block of every sequence to its tail CTAs (set per step)
   int *unit_done;    // [unit] attention splits finished this step (zero between steps); null = merge is a separate launch
   int *status;       // device status word
 };
@@ -51,6 +52,7 @@ struct ckv_ctx {
   size_t stage_q, stage_knew, stage_vnew, stage_out, stage_ids, stage_cnt;
   int64_t launches;
   int sm_count;
+  int tail_mode;   // ckv_tail_mode
 };
 
 cudaError_t ckv_configure_kernels();   // selection kernel attributes
@@ -78,10 +80,13 @@ struct CkvNewToken {
   int *seq_lens;              // read as the lengths before the append; holds the new lengths when the launch is over
   const void *k_new, *v_new;  // [batch][Hkv][128]
 };
-// max_len is an upper bound of the lengths the step works on (after the append, if there is one).
+// max_len is an upper bound of the lengths the step works on (after the append, if there is one).  The launch
+// follows c->dev.tail; a new token needs tail mode.
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
                             const CkvNewToken *fresh, int *grid_out, cudaStream_t st);
-bool ckv_scan_can_append(const ckv_ctx *c, int batch, int max_len);   // whether ckv_launch_scan should take the new token
+// Whether a step of this size should run in tail mode (the scan, select and attention launches of one step must
+// agree: the caller stores the answer in c->dev.tail before launching them).
+bool ckv_scan_wants_tail(const ckv_ctx *c, int batch, int max_len);
 cudaError_t ckv_launch_select(ckv_ctx *c, const int *seq_lens, int batch, int kcap, int scan_grid, int *sel_ids,
                               int *sel_cnt, cudaStream_t st);
 cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,
@@ -247,14 +252,14 @@ __device__ __forceinline__ float exp2_diff(float a, float b) {
   return (a == -CUDART_INF_F) ? 0.0f : exp2f(a - b);
 }
 
-// Which scan partials belong to `unit`.  The scan leaves the LAST block of every sequence (the one a new token
-// lands in) to its tail CTAs and cuts the other X - 1 blocks of all units into tiles of CKV_SCAN_TILE blocks; scan
-// CTA c gets the tiles [c * tpc, (c + 1) * tpc) and consumer warp w stores its partial for unit u in entry
+// Which scan partials belong to `unit`.  The scan cuts the blocks of all units into tiles of CKV_SCAN_TILE blocks;
+// scan CTA c gets the tiles [c * tpc, (c + 1) * tpc) and consumer warp w stores its partial for unit u in entry
 // (c + 2 u) * CKV_SCAN_WARPS + w.  The (c, u) pairs that occur form a monotone staircase, so with the factor 2 the
-// group behind a unit's last CTA is free: its first entry holds the last block's partial.  A unit's entries are
-// therefore contiguous: `first`, and `count` of them (zero for an empty sequence).
+// group behind a unit's last CTA is free.  In tail mode (P.tail) the scan CTAs leave the LAST block of every
+// sequence (the one a new token lands in) to the launch's tail CTAs, whose partial takes the first entry of that
+// free group.  Either way a unit's entries are contiguous: `first`, and `count` of them (zero for an empty sequence).
 // len_of(i) is the clamped length of sequence i.  Must be called by all 32 lanes of a warp; every lane gets the result.
-__device__ __forceinline__ int ckv_scan_blocks(int n, int bs) { return max((n + bs - 1) / bs - 1, 0); }
+__device__ __forceinline__ int ckv_scan_blocks(int n, int bs, int tail) { return max((n + bs - 1) / bs - tail, 0); }
 template <class LenFn>
 __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of, int units, int unit, int scan_grid,
                                                   int lane, int &first, int &count) {
@@ -262,7 +267,7 @@ __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of,
   unsigned tot = 0, before = 0, mine = 0, n_mine = 0;
   for (int i = lane; i < batch; i += 32) {
     const int n = len_of(i);
-    const unsigned t = (unsigned)((ckv_scan_blocks(n, P.bs) + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE);
+    const unsigned t = (unsigned)((ckv_scan_blocks(n, P.bs, P.tail) + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE);
     tot += t;
     if (i < s) before += t;
     if (i == s) { mine = t; n_mine = (unsigned)n; }
@@ -277,7 +282,7 @@ __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of,
   const int cfirst = (int)(T0 / tpc);
   const int ccount = mine == 0 ? 0 : (int)((T0 + mine - 1) / tpc) - cfirst + 1;
   first = (cfirst + 2 * unit) * CKV_SCAN_WARPS;
-  count = n_mine == 0 ? 0 : ccount * CKV_SCAN_WARPS + 1;
+  count = ccount * CKV_SCAN_WARPS + ((P.tail && n_mine > 0) ? 1 : 0);
 }
 // The usual length source: the device array, clamped to the cache's capacity.
 struct CkvClampedLens {

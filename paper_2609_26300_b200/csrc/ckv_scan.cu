@@ -49,7 +49,7 @@ constexpr int kConsumerWarps = CKV_SCAN_WARPS;
 constexpr int kThreads = kConsumerWarps * 32 + 32;   // plus the producer warp
 constexpr int kMaxSeqs = 1024;      // sequence lengths are staged in shared memory up to this many sequences
 
-struct UnitInfo { int N, X, tiles; };   // X: the blocks the scan CTAs cover, all but the sequence's last one
+struct UnitInfo { int N, X, tiles; };   // X: the blocks the scan CTAs cover (in tail mode all but the sequence's last one)
 
 // s_len holds the clamped lengths (after this step's append, if any) of the first kMaxSeqs sequences, staged once
 // per CTA; longer batches never come with an append and read the device array
@@ -59,13 +59,13 @@ __device__ __forceinline__ int seq_len_of(const CkvDev &P, const int *s_len, con
 __device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *s_len, const int *__restrict__ seq_lens, int u) {
   UnitInfo ui;
   ui.N = seq_len_of(P, s_len, seq_lens, u / P.Hkv);
-  ui.X = ckv_scan_blocks(ui.N, P.bs);
+  ui.X = ckv_scan_blocks(ui.N, P.bs, P.tail);
   ui.tiles = (ui.X + TB - 1) / TB;
   return ui;
 }
 
 __device__ __forceinline__ int seq_tiles(const int *s_len, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
-  return (ckv_scan_blocks(seq_len_of(P, s_len, seq_lens, i), P.bs) + TB - 1) / TB;
+  return (ckv_scan_blocks(seq_len_of(P, s_len, seq_lens, i), P.bs, P.tail) + TB - 1) / TB;
 }
 
 constexpr int kLenCounter = 16;   // word of the status region that counts the CTAs which have read the lengths
@@ -173,7 +173,7 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
         }
         __syncwarp();
         const size_t row = (size_t)u * P.max_blocks + b;
-        block_stats_warp<QT, false, true>(P, k_pool, v_pool, pt_row, h, b, cnt, sq, P.kmean + row * P.row_elems,
+        block_stats_warp<QT, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq, P.kmean + row * P.row_elems,
                                     P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
       }
     }
@@ -365,6 +365,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     float *sw = sw_all + (size_t)warp * P.r * G;   // [t][g], r != 4 only
     const float log_bs = logf((float)P.bs);
     const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;
+    float log_last = 0.f;   // log of the token count of the unit's last block, when the scan CTAs cover it
     const bool pair_ok = (P.max_blocks & 1) == 0;   // rows of the per-block outputs start on 8-byte boundaries
     const int ulast = s_ulast;
     int u = s_u0, tl = s_tl0, cur = -1, next_empty = s_u0;
@@ -481,6 +482,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
 #pragma unroll
         for (int t = 0; t < 16; ++t) { acc[t][0] = 0.f; acc[t][1] = 0.f; }
         m_ref = -CUDART_INF_F; l_acc = 0.f; lp_acc = 0.f;
+        log_last = logf((float)(ui.N - (ui.X - 1) * P.bs));
         const size_t row0 = (size_t)u * P.max_blocks;
         lu = P.lu + row0 * G;   // [head][block] within the unit
         lz = P.lz + row0 * G;
@@ -578,8 +580,9 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
             }
             sig[nt][e] = sg;
             const float zbar = z[nt][e] * P.scale;
-            ell[e] = log_bs + zbar + P.half_var * sg;   // every block the scan CTAs see is full
-            zl2[nt][e] = val[nt][e] ? (zbar + log_bs) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
+            const float logc = (!P.tail && b == ui.X - 1) ? log_last : log_bs;   // in tail mode every block here is full
+            ell[e] = logc + zbar + P.half_var * sg;
+            zl2[nt][e] = val[nt][e] ? (zbar + logc) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
             tmax = fmaxf(tmax, zl2[nt][e]);
           }
           // what the later kernels read, both in log2 units: the head's term of the block score, e^l sigma^2 (e^l
@@ -730,21 +733,18 @@ namespace {
 // of three or four dependent cache misses, each of which costs several microseconds once the scan CTAs have
 // saturated DRAM (two rounds for 32 units made the whole step 7 us slower than one).
 int tail_ctas(const ckv_ctx *c, int batch) {
+  if (!c->dev.tail) return 0;
   const int units = batch * c->dev.Hkv;
   const int one_round = (units + 7) / 8;
   if (one_round <= 16) return std::max(1, one_round);
   return std::min((units + 15) / 16, std::max(16, c->sm_count / 4));   // many units: two rounds, at most a quarter of the SMs
-}
-int tail_rounds(const ckv_ctx *c, int batch) {
-  const int units = batch * c->dev.Hkv;
-  return (units + 8 * tail_ctas(c, batch) - 1) / (8 * tail_ctas(c, batch));
 }
 }  // namespace
 
 // Scan CTAs of a step: one persistent CTA per SM the tail CTAs leave free, never more CTAs than tiles.
 int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
   const CkvDev &P = c->dev;
-  const int xmax = std::max((max_len + P.bs - 1) / P.bs - 1, 0);   // the last block of a sequence is the tail CTAs'
+  const int xmax = std::max((max_len + P.bs - 1) / P.bs - P.tail, 0);   // in tail mode the last block is the tail CTAs'
   const long long tiles = (long long)batch * P.Hkv * ((xmax + TB - 1) / TB);
   long long grid = c->sm_count - tail_ctas(c, batch);
   if (grid > CKV_MAX_SCAN_CTAS) grid = CKV_MAX_SCAN_CTAS;
@@ -752,16 +752,20 @@ int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
   return (int)(grid < 1 ? 1 : grid);
 }
 
-// Whether the step's append should ride in the scan launch: the lengths must fit the staging array, and the tail
-// CTAs' rounds (about 20 us each under load) must hide behind the scan (about 5 MB per us), otherwise the
-// stand-alone append launch, whose warps all run at once, is the shorter way.
-bool ckv_scan_can_append(const ckv_ctx *c, int batch, int max_len) {
-  if (batch > kMaxSeqs) return false;
+// Tail mode pays when the scan is long enough to hide the tail CTAs: a tail warp's work is a chain of dependent
+// cache misses and of instructions fetched once (9 - 20 us without a new token, 15 - 35 us with one, per round),
+// whereas the scan streams about 5 MB per microsecond.  Below that size the scan CTAs cover every block and the
+// append is a launch of its own, whose warps all run at once.
+bool ckv_scan_wants_tail(const ckv_ctx *c, int batch, int max_len) {
+  if (batch > kMaxSeqs || c->tail_mode == CKV_TAIL_OFF) return false;   // the lengths must fit the staging array
+  if (c->tail_mode == CKV_TAIL_ON) return true;
   const CkvDev &P = c->dev;
-  const int rounds = tail_rounds(c, batch);
-  if (rounds == 1) return true;
-  const double bytes = (double)batch * P.Hkv * ((max_len + P.bs - 1) / P.bs) * (2.0 * P.row_elems * 2 + 4.0 * P.r);
-  return bytes / 5.0e6 >= 30.0 * rounds;   // scan microseconds against tail microseconds, with a margin
+  const int units = batch * P.Hkv;
+  const int one_round = (units + 7) / 8;
+  const int n_tail = one_round <= 16 ? std::max(1, one_round) : std::min((units + 15) / 16, std::max(16, c->sm_count / 4));
+  const int rounds = (units + 8 * n_tail - 1) / (8 * n_tail);
+  const double bytes = (double)units * ((max_len + P.bs - 1) / P.bs) * (2.0 * P.row_elems * 2 + 4.0 * P.r);
+  return bytes / 5.0e6 >= 40.0 * rounds;
 }
 
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
@@ -772,7 +776,7 @@ cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int 
   const int grid = n_tail + n_scan;
   CkvNewToken fresh = {};
   if (fresh_in != nullptr) {
-    if (!ckv_scan_can_append(c, batch, max_len)) return cudaErrorInvalidValue;
+    if (!P.tail || batch > kMaxSeqs) return cudaErrorInvalidValue;   // the new token is the tail CTAs' job
     fresh = *fresh_in;
   }
   *grid_out = n_scan;

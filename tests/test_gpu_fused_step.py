@@ -26,11 +26,14 @@ def rows(d, t):
             torch.from_numpy(v_new).to(d.dtype).cuda())
 
 
-def run_both(w, steps, dtype=torch.bfloat16, step_launches=3, **layout):
+def run_both(w, steps, dtype=torch.bfloat16, step_launches=3, tail=binding.CKV_TAIL_ON, **layout):
     """Two identical caches: one stepped with ckv_step, one with ckv_append + ckv_decode.  The summaries, pages,
-    lengths and selected ids must be identical; the outputs agree bit for bit (same kernels, same order)."""
+    lengths and selected ids must be identical; the outputs agree bit for bit (same kernels, same order).  The
+    caches here are small, so the mode the library would pick by itself is the two-call one: tail mode (the
+    append inside the scan launch) is switched on explicitly unless a test says otherwise."""
     a, b = setup(w, dtype, **layout), setup(w, dtype, **layout)
     for d in (a, b):
+        d.ckv.set_tail_mode(tail)
         d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
     for t in range(steps):
         q, kn, vn = rows(a, t)
@@ -79,6 +82,7 @@ def test_step_equals_append_then_decode_bf16_summaries():
 def test_step_launch_count_is_three():
     w = small(decode_steps=2)
     d = setup(w)
+    d.ckv.set_tail_mode(binding.CKV_TAIL_ON)
     d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
     torch.cuda.synchronize()
     n0 = d.ckv.launch_count()
@@ -96,17 +100,25 @@ def test_many_units_one_round_of_tail_warps():
 
 
 def test_more_units_than_one_round_of_tail_warps():
-    """136 units: the tail warps go round twice, and the cache is long enough (35K tokens per sequence) for the
-    library to keep the append inside the scan launch (short caches with this many units take the two-call route,
-    which the second half checks)."""
-    w = small(batch=17, num_q_heads=8, num_kv_heads=8, ctx_min=16 * 2100, ctx=16 * 2200 + 5, decode_steps=3,
-              budget_tokens=16 * 8, needles=0, outlier_dims=0)
-    a = run_both(w, 3)   # three launches per step: scan (with the append), select, attention + merge
-    del a
-    torch.cuda.empty_cache()
+    """136 units: the tail warps go round twice."""
     w = small(batch=17, num_q_heads=8, num_kv_heads=8, ctx_min=16 * 8 + 1, ctx=16 * 20 + 3, decode_steps=6,
               budget_tokens=16 * 6, needles=0)
-    run_both(w, 6, step_launches=4)   # append, scan, select, attention + merge
+    run_both(w, 6)
+
+
+def test_small_steps_take_the_two_call_route_by_default_and_agree_with_tail_mode():
+    """Left to itself the library appends in a launch of its own when the scan is too short to hide the tail CTAs
+    (four launches); the result agrees with tail mode to rounding: same ids, outputs within the bf16 tolerance."""
+    w = small(ctx_min=16 * 20 + 1, ctx=16 * 70 + 5, decode_steps=10)
+    a = run_both(w, 10, step_launches=4, tail=binding.CKV_TAIL_AUTO)
+    b = run_both(w, 10, step_launches=3, tail=binding.CKV_TAIL_ON)
+    q = torch.from_numpy(synth.queries(w, 9)).to(a.dtype).cuda()
+    oa, la, ia, ca = a.ckv.decode(q, a.k_pool, a.v_pool, a.table, a.lens, a.max_len + 10, w.budget_tokens)
+    ob, lb, ib, cb = b.ckv.decode(q, b.k_pool, b.v_pool, b.table, b.lens, b.max_len + 10, w.budget_tokens)
+    torch.cuda.synchronize()
+    assert torch.equal(ia, ib) and torch.equal(ca, cb)
+    assert float((oa.float() - ob.float()).abs().max()) <= 2e-2 * float(ob.float().abs().max())
+    assert float((la - lb).abs().max()) <= 1e-4
 
 
 def test_step_on_full_sequence_sets_status_and_keeps_length():
@@ -116,6 +128,7 @@ def test_step_on_full_sequence_sets_status_and_keeps_length():
     a, b = setup(w), setup(w)
     cap = a.table.shape[1] * 16
     for d in (a, b):
+        d.ckv.set_tail_mode(binding.CKV_TAIL_ON)
         d.lens[0] = cap                                  # sequence 0 fills its page table completely
         d.lens[1] = cap - 21
         d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, cap)
@@ -140,6 +153,7 @@ def test_step_replayed_in_a_cuda_graph_advances_lengths():
     w = small(ctx=16 * 30 + 7, decode_steps=12)
     a, b = setup(w), setup(w)
     for d in (a, b):
+        d.ckv.set_tail_mode(binding.CKV_TAIL_ON)
         d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
     q, kn, vn = rows(a, 0)
     max_len = a.max_len + 12

@@ -332,8 +332,13 @@ def test_append_past_capacity_sets_status():
 
 # ---- decode steps with appends ----------------------------------------------------------------------------------------
 
-def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False, fused=False, **ck):
+def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False, fused=False, tail_on=None, **ck):
+    from paper_2609_26300_b200 import binding
     w = d.w
+    # these caches are small: left to itself the library would take the two-call route for every step, so the
+    # ckv_step tests switch tail mode (the append inside the scan launch) on explicitly
+    if fused or tail_on:
+        d.ckv.set_tail_mode(binding.CKV_TAIL_ON)
     n0 = d.lens.cpu().numpy().copy()
     d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
     for t in range(steps):
@@ -385,6 +390,13 @@ def test_decode_loop_small_with_appends():
     w = small(ctx_min=16 * 30 + 1, ctx=16 * 60, decode_steps=36)
     d = setup(w)
     decode_loop(d, 36, w.budget_tokens, set(range(36)), all_units(w))
+
+
+def test_decode_loop_two_calls_in_tail_mode():
+    """ckv_append + ckv_decode with the last block of every sequence left to the scan launch's tail CTAs."""
+    w = small(ctx_min=16 * 30 + 1, ctx=16 * 60, decode_steps=20)
+    d = setup(w)
+    decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), tail_on=True)
 
 
 @pytest.mark.parametrize("bs,r", [(16, 4), (32, 4), (64, 4), (16, 128), (16, 8)])
