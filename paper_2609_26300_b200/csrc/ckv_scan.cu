@@ -146,6 +146,7 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
   __syncthreads();
   auto len_of = [&](int i) { return seq_len_of(P, s_len, seq_lens, i); };
 
+#pragma unroll 1
   for (int u = u_first; u < units; u += n_tail * 8) {
     const int s = u / P.Hkv, h = u % P.Hkv;
     if (u != u_first) {
@@ -188,9 +189,14 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
     if (P.r == CKV_D) {
       load_split8<false>(reinterpret_cast<const __nv_bfloat16 *>(P.dbar + row * CKV_D), li, b, dx);
     } else {
+      // group of coordinate c: c / (128 / r), or ((c mod 64) / (64 / r)) in the half-split layout; r is a power of two
       const float *drow = P.dbar + row * P.r;
+      const int sh = 31 - __clz(CKV_D / P.r);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) dx[i] = drow[group_of(8 * li + i, P.r, P.glayout)];
+      for (int i = 0; i < 8; ++i) {
+        const int c = 8 * li + i;
+        dx[i] = drow[P.glayout == 0 ? c >> sh : (c & (CKV_D / 2 - 1)) >> (sh - 1)];
+      }
     }
     int first = 0, count = 0;
     unit_scan_entries(P, len_of, units, u, nscan, lane, first, count);
