@@ -20,13 +20,12 @@
 //
 // Merge.  The scan's partials of the unit (one per scan CTA and consumer warp) exist before this kernel
 // starts, so the unit's active CTAs share them out, fetch their share while their last page is in flight and
-// fold it into their own partial.  What is left is one partial (m, l, acc[128]) per head and warp or CTA:
-//   * sparse mode launches the unit's splits (at most 8) as one thread-block cluster: every WARP folds its share
-//     of the scan partials into its own accumulators and stores its partial of head g, straight from registers,
-//     into the shared memory of CTA g mod cluster size (distributed-shared-memory stores); after one cluster
-//     barrier that CTA reduces the head from its own shared memory and writes the output row and the log-sum-exp.
-//     No warp waits for the other warps of its CTA, nobody's shared memory is read remotely, so no CTA waits for
-//     another before it leaves (the pull version, remote loads between two barriers, was 3 us slower per step);
+// fold it into their own partial.  What is left is one partial (m, l, acc[128]) per head and CTA:
+//   * sparse mode launches the unit's splits (at most 8) as one thread-block cluster: every CTA stores its
+//     partial of head g into the shared memory of CTA g mod cluster size (distributed-shared-memory stores), and
+//     after one cluster barrier that CTA reduces the head from its own shared memory and writes the output row
+//     and the log-sum-exp.  Nobody's shared memory is read remotely, so no CTA waits for another before it
+//     leaves (the pull version, remote loads between two barriers, was 3 us slower per step);
 //   * dense mode (more splits than a cluster holds), and sparse mode when a cluster cannot be placed, publish the
 //     partials in global memory and bump the unit's counter; the CTA that finds the counter complete reads them
 //     back and writes the output.  The counter is left at zero for the next step.
@@ -71,11 +70,9 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   extern __shared__ __align__(128) unsigned char smem[];   // [W warps][2 buffers][K tile | V tile], then [W warps][aux]
   __shared__ float s_M[G], s_den[G];
   __shared__ int s_last;
-  // Cluster merge: where the warps of all splits of the unit deposit their partials of the heads this CTA reduces.
-  // Entry ((j * cluster size + source rank) * W + source warp) belongs to head (this rank + j * cluster size).
-  // (heads are dealt round-robin to the cluster's CTAs: a CTA reduces at most ceil(G / size) heads, size <= 8)
-  constexpr int kRecvEntries = (G + kMaxCluster - 1) * W;
-  __shared__ __align__(16) float s_recv[CL ? kRecvEntries * CKV_PART_STRIDE : 4];
+  // Cluster merge: where the other splits of the unit deposit their partials of the heads this CTA reduces.
+  // Entry (j * cluster size + source rank) belongs to head (this rank + j * cluster size).
+  __shared__ __align__(16) float s_recv[CL ? (G + kMaxCluster) * CKV_PART_STRIDE : 4];
   if (CL) cluster_arrive_relaxed();   // first phase of the cluster barrier: "this CTA runs, its shared memory exists"
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -100,40 +97,46 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   const bool comp = !DENSE && nsel < X && !(P.variant & CKV_VARIANT_DROP);
   const int p1 = min(p0 + pages_per_split, total);
   float *part = P.attn_part + ((size_t)unit * CKV_MAX_SPLITS + blockIdx.x) * G * CKV_PART_STRIDE;
-  // Cluster merge: CTA r of the cluster (= split r of the unit) reduces heads r, r + cluster size, ...  Every WARP
-  // of every CTA stores its partial of a head (running maximum, normaliser, 128 numerators, straight from its
-  // accumulator registers) into the shared memory of the CTA that reduces that head; one cluster barrier later
-  // the data is local there.  No warp waits for the other warps of its CTA, no CTA's shared memory is read
-  // remotely, so nobody has to wait before leaving.  acc == nullptr: a split without pages announces empty partials.
-  auto cluster_merge = [&](const float (*acc)[2], float m_w, float l_w) {
-    const int head = lane >> 2, qd = lane & 3;
+  // Cluster merge: CTA r of the cluster (= split r of the unit) reduces heads r, r + cluster size, ...  Every CTA
+  // stores its partial of a head into the shared memory of the CTA that reduces it; one cluster barrier later the
+  // data is local there.  No CTA's shared memory is read remotely, so nobody has to wait before leaving.
+  // `num` holds this CTA's numerators (thread t: element t, t + W * 32, ... of [G][CKV_D]); `have` is false for a
+  // split without pages, which only announces an empty partial.
+  auto cluster_merge = [&](const float *num, bool have) {
     cluster_wait();   // every CTA of the cluster has started
     const uint32_t rank = cluster_rank(), csize = cluster_size();
     const uint32_t recv0 = (uint32_t)__cvta_generic_to_shared(s_recv);
-    if (head < G) {
-      const uint32_t ent = (((uint32_t)head / csize) * csize + rank) * W + warp;
-      const uint32_t dst = cluster_map(recv0 + ent * kPartBytes, (uint32_t)head % csize);
-      if (acc != nullptr) {
+    constexpr int NP = (G * CKV_D + W * 32 - 1) / (W * 32);
+    if (have) {
 #pragma unroll
-        for (int t = 0; t < 16; ++t) st_cluster_f32x2(dst + (4 + 8 * t + 2 * qd) * 4, acc[t][0], acc[t][1]);
+      for (int it = 0; it < NP; ++it) {
+        const int idx = tid + it * W * 32;
+        if (idx < G * CKV_D) {
+          const uint32_t g = idx / CKV_D, c = idx % CKV_D;
+          const uint32_t ent = (g / csize) * csize + rank;
+          st_cluster_f32(cluster_map(recv0 + (ent * CKV_PART_STRIDE + 4 + c) * 4, g % csize), num[it]);
+        }
       }
-      if (qd == 0) st_cluster_f32x2(dst, acc != nullptr ? m_w : -CUDART_INF_F, acc != nullptr ? l_w : 0.f);
+    }
+    if (tid < G) {
+      const uint32_t ent = ((uint32_t)tid / csize) * csize + rank;
+      st_cluster_f32x2(cluster_map(recv0 + ent * kPartBytes, (uint32_t)tid % csize),
+                       have ? s_M[tid] : -CUDART_INF_F, have ? s_den[tid] : 0.f);
     }
     cluster_sync_all();   // release the stores, acquire everybody else's
-    const int n_ent = (int)csize * W;   // entries per head: at most 32, one per lane
     for (int g = (int)rank, j = 0; g < G; g += (int)csize, ++j) {
-      const float *e0 = s_recv + (size_t)j * n_ent * CKV_PART_STRIDE;
+      const float *e0 = s_recv + (size_t)j * csize * CKV_PART_STRIDE;
       float2 ml = make_float2(-CUDART_INF_F, 0.f);
-      if (lane < n_ent) ml = *reinterpret_cast<const float2 *>(e0 + lane * CKV_PART_STRIDE);
+      if (lane < (int)csize) ml = *reinterpret_cast<const float2 *>(e0 + lane * CKV_PART_STRIDE);
       const float M = warp_max(ml.x);
       const float sc = exp2_diff(ml.x, M);
       const float den = warp_sum(ml.y * sc);
       for (int c = tid; c < CKV_D; c += W * 32) {
         float o = 0.f;
-#pragma unroll 8
-        for (int e = 0; e < n_ent; ++e) {
+#pragma unroll
+        for (int e = 0; e < kMaxCluster; ++e) {
           const float sce = __shfl_sync(0xffffffffu, sc, e);
-          if (sce != 0.f) o = fmaf(e0[e * CKV_PART_STRIDE + 4 + c], sce, o);
+          if (e < (int)csize && sce != 0.f) o = fmaf(e0[e * CKV_PART_STRIDE + 4 + c], sce, o);
         }
         out[((size_t)s * P.Hq + h * G + g) * CKV_D + c] = __float2bfloat16_rn(o / den);
       }
@@ -149,7 +152,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
       }
       return;
     }
-    if (CL) cluster_merge(nullptr, 0.f, 0.f);   // it still takes part in the cluster's merge, with empty partials
+    if (CL) cluster_merge(nullptr, false);   // it still takes part in the cluster's merge, with an empty partial
     return;
   }
   const int n_active = (total + pages_per_split - 1) / pages_per_split;   // splits of this unit that have pages
@@ -451,45 +454,6 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   __syncwarp();
   if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
 
-  if constexpr (CL) {
-    // ---- cluster path: the warp folds its own share of the scan partials (they sit in its idle page buffer, or
-    //      arrive there round by round) into its accumulators and hands the result to the reducing CTAs ----
-    const int ent_buf = (n_mine > 0 ? (n_mine - 1) & 1 : 0) ^ 1;
-    const float *ents = reinterpret_cast<const float *>(wtiles + (size_t)ent_buf * kPageBytes);
-    for (int base = 0; base < my_cnt; base += kSlots) {
-      if (base > 0) {
-        __syncwarp();   // the entries of the round before have been read
-        issue_comp(ent_buf, base);
-        cp_async_commit();
-        cp_async_wait<0>();
-        __syncwarp();
-      }
-#pragma unroll 1
-      for (int k = 0; k < kSlotsPerWarp; ++k) {
-        if (base + warp * kSlotsPerWarp + k >= my_cnt) break;   // warp-uniform
-        if (hv) {
-          const float *eh = ents + (size_t)k * G * CKV_PART_STRIDE + head * CKV_PART_STRIDE;
-          const float me = eh[0];
-          if (me != -CUDART_INF_F) {
-            const float M = fmaxf(m_ref, me);
-            const float s0 = exp2_diff(m_ref, M), s1 = exp2f(me - M);
-            l_acc = fmaf(l_acc, s0, qd == 0 ? eh[1] * s1 : 0.f);   // the entry's normaliser enters once per head
-#pragma unroll
-            for (int t = 0; t < 16; ++t) {
-              const float2 a = *reinterpret_cast<const float2 *>(eh + 4 + 8 * t + 2 * qd);
-              acc[t][0] = fmaf(acc[t][0], s0, a.x * s1);
-              acc[t][1] = fmaf(acc[t][1], s0, a.y * s1);
-            }
-            m_ref = M;
-          }
-        }
-      }
-    }
-    l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 1);
-    l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 2);
-    cluster_merge(acc, m_ref, l_acc);
-  } else {
-
   // ---- CTA partial: fold the warps (each with its own running maximum) and this CTA's scan partials ----
   // A warp's partial [G][CKV_PART_STRIDE] goes into the buffer of its last page; the other buffer holds its
   // share of the scan partials.  Entry e < W is warp e's partial, entry W + c is scan-partial slot c.
@@ -568,7 +532,10 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     cp_async_commit();
     cp_async_wait<0>();
   }
-  {
+  if constexpr (CL) {
+    cluster_merge(num, true);
+    return;
+  } else {
 #pragma unroll
   for (int it = 0; it < NI; ++it) {
     const int idx = tid + it * W * 32;
@@ -624,7 +591,6 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     o2.y = pack_bf16(o.z * inv, o.w * inv);
     *reinterpret_cast<uint2 *>(out + ((size_t)s * P.Hq + h * G + g) * CKV_D + c4) = o2;
     if (lse != nullptr && lane == 0) lse[(size_t)s * P.Hq + h * G + g] = (M + log2f(den)) * kLn2;
-  }
   }
   }   // !CL
 }
