@@ -249,7 +249,7 @@ def main():
     # ---- inputs: every rank holds a full replica of the workload (the path does not shard) ----
     k_pool, v_pool, table, lens = synth.make_pools(w, threads=min(8, os.cpu_count() or 1))
     q_np, kn_np, vn_np = step_inputs(w, total)
-    max_blocks = synth.pages_per_seq(w)
+    max_blocks = synth.pages_per_seq(w) * w.page_size // w.block_size   # the table row holds whole blocks
     ckv = binding.CompKV(w.num_q_heads, w.num_kv_heads, w.batch, max_blocks, k_pool.shape[0],
                          block_size=w.block_size, var_groups=w.var_groups, device=str(dev),
                          stat_bf16=int(args.stat_bf16))

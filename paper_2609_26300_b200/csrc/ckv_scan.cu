@@ -770,8 +770,11 @@ bool ckv_scan_wants_tail(const ckv_ctx *c, int batch, int max_len) {
   const int one_round = (units + 7) / 8;
   const int n_tail = one_round <= 16 ? std::max(1, one_round) : std::min((units + 15) / 16, std::max(16, c->sm_count / 4));
   const int rounds = (units + 8 * n_tail - 1) / (8 * n_tail);
-  const double bytes = (double)units * ((max_len + P.bs - 1) / P.bs) * (2.0 * P.row_elems * 2 + 4.0 * P.r);
-  return bytes / 5.0e6 >= 40.0 * rounds;
+  const double blocks = (double)units * ((max_len + P.bs - 1) / P.bs);
+  const double bytes = blocks * (2.0 * P.row_elems * 2 + 4.0 * P.r);
+  // scan microseconds: bandwidth-bound at about 5 MB/us, or issue-bound at about 6000 blocks/us (bf16 summaries)
+  const double scan_us = std::max(bytes / 5.0e6, blocks / 6.0e3);
+  return scan_us >= 40.0 * rounds;
 }
 
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
