@@ -9,12 +9,56 @@
 #define CKV_BLOCKSTATS_CUH_
 #include "ckv_internal.cuh"
 
+// Second half of the block routine, shared by its variants: the half warps' squared deviations are combined, the
+// three summary rows are written (hw 0: mean key and variances, hw 1: mean value).  km: mean key, vs: value sums,
+// sq: this half warp's squared deviations, all for the lane's 8 coordinates.
+__device__ __forceinline__ void block_stats_finish(const CkvDev &P, int b, float fc, const float (&km)[8],
+                                                   const float (&vs)[8], float (&sq)[8], float *sq_smem,
+                                                   __nv_bfloat16 *kmean_row, float *dbar_row,
+                                                   __nv_bfloat16 *vmean_row, int lane, bool bad) {
+  const int hw = lane >> 4, li = lane & 15;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], 16);
+  if (hw == 0) {
+    store_split8(kmean_row, li, b, km, P.row_elems == CKV_ROW_ELEMS);
+    if (P.r == CKV_D) {
+      // one group per coordinate: the variance row has the mean rows' layout (split bf16 pairs, swizzled chunks),
+      // so that the scan can project it with the same tensor-core product as the mean keys
+      float dv[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) dv[i] = sq[i] / fc;
+      store_split8(reinterpret_cast<__nv_bfloat16 *>(dbar_row), li, b, dv);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sq_smem[8 * li + i] = sq[i];
+    }
+  } else {
+    float vm[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) vm[i] = vs[i] / fc;
+    store_split8(vmean_row, li, b, vm, P.row_elems == CKV_ROW_ELEMS);
+  }
+  __syncwarp();
+  // grouped variance: average of the per-coordinate population variances of each group (Eq. 8)
+  const int gs = CKV_D / P.r;
+  for (int t = lane; t < P.r && P.r != CKV_D; t += 32) {
+    float s = 0.f;
+    if (P.glayout == 0) {
+      for (int i = 0; i < gs; ++i) s += sq_smem[t * gs + i];
+    } else {
+      const int hg = gs / 2;
+      for (int i = 0; i < hg; ++i) s += sq_smem[t * hg + i];
+      for (int i = 0; i < hg; ++i) s += sq_smem[CKV_D / 2 + t * hg + i];
+    }
+    dbar_row[t] = s / (fc * (float)gs);
+  }
+  __syncwarp();
+  if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
+}
+
 // NC: the pools are read-only for the whole kernel (loads may use the non-coherent path).
-// SMALL: compact code for callers that are bound by memory latency and share their kernel with a hot loop whose
-// instructions should stay cached: loops are not unrolled and the register-resident one-page path is left out
-// (the general path performs the same operations in the same order, hence the same bits).
 // sq_smem: 128 floats of shared memory owned by the calling warp.
-template <typename T, bool NC, bool SMALL = false>
+template <typename T, bool NC>
 __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__restrict__ k_pool,
                                                  const T *__restrict__ v_pool, const int *__restrict__ pt_row,
                                                  int h, int b, int cnt, float *sq_smem, __nv_bfloat16 *kmean_row,
@@ -28,7 +72,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
   const float fc = (float)cnt;
   float km[8], sq[8];
   bool done = false;
-  if constexpr (sizeof(T) == 2 && !SMALL) {
+  if constexpr (sizeof(T) == 2) {
     if (npages == 1) {
       // One page of bf16 rows (every block of the default 16-token layout): the key rows stay in registers between
       // the two passes, so the cache is read exactly once.  Same operations in the same order as the general path
@@ -83,7 +127,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
       if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
       const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
       const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
-#pragma unroll(SMALL ? 1 : 8)
+#pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int t = hw + 2 * j;
         if (t < ntok) {
@@ -107,7 +151,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
       if (phys < 0 || phys >= P.num_pages) continue;
       const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
       const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
-#pragma unroll(SMALL ? 1 : 8)
+#pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int t = hw + 2 * j;
         if (t < ntok) {
@@ -119,43 +163,89 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
       }
     }
   }
+  block_stats_finish(P, b, fc, km, vs, sq, sq_smem, kmean_row, dbar_row, vmean_row, lane, bad);
+}
+
+// The same block routine for a caller whose time goes into instruction fetch rather than arithmetic (the tail
+// warps of the scan launch run this code once per launch, next to a kernel that saturates DRAM): the rows of a
+// page are brought into shared memory with asynchronous 16-byte copies issued from a rolled loop (all in flight
+// together, no load waits for another), and both passes are rolled loops over the staged rows.  Same operations
+// in the same order as block_stats_warp, hence the same bits; a third of its code.
+// stage: 2 * CKV_PAGE * CKV_D * sizeof(T) bytes of shared memory owned by the calling warp, 16-byte aligned.
+template <typename T>
+__device__ __forceinline__ void block_stats_warp_staged(const CkvDev &P, const T *k_pool, const T *v_pool,
+                                                        const int *pt_row, int h, int b, int cnt,
+                                                        unsigned char *stage, float *sq_smem,
+                                                        __nv_bfloat16 *kmean_row, float *dbar_row,
+                                                        __nv_bfloat16 *vmean_row, int lane) {
+  const int hw = lane >> 4, li = lane & 15;
+  constexpr int kPageElems = CKV_PAGE * CKV_D;
+  constexpr int kPieces = (int)(kPageElems * sizeof(T) / 16);   // 16-byte pieces of one head's K (or V) page
+  const T *sk = reinterpret_cast<const T *>(stage), *sv = sk + kPageElems;
+  const uint32_t stage_u32 = (uint32_t)__cvta_generic_to_shared(stage);
+  float ks[8], vs[8], km[8], sq[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], 16);
-  if (hw == 0) {
-    store_split8(kmean_row, li, b, km, P.row_elems == CKV_ROW_ELEMS);
-    if (P.r == CKV_D) {
-      // one group per coordinate: the variance row has the mean rows' layout (split bf16 pairs, swizzled chunks),
-      // so that the scan can project it with the same tensor-core product as the mean keys
-      float dv[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) dv[i] = sq[i] / fc;
-      store_split8(reinterpret_cast<__nv_bfloat16 *>(dbar_row), li, b, dv);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) sq_smem[8 * li + i] = sq[i];
+  for (int i = 0; i < 8; ++i) { ks[i] = 0.f; vs[i] = 0.f; }
+  const int npages = (cnt + CKV_PAGE - 1) / CKV_PAGE;
+  const float fc = (float)cnt;
+  bool bad = false;
+  auto stage_page = [&](int pg, bool with_v) -> bool {   // false: the page id is bad, nothing staged
+    const int phys = pt_row[b * P.ppb + pg];
+    if (phys < 0 || phys >= P.num_pages) return false;
+    const size_t base = ((size_t)phys * P.Hkv + h) * kPageElems;
+    const char *gk = reinterpret_cast<const char *>(k_pool + base), *gv = reinterpret_cast<const char *>(v_pool + base);
+    const int n = with_v ? 2 * kPieces : kPieces;
+#pragma unroll 1
+    for (int p = lane; p < n; p += 32) {
+      const char *src = p < kPieces ? gk + (size_t)p * 16 : gv + (size_t)(p - kPieces) * 16;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_u32 + (uint32_t)p * 16u), "l"(src) : "memory");
     }
-  } else {
-    float vm[8];
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    return true;
+  };
+#pragma unroll 1
+  for (int pg = 0; pg < npages; ++pg) {
+    if (!stage_page(pg, true)) { bad = true; continue; }
+    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+#pragma unroll 1
+    for (int j = 0; j < 8; ++j) {
+      const int t = hw + 2 * j;
+      if (t < ntok) {
+        float a[8], c[8];
+        load8<false>(sk + t * CKV_D + 8 * li, a);
+        load8<false>(sv + t * CKV_D + 8 * li, c);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) vm[i] = vs[i] / fc;
-    store_split8(vmean_row, li, b, vm, P.row_elems == CKV_ROW_ELEMS);
-  }
-  __syncwarp();
-  // grouped variance: average of the per-coordinate population variances of each group (Eq. 8)
-  const int gs = CKV_D / P.r;
-  for (int t = lane; t < P.r && P.r != CKV_D; t += 32) {
-    float s = 0.f;
-    if (P.glayout == 0) {
-      for (int i = 0; i < gs; ++i) s += sq_smem[t * gs + i];
-    } else {
-      const int hg = gs / 2;
-      for (int i = 0; i < hg; ++i) s += sq_smem[t * hg + i];
-      for (int i = 0; i < hg; ++i) s += sq_smem[CKV_D / 2 + t * hg + i];
+        for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+      }
     }
-    dbar_row[t] = s / (fc * (float)gs);
+    __syncwarp();   // the stage may be overwritten
   }
-  __syncwarp();
-  if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
+    vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
+    km[i] = ks[i] / fc;
+    sq[i] = 0.f;
+  }
+#pragma unroll 1
+  for (int pg = 0; pg < npages; ++pg) {
+    if (npages > 1 && !stage_page(pg, false)) continue;   // a one-page block is still staged from the first pass
+    if (npages == 1 && bad) continue;
+    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+#pragma unroll 1
+    for (int j = 0; j < 8; ++j) {
+      const int t = hw + 2 * j;
+      if (t < ntok) {
+        float a[8];
+        load8<false>(sk + t * CKV_D + 8 * li, a);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+      }
+    }
+    __syncwarp();
+  }
+  block_stats_finish(P, b, fc, km, vs, sq, sq_smem, kmean_row, dbar_row, vmean_row, lane, bad);
 }
 
 #endif  // CKV_BLOCKSTATS_CUH_

@@ -116,7 +116,7 @@ __device__ __noinline__ void lens_arrive(int *counter, const int *seq_lens, int 
 template <int G, typename QT>
 __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q, const int *seq_lens, int *s_len,
                                        int len_mine, int units, int nscan, const CkvNewToken fresh, int n_tail,
-                                       float *smem_f) {
+                                       float *smem_f, int smem_bytes) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, hw = lane >> 4, li = lane & 15;
   const int batch = units / P.Hkv, cap = P.max_blocks * P.bs;
   const bool append = fresh.k_new != nullptr;
@@ -174,8 +174,15 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
         }
         __syncwarp();
         const size_t row = (size_t)u * P.max_blocks + b;
-        block_stats_warp<QT, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq, P.kmean + row * P.row_elems,
-                                    P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
+        // rows staged in this warp's slice of the (otherwise unused) ring memory when it is large enough
+        constexpr int kStageBytes = 2 * CKV_PAGE * CKV_D * (int)sizeof(QT);
+        if (smem_bytes >= 8 * CKV_D * 4 + 8 * kStageBytes)
+          block_stats_warp_staged<QT>(P, k_pool, v_pool, pt_row, h, b, cnt,
+                                      reinterpret_cast<unsigned char *>(smem_f + 8 * CKV_D) + (size_t)warp * kStageBytes, sq,
+                                      P.kmean + row * P.row_elems, P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
+        else
+          block_stats_warp<QT, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq, P.kmean + row * P.row_elems,
+                                      P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
       }
     }
     const int N = len_of(s);
@@ -269,7 +276,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   if ((int)blockIdx.x < n_tail) {
     // ---------------- tail CTAs: the new token and the last block of every unit ----------------
     scan_tail<G, QT>(P, q, seq_lens, s_len, len_mine, units, (int)gridDim.x - n_tail, fresh, n_tail,
-                     reinterpret_cast<float *>(stage_mem));
+                     reinterpret_cast<float *>(stage_mem), stages * stage_bytes);
     if (append) lens_arrive(P.status + kLenCounter, seq_lens, fresh.seq_lens, batch, cap, (int)gridDim.x, /*whole_cta=*/true);
     return;
   }
@@ -758,10 +765,11 @@ int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
   return (int)(grid < 1 ? 1 : grid);
 }
 
-// Tail mode pays when the scan is long enough to hide the tail CTAs: a tail warp's work is a chain of dependent
-// cache misses and of instructions fetched once (9 - 20 us without a new token, 15 - 35 us with one, per round),
-// whereas the scan streams about 5 MB per microsecond.  Below that size the scan CTAs cover every block and the
-// append is a launch of its own, whose warps all run at once.
+// Tail mode pays when the scan is long enough to hide the tail CTAs.  A tail warp's work is a chain of dependent
+// cache misses behind the scan's traffic plus a few thousand instructions run once by a single warp: measured from
+// launch, a round of tail work ends after 15 - 20 us without a new token and after 27 us (idle DRAM, 32K cache) to
+// 45 us (beside a saturating 128K scan) with one, whereas the scan streams about 5 MB per microsecond.  Below that
+// size the scan CTAs cover every block and the append is a launch of its own, whose warps all run at once.
 bool ckv_scan_wants_tail(const ckv_ctx *c, int batch, int max_len) {
   if (batch > kMaxSeqs || c->tail_mode == CKV_TAIL_OFF) return false;   // the lengths must fit the staging array
   if (c->tail_mode == CKV_TAIL_ON) return true;
