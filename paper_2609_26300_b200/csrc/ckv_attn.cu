@@ -470,7 +470,9 @@ cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k
     // Up to 8 splits of a unit run as one cluster and merge in shared memory.  With so few units that 8 splits each
     // would leave most SMs idle, many short splits (merged through global memory) finish sooner.
     // (measured: about 1.75 CTAs per SM is the best grid there; more, shorter splits cost more in the merge)
-    const int by_sm = max(1, 3 * sms / units);
+    // Two of these CTAs fit an SM (shared memory): more than 2 * sms CTAs would run as two waves, the second one
+    // waiting for the first (128 units: 3 splits each took 43 us, 2 splits each 34 us).
+    const int by_sm = max(1, 2 * sms / units);
     n_splits = (by_sm > 8 && units * 16 <= sms) ? (7 * sms / 4 + units - 1) / units : min(by_sm, 8);
   }
   // at least one page per warp of a split: 8-warp CTAs everywhere except the tensor-core kernel's sparse mode (4 warps)
