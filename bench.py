@@ -527,7 +527,7 @@ def main():
                      "traffic": None if SCAN_TRAFFIC_RATIO is None else SCAN_TRAFFIC_RATIO * stats_b},
         "clocks": clocks,
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "call": "ckv_step_host (pinned host q/k_new/v_new in, out/sel_ids/sel_cnt back, stream sync)"},
+                "call": "ckv_step_host (pinned host q/k_new/v_new in, out/sel_ids/sel_cnt back; returns when the results are complete in the host buffers)"},
         "gpu_launches": int(launches_per_step * K),
         "wall_s_timed_region": t_wall,
         "paper_context": PAPER_CONTEXT,

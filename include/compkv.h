@@ -248,10 +248,13 @@ int ckv_exact_blocks(ckv_ctx *ctx, const void *q, const void *k_pool, const int3
  * Mandatory blocks carry their score too (they are excluded from the ranking, not from Eq. 9). */
 int ckv_copy_scores(ckv_ctx *ctx, float *dst, int batch, ckv_stream stream);
 
-/* One whole decode step from HOST buffers: copies q, k_new, v_new to the device, runs
- * ckv_append then ckv_decode, copies out / sel_ids / sel_cnt back and synchronises the stream.
- * Host buffers should be pinned; device staging comes out of the workspace.  seq_lens (device)
- * is incremented.  max_seq_len_host bounds the lengths AFTER the append.  The id staging area holds
+/* One whole decode step from HOST buffers: brings q, k_new, v_new to the device, runs ckv_step,
+ * brings out / sel_ids / sel_cnt back and returns when they are complete in the caller's buffers
+ * (all work the call put on the stream has then finished).  Host buffers should be pinned: buffers the
+ * device can address (pinned, registered or managed memory, 16-byte aligned) are moved by two small
+ * kernels of the library and the call waits on a pinned word its last kernel stores; pageable buffers
+ * take six copies and a stream synchronisation (about 20 us more per call).  Device staging comes out of
+ * the workspace.  seq_lens (device) is incremented.  max_seq_len_host bounds the lengths AFTER the append.  The id staging area holds
  * max_blocks_per_seq ids per unit: budget_tokens / block_size beyond that is CKV_ERR_INVALID_ARG. */
 int ckv_step_host(ckv_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
                   void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens, int batch,

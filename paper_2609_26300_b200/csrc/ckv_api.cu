@@ -3,6 +3,8 @@
 #include <new>
 #include <string.h>
 
+#include <algorithm>
+
 #include "ckv_internal.cuh"
 
 namespace {
@@ -168,11 +170,26 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev_id);
   if (e == cudaSuccess) e = cudaMemsetAsync(P.status, 0, R.ls - R.status, (cudaStream_t)stream);   // status word, split counters
   if (e != cudaSuccess) { delete c; return cuda_fail(e); }
+  // one pinned word for ckv_step_host: its last kernel stores the call's number there and the host waits on the
+  // word instead of on the driver (without it the call falls back to a stream synchronisation)
+  void *flag = nullptr;
+  if (cudaHostAlloc(&flag, 64, cudaHostAllocMapped | cudaHostAllocPortable) == cudaSuccess) {
+    c->host_flag = (volatile int *)flag;
+    *c->host_flag = 0;
+    void *dflag = nullptr;
+    if (cudaHostGetDevicePointer(&dflag, flag, 0) == cudaSuccess) c->host_flag_dev = (int *)dflag;
+    else { cudaFreeHost(flag); c->host_flag = nullptr; }
+  } else {
+    (void)cudaGetLastError();
+  }
   *out = c;
   return CKV_OK;
 }
 
-void ckv_destroy(ckv_ctx *ctx) { delete ctx; }
+void ckv_destroy(ckv_ctx *ctx) {
+  if (ctx != nullptr && ctx->host_flag != nullptr) cudaFreeHost((void *)ctx->host_flag);
+  delete ctx;
+}
 
 int ckv_stats_build(ckv_ctx *c, const void *k_pool, const void *v_pool, const int32_t *page_table,
                     const int32_t *seq_lens, int batch, int max_seq_len_host, ckv_stream stream) {
@@ -211,6 +228,65 @@ int ckv_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int32_t *page_tabl
 }
 
 namespace {
+
+// ---- host-buffer entry point: device-visible host memory is moved by kernels, not by the copy engines ----
+
+// The address under which the GPU can reach a host buffer, if it can (pinned or registered memory, managed
+// memory; a device pointer passes through).  Pageable memory: false.
+bool device_view(const void *host, void **dev) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, host) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+  if (a.type == cudaMemoryTypeUnregistered || a.devicePointer == nullptr) return false;
+  *dev = a.devicePointer;
+  return true;
+}
+bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+// three source ranges to three destination ranges, 16 bytes per thread and iteration (sizes are multiples of 16)
+__global__ void __launch_bounds__(1024) ckv_move3_kernel(const uint4 *__restrict__ a, uint4 *__restrict__ da, int na,
+                                                        const uint4 *__restrict__ b, uint4 *__restrict__ db, int nb,
+                                                        const uint4 *__restrict__ c, uint4 *__restrict__ dc, int nc,
+                                                        const int *__restrict__ tail_src, int *__restrict__ tail_dst,
+                                                        int n_tail, int *done_flag, int done_value) {
+  const int stride = gridDim.x * blockDim.x;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < na + nb + nc; i += stride) {
+    if (i < na) da[i] = a[i];
+    else if (i < na + nb) db[i - na] = b[i - na];
+    else dc[i - na - nb] = c[i - na - nb];
+  }
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_tail; i += stride) tail_dst[i] = tail_src[i];   // 4-byte leftovers
+  if (done_flag != nullptr) {   // single-CTA launches only: everything above is in host memory before the word is
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x == 0) { *(volatile int *)done_flag = done_value; __threadfence_system(); }
+  }
+}
+
+cudaError_t ckv_launch_host_in(ckv_ctx *c, const void *hq, const void *hk, const void *hv, void *dq, void *dk, void *dv,
+                               size_t q_bytes, size_t kv_bytes, cudaStream_t s) {
+  const int nq = (int)(q_bytes / 16), nkv = (int)(kv_bytes / 16);
+  const int grid = std::max(1, std::min((nq + 2 * nkv + 255) / 256, 64));
+  ckv_move3_kernel<<<grid, 256, 0, s>>>((const uint4 *)hq, (uint4 *)dq, nq, (const uint4 *)hk, (uint4 *)dk, nkv,
+                                        (const uint4 *)hv, (uint4 *)dv, nkv, nullptr, nullptr, 0, nullptr, 0);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+cudaError_t ckv_launch_host_out(ckv_ctx *c, const void *dout, const int32_t *dids, const int32_t *dcnt, void *ho, void *hi,
+                                void *hc, size_t out_bytes, size_t ids_bytes, size_t cnt_bytes, int *done_flag,
+                                int done_value, cudaStream_t s) {
+  // out rows are multiples of 16 bytes; the id array is moved in 16-byte pieces with a 4-byte remainder; the counts
+  // (one int per unit) go as the 4-byte tail of the same launch.  One CTA: a few tens of KB, and the completion
+  // word must follow every store of the launch.
+  const int no = (int)(out_bytes / 16), ni = (int)(ids_bytes / 16);
+  if (ids_bytes % 16 != 0)   // at most three ids
+    ckv_move3_kernel<<<1, 32, 0, s>>>(nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr, 0,
+                                      dids + ni * 4, (int *)hi + ni * 4, (int)((ids_bytes % 16) / 4), nullptr, 0);
+  ckv_move3_kernel<<<1, 1024, 0, s>>>((const uint4 *)dout, (uint4 *)ho, no, (const uint4 *)dids, (uint4 *)hi, ni,
+                                      nullptr, nullptr, 0, dcnt, (int *)hc, (int)(cnt_bytes / 4), done_flag, done_value);
+  c->launches++;
+  return cudaGetLastError();
+}
 
 // The launches of a sparse decode step; ev (may be null) receives 5 events bracketing them.  With `fresh` the
 // scan launch also appends the step's new token (its tail CTAs do, beside the scan CTAs).
@@ -372,15 +448,40 @@ int ckv_step_host(ckv_ctx *c, const void *q_host, const void *k_new_host, const 
   void *dq = c->work + c->stage_q, *dk = c->work + c->stage_knew, *dv = c->work + c->stage_vnew;
   void *dout = c->work + c->stage_out;
   int32_t *dids = (int32_t *)(c->work + c->stage_ids), *dcnt = (int32_t *)(c->work + c->stage_cnt);
-  CKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
-  CKV_CUDA(cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
-  CKV_CUDA(cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+  // Pinned (or otherwise device-visible) host buffers are read and written by two small kernels of the library,
+  // one before and one after the step, instead of three copy-engine transfers each way: the six transfers cost
+  // about 40 us of a 145 us call.  Pageable buffers take the copies.
+  void *hq = nullptr, *hk = nullptr, *hv = nullptr, *ho = nullptr, *hi = nullptr, *hc = nullptr;
+  // (asked on every call: a buffer may have been freed and its address reused by pageable memory since the last one)
+  const bool direct = device_view(q_host, &hq) && device_view(k_new_host, &hk) && device_view(v_new_host, &hv) &&
+                      device_view(out_host, &ho) && device_view(sel_ids_host, &hi) && device_view(sel_cnt_host, &hc) &&
+                      aligned16(hq) && aligned16(hk) && aligned16(hv) && aligned16(ho) && aligned16(hi);
+  if (direct) {
+    CKV_CUDA(ckv_launch_host_in(c, hq, hk, hv, dq, dk, dv, q_bytes, kv_bytes, s));
+  } else {
+    CKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+  }
   const int r = ckv_step(c, dq, dk, dv, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, dout,
                          nullptr, dids, dcnt, stream);
   if (r != CKV_OK) return r;
-  CKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s));
-  CKV_CUDA(cudaMemcpyAsync(sel_ids_host, dids, ids_bytes, cudaMemcpyDeviceToHost, s));
-  CKV_CUDA(cudaMemcpyAsync(sel_cnt_host, dcnt, cnt_bytes, cudaMemcpyDeviceToHost, s));
+  if (direct) {
+    const bool flagged = c->host_flag != nullptr;
+    const int epoch = ++c->host_epoch;
+    CKV_CUDA(ckv_launch_host_out(c, dout, dids, dcnt, ho, hi, hc, q_bytes, ids_bytes, cnt_bytes,
+                                 flagged ? c->host_flag_dev : nullptr, epoch, s));
+    if (flagged) {
+      // wait on the word the last kernel stores (its stores to the caller's buffers precede it); if it does not
+      // show up in a long while something failed: let the stream synchronisation below report it
+      for (long long spin = 0; spin < 200000000ll; ++spin)
+        if (*c->host_flag == epoch) return CKV_OK;
+    }
+  } else {
+    CKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaMemcpyAsync(sel_ids_host, dids, ids_bytes, cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaMemcpyAsync(sel_cnt_host, dcnt, cnt_bytes, cudaMemcpyDeviceToHost, s));
+  }
   CKV_CUDA(cudaStreamSynchronize(s));
   return CKV_OK;
 }

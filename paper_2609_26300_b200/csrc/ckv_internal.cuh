@@ -53,6 +53,9 @@ struct ckv_ctx {
   int64_t launches;
   int sm_count;
   int tail_mode;   // ckv_tail_mode
+  volatile int *host_flag;   // pinned word ckv_step_host waits on (null: stream synchronisation instead)
+  int *host_flag_dev;        // the same word as the device sees it
+  int host_epoch;            // number of the last ckv_step_host call that used the word
 };
 
 cudaError_t ckv_configure_kernels();   // selection kernel attributes

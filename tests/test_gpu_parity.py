@@ -442,3 +442,30 @@ def test_decode_loop_through_host_buffer_call():
     w = small(ctx=16 * 50 + 15, decode_steps=20)
     d = setup(w)
     decode_loop(d, 20, w.budget_tokens, {0, 1, 2, 16, 17, 19}, all_units(w), use_host_call=True)
+
+
+def test_host_buffer_call_pinned_and_pageable_buffers_agree():
+    """ckv_step_host moves pinned buffers with kernels of its own and pageable ones with copies: same results."""
+    w = small(ctx=16 * 40 + 3, decode_steps=4, budget_tokens=16 * 9 + 16)   # 10 ids per unit: a 40-byte id row
+    a, b = setup(w), setup(w)
+    kcap = w.budget_tokens // w.block_size
+    for d in (a, b):
+        d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    for t in range(4):
+        k_new, v_new = synth.appended_rows(w, t)
+        q = synth.queries(w, t)
+        res = []
+        for d, pin in ((a, True), (b, False)):
+            mk = (lambda x: x.pin_memory()) if pin else (lambda x: x)
+            hq = mk(torch.from_numpy(q).to(d.dtype)); hk = mk(torch.from_numpy(k_new).to(d.dtype))
+            hv = mk(torch.from_numpy(v_new).to(d.dtype))
+            ho = mk(torch.zeros(w.batch, w.num_q_heads, 128, dtype=d.dtype))
+            hi = mk(torch.zeros(w.batch, w.num_kv_heads, kcap, dtype=torch.int32))
+            hc = mk(torch.zeros(w.batch, w.num_kv_heads, dtype=torch.int32))
+            d.ckv.step_host(hq, hk, hv, d.k_pool, d.v_pool, d.table, d.lens, d.max_len + t + 1, w.budget_tokens,
+                            ho, hi, hc)
+            res.append((ho.clone(), hi.clone(), hc.clone()))
+        for x, y in zip(*res):
+            assert torch.equal(x, y), t
+        assert int(res[0][2].min()) == kcap
+    assert a.ckv.read_status() == 0 and b.ckv.read_status() == 0
