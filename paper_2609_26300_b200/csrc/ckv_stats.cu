@@ -10,6 +10,11 @@
 
 namespace {
 
+constexpr int kBuildRounds = 8;   // blocks per warp of the build kernel
+
+// A warp takes kBuildRounds blocks, eight blocks apart, and asks the L2 for the pages of its next block before it
+// works on the current one: the block routine waits for all rows of a block at once, so without the request every
+// block would cost a full DRAM round trip with nothing else in flight for that warp.
 template <typename T>
 __global__ void __launch_bounds__(256, 3) ckv_stats_build_kernel(CkvDev P, const T *__restrict__ k_pool,
                                                               const T *__restrict__ v_pool,
@@ -20,13 +25,26 @@ __global__ void __launch_bounds__(256, 3) ckv_stats_build_kernel(CkvDev P, const
   const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
   const int N = min(seq_lens[s], P.max_blocks * P.bs);
   const int X = (N + P.bs - 1) / P.bs;
-  const int b = blockIdx.x * 8 + warp;
-  if (b >= X) return;
-  const int cnt = min(P.bs, N - b * P.bs);
-  const size_t row = (size_t)unit * P.max_blocks + b;
-  block_stats_warp<T, true>(P, k_pool, v_pool, page_table + (size_t)s * P.max_pages_per_seq, h, b, cnt,
-                            sq_smem[warp], P.kmean + row * P.row_elems, P.dbar + row * P.r,
-                            P.vmean + row * P.row_elems, lane);
+  const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
+  constexpr unsigned kPageBytes = CKV_PAGE * CKV_D * sizeof(T);
+#pragma unroll 1
+  for (int i = 0; i < kBuildRounds; ++i) {
+    const int b = (blockIdx.x * kBuildRounds + i) * 8 + warp;
+    if (b >= X) return;
+    const int bn = b + 8;
+    if (i + 1 < kBuildRounds && bn < X && lane < P.ppb && bn * P.bs + lane * CKV_PAGE < N) {
+      const int phys = pt_row[bn * P.ppb + lane];
+      if (phys >= 0 && phys < P.num_pages) {
+        const size_t off = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D;
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(k_pool + off), "r"(kPageBytes) : "memory");
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(v_pool + off), "r"(kPageBytes) : "memory");
+      }
+    }
+    const int cnt = min(P.bs, N - b * P.bs);
+    const size_t row = (size_t)unit * P.max_blocks + b;
+    block_stats_warp<T, true>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * P.row_elems,
+                              P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
+  }
 }
 
 // One CTA per sequence, one warp per KV head (looping when there are more heads than warps).
@@ -186,7 +204,7 @@ cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v
   const CkvDev &P = c->dev;
   const int xmax = (max_len + P.bs - 1) / P.bs;
   if (xmax <= 0 || batch <= 0) return cudaSuccess;
-  dim3 grid((xmax + 7) / 8, batch * P.Hkv);
+  dim3 grid((xmax + 8 * kBuildRounds - 1) / (8 * kBuildRounds), batch * P.Hkv);
   if (c->layout.kv_dtype == CKV_BF16)
     ckv_stats_build_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16 *)k_pool,
                                                                 (const __nv_bfloat16 *)v_pool, page_table, seq_lens);
