@@ -31,6 +31,9 @@ int check_layout(const ckv_layout *L) {
   if (!(L->sm_scale >= 0.f) || !isfinite(L->sm_scale)) return CKV_ERR_BAD_LAYOUT;
   if (L->variant & ~(CKV_VARIANT_FIRST_ORDER_MASS | CKV_VARIANT_RANK_BY_MASS | CKV_VARIANT_DROP)) return CKV_ERR_BAD_LAYOUT;
   if (L->stat_bf16 != 0 && L->stat_bf16 != 1) return CKV_ERR_BAD_LAYOUT;
+  // the kernels count the scan tiles (32 blocks each) of a whole step in 32 bits
+  if ((long long)L->max_batch * L->num_kv_heads * ((L->max_blocks_per_seq + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE) >= (1ll << 30))
+    return CKV_ERR_BAD_LAYOUT;
   if (L->stat_bf16 == 1 && (L->kv_dtype != CKV_BF16 || L->var_groups == CKV_D)) return CKV_ERR_BAD_LAYOUT;
   return CKV_OK;
 }

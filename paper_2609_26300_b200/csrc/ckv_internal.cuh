@@ -279,19 +279,11 @@ __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of,
   before = __reduce_add_sync(0xffffffffu, before);
   mine = __reduce_add_sync(0xffffffffu, mine);
   n_mine = __reduce_add_sync(0xffffffffu, n_mine);
-  const long long T = (long long)tot * P.Hkv;
-  const long long T0 = (long long)before * P.Hkv + (long long)h * mine;
-  int cfirst, ccount;
-  if (T < 0x40000000ll) {   // the usual case in 32-bit arithmetic: the callers have this on their critical path
-    const unsigned t = (unsigned)T, t0 = (unsigned)T0;
-    const unsigned tpc = max((t + (unsigned)scan_grid - 1u) / (unsigned)scan_grid, 1u);
-    cfirst = (int)(t0 / tpc);
-    ccount = mine == 0 ? 0 : (int)((t0 + mine - 1u) / tpc) - cfirst + 1;
-  } else {
-    const long long tpc = max((T + scan_grid - 1) / scan_grid, 1ll);
-    cfirst = (int)(T0 / tpc);
-    ccount = mine == 0 ? 0 : (int)((T0 + mine - 1) / tpc) - cfirst + 1;
-  }
+  // 32-bit arithmetic: ckv_create refuses layouts whose tiles per step would not fit (2^30)
+  const unsigned T = tot * (unsigned)P.Hkv, T0 = before * (unsigned)P.Hkv + (unsigned)h * mine;
+  const unsigned tpc = max((T + (unsigned)scan_grid - 1u) / (unsigned)scan_grid, 1u);
+  const int cfirst = (int)(T0 / tpc);
+  const int ccount = mine == 0 ? 0 : (int)((T0 + mine - 1u) / tpc) - cfirst + 1;
   first = (cfirst + 2 * unit) * CKV_SCAN_WARPS;
   count = ccount * CKV_SCAN_WARPS + ((P.tail && n_mine > 0) ? 1 : 0);
 }
