@@ -66,7 +66,9 @@ def test_sizes_follow_the_summary_layout():
                                  dict(max_batch=0), dict(num_pages=0), dict(sink_blocks=-1),
                                  dict(sm_scale=float("nan")), dict(max_blocks_per_seq=0), dict(variant=8),
                                  dict(variant=-1), dict(stat_bf16=2), dict(stat_bf16=1, kv_dtype=binding.CKV_F32),
-                                 dict(stat_bf16=1, var_groups=128)])
+                                 dict(stat_bf16=1, var_groups=128),
+                                 # more scan tiles per step than the kernels count in 32 bits
+                                 dict(max_batch=1 << 16, max_blocks_per_seq=1 << 21)])
 def test_bad_layouts_are_rejected(bad):
     with pytest.raises(binding.CompKVError) as e:
         binding.query_sizes(layout(**bad))
