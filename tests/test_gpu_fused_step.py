@@ -226,3 +226,37 @@ def test_tail_modes_agree_on_random_shapes(seed):
     for x, y in zip(a.ckv.export_stats(), b.ckv.export_stats()):
         assert torch.equal(x, y)
     assert a.ckv.read_status() == 0 and b.ckv.read_status() == 0
+
+
+def test_step_with_fewer_sequences_than_the_context_allows():
+    """A context sized for 5 sequences stepping 2 of them (the first two rows of every array): both arrangements."""
+    w5 = small(batch=5, ctx_min=16 * 20 + 1, ctx=16 * 45 + 5, decode_steps=6)
+    w2 = w5.with_(batch=2)
+    for mode in (binding.CKV_TAIL_ON, binding.CKV_TAIL_OFF):
+        big, ref = setup(w5), setup(w2)
+        # the generator keys rows by (seed, sequence, head): the two-sequence workload is the first two sequences of
+        # the five-sequence one (different pages, same contents)
+        for d in (big, ref):
+            d.ckv.set_tail_mode(mode)
+        big.ckv.stats_build(big.k_pool, big.v_pool, big.table, big.lens, big.max_len)
+        ref.ckv.stats_build(ref.k_pool, ref.v_pool, ref.table, ref.lens, ref.max_len)
+        torch.cuda.synchronize()
+        if not torch.equal(big.lens[:2], ref.lens):
+            pytest.skip("the generator does not key sequences independently of the batch size")
+        for t in range(6):
+            q5, kn5, vn5 = rows(big, t)
+            q2, kn2, vn2 = rows(ref, t)
+            assert torch.equal(q5[:2], q2)
+            ob, lb, ib, cb = big.ckv.step(q5[:2].contiguous(), kn5[:2].contiguous(), vn5[:2].contiguous(), big.k_pool,
+                                          big.v_pool, big.table, big.lens, big.max_len + t + 1, w5.budget_tokens)
+            orf, lr, ir, cr = ref.ckv.step(q2, kn2, vn2, ref.k_pool, ref.v_pool, ref.table, ref.lens,
+                                           ref.max_len + t + 1, w2.budget_tokens)
+            torch.cuda.synchronize()
+            assert torch.equal(big.lens[:2], ref.lens) and int(big.lens[2]) == int(setup_len(w5, 2))
+            assert torch.equal(ib, ir) and torch.equal(cb, cr)
+            assert torch.equal(ob, orf) and torch.equal(lb, lr)
+        assert big.ckv.read_status() == 0 and ref.ckv.read_status() == 0
+
+
+def setup_len(w, s):
+    return int(synth.seq_lens(w)[s])
