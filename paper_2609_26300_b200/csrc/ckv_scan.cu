@@ -285,40 +285,41 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   // never arbitrary bit patterns (a NaN times a zero weight would poison the accumulators)
   for (int i = tid; i < stages * stage_bytes / 16; i += kThreads) reinterpret_cast<uint4 *>(stage_mem)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async();
+  if (tid == 0) {   // also done while the lengths are on their way: the barriers of the ring
+    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], kConsumerWarps); }
+    fence_barrier_init();
+  }
   if (tid < batch) s_len[tid] = eff_len(len_mine);
   for (int i = tid + kThreads; i < batch && i < kMaxSeqs; i += kThreads) s_len[i] = eff_len(seq_lens[i]);
   __syncthreads();
   if (tid == 0) {
-    long long T = 0;
-    for (int i = 0; i < batch; ++i) T += (long long)seq_tiles(s_len, seq_lens, P, i) * P.Hkv;
-    const long long tpc = (T + nscan - 1) / nscan;
-    const long long first = (long long)bid * tpc;
-    long long cnt = T - first;
-    if (cnt > tpc) cnt = tpc;
-    if (cnt < 0) cnt = 0;
+    // this CTA's range of the tiles (32-bit arithmetic: a step has fewer than 2^30 tiles, checked at creation)
+    unsigned T = 0;
+    for (int i = 0; i < batch; ++i) T += (unsigned)seq_tiles(s_len, seq_lens, P, i) * (unsigned)P.Hkv;
+    const unsigned tpc = (T + (unsigned)nscan - 1u) / (unsigned)nscan;
+    const unsigned first = (unsigned)bid * tpc;
+    const unsigned cnt = first >= T ? 0u : min(T - first, tpc);
     int u0 = 0, tl0 = 0, ulast = 0;
     if (cnt > 0) {
-      long long accum = 0;
+      unsigned accum = 0;
       bool have_first = false;
       for (int i = 0; i < batch; ++i) {
-        const long long t = seq_tiles(s_len, seq_lens, P, i);
+        const unsigned t = (unsigned)seq_tiles(s_len, seq_lens, P, i);
         if (t > 0) {
-          if (!have_first && first < accum + t * P.Hkv) {
-            const long long off = first - accum;
+          if (!have_first && first < accum + t * (unsigned)P.Hkv) {
+            const unsigned off = first - accum;
             u0 = i * P.Hkv + (int)(off / t); tl0 = (int)(off % t);
             have_first = true;
           }
-          if (first + cnt - 1 < accum + t * P.Hkv) {
-            ulast = i * P.Hkv + (int)((first + cnt - 1 - accum) / t);
+          if (first + cnt - 1u < accum + t * (unsigned)P.Hkv) {
+            ulast = i * P.Hkv + (int)((first + cnt - 1u - accum) / t);
             break;
           }
         }
-        accum += t * P.Hkv;
+        accum += t * (unsigned)P.Hkv;
       }
     }
     s_u0 = u0; s_tl0 = tl0; s_ulast = ulast; s_count = (int)cnt; s_abort = 0; s_issued = 0;
-    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], kConsumerWarps); }
-    fence_barrier_init();
   }
   __syncthreads();
   const int count = s_count;
