@@ -253,8 +253,11 @@ int ckv_copy_scores(ckv_ctx *ctx, float *dst, int batch, ckv_stream stream);
  * (all work the call put on the stream has then finished).  Host buffers should be pinned: buffers the
  * device can address (pinned, registered or managed memory, 16-byte aligned) are moved by two small
  * kernels of the library and the call waits on a pinned word its last kernel stores; pageable buffers
- * take six copies and a stream synchronisation (about 20 us more per call).  Device staging comes out of
- * the workspace.  seq_lens (device) is incremented.  max_seq_len_host bounds the lengths AFTER the append.  The id staging area holds
+ * take six copies and a stream synchronisation (about 20 us more per call).  A caller that comes back with the
+ * same buffers, arrays and sizes on a stream of its own (not the default stream, not a capturing one) has its
+ * second such call captured as a CUDA graph and the later ones replayed (the length bound is rounded up to a
+ * multiple of 1024 inside, so the graph lasts that many steps); the graph is the context's and goes with it.
+ * Device staging comes out of the workspace.  seq_lens (device) is incremented.  max_seq_len_host bounds the lengths AFTER the append.  The id staging area holds
  * max_blocks_per_seq ids per unit: budget_tokens / block_size beyond that is CKV_ERR_INVALID_ARG. */
 int ckv_step_host(ckv_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
                   void *k_pool, void *v_pool, const int32_t *page_table, int32_t *seq_lens, int batch,

@@ -190,6 +190,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
 }
 
 void ckv_destroy(ckv_ctx *ctx) {
+  if (ctx != nullptr && ctx->hg_exec != nullptr) cudaGraphExecDestroy((cudaGraphExec_t)ctx->hg_exec);
   if (ctx != nullptr && ctx->host_flag != nullptr) cudaFreeHost((void *)ctx->host_flag);
   delete ctx;
 }
@@ -244,13 +245,14 @@ bool device_view(const void *host, void **dev) {
   return true;
 }
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+constexpr int kHostEpochWord = 20;   // word of the status region that counts the ckv_step_host calls completed on the device
 
 // three source ranges to three destination ranges, 16 bytes per thread and iteration (sizes are multiples of 16)
 __global__ void __launch_bounds__(1024) ckv_move3_kernel(const uint4 *__restrict__ a, uint4 *__restrict__ da, int na,
                                                         const uint4 *__restrict__ b, uint4 *__restrict__ db, int nb,
                                                         const uint4 *__restrict__ c, uint4 *__restrict__ dc, int nc,
                                                         const int *__restrict__ tail_src, int *__restrict__ tail_dst,
-                                                        int n_tail, int *done_flag, int done_value) {
+                                                        int n_tail, int *done_flag, int *done_count) {
   const int stride = gridDim.x * blockDim.x;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < na + nb + nc; i += stride) {
     if (i < na) da[i] = a[i];
@@ -261,7 +263,8 @@ __global__ void __launch_bounds__(1024) ckv_move3_kernel(const uint4 *__restrict
   if (done_flag != nullptr) {   // single-CTA launches only: everything above is in host memory before the word is
     __threadfence_system();
     __syncthreads();
-    if (threadIdx.x == 0) { *(volatile int *)done_flag = done_value; __threadfence_system(); }
+    // the call's number is counted on the device, so that a captured launch can be replayed
+    if (threadIdx.x == 0) { const int e = *done_count + 1; *done_count = e; *(volatile int *)done_flag = e; __threadfence_system(); }
   }
 }
 
@@ -270,23 +273,23 @@ cudaError_t ckv_launch_host_in(ckv_ctx *c, const void *hq, const void *hk, const
   const int nq = (int)(q_bytes / 16), nkv = (int)(kv_bytes / 16);
   const int grid = std::max(1, std::min((nq + 2 * nkv + 255) / 256, 64));
   ckv_move3_kernel<<<grid, 256, 0, s>>>((const uint4 *)hq, (uint4 *)dq, nq, (const uint4 *)hk, (uint4 *)dk, nkv,
-                                        (const uint4 *)hv, (uint4 *)dv, nkv, nullptr, nullptr, 0, nullptr, 0);
+                                        (const uint4 *)hv, (uint4 *)dv, nkv, nullptr, nullptr, 0, nullptr, nullptr);
   c->launches++;
   return cudaGetLastError();
 }
 
 cudaError_t ckv_launch_host_out(ckv_ctx *c, const void *dout, const int32_t *dids, const int32_t *dcnt, void *ho, void *hi,
                                 void *hc, size_t out_bytes, size_t ids_bytes, size_t cnt_bytes, int *done_flag,
-                                int done_value, cudaStream_t s) {
+                                int *done_count, cudaStream_t s) {
   // out rows are multiples of 16 bytes; the id array is moved in 16-byte pieces with a 4-byte remainder; the counts
   // (one int per unit) go as the 4-byte tail of the same launch.  One CTA: a few tens of KB, and the completion
   // word must follow every store of the launch.
   const int no = (int)(out_bytes / 16), ni = (int)(ids_bytes / 16);
   if (ids_bytes % 16 != 0)   // at most three ids
     ckv_move3_kernel<<<1, 32, 0, s>>>(nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr, 0,
-                                      dids + ni * 4, (int *)hi + ni * 4, (int)((ids_bytes % 16) / 4), nullptr, 0);
+                                      dids + ni * 4, (int *)hi + ni * 4, (int)((ids_bytes % 16) / 4), nullptr, nullptr);
   ckv_move3_kernel<<<1, 1024, 0, s>>>((const uint4 *)dout, (uint4 *)ho, no, (const uint4 *)dids, (uint4 *)hi, ni,
-                                      nullptr, nullptr, 0, dcnt, (int *)hc, (int)(cnt_bytes / 4), done_flag, done_value);
+                                      nullptr, nullptr, 0, dcnt, (int *)hc, (int)(cnt_bytes / 4), done_flag, done_count);
   c->launches++;
   return cudaGetLastError();
 }
@@ -459,32 +462,84 @@ int ckv_step_host(ckv_ctx *c, const void *q_host, const void *k_new_host, const 
   const bool direct = device_view(q_host, &hq) && device_view(k_new_host, &hk) && device_view(v_new_host, &hv) &&
                       device_view(out_host, &ho) && device_view(sel_ids_host, &hi) && device_view(sel_cnt_host, &hc) &&
                       aligned16(hq) && aligned16(hk) && aligned16(hv) && aligned16(ho) && aligned16(hi);
-  if (direct) {
-    CKV_CUDA(ckv_launch_host_in(c, hq, hk, hv, dq, dk, dv, q_bytes, kv_bytes, s));
-  } else {
-    CKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
-    CKV_CUDA(cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
-    CKV_CUDA(cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
-  }
-  const int r = ckv_step(c, dq, dk, dv, k_pool, v_pool, page_table, seq_lens, batch, max_seq_len_host, budget_tokens, dout,
-                         nullptr, dids, dcnt, stream);
-  if (r != CKV_OK) return r;
-  if (direct) {
-    const bool flagged = c->host_flag != nullptr;
-    const int epoch = ++c->host_epoch;
-    CKV_CUDA(ckv_launch_host_out(c, dout, dids, dcnt, ho, hi, hc, q_bytes, ids_bytes, cnt_bytes,
-                                 flagged ? c->host_flag_dev : nullptr, epoch, s));
-    if (flagged) {
-      // wait on the word the last kernel stores (its stores to the caller's buffers precede it); if it does not
-      // show up in a long while something failed: let the stream synchronisation below report it
-      for (long long spin = 0; spin < 200000000ll; ++spin)
-        if (*c->host_flag == epoch) return CKV_OK;
+  const bool flagged = direct && c->host_flag != nullptr;
+  int *done_count = c->dev.status + kHostEpochWord;
+  // the three parts of the call as launches on `on`: inputs in, the step, results out (+ completion word)
+  auto enqueue = [&](cudaStream_t on, int max_len) -> int {
+    if (direct) {
+      CKV_CUDA(ckv_launch_host_in(c, hq, hk, hv, dq, dk, dv, q_bytes, kv_bytes, on));
+    } else {
+      CKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, on));
+      CKV_CUDA(cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, on));
+      CKV_CUDA(cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, on));
     }
-  } else {
-    CKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s));
-    CKV_CUDA(cudaMemcpyAsync(sel_ids_host, dids, ids_bytes, cudaMemcpyDeviceToHost, s));
-    CKV_CUDA(cudaMemcpyAsync(sel_cnt_host, dcnt, cnt_bytes, cudaMemcpyDeviceToHost, s));
+    const int r = ckv_step(c, dq, dk, dv, k_pool, v_pool, page_table, seq_lens, batch, max_len, budget_tokens, dout, nullptr,
+                           dids, dcnt, (ckv_stream)on);
+    if (r != CKV_OK) return r;
+    if (direct) {
+      CKV_CUDA(ckv_launch_host_out(c, dout, dids, dcnt, ho, hi, hc, q_bytes, ids_bytes, cnt_bytes,
+                                   flagged ? c->host_flag_dev : nullptr, done_count, on));
+    } else {
+      CKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, on));
+      CKV_CUDA(cudaMemcpyAsync(sel_ids_host, dids, ids_bytes, cudaMemcpyDeviceToHost, on));
+      CKV_CUDA(cudaMemcpyAsync(sel_cnt_host, dcnt, cnt_bytes, cudaMemcpyDeviceToHost, on));
+    }
+    return CKV_OK;
+  };
+  // wait on the word the last kernel stores (its stores to the caller's buffers precede it); if it does not show
+  // up in a long while something failed: the stream synchronisation reports it
+  auto wait_done = [&]() -> int {
+    const int epoch = ++c->host_epoch;
+    for (long long spin = 0; spin < 200000000ll; ++spin)
+      if (*c->host_flag == epoch) return CKV_OK;
+    CKV_CUDA(cudaStreamSynchronize(s));
+    c->host_epoch = *c->host_flag;
+    return CKV_OK;
+  };
+
+  // A caller that comes back with the same buffers and sizes (a decode loop) gets its second call captured as a
+  // CUDA graph and every later one replayed: one driver call instead of five launches.  The length bound is part
+  // of the captured launches, so it is rounded up (it only has to be an upper bound) and the graph lasts 1024 steps.
+  cudaStreamCaptureStatus cap_state = cudaStreamCaptureStatusActive;
+  const bool own_stream = s != nullptr && s != cudaStreamLegacy && s != cudaStreamPerThread &&
+                          cudaStreamIsCapturing(s, &cap_state) == cudaSuccess && cap_state == cudaStreamCaptureStatusNone;
+  if (flagged && own_stream && !c->hg_disabled) {
+    const int cap_tokens = L.max_blocks_per_seq * L.block_size;
+    const int len_r = std::min((max_seq_len_host + 1023) / 1024 * 1024, cap_tokens);
+    const void *key[10] = {q_host, k_new_host, v_new_host, out_host, sel_ids_host, sel_cnt_host, k_pool, v_pool, page_table, seq_lens};
+    const int ints[4] = {batch, len_r, budget_tokens, c->tail_mode};
+    const bool same = c->hg_key_valid && memcmp(key, c->hg_key, sizeof(key)) == 0 && memcmp(ints, c->hg_ints, sizeof(ints)) == 0;
+    if (same && c->hg_exec == nullptr) {   // second call in a row with this key: capture it
+      const int64_t before = c->launches;
+      cudaGraph_t graph = nullptr;
+      cudaGraphExec_t exec = nullptr;
+      bool ok = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+      if (ok) {
+        ok = enqueue(s, len_r) == CKV_OK;
+        ok = (cudaStreamEndCapture(s, &graph) == cudaSuccess) && ok && graph != nullptr;
+      }
+      if (ok) ok = cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess;
+      if (graph != nullptr) cudaGraphDestroy(graph);
+      c->hg_launches = (int)(c->launches - before);
+      c->launches = before;
+      if (ok) c->hg_exec = exec;
+      else { (void)cudaGetLastError(); c->hg_disabled = true; }
+    }
+    if (same && c->hg_exec != nullptr) {
+      CKV_CUDA(cudaGraphLaunch((cudaGraphExec_t)c->hg_exec, s));
+      c->launches += c->hg_launches;
+      return wait_done();
+    }
+    if (!same) {   // a new key: remember it, drop the graph of the old one
+      if (c->hg_exec != nullptr) { cudaGraphExecDestroy((cudaGraphExec_t)c->hg_exec); c->hg_exec = nullptr; }
+      memcpy(c->hg_key, key, sizeof(key));
+      memcpy(c->hg_ints, ints, sizeof(ints));
+      c->hg_key_valid = true;
+    }
   }
+  const int r = enqueue(s, max_seq_len_host);
+  if (r != CKV_OK) return r;
+  if (flagged) return wait_done();
   CKV_CUDA(cudaStreamSynchronize(s));
   return CKV_OK;
 }

@@ -56,6 +56,12 @@ struct ckv_ctx {
   volatile int *host_flag;   // pinned word ckv_step_host waits on (null: stream synchronisation instead)
   int *host_flag_dev;        // the same word as the device sees it
   int host_epoch;            // number of the last ckv_step_host call that used the word
+  // ckv_step_host replays a captured graph when it is called again with the same buffers and sizes
+  void *hg_exec;             // cudaGraphExec_t, or null
+  const void *hg_key[10];    // the six host buffers, pools, page table, lengths array
+  int hg_ints[4];            // batch, rounded length bound, budget, tail mode
+  int hg_launches;           // kernel launches one replay stands for
+  bool hg_key_valid, hg_disabled;
 };
 
 cudaError_t ckv_configure_kernels();   // selection kernel attributes

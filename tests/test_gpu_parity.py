@@ -444,6 +444,39 @@ def test_decode_loop_through_host_buffer_call():
     decode_loop(d, 20, w.budget_tokens, {0, 1, 2, 16, 17, 19}, all_units(w), use_host_call=True)
 
 
+def test_host_buffer_call_replayed_from_fixed_buffers():
+    """A decode loop that reuses its pinned buffers on a stream of its own: ckv_step_host captures its second call
+    and replays it afterwards (the length bound is rounded up inside); results equal ckv_step's, step by step."""
+    w = small(ctx=16 * 40 + 3, decode_steps=24)
+    a, b = setup(w), setup(w)
+    kcap = w.budget_tokens // w.block_size
+    for d in (a, b):
+        d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    hq = torch.zeros(w.batch, w.num_q_heads, 128, dtype=a.dtype).pin_memory()
+    hk = torch.zeros(w.batch, w.num_kv_heads, 128, dtype=a.dtype).pin_memory()
+    hv = torch.zeros_like(hk).pin_memory()
+    ho = torch.zeros_like(hq).pin_memory()
+    hi = torch.zeros(w.batch, w.num_kv_heads, kcap, dtype=torch.int32).pin_memory()
+    hc = torch.zeros(w.batch, w.num_kv_heads, dtype=torch.int32).pin_memory()
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    n_before = a.ckv.launch_count()
+    for t in range(24):
+        k_new, v_new = synth.appended_rows(w, t)
+        q = synth.queries(w, t)
+        hq.copy_(torch.from_numpy(q).to(a.dtype)); hk.copy_(torch.from_numpy(k_new).to(a.dtype))
+        hv.copy_(torch.from_numpy(v_new).to(a.dtype))
+        with torch.cuda.stream(side):
+            a.ckv.step_host(hq, hk, hv, a.k_pool, a.v_pool, a.table, a.lens, a.max_len + t + 1, w.budget_tokens, ho, hi, hc)
+        ob, lb, ib, cb = b.ckv.step(hq.cuda(), hk.cuda(), hv.cuda(), b.k_pool, b.v_pool, b.table, b.lens,
+                                    b.max_len + t + 1, w.budget_tokens)
+        torch.cuda.synchronize()
+        assert torch.equal(ho, ob.cpu()) and torch.equal(hi, ib.cpu()) and torch.equal(hc, cb.cpu()), t
+        assert torch.equal(a.lens, b.lens), t
+    assert a.ckv.launch_count() - n_before == 24 * 6   # in, append, scan, select, attention, out: replays count too
+    assert a.ckv.read_status() == 0 and b.ckv.read_status() == 0
+
+
 def test_host_buffer_call_pinned_and_pageable_buffers_agree():
     """ckv_step_host moves pinned buffers with kernels of its own and pageable ones with copies: same results."""
     w = small(ctx=16 * 40 + 3, decode_steps=4, budget_tokens=16 * 9 + 16)   # 10 ids per unit: a 40-byte id row
