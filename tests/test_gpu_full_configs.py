@@ -118,3 +118,24 @@ def test_config2_other_layouts(kw, ck):
         assert d.ckv.read_status() == 0
         for h in (1, 6):
             check_unit_decode(d, 0, h, w.ctx + t + 1, t, w.budget_tokens, out, lse, ids, cnt, scores, **ck)
+
+
+@pytest.mark.parametrize("cfg", [2, 3])
+def test_results_are_a_pure_function_of_the_inputs(cfg):
+    """The same decode twice, and the same dense decode twice, on a full-size cache (148 scan CTAs, clusters of
+    eight splits, counter-based merges): every output bit, id and score repeats."""
+    w = synth.CONFIGS[cfg]
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    q = dev_q(d)
+    runs = []
+    for _ in range(3):
+        out, lse, ids, cnt = d.ckv.decode(q, d.k_pool, d.v_pool, d.table, d.lens, d.max_len, w.budget_tokens)
+        scores = d.ckv.copy_scores(w.batch)
+        dout, dlse = d.ckv.dense_decode(q, d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+        torch.cuda.synchronize()
+        runs.append([t.clone() for t in (out, lse, ids, cnt, scores, dout, dlse)])
+    for r in runs[1:]:
+        for x, y in zip(runs[0], r):
+            assert torch.equal(x, y)
+    assert d.ckv.read_status() == 0
