@@ -407,6 +407,15 @@ def test_fused_step_loop(bs, r):
     decode_loop(d, 36, w.budget_tokens, set(range(36)), all_units(w), fused=True, var_groups=r)
 
 
+def test_fused_step_custom_scale_group_layout_and_mandatory_counts():
+    """Tail mode with a logit scale of the caller's, contiguous coordinate groups, two sink and three recent blocks:
+    the last block's terms come from the tail warps' own arithmetic and must follow the same layout switches."""
+    w = small(ctx_min=16 * 25 + 3, ctx=16 * 50 + 9, decode_steps=18)
+    d = setup(w, sink=2, recent=3, sm_scale=0.05, group_layout=0, var_groups=8)
+    decode_loop(d, 18, w.budget_tokens, set(range(18)), all_units(w), fused=True, sink=2, recent=3, scale=0.05,
+                group_layout=0, var_groups=8)
+
+
 @pytest.mark.parametrize("hq,hkv", [(2, 2), (16, 2)])   # G = 1 and 8
 def test_fused_step_group_sizes(hq, hkv):
     w = small(ctx=16 * 40 + 9, decode_steps=20, num_q_heads=hq, num_kv_heads=hkv)
