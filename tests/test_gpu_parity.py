@@ -399,7 +399,7 @@ def test_decode_loop_two_calls_in_tail_mode():
     decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), tail_on=True)
 
 
-@pytest.mark.parametrize("bs,r", [(16, 4), (32, 4), (64, 4), (16, 128), (16, 8)])
+@pytest.mark.parametrize("bs,r", [(16, 4), (32, 4), (64, 4), (16, 128), (16, 8), (16, 64), (16, 1), (32, 32)])
 def test_fused_step_loop(bs, r):
     """ckv_step over block roll-overs, one-token blocks and ragged lengths: every unit, every step."""
     w = small(ctx_min=16 * 30 + 1, ctx=16 * 60, decode_steps=36, block_size=bs, budget_tokens=bs * 7)
