@@ -122,6 +122,20 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
     }
   }
   if (!done) {
+    if constexpr (!NC) {
+      // A block of several pages (32- or 64-token blocks) is read page after page, twice: when the caller works on
+      // one block only (the append, the chunked prefill) the L2 is asked for all of its pages first, so that only
+      // the first page costs a DRAM round trip.  (The build kernel asks for its next block itself.)
+      if (npages > 1 && lane < npages) {
+        const int phys = pt_row[b * P.ppb + lane];
+        if (phys >= 0 && phys < P.num_pages) {
+          const size_t off = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D;
+          const unsigned bytes = CKV_PAGE * CKV_D * sizeof(T);
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(k_pool + off), "r"(bytes) : "memory");
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(v_pool + off), "r"(bytes) : "memory");
+        }
+      }
+    }
     for (int pg = 0; pg < npages; ++pg) {
       const int phys = pt_row[b * P.ppb + pg];
       if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
