@@ -139,3 +139,29 @@ def test_results_are_a_pure_function_of_the_inputs(cfg):
         for x, y in zip(runs[0], r):
             assert torch.equal(x, y)
     assert d.ckv.read_status() == 0
+
+
+def test_config4_qwen_steps_in_tail_mode():
+    """The ragged 16-sequence, group-of-8 configuration stepped with ckv_step: at this size the library runs the
+    append inside the scan launch (16 tail CTAs, 128 units), clusters of two attention splits per unit."""
+    w = synth.CONFIGS[4].with_(decode_steps=6)
+    d = setup(w)
+    lens0 = d.lens.cpu().numpy().copy()
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    sample = [(int(lens0.argmin()), 1), (int(lens0.argmax()), 6), (7, 3)]
+    for t in range(6):
+        k_new, v_new = synth.appended_rows(w, t)
+        n_before = d.ckv.launch_count()
+        out, lse, ids, cnt = d.ckv.step(torch.from_numpy(synth.queries(w, t)).bfloat16().cuda(),
+                                        torch.from_numpy(k_new).bfloat16().cuda(),
+                                        torch.from_numpy(v_new).bfloat16().cuda(), d.k_pool, d.v_pool, d.table,
+                                        d.lens, d.max_len + t + 1, w.budget_tokens)
+        assert d.ckv.launch_count() - n_before == 3
+        if t in (0, 5):
+            scores = d.ckv.copy_scores(w.batch)
+            torch.cuda.synchronize()
+            for s, h in sample:
+                check_unit_decode(d, s, h, int(lens0[s]) + t + 1, t, w.budget_tokens, out, lse, ids, cnt, scores)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() == 0
+    assert np.array_equal(d.lens.cpu().numpy(), lens0 + 6)
