@@ -280,6 +280,17 @@ int64_t ckv_launch_count(const ckv_ctx *ctx);
 enum ckv_tail_mode { CKV_TAIL_AUTO = 0, CKV_TAIL_OFF = 1, CKV_TAIL_ON = 2 };
 int ckv_set_tail_mode(ckv_ctx *ctx, int mode);
 
+/* ---- test hook ------------------------------------------------------------------------------------------------
+ * Every wait inside a kernel is bounded: after a number of polls it gives up, sets CKV_DEV_TIMEOUT, drains the
+ * copies it has in flight and the launch returns -- nothing traps and nothing waits for ever.  ckv_debug_set() lets
+ * a test make that happen without a fault: spin_limit replaces the number of polls (0 restores the default, 2^22),
+ * and CKV_DEBUG_SKIP_FILL makes the producer thread of the summary scan's first CTA announce its first
+ * shared-memory fill and never issue it, so that the waits on it run out.  The decode step that follows reports
+ * CKV_DEV_TIMEOUT through ckv_read_status() and its results are invalid; with the flag cleared the next step is
+ * correct again.  The paper has no counterpart.  Not for production use. */
+enum ckv_debug_flags { CKV_DEBUG_SKIP_FILL = 1 };
+int ckv_debug_set(ckv_ctx *ctx, uint32_t spin_limit, int flags);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,13 +21,14 @@ CKV_TAIL_AUTO, CKV_TAIL_OFF, CKV_TAIL_ON = 0, 1, 2
 CKV_OK = 0
 CKV_ERR_INVALID_ARG, CKV_ERR_BAD_LAYOUT, CKV_ERR_BUDGET_TOO_SMALL = -1, -2, -3
 CKV_ERR_CAPACITY, CKV_ERR_CUDA, CKV_ERR_TIMEOUT = -4, -5, -6
+CKV_DEBUG_SKIP_FILL = 1
 CKV_DEV_BAD_PAGE, CKV_DEV_SEQ_FULL, CKV_DEV_NONFINITE, CKV_DEV_TIMEOUT, CKV_DEV_BAD_COPY = 1, 2, 4, 8, 16
 
 EXPORTS = ["ckv_version", "ckv_strerror", "ckv_last_cuda_error", "ckv_query_sizes", "ckv_stats_offsets",
            "ckv_create", "ckv_destroy", "ckv_stats_build", "ckv_stats_export", "ckv_append", "ckv_prefill", "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode",
            "ckv_dense_decode_static",
            "ckv_exact_blocks", "ckv_copy_scores", "ckv_step_host", "ckv_read_status", "ckv_launch_count",
-           "ckv_set_tail_mode"]
+           "ckv_set_tail_mode", "ckv_debug_set"]
 
 
 class ckv_layout(ctypes.Structure):
@@ -94,6 +95,8 @@ def load() -> ctypes.CDLL:
     lib.ckv_launch_count.restype = ctypes.c_int64
     lib.ckv_set_tail_mode.argtypes = [vp, ctypes.c_int]
     lib.ckv_set_tail_mode.restype = ctypes.c_int
+    lib.ckv_debug_set.argtypes = [vp, ctypes.c_uint32, ctypes.c_int]
+    lib.ckv_debug_set.restype = ctypes.c_int
     for name in ("ckv_query_sizes", "ckv_stats_offsets", "ckv_create", "ckv_stats_build", "ckv_stats_export", "ckv_append",
                  "ckv_decode", "ckv_step", "ckv_decode_profile", "ckv_scan_profile", "ckv_dense_decode", "ckv_copy_scores", "ckv_step_host", "ckv_read_status"):
         getattr(lib, name).restype = i32
@@ -307,3 +310,7 @@ class CompKV:
     def set_tail_mode(self, mode: int) -> None:
         """ckv_set_tail_mode: CKV_TAIL_AUTO (default), CKV_TAIL_OFF, CKV_TAIL_ON."""
         _check(self.lib.ckv_set_tail_mode(self._ctx, int(mode)), "ckv_set_tail_mode")
+
+    def debug_set(self, spin_limit: int = 0, flags: int = 0) -> None:
+        """ckv_debug_set (test hook): polls a bounded device-side wait makes (0 = default), CKV_DEBUG_* flags."""
+        _check(self.lib.ckv_debug_set(self._ctx, int(spin_limit), int(flags)), "ckv_debug_set")

@@ -6,6 +6,7 @@
 #include <algorithm>
 
 #include "ckv_internal.cuh"
+#include "ckv_pipe.cuh"
 
 namespace {
 
@@ -160,6 +161,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.status = (int *)(wb + R.status); P.unit_done = (int *)(wb + R.done);
   P.lu = (float *)(wb + R.ls); P.lz = (float *)(wb + R.lz); P.scores = (float *)(wb + R.scores);
   P.comp_part = (float *)(wb + R.comp); P.attn_part = (float *)(wb + R.attn);
+  P.spin_limit = ckv_pipe::kSpinLimit; P.debug = 0;
   c->work = wb; c->work_bytes = work_bytes;
   c->stage_q = R.stage_q; c->stage_knew = R.stage_knew; c->stage_vnew = R.stage_vnew;
   c->stage_out = R.stage_out; c->stage_ids = R.stage_ids; c->stage_cnt = R.stage_cnt;
@@ -554,6 +556,13 @@ int ckv_read_status(ckv_ctx *c, int32_t *host_status, ckv_stream stream) {
 }
 
 int64_t ckv_launch_count(const ckv_ctx *c) { return c == nullptr ? 0 : c->launches; }
+
+int ckv_debug_set(ckv_ctx *c, uint32_t spin_limit, int flags) {
+  if (c == nullptr || (flags & ~CKV_DEBUG_SKIP_FILL) != 0) return CKV_ERR_INVALID_ARG;
+  c->dev.spin_limit = spin_limit == 0 ? ckv_pipe::kSpinLimit : spin_limit;
+  c->dev.debug = flags;
+  return CKV_OK;
+}
 
 int ckv_set_tail_mode(ckv_ctx *c, int mode) {
   if (c == nullptr || mode < CKV_TAIL_AUTO || mode > CKV_TAIL_ON) return CKV_ERR_INVALID_ARG;

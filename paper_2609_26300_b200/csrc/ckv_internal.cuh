@@ -41,6 +41,8 @@ struct CkvDev {
   int tail;          // 1: the scan launch leaves the last block of every sequence to its tail CTAs (set per step)
   int *unit_done;    // [unit] attention splits finished this step (zero between steps); null = merge is a separate launch
   int *status;       // device status word
+  uint32_t spin_limit;  // polls a bounded wait makes before it gives up (ckv_debug_set; default ckv_pipe::kSpinLimit)
+  int debug;         // ckv_debug_flags (test hooks; 0 in normal use)
 };
 
 struct ckv_ctx {

@@ -1,7 +1,8 @@
 // mbarrier and bulk-copy (TMA, untiled) primitives for shared-memory pipelines on sm_100a.
 //
-// Every wait is bounded: after kSpinLimit failed polls the wait gives up and returns false, and
-// the caller records CKV_DEV_TIMEOUT and drains its outstanding copies before leaving.
+// Every wait is bounded: after `limit` failed polls (kSpinLimit unless the context was given another value through
+// ckv_debug_set) the wait gives up and returns false, and the caller records CKV_DEV_TIMEOUT and drains its
+// outstanding copies before leaving.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -38,8 +39,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait for the phase with the given parity to complete.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t limit = kSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }

@@ -260,8 +260,9 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   __shared__ int s_len[kMaxSeqs];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool dbar_bulk = P.r >= 4;   // smaller rows cannot keep the 16-byte alignment bulk copies need
   const bool r4 = P.r == 4;          // the default: the variance projection is four FMAs on one 16-byte read
+  const bool dbar_bulk = P.r >= 4;   // smaller rows cannot keep the 16-byte alignment bulk copies need
+  constexpr int kParts = TB / 16;    // 16-block parts of a tile, each worked on by one consumer warp
   const int stage_bytes = TB * 2 * kRowBytes + (dbar_bulk ? TB * P.r * 4 : 0);
   // per-warp w_{g,t} table for r != 4, behind the ring
   float *sw_all = reinterpret_cast<float *>(stage_mem + (size_t)stages * stage_bytes);
@@ -338,7 +339,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
       uint32_t phase = 0;            // parity of the empty-barrier phase the next refill of stage `st` waits for
       UnitInfo ui = unit_info(P, s_len, seq_lens, u);
       for (int it = 0; it < count; ++it) {
-        if (it >= stages && !mbar_wait(&empty_bar[st], phase)) {
+        if (it >= stages && !mbar_wait(&empty_bar[st], phase, P.spin_limit)) {
           atomicOr(P.status, CKV_DEV_TIMEOUT);
           *(volatile int *)&s_abort = 1;
         }
@@ -353,11 +354,15 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
         const uint32_t lo = smem_u32(stage_mem), hi = lo + (uint32_t)stages * stage_bytes;
         bool ok = nb >= 1 && u < units && row + nb <= (size_t)units * P.max_blocks;
-        ok = ok && bulk_g2s_checked(sk, P.kmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
-        ok = ok && bulk_g2s_checked(sv, P.vmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
-        if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, &full_bar[st], lo, hi);
+        // test hook (ckv_debug_set): one fill is announced but never issued, so that the waits on it run out
+        const bool skip = (P.debug & CKV_DEBUG_SKIP_FILL) != 0 && it == 0 && bid == 0;
+        if (!skip) {
+          ok = ok && bulk_g2s_checked(sk, P.kmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
+          ok = ok && bulk_g2s_checked(sv, P.vmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
+          if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, &full_bar[st], lo, hi);
+          *(volatile int *)&s_issued = it + 1;
+        }
         if (!ok) atomicOr(P.status, CKV_DEV_BAD_COPY);
-        *(volatile int *)&s_issued = it + 1;
         if (++st == stages) { st = 0; if (it >= stages) phase ^= 1; }
         if (++tl == ui.tiles) {
           tl = 0;
@@ -427,12 +432,13 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         tl = 0;
         do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
       }
-      const int j0 = (2 * it) % kConsumerWarps;
-      const int half = j0 == warp ? 0 : ((j0 + 1) % kConsumerWarps == warp ? 1 : -1);
+      // part p of tile `it` belongs to warp (kParts * it + p) % W
+      int half = (warp - (kParts * it) % kConsumerWarps + kConsumerWarps) % kConsumerWarps;
+      if (half >= kParts) half = -1;
       // a wait that runs out marks the step invalid (`aborted`); the walk still runs to the end
       if (!aborted) {
         bool fail = *(volatile int *)&s_abort != 0;
-        if (!fail && !mbar_wait(&full_bar[st], phase)) {
+        if (!fail && !mbar_wait(&full_bar[st], phase, P.spin_limit)) {
           atomicOr(P.status, CKV_DEV_TIMEOUT);
           *(volatile int *)&s_abort = 1;
           fail = true;
@@ -671,7 +677,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     // leave no bulk copy in flight into this CTA's shared memory: wait (bounded) for every issued fill
     // (a completed phase is seen as complete again, so waiting on consumed stages returns at once)
     const int issued = s_issued;
-    for (int it = max(issued - stages, 0); it < issued; ++it) mbar_wait(&full_bar[it % stages], (it / stages) & 1);
+    for (int it = max(issued - stages, 0); it < issued; ++it) mbar_wait(&full_bar[it % stages], (it / stages) & 1, P.spin_limit);
   }
 }
 

@@ -100,6 +100,7 @@ def test_null_arguments_are_rejected_before_any_cuda_call():
     assert lib.ckv_exact_blocks(None, None, None, None, None, 1, 16, None, None, None, None) == bad
     assert lib.ckv_scan_profile(None, None, None, 1, 16, 1, None, None) == bad
     assert lib.ckv_set_tail_mode(None, binding.CKV_TAIL_ON) == bad
+    assert lib.ckv_debug_set(None, 0, 0) == bad
     assert lib.ckv_dense_decode(None, None, None, None, None, None, 1, 16, None, None, None) == bad
     assert lib.ckv_stats_build(None, None, None, None, None, 1, 16, None) == bad
     assert lib.ckv_dense_decode_static(None, None, None, None, None, None, 1, 16, None, None, None) == bad

@@ -318,6 +318,39 @@ def test_bad_page_id_sets_status_and_does_not_fault():
     assert d.ckv.read_status() == 0            # reading clears it
 
 
+def test_bounded_wait_runs_out_and_the_context_recovers():
+    """Failure detection without a fault: the scan's producer announces one shared-memory fill and never issues it
+    (a test hook), the poll limit of the bounded waits is lowered to 2^10, and the step must RETURN with
+    CKV_DEV_TIMEOUT in the status word -- nothing traps, nothing waits for ever, no copy is left in flight.  With the
+    hook cleared, the next step on the same context is correct against the oracle."""
+    from paper_2609_26300_b200 import binding
+    w = small(batch=1, num_q_heads=4, num_kv_heads=1, ctx=16 * 60 + 3, budget_tokens=16 * 8, decode_steps=0)
+    d = setup(w)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() == 0
+    d.ckv.debug_set(1 << 10, binding.CKV_DEBUG_SKIP_FILL)
+    d.ckv.decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len, w.budget_tokens)
+    torch.cuda.synchronize()                       # the launch came back
+    st = d.ckv.read_status()
+    assert st & binding.CKV_DEV_TIMEOUT, st
+    assert d.ckv.read_status() == 0                # reading cleared it
+    d.ckv.debug_set(0, 0)                          # default poll limit, no hook
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, int(d.lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores)
+    # the same through the fused step (the scan launch with its tail CTAs)
+    d.ckv.set_tail_mode(binding.CKV_TAIL_ON)
+    d.ckv.debug_set(1 << 10, binding.CKV_DEBUG_SKIP_FILL)
+    d.ckv.decode(dev_q(d), d.k_pool, d.v_pool, d.table, d.lens, d.max_len, w.budget_tokens)
+    torch.cuda.synchronize()
+    assert d.ckv.read_status() & binding.CKV_DEV_TIMEOUT
+    d.ckv.debug_set(0, 0)
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    for s, h in all_units(w):
+        check_unit_decode(d, s, h, int(d.lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores)
+
+
 def test_append_past_capacity_sets_status():
     from paper_2609_26300_b200 import binding
     w = small(batch=1, ctx=16 * 4, decode_steps=0)
