@@ -223,11 +223,16 @@ int ckv_dense_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void
  * plugin handed only the operation's own tensors, code under a memory pool or a capture that forbids
  * cudaMalloc, a process whose device memory is already committed to the KV cache.)
  * Same inputs, outputs and result as ckv_dense_decode(), with `layout` passed directly.  The split partials
- * live in a fixed device array inside the library image (4 MiB + 256 B, held by every GPU that loads the
- * library until the process exits); the call allocates nothing.  It returns CKV_ERR_CAPACITY, before launching
- * anything, when batch * num_q_heads * 528 B * 64 exceeds 4 MiB.  All calls share that array: calls that overlap
+ * live in a fixed device array inside the library image (4 MiB + 1 KiB, held by every GPU that loads the
+ * library until the process exits); the call allocates nothing.  Two limits, checked before anything is
+ * launched (CKV_ERR_CAPACITY): batch * num_q_heads * 528 B * 64 must fit in 4 MiB, and batch * num_kv_heads must
+ * not exceed 192 (one split counter per unit in the last KiB).  All calls share that array: calls that overlap
  * on the GPU (other streams, other host threads) race on it, so serialise them.  The first call on a device
- * looks up the array's device address and sets kernel attributes: make it outside any stream capture. */
+ * looks up the array's device address, and the first call with a given (device, group size, kv_dtype) sets the
+ * attributes of that layout's kernels: make those calls outside any stream capture.  Unlike the context calls,
+ * this one has no way of returning what only the device can see: a page id outside the pool is skipped (the
+ * page contributes nothing) and the status word that records it, which lives in the array, is cleared by the
+ * next call unread.  A failed CUDA call returns CKV_ERR_CUDA and leaves its code for ckv_last_cuda_error(). */
 int ckv_dense_decode_static(const ckv_layout *layout, const void *q, const void *k_pool, const void *v_pool,
                             const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
                             void *out, float *lse, ckv_stream stream);

@@ -84,6 +84,12 @@ inline int cuda_fail(cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail(e__);    \
   } while (0)
 
+}  // namespace
+
+int ckv_record_cuda_error(cudaError_t e) { return cuda_fail(e); }
+
+namespace {
+
 int check_step_args(const ckv_ctx *c, int batch, int max_len) {
   if (c == nullptr) return CKV_ERR_INVALID_ARG;
   if (batch <= 0 || batch > c->layout.max_batch) return CKV_ERR_INVALID_ARG;

@@ -29,6 +29,8 @@
 //   * dense mode (more splits than a cluster holds), and sparse mode when a cluster cannot be placed, publish the
 //     partials in global memory and bump the unit's counter; the CTA that finds the counter complete reads them
 //     back and writes the output.  The counter is left at zero for the next step.
+#include <mutex>
+
 #include "ckv_internal.cuh"
 #include "ckv_mma.cuh"
 #include "ckv_cluster.cuh"
@@ -601,7 +603,15 @@ constexpr int kSparseWarps = 4, kDenseWarps = 8;
 template <int G>
 bool cluster_fits(int n_splits, cudaStream_t st) {
   if (n_splits > kMaxCluster) return false;
-  static int cache[kMaxCluster + 1];   // 0 unknown, 1 fits, 2 does not (per G: the template instantiates one array each)
+  // the answer is a property of the device: cached per device (and per G: the template instantiates one table
+  // each), behind a mutex, since contexts on several devices or host threads may ask at once
+  constexpr int kMaxDev = 64;
+  static std::mutex mtx;
+  static int table[kMaxDev][kMaxCluster + 1];   // 0 unknown, 1 fits, 2 does not
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { (void)cudaGetLastError(); return false; }
+  std::lock_guard<std::mutex> lock(mtx);
+  int *cache = table[dev];
   if (cache[n_splits] != 0) return cache[n_splits] == 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_splits, 1, 1);

@@ -66,6 +66,7 @@ struct ckv_ctx {
   bool hg_key_valid, hg_disabled;
 };
 
+int ckv_record_cuda_error(cudaError_t e);   // remembers e for ckv_last_cuda_error() on this thread; returns CKV_ERR_CUDA
 cudaError_t ckv_configure_kernels();   // selection kernel attributes
 cudaError_t ckv_configure_scan(const ckv_ctx *c);   // scan kernel attributes
 cudaError_t ckv_configure_attn(const ckv_ctx *c);   // attention kernel attributes

@@ -11,14 +11,17 @@
 //   * the array is shared by every call: two calls that overlap on the GPU (different streams, or the same
 //     call from two host threads) race on it and produce garbage.  Serialise them;
 //   * a problem whose partials do not fit returns CKV_ERR_CAPACITY before anything is launched;
-//   * the first call on a device looks the array's device address up and sets kernel attributes; make that
-//     first call outside any stream capture.
+//   * the first call on a device looks the array's device address up, and the first call with a given
+//     (device, group size, kv_dtype) sets the attributes of the kernels that layout uses; make those first calls
+//     outside any stream capture;
+//   * problems only the device can see (a page id outside the pool) are skipped as everywhere else, but the
+//     status word they are recorded in lives in the array and no call returns it: check page tables beforehand.
 #include <mutex>
 
 #include "ckv_internal.cuh"
 
 #define CKV_STATIC_SCRATCH_BYTES (4u << 20)   // 4 MiB of split partials, followed by the words below
-#define CKV_STATIC_TAIL_BYTES 1024            // status word at +0, per-unit split counters at +256 (192 of them)
+#define CKV_STATIC_TAIL_BYTES 1024            // 1 KiB: status word at +0, per-unit split counters at +256 (192 of them)
 
 namespace {
 
@@ -30,6 +33,7 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
 void *g_scratch_ptr[kMaxDevices];   // device address of g_static_scratch on each device, null until looked up
 int g_sm_count[kMaxDevices];
+unsigned g_configured[kMaxDevices];  // bit (4 * kv_dtype + log2 G): the kernels of that layout have their attributes set
 
 }  // namespace
 
@@ -65,17 +69,27 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
 
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CKV_ERR_CUDA;
+  if (e != cudaSuccess) return ckv_record_cuda_error(e);
+  if (dev < 0 || dev >= kMaxDevices) return ckv_record_cuda_error(cudaErrorInvalidDevice);
   {
     std::lock_guard<std::mutex> lock(g_mutex);
     if (g_scratch_ptr[dev] == nullptr) {   // once per device, with that device current
       void *ptr = nullptr;
       e = cudaGetSymbolAddress(&ptr, g_static_scratch);
       if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
-      if (e == cudaSuccess) e = ckv_configure_attn(&c);
-      if (e == cudaSuccess) e = ckv_configure_attn_mma(&c);
-      if (e != cudaSuccess || ptr == nullptr) return CKV_ERR_CUDA;
+      if (e != cudaSuccess) return ckv_record_cuda_error(e);
+      if (ptr == nullptr) return ckv_record_cuda_error(cudaErrorInvalidSymbol);
       g_scratch_ptr[dev] = ptr;
+    }
+    // the attention kernels of this layout (one instantiation per group size and page type) opt in to their
+    // shared memory once per device: a later call with another layout must not find the opt-in missing
+    const int lg = P.G == 1 ? 0 : (P.G == 2 ? 1 : (P.G == 4 ? 2 : 3));
+    const unsigned bit = 1u << (4 * (layout->kv_dtype == CKV_BF16 ? 0 : 1) + lg);
+    if ((g_configured[dev] & bit) == 0) {
+      e = ckv_configure_attn(&c);
+      if (e == cudaSuccess) e = ckv_configure_attn_mma(&c);
+      if (e != cudaSuccess) return ckv_record_cuda_error(e);
+      g_configured[dev] |= bit;
     }
   }
   unsigned char *scratch = (unsigned char *)g_scratch_ptr[dev];
@@ -88,15 +102,15 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
   // the array keeps whatever the previous call left: the status word and the split counters must start at zero
   // (an interrupted call may have left counters behind); every partial that is read is rewritten by this call
   e = cudaMemsetAsync(P.status, 0, CKV_STATIC_TAIL_BYTES, s);
-  if (e != cudaSuccess) return CKV_ERR_CUDA;
+  if (e != cudaSuccess) return ckv_record_cuda_error(e);
   int n_splits = 0;
   bool merged = false;
   e = ckv_launch_attn(&c, true, q, k_pool, v_pool, page_table, seq_lens, nullptr, nullptr, 0, batch, max_seq_len_host,
                       0, out, lse, &n_splits, &merged, s);
-  if (e != cudaSuccess) return CKV_ERR_CUDA;
+  if (e != cudaSuccess) return ckv_record_cuda_error(e);
   if (!merged) {   // fp32 pages: the merge is a launch of its own
     e = ckv_launch_merge(&c, true, seq_lens, nullptr, n_splits, 0, batch, out, lse, s);
-    if (e != cudaSuccess) return CKV_ERR_CUDA;
+    if (e != cudaSuccess) return ckv_record_cuda_error(e);
   }
   return CKV_OK;
 }
