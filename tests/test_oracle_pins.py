@@ -357,6 +357,77 @@ def test_score_approaches_oracle_rule_in_small_variance_regime():
     assert gaps[0] < 0.05 and gaps[1] < gaps[0]
 
 
+
+def test_grouped_variance_follows_the_logit_scale():
+    """Eq. 8's 1/d is the squared logit scale (App. A.4 derives it from z - zbar = q (k - kbar)^T / sqrt(d)): at any
+    other scale s the statistic must still equal the exact logit variance in the case where Eq. 8 is exact (r = d,
+    within-block variation along one coordinate), i.e. sigma_hat^2 = s^2 sum_t w_t Dbar_t, and zbar scales with s."""
+    q, k, v = one_coordinate_unit(0.5, coord=77, g=3, seed=46)
+    st = O.stats(k, v, 16, r=128)
+    for s in (0.25, 1.0 / np.sqrt(D) * 3.0, 0.011):
+        sc = O.scores(q, st, scale=s)
+        for g in range(3):
+            eb = O.exact_blocks(q[g], k, 16, scale=s)
+            np.testing.assert_allclose(sc.sigma2[g], eb.sigma2, rtol=1e-9)
+            np.testing.assert_allclose(sc.zbar[g], st.kmean @ q[g].astype(np.float64) * s, rtol=1e-12, atol=1e-14)
+    # the scale really enters squared: sigma_hat^2(2 s) = 4 sigma_hat^2(s)
+    a, b = O.scores(q, st, scale=0.07), O.scores(q, st, scale=0.14)
+    np.testing.assert_allclose(b.sigma2, 4.0 * a.sigma2, rtol=1e-12)
+
+
+def test_block_score_closed_form_two_token_blocks():
+    """Eq. 9-10 by hand.  Blocks of two tokens k = c_b +- delta_b e_{i_b}: the mean key is c_b, the only non-zero
+    variance is delta_b^2 along i_b, so for head g (a = q_{g,i_b} delta_b scale)
+        zbar = q_g . c_b scale,  sigma_hat^2 = a^2  (r = d)  or  scale^2 w_{g,t} delta_b^2 / |G_t|  (r = 4),
+        l = log 2 + zbar + sigma_hat^2 / 2,  phat = softmax_b(l),  S_b = sum_g phat_{g,b} sigma_hat^2_{g,b},
+    and the exact block sum is Z_b = 2 e^{zbar} cosh(a).  All values are dyadic, so the summaries are exact."""
+    import math
+    r = np.random.default_rng(47)
+    nb, G = 6, 3
+    c = r.integers(-12, 13, size=(nb, D)) / 8.0
+    q = r.integers(-16, 17, size=(G, D)) / 16.0
+    coord = [3, 40, 64, 99, 127, 17]
+    delta = [0.5, 0.25, 1.0, 0.75, 0.125, 0.5]
+    k = np.zeros((2 * nb, D), np.float32)
+    for b in range(nb):
+        e = np.zeros(D); e[coord[b]] = delta[b]
+        k[2 * b], k[2 * b + 1] = c[b] + e, c[b] - e
+    v = r.standard_normal((2 * nb, D)).astype(np.float32)
+    scale = 1.0 / math.sqrt(D)
+    for rr, layout in ((128, 1), (4, 0), (4, 1)):
+        st = O.stats(k, v, 2, r=rr, layout=layout)
+        sc = O.scores(q.astype(np.float32), st)
+        zbar = [[sum(q[g, i] * c[b, i] for i in range(D)) * scale for b in range(nb)] for g in range(G)]
+        sig = [[0.0] * nb for _ in range(G)]
+        for g in range(G):
+            for b in range(nb):
+                if rr == 128:
+                    sig[g][b] = (q[g, coord[b]] * delta[b] * scale) ** 2
+                else:
+                    members = next(m for m in groups_literal(D, 4, layout) if coord[b] in m)
+                    w = sum(q[g, i] ** 2 for i in members)
+                    sig[g][b] = scale ** 2 * w * delta[b] ** 2 / len(members)
+        S = [0.0] * nb
+        for g in range(G):
+            ell = [math.log(2.0) + zbar[g][b] + 0.5 * sig[g][b] for b in range(nb)]
+            m = max(ell)
+            den = sum(math.exp(x - m) for x in ell)
+            for b in range(nb):
+                ph = math.exp(ell[b] - m) / den
+                assert abs(sc.phat[g][b] - ph) <= 1e-12 * ph
+                assert abs(sc.sigma2[g][b] - sig[g][b]) <= 1e-12 * max(sig[g][b], 1e-300)
+                assert abs(sc.zbar[g][b] - zbar[g][b]) <= 1e-12 * max(abs(zbar[g][b]), 1.0)
+                S[b] += ph * sig[g][b]
+            if rr == 128:   # the exact block sums of the same construction
+                eb = O.exact_blocks(q[g].astype(np.float32), k, 2)
+                for b in range(nb):
+                    a = q[g, coord[b]] * delta[b] * scale
+                    assert abs(eb.logZ[b] - (math.log(2.0) + zbar[g][b] + math.log(math.cosh(a)))) <= 1e-12
+        for b in range(nb):
+            assert abs(sc.S[b] - S[b]) <= 1e-12 * S[b]
+        # a head index or a mass taken from the wrong head must change S: the heads' terms differ
+        assert max(abs(sc.phat[0][b] * sc.sigma2[0][b] - sc.phat[1][b] * sc.sigma2[1][b]) / S[b] for b in range(nb)) > 1e-3
+
 def test_scores_invariances():
     q, k, v = make_unit(16 * 10 + 4, 4, noise=0.3, seed=46)
     st = O.stats(k, v, 16)
@@ -400,6 +471,30 @@ def brute_select(S, K, sink=1, recent=2):
     F = {b for b in range(x) if b < sink or b >= x - recent}
     rest = sorted((b for b in range(x) if b not in F), key=lambda b: (-S[b], b))
     return sorted(F | set(rest[:K - len(F)]))
+
+
+def test_select_with_other_mandatory_counts_matches_brute_force():
+    """Eq. 11 with sink and recent counts other than (1, 2), 0 included, on sequences short enough for the two
+    mandatory ends to overlap ("counting any overlap once")."""
+    r = np.random.default_rng(52)
+    seen = set()
+    for trial in range(1500):
+        sink, recent = int(r.integers(0, 4)), int(r.integers(0, 4))
+        x = int(r.integers(1, 14))
+        S = r.choice([0.0, 0.5, 1.0, 2.0], size=x) if trial % 3 == 0 else r.random(x)
+        K = int(r.integers(1, 16))
+        F = {b for b in range(x) if b < sink or b >= x - recent}
+        if K < x and K < len(F):
+            with pytest.raises(ValueError):
+                O.select(S, K, sink, recent)
+            continue
+        ids = list(O.select(S, K, sink, recent))
+        assert ids == brute_select(S, K, sink, recent), (sink, recent, x, K)
+        assert len(ids) == min(K, x) and ids == sorted(set(ids))
+        if K < x:
+            assert F <= set(ids)
+        seen.add((sink, recent, sink + recent > x))
+    assert len({(a, b) for a, b, _ in seen}) == 16 and any(o for _, _, o in seen)
 
 
 def test_select_matches_brute_force_with_ties():
