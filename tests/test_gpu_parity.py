@@ -138,7 +138,12 @@ def test_bf16_summaries_layout(bs, hq):
             assert np.all(err <= 2.0 ** -7 * np.abs(ref) + 1e-30)          # at most one bf16 ulp (a rounding flip)
             assert np.mean(err == 0.0) > 0.99                                # and almost always none
         assert np.allclose(db[s, h, :x].double().cpu().numpy(), st.Dbar, rtol=1e-5, atol=1e-12)
-    decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), fused=True, stat_bf16=True)
+    checked, identical = decode_loop(d, 20, w.budget_tokens, set(range(20)), all_units(w), fused=True, stat_bf16=True)
+    # this layout's near-tie rule is 500 times wider than the default one (helpers.SCORE_RTOL_STAT_BF16): say how
+    # often it was needed at all (run with -s to see it), and require that it is the exception
+    print("bf16 summaries, block %d, %d heads: selected ids identical to the oracle's on %d of %d unit-steps"
+          % (bs, hq, identical, checked))
+    assert identical >= 0.9 * checked
 
 
 @pytest.mark.parametrize("blocks", [70, 71, 72, 73])
@@ -374,6 +379,7 @@ def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False
         d.ckv.set_tail_mode(binding.CKV_TAIL_ON)
     n0 = d.lens.cpu().numpy().copy()
     d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    checked = identical = 0
     for t in range(steps):
         k_new, v_new = synth.appended_rows(w, t)
         q = synth.queries(w, t)
@@ -413,10 +419,13 @@ def decode_loop(d, steps, budget, check_steps, sample_units, use_host_call=False
                     ref, _ = O.sparse(qq, K, V, st, ref_ids if same else got)
                     assert rel_inf(out[s, h * G:(h + 1) * G].double().numpy(), ref) <= OUT_TOL[d.dtype]
                 else:
-                    check_unit_decode(d, s, h, int(n0[s]) + t + 1, t, budget, out, lse, ids, cnt, scores, **ck)
+                    res = check_unit_decode(d, s, h, int(n0[s]) + t + 1, t, budget, out, lse, ids, cnt, scores, **ck)
+                    checked += 1
+                    identical += int(res["ids_identical"])
     torch.cuda.synchronize()
     assert d.ckv.read_status() == 0
     assert np.array_equal(d.lens.cpu().numpy(), n0 + steps)
+    return checked, identical
 
 
 def test_decode_loop_small_with_appends():
