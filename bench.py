@@ -34,8 +34,12 @@ FALLBACK_HBM_GBS = 6650.0
 PAPER_CONTEXT = {"speedup_vs_full": 6.85, "hardware": "NVIDIA H100 80GB HBM3, CPU-offload pipeline, batch 1",
                  "setting": "128K endpoint, budget 512, r=4 (1.456 ms vs 9.966 ms)", "note": "context only"}
 # DRAM traffic (reads + writes) per algorithmic byte of the summary-scan kernel, from the committed ncu capture
-# (profiles/ckv_scan_kernel_llama8b_128k_b4.md): 272.84 MB read + 10.04 MB written for 272.9 MB of summaries.
-SCAN_TRAFFIC_RATIO = 1.037
+# (profiles/ckv_scan_kernel_llama8b_128k_b4.md): 272.97 MB read + 9.33 - 9.51 MB written for 272.9 MB of summaries.
+SCAN_TRAFFIC_RATIO = (272.97 + 9.42) / 272.9
+# What is stored and multiplied (the line's `dtype`): K/V pages are bf16; mean keys and mean values keep fp32
+# precision as split bf16 pairs (hi = bf16(x), lo = bf16(x - hi), relative error <= 2^-18), variances are fp32; the
+# contractions run on bf16 tensor-core tiles (mma.sync) with fp32 accumulation, everything else is fp32.
+DTYPE = "bf16 mma operands (bf16 K/V; summaries as split-bf16 pairs hi+lo, rel. error 2^-18; fp32 variances), fp32 accumulate"
 
 
 def measured_peak():
@@ -117,8 +121,9 @@ def describe(w, default: bool) -> str:
     head = "configs[2] " if default else "sweep point of "
     ctx = "ctx %d" % w.ctx if w.ctx_min is None else "ctx %d..%d (ragged)" % (w.ctx_min, w.ctx)
     return ("%s%s: batch %d, %dq/%dkv heads, d%d, %s (+ appended tokens), block %d, budget %d, r=%d, "
-            "fp32 summaries, bf16 paged KV" % (head, w.name, w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, ctx,
-                                               w.block_size, w.budget_tokens, w.var_groups))
+            "fp32-precision summaries stored as split bf16 pairs, bf16 paged KV"
+            % (head, w.name, w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, ctx, w.block_size, w.budget_tokens,
+               w.var_groups))
 
 
 def step_inputs(w, n_steps: int):
@@ -147,6 +152,94 @@ def oracle_sample_setup(w):
         n0 = int(synth.seq_lens(w)[0])
         stats = list(ex.map(lambda i: O.stats(kv[i][0][:n0], kv[i][1][:n0], w.block_size, w.var_groups), heads))
     return kv, stats, n0, cores
+
+
+def oracle_dense_step(w, kv, n0, cores, step: int):
+    """The oracle's dense attention over the same sample units (Eq. 12 with every block selected); wall seconds."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import compkv_oracle as O
+    from paper_2609_26300_b200 import synth
+    q = synth.queries(w, step)[0]
+    n = n0 + step + 1
+    G = w.group
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(cores) as ex:
+        list(ex.map(lambda h: O.dense(q[h * G:(h + 1) * G], kv[h][0][:n], kv[h][1][:n]), range(len(kv))))
+    return time.perf_counter() - t0
+
+
+def sweep_config5(dev, peak, steps: int = 16):
+    """Benchmark configs[4]: batch 1, 128K context, block size {16, 32, 64} x budget {512, 1024, 2048, 4096} and
+    the stats build per block size, against the dense decode of the same cache.  One cache for all points; every
+    point is ckv_step captured as a CUDA graph, 3 warm-up + `steps` timed replays, L2 flushed before each."""
+    import torch
+    from paper_2609_26300_b200 import binding, synth
+    base = synth.CONFIGS[5].with_(decode_steps=400)
+    k_pool, v_pool, table, lens0 = synth.make_pools(base, threads=min(8, os.cpu_count() or 1))
+    k_pool, v_pool, table = k_pool.to(dev), v_pool.to(dev), table.to(dev)
+    n0 = int(lens0.max())
+    max_len = n0 + 400
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    clean = torch.zeros(64 << 20, dtype=torch.float32, device=dev)
+    q = torch.from_numpy(synth.queries(base, 0)).to(torch.bfloat16).to(dev)
+    kn, vn = (torch.from_numpy(a).to(torch.bfloat16).to(dev) for a in synth.appended_rows(base, 0))
+    points, builds = [], []
+    dense_us = None
+    for bs in synth.SWEEP_BLOCK_SIZES:
+        w = base.with_(block_size=bs)
+        lens = lens0.clone().to(dev)
+        max_blocks = synth.pages_per_seq(w) * w.page_size // bs
+        ckv = binding.CompKV(w.num_q_heads, w.num_kv_heads, w.batch, max_blocks, k_pool.shape[0], block_size=bs,
+                             var_groups=w.var_groups, device=str(dev))
+        ms = []
+        for i in range(4):
+            flush.zero_(); clean.sum()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); ckv.stats_build(k_pool, v_pool, table, lens, n0); e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        b_us = float(np.median(ms[1:])) * 1e3
+        b_bytes = n0 * w.num_kv_heads * 2 * w.head_dim * 2 + required_bytes(w, [n0], 0)[0]
+        builds.append({"block_size": bs, "us": b_us, "bytes": b_bytes, "gbs": b_bytes / (b_us * 1e-6) / 1e9,
+                       "frac_of_peak": b_bytes / (b_us * 1e-6) / 1e9 / peak})
+        if dense_us is None:
+            dms = []
+            for i in range(6):
+                flush.zero_(); clean.sum()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); ckv.dense_decode(q, k_pool, v_pool, table, lens, max_len); e1.record()
+                torch.cuda.synchronize()
+                dms.append(e0.elapsed_time(e1))
+            dense_us = float(np.median(dms[2:])) * 1e3
+        for budget in synth.SWEEP_BUDGETS:
+            outs = ckv.alloc_outputs(w.batch, budget)
+            ckv.step(q, kn, vn, k_pool, v_pool, table, lens, max_len, budget, outs)   # eager warm-up
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                ckv.step(q, kn, vn, k_pool, v_pool, table, lens, max_len, budget, outs)
+            ev = []
+            for i in range(3 + steps):
+                flush.zero_(); clean.sum()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); g.replay(); e1.record()
+                ev.append((e0, e1))
+            torch.cuda.synchronize()
+            us = float(np.mean([a.elapsed_time(b) for a, b in ev[3:]])) * 1e3
+            sel = outs[3].cpu().numpy()
+            stats_b, sel_b = required_bytes(w, lens.cpu().numpy(), sel * bs)
+            req = stats_b + sel_b
+            points.append({"block_size": bs, "budget": budget, "us_per_step": us, "required_bytes": req,
+                           "hbm_gbs": req / (us * 1e-6) / 1e9, "frac_of_peak": req / (us * 1e-6) / 1e9 / peak,
+                           "speedup_vs_dense": dense_us / us})
+            del g
+        assert ckv.read_status() == 0
+        del ckv
+    del k_pool, v_pool, flush, clean
+    torch.cuda.empty_cache()
+    return {"workload": "configs[4]: batch 1, 32q/8kv heads, d128, ctx 131072, block {16,32,64} x budget {512,1024,2048,4096}",
+            "steps_per_point": steps, "dense_us": dense_us, "dense_bytes": n0 * 8 * 2 * 128 * 2,
+            "points": points, "stats_build": builds}
 
 
 def oracle_step(w, kv, stats, n0, cores, step: int):
@@ -216,6 +309,7 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=48)
     ap.add_argument("--e2e-steps", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the batch-1 128K sweep (configs[4])")
     # sweep points (the default line is configs[2]; these leave the metric's workload)
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5], help="synth.CONFIGS index")
     ap.add_argument("--block-size", type=int, default=0)
@@ -501,7 +595,7 @@ def main():
     line = {
         "metric": METRIC if is_default else "sparse decode-attn us/step (append + decode)", "value": us_per_step, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": DTYPE, "data": "synthetic",
         "config": {"workload": describe(w, is_default).replace("fp32 summaries", "bf16 summaries") if args.stat_bf16
                    else describe(w, is_default),
                    "step": "ckv_step (summary scan with the new token's append in its tail CTAs, select, attention + merge: three launches) replayed as one CUDA graph; CUDA events around each replay",
@@ -530,12 +624,21 @@ def main():
         "stats_build": {"us": build_us, "gbs": build_bytes / (build_us * 1e-6) / 1e9, "bytes": build_bytes},
         "roofline": {"kernel": "ckv_scan_kernel", "bound": "hbm", "achieved": scan_gbs, "peak": peak,
                      "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": scan_gbs / peak,
+                     "frac_step": step_gbs / peak, "frac_step_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+                     "frac_step_note": "the whole step (scan, select, attention + merge) on its required bytes; "
+                                       "`frac` is the dominant kernel alone",
+                     "scan_form": "the launch timed here is the decode-only form (its tail CTAs redo the last "
+                                  "block's terms but append nothing); in the timed step the same launch also "
+                                  "appends the new token",
                      "algorithmic_bytes": stats_b, "launch_us": scan_us,
                      "timing": "average of 16 back-to-back launches between two CUDA events on the launching stream "
                                "(median of 5 such runs); inside an eager step, between events, the same kernel "
                                "takes launch_us_in_eager_step",
                      "launch_us_in_eager_step": scan_eager_us,
-                     "traffic": None if SCAN_TRAFFIC_RATIO is None else SCAN_TRAFFIC_RATIO * stats_b},
+                     "traffic": SCAN_TRAFFIC_RATIO * stats_b,
+                     "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this launch "
+                                       "configuration (profiles/ckv_scan_kernel_llama8b_128k_b4.md: 272.97 MB + "
+                                       "9.33 - 9.51 MB for 272.9 MB of summaries), scaled by the algorithmic bytes"},
         "clocks": clocks,
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "call": "ckv_step_host on the caller's own stream: the step's q/k_new/v_new are written into one set of pinned staging buffers (inside the timed region), out/sel_ids/sel_cnt come back into pinned buffers; returns when the results are complete in the host buffers"},
@@ -543,15 +646,33 @@ def main():
         "wall_s_timed_region": t_wall,
         "paper_context": PAPER_CONTEXT,
     }
+    if world == 1 and is_default and not args.no_sweep:
+        sw = sweep_config5(dev, peak)
+        line["sweep"] = sw
+        b1 = next(p for p in sw["points"] if p["block_size"] == 16 and p["budget"] == 2048)
+        line["batch1_128k"] = {"workload": "configs[4] point: batch 1, ctx 131072, block 16, budget 2048 (the paper's "
+                                           "latency table is batch 1 throughout)",
+                               "us_per_step": b1["us_per_step"], "required_mb": b1["required_bytes"] / 1e6,
+                               "frac_of_%s_peak" % peak_kind: b1["frac_of_peak"], "dense_us": sw["dense_us"],
+                               "speedup_vs_dense": b1["speedup_vs_dense"]}
     if world == 1 and not args.no_cpu_baseline:
         kv, stats, n0s, cores = oracle_sample_setup(w)
         reps = 6
         oracle_step(w, kv, stats, n0s, cores, 0)
         ts = [oracle_step(w, kv, stats, n0s, cores, 1 + i) for i in range(reps)]
         cpu_us = float(np.mean(ts)) * 1e6 * w.batch
+        t1 = [oracle_step(w, kv, stats, n0s, 1, 1 + reps + i) for i in range(2)]
+        td = [oracle_dense_step(w, kv, n0s, cores, i) for i in range(3)]
+        td1 = [oracle_dense_step(w, kv, n0s, 1, i) for i in range(1)]
         line["cpu_baseline"] = {"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "value_1thread": float(np.mean(t1)) * 1e6 * w.batch,
+                                "dense_value": float(np.mean(td[1:])) * 1e6 * w.batch,
+                                "dense_value_1thread": float(np.mean(td1)) * 1e6 * w.batch,
+                                "host_cores": os.cpu_count(),
                                 "sample": "oracle decode step (summary update, scores, top-k, compensated attention) "
-                                          "on the %d KV heads of sequence 0, %d steps, wall time x %d sequences"
+                                          "on the %d KV heads of sequence 0, %d steps, wall time x %d sequences; "
+                                          "dense_value: the oracle's dense attention over the same units; "
+                                          "`cores` = threads used (one per KV head), the *_1thread values use one"
                                           % (w.num_kv_heads, reps, w.batch)}
     print(json.dumps(line))
     rep.close()
