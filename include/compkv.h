@@ -17,6 +17,10 @@
  *     host object.
  *   - All calls that take a stream enqueue work on it and return without synchronising
  *     (ckv_step_host and ckv_read_status synchronise the stream before returning).
+ *   - One context is used from one stream at a time: every call works in the context's workspace (block terms,
+ *     partials, split counters, staging) and some keep per-call state in the host object, so two calls on the
+ *     same context must not overlap on the GPU, nor be issued from two host threads at once.  Use one context
+ *     per concurrent stream; contexts are independent.
  *   - Return value: 0 (CKV_OK) or a negative ckv_status.  Nothing throws or aborts.
  *     Problems only the device can see (a page id outside the pool, a sequence that outgrew
  *     its page table, a non-finite score) set a bit in a device status word and the
@@ -195,23 +199,6 @@ int ckv_step(ckv_ctx *ctx, const void *q, const void *k_new, const void *v_new, 
              const int32_t *page_table, int32_t *seq_lens, int batch, int max_seq_len_host, int budget_tokens,
              void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt, ckv_stream stream);
 
-/* ckv_decode with CUDA events recorded on `stream` between its four kernels (summary scan, score +
- * top-k selection, exact attention on the selected blocks, merge; the bf16 layout merges inside the attention
- * kernel, its fourth duration is then an empty interval).  Waits for the step to finish and writes the four
- * durations in milliseconds to stage_ms_host[0..3] (host).  For measurement only. */
-int ckv_decode_profile(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_pool,
-                       const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
-                       int budget_tokens, void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt,
-                       ckv_stream stream, float *stage_ms_host);
-
-/* The summary scan of ckv_decode (Eq. 8-10 logits and the all-block compensation sums of Eq. 12) launched
- * `reps` times back to back between two CUDA events on `stream`; waits, and writes the average duration of
- * one launch in milliseconds to *avg_ms_host (host).  The scan only rewrites its own workspace rows, so the
- * repetitions are idempotent; the summaries of the bench workloads exceed L2, so every launch streams them
- * from HBM.  For measurement only (the roofline figure of the dominant kernel). */
-int ckv_scan_profile(ckv_ctx *ctx, const void *q, const int32_t *seq_lens, int batch, int max_seq_len_host,
-                     int reps, ckv_stream stream, float *avg_ms_host);
-
 /* Dense decode attention over the whole paged cache (Sec. 3.1; Eq. 12 with S = all blocks),
  * split along the sequence with a log-sum-exp merge.  Same tile code as the sparse path. */
 int ckv_dense_decode(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_pool,
@@ -272,9 +259,6 @@ int ckv_step_host(ckv_ctx *ctx, const void *q_host, const void *k_new_host, cons
 /* Read and clear the device status word (bits of ckv_device_status); synchronises `stream`. */
 int ckv_read_status(ckv_ctx *ctx, int32_t *host_status, ckv_stream stream);
 
-/* Number of kernel launches the library has enqueued through this context so far. */
-int64_t ckv_launch_count(const ckv_ctx *ctx);
-
 /* How the decode step treats the last block of every sequence (the only block a step can change).  In "tail
  * mode" a few CTAs of the scan launch own that block -- and, in ckv_step, append the new token to it inside the
  * same launch -- while the other CTAs stream the remaining summaries; otherwise the scan covers every block and
@@ -284,6 +268,30 @@ int64_t ckv_launch_count(const ckv_ctx *ctx);
  * (honoured up to 1024 sequences).  Returns CKV_ERR_INVALID_ARG for a null context or an unknown mode. */
 enum ckv_tail_mode { CKV_TAIL_AUTO = 0, CKV_TAIL_OFF = 1, CKV_TAIL_ON = 2 };
 int ckv_set_tail_mode(ckv_ctx *ctx, int mode);
+
+/* ---- measurement ---------------------------------------------------------------------------------------------
+ * Not part of the decode path: these calls exist so that a benchmark can time the library's own launches with
+ * CUDA events on the launching stream, and count them. */
+
+/* ckv_decode with CUDA events recorded on `stream` between its four kernels (summary scan, score +
+ * top-k selection, exact attention on the selected blocks, merge; the bf16 layout merges inside the attention
+ * kernel, its fourth duration is then an empty interval).  Waits for the step to finish and writes the four
+ * durations in milliseconds to stage_ms_host[0..3] (host).  For measurement only. */
+int ckv_decode_profile(ckv_ctx *ctx, const void *q, const void *k_pool, const void *v_pool,
+                       const int32_t *page_table, const int32_t *seq_lens, int batch, int max_seq_len_host,
+                       int budget_tokens, void *out, float *lse, int32_t *sel_ids, int32_t *sel_cnt,
+                       ckv_stream stream, float *stage_ms_host);
+
+/* The summary scan of ckv_decode (Eq. 8-10 logits and the all-block compensation sums of Eq. 12) launched
+ * `reps` times back to back between two CUDA events on `stream`; waits, and writes the average duration of
+ * one launch in milliseconds to *avg_ms_host (host).  The scan only rewrites its own workspace rows, so the
+ * repetitions are idempotent; the summaries of the bench workloads exceed L2, so every launch streams them
+ * from HBM.  For measurement only (the roofline figure of the dominant kernel). */
+int ckv_scan_profile(ckv_ctx *ctx, const void *q, const int32_t *seq_lens, int batch, int max_seq_len_host,
+                     int reps, ckv_stream stream, float *avg_ms_host);
+
+/* Number of kernel launches the library has enqueued through this context so far. */
+int64_t ckv_launch_count(const ckv_ctx *ctx);
 
 /* ---- test hook ------------------------------------------------------------------------------------------------
  * Every wait inside a kernel is bounded: after a number of polls it gives up, sets CKV_DEV_TIMEOUT, drains the
