@@ -12,7 +12,10 @@
 #define CKV_PAGE 16           // tokens per page
 #define CKV_ROW_ELEMS 256     // bf16 elements of one mean-key / mean-value summary row (128 hi halves + 128 lo halves)
 #define CKV_PART_STRIDE 132   // floats per split partial: m, l, pad, pad, acc[128]
-#define CKV_SCAN_TILE 32      // blocks per scan tile
+#define CKV_SCAN_TILE 32      // blocks per scan tile (rows of 512 bytes: two 16 KB bulk copies and the variances per tile)
+#define CKV_SCAN_TILE_HS 64   // ... with bf16 summaries (rows of 256 bytes): the same bytes per copy.  An SM's copy engine
+                              // takes about 3.8 bulk copies per microsecond whatever their size (measured), so halving
+                              // the rows without doubling the tile left the scan exactly as slow as before
 #define CKV_SCAN_WARPS 7       // consumer warps of a scan CTA (plus one producer warp: 256 threads), each with a partial of its own
 #define CKV_MAX_SCAN_CTAS 160 // persistent scan grid is capped at this many CTAs
 #define CKV_MAX_SPLITS 64     // attention partials per unit
@@ -38,6 +41,7 @@ struct CkvDev {
   int row_elems;     // bf16 elements of one mean-key / mean-value row: CKV_ROW_ELEMS, or CKV_D when only hi halves are kept
   int variant;       // ckv_variant bits
   float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
+  int scan_tile;     // blocks per scan tile: CKV_SCAN_TILE, or CKV_SCAN_TILE_HS with bf16 summaries
   int tail;          // 1: the scan launch leaves the last block of every sequence to its tail CTAs (set per step)
   int *unit_done;    // [unit] attention splits finished this step (zero between steps); null = merge is a separate launch
   int *status;       // device status word
@@ -264,7 +268,7 @@ __device__ __forceinline__ float exp2_diff(float a, float b) {
   return (a == -CUDART_INF_F) ? 0.0f : exp2f(a - b);
 }
 
-// Which scan partials belong to `unit`.  The scan cuts the blocks of all units into tiles of CKV_SCAN_TILE blocks;
+// Which scan partials belong to `unit`.  The scan cuts the blocks of all units into tiles of P.scan_tile blocks;
 // scan CTA c gets the tiles [c * tpc, (c + 1) * tpc) and consumer warp w stores its partial for unit u in entry
 // (c + 2 u) * CKV_SCAN_WARPS + w.  The (c, u) pairs that occur form a monotone staircase, so with the factor 2 the
 // group behind a unit's last CTA is free.  In tail mode (P.tail) the scan CTAs leave the LAST block of every
@@ -279,7 +283,7 @@ __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of,
   unsigned tot = 0, before = 0, mine = 0, n_mine = 0;
   for (int i = lane; i < batch; i += 32) {
     const int n = len_of(i);
-    const unsigned t = (unsigned)((ckv_scan_blocks(n, P.bs, P.tail) + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE);
+    const unsigned t = (unsigned)((ckv_scan_blocks(n, P.bs, P.tail) + P.scan_tile - 1) / P.scan_tile);
     tot += t;
     if (i < s) before += t;
     if (i == s) { mine = t; n_mine = (unsigned)n; }

@@ -43,7 +43,7 @@ namespace {
 
 using namespace ckv_pipe;
 
-constexpr int TB = CKV_SCAN_TILE;   // blocks per tile
+template <bool HS> struct ScanTile { static constexpr int TB = HS ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE; };   // blocks per tile
 constexpr int kMaxStages = 8;
 constexpr int kConsumerWarps = CKV_SCAN_WARPS;
 constexpr int kThreads = kConsumerWarps * 32 + 32;   // plus the producer warp
@@ -60,12 +60,12 @@ __device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *s_len,
   UnitInfo ui;
   ui.N = seq_len_of(P, s_len, seq_lens, u / P.Hkv);
   ui.X = ckv_scan_blocks(ui.N, P.bs, P.tail);
-  ui.tiles = (ui.X + TB - 1) / TB;
+  ui.tiles = (ui.X + P.scan_tile - 1) / P.scan_tile;
   return ui;
 }
 
 __device__ __forceinline__ int seq_tiles(const int *s_len, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
-  return (ckv_scan_blocks(seq_len_of(P, s_len, seq_lens, i), P.bs, P.tail) + TB - 1) / TB;
+  return (ckv_scan_blocks(seq_len_of(P, s_len, seq_lens, i), P.bs, P.tail) + P.scan_tile - 1) / P.scan_tile;
 }
 
 constexpr int kLenCounter = 16;   // word of the status region that counts the CTAs which have read the lengths
@@ -254,6 +254,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
                 int n_tail) {
   constexpr bool QS = QSplit<QT>::value;   // fp32 queries are split into hi + lo like the summaries
   constexpr int kRowBytes = HS ? CKV_D * 2 : CKV_ROW_ELEMS * 2;   // bytes of one mean-key / mean-value row
+  constexpr int TB = ScanTile<HS>::TB;
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
   __shared__ int s_u0, s_tl0, s_count, s_ulast, s_abort, s_issued;
@@ -518,7 +519,10 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         const float *sd = reinterpret_cast<const float *>(stage_mem + (size_t)st * stage_bytes + 2 * TB * kRowBytes);
 
         // ---- Z^T = Q Kbar^T: heads x 16 blocks (two n-tiles of 8 blocks), hi and lo planes into one accumulator ----
-        float z[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, zlo[2][2] = {{0.f, 0.f}, {0.f, 0.f}};   // two chains per n-tile
+        // four accumulation chains per n-tile (hi / lo plane x even / odd 16-coordinate step): the products of a chain
+        // depend on one another, and a warp has little else to issue while it waits for them
+        float z[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, zlo[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        float z2[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, zlo2[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
         {
           // ldmatrix lane roles: matrix lane / 8 -> 8-coordinate chunk, row lane % 8
           const int lrow = lane & 7, lmat = lane >> 3;
@@ -532,18 +536,19 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
               uint32_t bh[4], bl[4];
               ldmatrix_x4(bh, rowaddr + coff);
               mma_rows8(z[nt][0], z[nt][1], qa[2 * j][0], qa[2 * j][1], bh[0], bh[1]);
-              mma_rows8(z[nt][0], z[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bh[2], bh[3]);
+              mma_rows8(z2[nt][0], z2[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bh[2], bh[3]);
               if (!HS) {
                 ldmatrix_x4(bl, rowaddr + 256 + coff);
                 mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j][0], qa[2 * j][1], bl[0], bl[1]);
-                mma_rows8(zlo[nt][0], zlo[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bl[2], bl[3]);
+                mma_rows8(zlo2[nt][0], zlo2[nt][1], qa[2 * j + 1][0], qa[2 * j + 1][1], bl[2], bl[3]);
               }
               if (QS) {
                 mma_rows8(zlo[nt][0], zlo[nt][1], qb[QS ? 2 * j : 0][0], qb[QS ? 2 * j : 0][1], bh[0], bh[1]);
                 mma_rows8(zlo[nt][0], zlo[nt][1], qb[QS ? 2 * j + 1 : 0][0], qb[QS ? 2 * j + 1 : 0][1], bh[2], bh[3]);
               }
             }
-            z[nt][0] += zlo[nt][0]; z[nt][1] += zlo[nt][1];
+            z[nt][0] = (z[nt][0] + z2[nt][0]) + (zlo[nt][0] + zlo2[nt][0]);
+            z[nt][1] = (z[nt][1] + z2[nt][1]) + (zlo[nt][1] + zlo2[nt][1]);
           }
         }
         float sgm[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
@@ -684,7 +689,8 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
 struct ScanCfg { int stages; size_t smem; };
 
 ScanCfg scan_cfg(const CkvDev &P, int G) {
-  const size_t stage_bytes = (size_t)TB * 2 * (P.row_elems * 2) + (P.r >= 4 ? (size_t)TB * P.r * 4 : 0);
+  const size_t TB = (size_t)P.scan_tile;
+  const size_t stage_bytes = TB * 2 * (P.row_elems * 2) + (P.r >= 4 ? TB * P.r * 4 : 0);
   const size_t sw_bytes = (P.r == 4 || P.r == CKV_D) ? 0 : (size_t)kConsumerWarps * P.r * G * 4;   // weight table of the generic path
   const size_t budget = 220 * 1024 - 8 * 1024 - sw_bytes;   // static shared memory stays below 8 KB
   int stages = (int)(budget / stage_bytes);
@@ -765,7 +771,7 @@ int tail_ctas(const ckv_ctx *c, int batch) {
 int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
   const CkvDev &P = c->dev;
   const int xmax = std::max((max_len + P.bs - 1) / P.bs - P.tail, 0);   // in tail mode the last block is the tail CTAs'
-  const long long tiles = (long long)batch * P.Hkv * ((xmax + TB - 1) / TB);
+  const long long tiles = (long long)batch * P.Hkv * ((xmax + P.scan_tile - 1) / P.scan_tile);
   long long grid = c->sm_count - tail_ctas(c, batch);
   if (grid > CKV_MAX_SCAN_CTAS) grid = CKV_MAX_SCAN_CTAS;
   if (grid > tiles) grid = tiles;
