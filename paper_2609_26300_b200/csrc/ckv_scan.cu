@@ -256,7 +256,8 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   constexpr int kRowBytes = HS ? CKV_D * 2 : CKV_ROW_ELEMS * 2;   // bytes of one mean-key / mean-value row
   constexpr int TB = ScanTile<HS>::TB;
   extern __shared__ __align__(128) unsigned char stage_mem[];
-  __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
+  __shared__ __align__(8) uint64_t full_bar[2][kMaxStages], empty_bar[kMaxStages];
+  __shared__ __align__(16) unsigned char s_zero_row[512];   // what mean-value rows past a unit's last block are read as
   __shared__ int s_u0, s_tl0, s_count, s_ulast, s_abort, s_issued;
   __shared__ int s_len[kMaxSeqs];
 
@@ -283,12 +284,12 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     return;
   }
   const int bid = (int)blockIdx.x - n_tail, nscan = (int)gridDim.x - n_tail;   // this CTA among the scan CTAs
-  // rows past a unit's last block are never copied: clear the ring once so that they hold zeros or old summaries,
-  // never arbitrary bit patterns (a NaN times a zero weight would poison the accumulators)
-  for (int i = tid; i < stages * stage_bytes / 16; i += kThreads) reinterpret_cast<uint4 *>(stage_mem)[i] = make_uint4(0u, 0u, 0u, 0u);
-  fence_proxy_async();
+  // rows of a stage past a unit's last block are never copied and the ring is never cleared: the products over
+  // blocks read such mean-value rows from a row of zeros instead (a stale NaN pattern times a zero weight would
+  // poison the accumulators); everywhere else a block is an output column, and those columns are discarded
+  if (tid < 32) reinterpret_cast<uint4 *>(s_zero_row)[tid] = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) {   // also done while the lengths are on their way: the barriers of the ring
-    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], kConsumerWarps); }
+    for (int st = 0; st < stages; ++st) { mbar_init(&full_bar[0][st], 1); mbar_init(&full_bar[1][st], 1); mbar_init(&empty_bar[st], kParts); }
     fence_barrier_init();
   }
   if (tid < batch) s_len[tid] = eff_len(len_mine);
@@ -338,6 +339,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     if (lane == 0) {
       int u = s_u0, tl = s_tl0, st = 0;
       uint32_t phase = 0;            // parity of the empty-barrier phase the next refill of stage `st` waits for
+      uint32_t round = 0;            // times the ring has wrapped: fill `it` uses the full barrier [round & 1][st]
       UnitInfo ui = unit_info(P, s_len, seq_lens, u);
       for (int it = 0; it < count; ++it) {
         if (it >= stages && !mbar_wait(&empty_bar[st], phase, P.spin_limit)) {
@@ -352,19 +354,20 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         unsigned char *sv = sk + TB * kRowBytes;
         const uint32_t kbytes = (uint32_t)nb * kRowBytes;
         const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
-        mbar_arrive_expect_tx(&full_bar[st], 2 * kbytes + dbytes);
+        uint64_t *fb = &full_bar[round & 1][st];
+        mbar_arrive_expect_tx(fb, 2 * kbytes + dbytes);
         const uint32_t lo = smem_u32(stage_mem), hi = lo + (uint32_t)stages * stage_bytes;
         bool ok = nb >= 1 && u < units && row + nb <= (size_t)units * P.max_blocks;
         // test hook (ckv_debug_set): one fill is announced but never issued, so that the waits on it run out
         const bool skip = (P.debug & CKV_DEBUG_SKIP_FILL) != 0 && it == 0 && bid == 0;
         if (!skip) {
-          ok = ok && bulk_g2s_checked(sk, P.kmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
-          ok = ok && bulk_g2s_checked(sv, P.vmean + row * P.row_elems, kbytes, &full_bar[st], lo, hi);
-          if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, &full_bar[st], lo, hi);
+          ok = ok && bulk_g2s_checked(sk, P.kmean + row * P.row_elems, kbytes, fb, lo, hi);
+          ok = ok && bulk_g2s_checked(sv, P.vmean + row * P.row_elems, kbytes, fb, lo, hi);
+          if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, fb, lo, hi);
           *(volatile int *)&s_issued = it + 1;
         }
         if (!ok) atomicOr(P.status, CKV_DEV_BAD_COPY);
-        if (++st == stages) { st = 0; if (it >= stages) phase ^= 1; }
+        if (++st == stages) { st = 0; ++round; if (it >= stages) phase ^= 1; }
         if (++tl == ui.tiles) {
           tl = 0;
           do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
@@ -422,24 +425,29 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         if (unit_info(P, s_len, seq_lens, next_empty).tiles > 0) write_partial(next_empty, false);
     };
 
-    // Half tile j = 2 * tile + half belongs to warp j % W.  A parity wait can only tell a fill of a stage from
-    // the one before it, so every warp passes over ALL tiles in order -- waits for the tile's data, works on it
-    // if one of its halves is this warp's, then releases it -- and a stage is refilled only after all W warps
-    // have released it: no warp is ever more than one fill away from a barrier it waits on.
-    int st = 0;
-    uint32_t phase = 0;              // parity of the full-barrier phase of stage `st` this pass over the ring
-    for (int it = 0; it < count; ++it) {
-      if (it > 0 && ++tl == ui.tiles) {
-        tl = 0;
-        do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
+    // Part j = kParts * tile + part-of-tile belongs to warp j % W, and a warp visits only the tiles that hold one
+    // of its parts: it waits for the tile's fill, works on its part and releases the stage; a stage is refilled
+    // once the kParts owners of its parts have released it.  A warp's next part is at most W parts (four tiles)
+    // ahead, and fill f is only issued after fill f - stages has landed and been released, so the stage a warp
+    // waits on is at most two fills behind the one it wants.  A parity wait can only tell a fill from the one
+    // before it, hence the two sets of full barriers used by alternate rounds of the ring: together they tell four
+    // consecutive fills of a stage apart.
+    int it_at = 0;   // tile the (u, tl) walk stands at
+    for (int pidx = warp; pidx < kParts * count; pidx += kConsumerWarps) {
+      const int it = pidx / kParts;
+      int half = pidx - it * kParts;
+      for (; it_at < it; ++it_at) {
+        if (++tl == ui.tiles) {
+          tl = 0;
+          do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
+        }
       }
-      // part p of tile `it` belongs to warp (kParts * it + p) % W
-      int half = (warp - (kParts * it) % kConsumerWarps + kConsumerWarps) % kConsumerWarps;
-      if (half >= kParts) half = -1;
+      const uint32_t round = (uint32_t)(it / stages);
+      const int st = it - (int)round * stages;
       // a wait that runs out marks the step invalid (`aborted`); the walk still runs to the end
       if (!aborted) {
         bool fail = *(volatile int *)&s_abort != 0;
-        if (!fail && !mbar_wait(&full_bar[st], phase, P.spin_limit)) {
+        if (!fail && !mbar_wait(&full_bar[round & 1][st], (round >> 1) & 1, P.spin_limit)) {
           atomicOr(P.status, CKV_DEV_TIMEOUT);
           *(volatile int *)&s_abort = 1;
           fail = true;
@@ -650,11 +658,12 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         {
           // ldmatrix.trans lane roles: matrix lane / 8 -> (block half, coordinate chunk parity), row lane % 8
           const int r = rb + ((lane >> 3) & 1) * 8 + (lane & 7);
-          const uint32_t rowaddr = sv + r * kRowBytes;
+          const bool real = r < nb;   // rows past the unit's last block: zeros
+          const uint32_t rowaddr = real ? sv + r * kRowBytes : smem_u32(s_zero_row);
           const int cpar = lane >> 4;
 #pragma unroll
           for (int t2 = 0; t2 < 8; ++t2) {   // two 8-coordinate n-tiles per ldmatrix.x4
-            const uint32_t coff = (uint32_t)swz_chunk(2 * t2 + cpar, r) * 16;
+            const uint32_t coff = real ? (uint32_t)swz_chunk(2 * t2 + cpar, r) * 16 : 0u;
             uint32_t vh[4], vl[4];
             ldmatrix_x4_trans(vh, rowaddr + coff);
             mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vh[0], vh[1]);
@@ -662,17 +671,16 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
             mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vh[2], vh[3]);
             mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wl[0], wl[1], vh[2], vh[3]);
             if (!HS) {
-              ldmatrix_x4_trans(vl, rowaddr + 256 + coff);
+              ldmatrix_x4_trans(vl, rowaddr + (real ? 256u : 0u) + coff);
               mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vl[0], vl[1]);
               mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vl[2], vl[3]);
             }
           }
         }
       }
-      }   // own half tile
+      }   // own part
       __syncwarp();
       if (lane == 0 && !aborted) mbar_arrive(&empty_bar[st]);
-      if (++st == stages) { st = 0; phase ^= 1; }
     }
     if (cur >= 0) { write_partial(cur, true); next_empty = cur + 1; }
     fill_empty_upto(ulast + 1);
@@ -682,7 +690,8 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     // leave no bulk copy in flight into this CTA's shared memory: wait (bounded) for every issued fill
     // (a completed phase is seen as complete again, so waiting on consumed stages returns at once)
     const int issued = s_issued;
-    for (int it = max(issued - stages, 0); it < issued; ++it) mbar_wait(&full_bar[it % stages], (it / stages) & 1, P.spin_limit);
+    for (int it = max(issued - stages, 0); it < issued; ++it)
+      mbar_wait(&full_bar[(it / stages) & 1][it % stages], ((it / stages) >> 1) & 1, P.spin_limit);
   }
 }
 
