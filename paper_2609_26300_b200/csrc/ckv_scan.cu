@@ -260,6 +260,12 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   __shared__ __align__(16) unsigned char s_zero_row[512];   // what mean-value rows past a unit's last block are read as
   __shared__ int s_u0, s_tl0, s_count, s_ulast, s_abort, s_issued;
   __shared__ int s_len[kMaxSeqs];
+  // Query rows and variance weights of the first kStagedUnits units of this CTA's range (a CTA's range rarely
+  // spans more than two), staged by the consumer warps while the first fills are on their way: a warp that moves
+  // on to another unit then sets up from shared memory instead of paying a round trip to global memory.
+  constexpr int kStagedUnits = 4;
+  __shared__ __align__(16) __nv_bfloat16 s_q[kStagedUnits][G][CKV_D];
+  __shared__ float s_w[kStagedUnits][G][4];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool r4 = P.r == 4;          // the default: the variance projection is four FMAs on one 16-byte read
@@ -380,6 +386,33 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     // ---------------- consumer warps: half tile j = warp, warp + 8, ... of the CTA's range ----------------
     const int head = lane >> 2, qd = lane & 3;   // this thread's accumulator row (head) and column pair
     const bool hv = head < G;
+    const bool staged = !QS && !RD && P.r == 4;   // bf16 queries, four variance groups: the staged setup below
+    if (staged) {
+      constexpr int kPieces = G * CKV_D * 2 / 16;   // 16-byte pieces of a unit's G query rows
+      for (int idx = tid; idx < kStagedUnits * kPieces; idx += kConsumerWarps * 32) {
+        const int k = idx / kPieces, pc = idx % kPieces, uu = s_u0 + k;
+        if (uu <= s_ulast && uu < units) {
+          const int s2 = uu / P.Hkv, h2 = uu % P.Hkv;
+          const uint4 *src = reinterpret_cast<const uint4 *>(q + ((size_t)s2 * P.Hq + h2 * G) * CKV_D);
+          reinterpret_cast<uint4 *>(&s_q[k][0][0])[pc] = __ldg(src + pc);
+        }
+      }
+      named_barrier(1, kConsumerWarps * 32);
+      // w_{g,t} of Eq. 8: sums of squared query coordinates per variance group, times the squared logit scale
+      for (int idx = tid; idx < kStagedUnits * G * 4; idx += kConsumerWarps * 32) {
+        const int k = idx / (G * 4), g = (idx / 4) % G, t = idx % 4;
+        if (s_u0 + k <= s_ulast) {
+          float w = 0.f;
+          for (int i = 0; i < CKV_D / 4; ++i) {   // the group's 32 coordinates: one run, or two runs of 16
+            const int c = P.glayout == 0 ? 32 * t + i : (i < 16 ? 16 * t + i : CKV_D / 2 + 16 * t + (i - 16));
+            const float x = __bfloat162float(s_q[k][g][c]);
+            w = fmaf(x, x, w);
+          }
+          s_w[k][g][t] = w * (P.scale * P.scale);
+        }
+      }
+      named_barrier(1, kConsumerWarps * 32);
+    }
     uint32_t qa[8][2], qb[QS ? 8 : 1][2];        // A fragments of the unit's queries (rows 0..7), per 16-coordinate step
     uint32_t qsh[RD ? 8 : 1][2], qsl[RD ? 8 : 1][2];   // (scale q)^2 as hi and lo halves, same fragment positions
     float acc[16][2];                            // W Vbar accumulator: head `head`, coordinates 8 t + 2 qd + {0, 1}
@@ -461,6 +494,17 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         // per-unit setup: query fragments, variance weights, fresh accumulators
         const int s = u / P.Hkv, h = u % P.Hkv;
         const QT *qrow = q + ((size_t)s * P.Hq + h * G + (hv ? head : 0)) * CKV_D;
+        const int uk = u - s_u0;
+        const bool from_smem = staged && uk < kStagedUnits;
+        if (from_smem) {
+          const uint32_t *srow = reinterpret_cast<const uint32_t *>(&s_q[uk][hv ? head : 0][0]);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) qa[ks][hh] = hv ? srow[(16 * ks + 8 * hh + 2 * qd) / 2] : 0u;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) wown[t] = hv ? s_w[uk][head][t] : 0.f;
+        } else {
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
 #pragma unroll
@@ -476,7 +520,10 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
             }
           }
         }
-        if (RD) {
+        }
+        if (from_smem) {
+          // set up above
+        } else if (RD) {
           // nothing to tabulate: the weights are the squared queries held above
         } else if (r4) {
           // w_{g,t} for this thread's head: every lane of the quad sums all 128 coordinates (once per unit)
