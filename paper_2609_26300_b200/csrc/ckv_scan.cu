@@ -386,6 +386,11 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     // ---------------- consumer warps: half tile j = warp, warp + 8, ... of the CTA's range ----------------
     const int head = lane >> 2, qd = lane & 3;   // this thread's accumulator row (head) and column pair
     const bool hv = head < G;
+    constexpr bool SP = (G <= 4) && !RD;   // the per-(head, block) arithmetic is shared between the half warps
+    constexpr int NE = SP ? 1 : 2;          // n-tiles a lane works on there
+    const int hsel = lane >> 4;             // ... and which one: the lower half warp the first, the upper the second
+    const int ehead = SP ? (head & 3) : head;
+    const bool ehv = ehead < G;
     const bool staged = !QS && !RD && P.r == 4;   // bf16 queries, four variance groups: the staged setup below
     if (staged) {
       constexpr int kPieces = G * CKV_D * 2 / 16;   // 16-byte pieces of a unit's G query rows
@@ -444,6 +449,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
       float l = l_acc, lp = lp_acc;
       l += __shfl_xor_sync(0xffffffffu, l, 1); l += __shfl_xor_sync(0xffffffffu, l, 2);
       lp += __shfl_xor_sync(0xffffffffu, lp, 1); lp += __shfl_xor_sync(0xffffffffu, lp, 2);
+      if (SP) { l += __shfl_xor_sync(0xffffffffu, l, 16); lp += __shfl_xor_sync(0xffffffffu, lp, 16); }
       if (hv) {
         float *pg = part + head * CKV_PART_STRIDE;
 #pragma unroll
@@ -503,7 +509,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) qa[ks][hh] = hv ? srow[(16 * ks + 8 * hh + 2 * qd) / 2] : 0u;
 #pragma unroll
-          for (int t = 0; t < 4; ++t) wown[t] = hv ? s_w[uk][head][t] : 0.f;
+          for (int t = 0; t < 4; ++t) wown[t] = ehv ? s_w[uk][ehead][t] : 0.f;
         } else {
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
@@ -528,10 +534,11 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         } else if (r4) {
           // w_{g,t} for this thread's head: every lane of the quad sums all 128 coordinates (once per unit)
           float wsum[4] = {0.f, 0.f, 0.f, 0.f};
+          const QT *qrow_e = q + ((size_t)s * P.Hq + h * G + (ehv ? ehead : 0)) * CKV_D;
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
             float x[8];
-            load8<true>(qrow + 8 * c, x);
+            load8<true>(qrow_e + 8 * c, x);
             float s8 = 0.f;
 #pragma unroll
             for (int i = 0; i < 8; ++i) s8 = fmaf(x[i], x[i], s8);
@@ -540,7 +547,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
             wsum[0] += t == 0 ? s8 : 0.f; wsum[1] += t == 1 ? s8 : 0.f;
             wsum[2] += t == 2 ? s8 : 0.f; wsum[3] += t == 3 ? s8 : 0.f;
           }
-          if (!hv) { wsum[0] = wsum[1] = wsum[2] = wsum[3] = 0.f; }
+          if (!ehv) { wsum[0] = wsum[1] = wsum[2] = wsum[3] = 0.f; }
 #pragma unroll
           for (int t = 0; t < 4; ++t) wown[t] = wsum[t] * (P.scale * P.scale);   // Eq. 8's 1/d is the squared logit scale
         } else {
@@ -633,54 +640,69 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         }
 
         // ---- per (head, block): variance projection, l, running maximum, compensation weight ----
-        float zl2[2][2], sig[2][2], wt[2][2];
-        bool val[2][2];
+        // The products leave this part's 16 blocks x G heads in the lanes of rows 0..G-1 (four values per lane).
+        // With G <= 4 those are lanes 0-15 only, so the upper half warp takes over the second n-tile: every lane
+        // then works on one n-tile's pair of blocks (half the dependent chain), and the weights travel back to
+        // the lower lanes, which hold the A operand of the next product.
+        float zin[NE][2];
+        if constexpr (SP) {
+          const float t0 = __shfl_sync(0xffffffffu, z[1][0], lane & 15), t1 = __shfl_sync(0xffffffffu, z[1][1], lane & 15);
+          zin[0][0] = hsel ? t0 : z[0][0];
+          zin[0][1] = hsel ? t1 : z[0][1];
+        } else {
+#pragma unroll
+          for (int k = 0; k < NE; ++k) { zin[k][0] = z[k][0]; zin[k][1] = z[k][1]; }
+        }
+        float zl2[NE][2], sig[NE][2], wt[NE][2];
+        bool val[NE][2];
         float tmax = -CUDART_INF_F;
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
+        for (int k = 0; k < NE; ++k) {
+          const int nt = SP ? hsel : k;
           const int r0 = rb + nt * 8 + 2 * qd;     // this thread's two blocks of the n-tile: rows r0, r0 + 1
           float ell[2];
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             const int r = r0 + e, b = b0 + r;
-            val[nt][e] = hv && r < nb;
+            val[k][e] = ehv && r < nb;
             float sg = 0.f;
-            if (val[nt][e]) {
+            if (val[k][e]) {
               if (RD) {
-                sg = fmaxf(sgm[nt][e], 0.f);
+                sg = fmaxf(sgm[RD ? k : 0][e], 0.f);
               } else if (r4) {
                 const float4 dv = *reinterpret_cast<const float4 *>(sd + r * 4);
                 sg = fmaf(wown[0], dv.x, fmaf(wown[1], dv.y, fmaf(wown[2], dv.z, wown[3] * dv.w)));
               } else {
                 for (int t = 0; t < P.r; ++t) {
                   const float dv = dbar_bulk ? sd[r * P.r + t] : __ldg(db + (size_t)b * P.r + t);
-                  sg = fmaf(sw[t * G + head], dv, sg);
+                  sg = fmaf(sw[t * G + ehead], dv, sg);
                 }
               }
             }
-            sig[nt][e] = sg;
-            const float zbar = z[nt][e] * P.scale;
+            sig[k][e] = sg;
+            const float zbar = zin[k][e] * P.scale;
             const float logc = (!P.tail && b == ui.X - 1) ? log_last : log_bs;   // in tail mode every block here is full
             ell[e] = logc + zbar + P.half_var * sg;
-            zl2[nt][e] = val[nt][e] ? (zbar + logc) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
-            tmax = fmaxf(tmax, zl2[nt][e]);
+            zl2[k][e] = val[k][e] ? (zbar + logc) * kLog2e : -CUDART_INF_F;   // log2 of |b| e^{zbar}
+            tmax = fmaxf(tmax, zl2[k][e]);
           }
           // what the later kernels read, both in log2 units: the head's term of the block score, e^l sigma^2 (e^l
           // alone when blocks are ranked by mass), and the block's mean-compensation weight |b| e^{zbar}.  The
           // thread's two blocks are neighbours: one 8-byte store each when the rows are 8-byte aligned.
-          const size_t o = (size_t)head * P.max_blocks + b0 + r0;
-          const float u0 = fmaf(ell[0], kLog2e, by_mass ? 0.f : __log2f(sig[nt][0]));
-          const float u1 = fmaf(ell[1], kLog2e, by_mass ? 0.f : __log2f(sig[nt][1]));
-          if (pair_ok && val[nt][1]) {
+          const size_t o = (size_t)ehead * P.max_blocks + b0 + r0;
+          const float u0 = fmaf(ell[0], kLog2e, by_mass ? 0.f : __log2f(sig[k][0]));
+          const float u1 = fmaf(ell[1], kLog2e, by_mass ? 0.f : __log2f(sig[k][1]));
+          if (pair_ok && val[k][1]) {
             *reinterpret_cast<float2 *>(lu + o) = make_float2(u0, u1);
-            *reinterpret_cast<float2 *>(lz + o) = make_float2(zl2[nt][0], zl2[nt][1]);
+            *reinterpret_cast<float2 *>(lz + o) = make_float2(zl2[k][0], zl2[k][1]);
           } else {
-            if (val[nt][0]) { lu[o] = u0; lz[o] = zl2[nt][0]; }
-            if (val[nt][1]) { lu[o + 1] = u1; lz[o + 1] = zl2[nt][1]; }
+            if (val[k][0]) { lu[o] = u0; lz[o] = zl2[k][0]; }
+            if (val[k][1]) { lu[o + 1] = u1; lz[o + 1] = zl2[k][1]; }
           }
         }
         tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
         tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        if (SP) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
         if (tmax > m_ref + CKV_RESCALE_SLACK) {   // the running maximum is only raised when exceeded by a slack
           const float sc = exp2_diff(m_ref, tmax);
           m_ref = tmax;
@@ -688,17 +710,28 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
 #pragma unroll
           for (int t = 0; t < 16; ++t) { acc[t][0] *= sc; acc[t][1] *= sc; }
         }
-        uint32_t wh[2], wl[2];   // A fragments of the weights: k = blocks 2 qd + {0, 1} (+ 8), hi and lo halves
+        uint32_t whm[NE], wlm[NE];
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
+        for (int k = 0; k < NE; ++k) {
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            wt[nt][e] = val[nt][e] ? fast_exp2(zl2[nt][e] - m_ref) : 0.f;
-            l_acc += wt[nt][e];
-            lp_acc = fmaf(wt[nt][e], fast_exp2(P.half_var * kLog2e * sig[nt][e]), lp_acc);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
+            wt[k][e] = val[k][e] ? fast_exp2(zl2[k][e] - m_ref) : 0.f;
+            l_acc += wt[k][e];
+            lp_acc = fmaf(wt[k][e], fast_exp2(P.half_var * kLog2e * sig[k][e]), lp_acc);   // e^{l - m} = e^{zbar + log|b| - m} e^{sigma^2/2}
           }
-          wh[nt] = pack_bf16(wt[nt][0], wt[nt][1]);
-          wl[nt] = pack_bf16(wt[nt][0] - bf16_round(wt[nt][0]), wt[nt][1] - bf16_round(wt[nt][1]));
+          whm[k] = pack_bf16(wt[k][0], wt[k][1]);
+          wlm[k] = pack_bf16(wt[k][0] - bf16_round(wt[k][0]), wt[k][1] - bf16_round(wt[k][1]));
+        }
+        uint32_t wh[2], wl[2];   // A fragments of the weights: k = blocks 2 qd + {0, 1} (+ 8), hi and lo halves
+        if constexpr (SP) {
+          // rows 0..3 (lanes 0-15) get their second n-tile from the lane 16 above; rows 4..7 carry zero weights
+          const uint32_t oh = __shfl_sync(0xffffffffu, whm[0], (lane & 15) + 16);
+          const uint32_t ol = __shfl_sync(0xffffffffu, wlm[0], (lane & 15) + 16);
+          wh[0] = hsel ? 0u : whm[0]; wl[0] = hsel ? 0u : wlm[0];
+          wh[1] = hsel ? 0u : oh;     wl[1] = hsel ? 0u : ol;
+        } else {
+#pragma unroll
+          for (int k = 0; k < NE; ++k) { wh[k] = whm[k]; wl[k] = wlm[k]; }
         }
 
         // ---- acc += W Vbar: heads x 128 coordinates, k = this half tile's 16 blocks ----
