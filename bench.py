@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 PAPER_CONTEXT = {"speedup_vs_full": 6.85, "hardware": "NVIDIA H100 80GB HBM3, CPU-offload pipeline, batch 1",
                  "setting": "128K endpoint, budget 512, r=4 (1.456 ms vs 9.966 ms)", "note": "context only"}
 # DRAM traffic (reads + writes) per algorithmic byte of the summary-scan kernel, from the committed ncu capture
-# (profiles/ckv_scan_kernel_llama8b_128k_b4.md): 272.97 MB read + 9.33 - 9.51 MB written for 272.9 MB of summaries.
-SCAN_TRAFFIC_RATIO = (272.97 + 9.42) / 272.9
+# (profiles/ckv_scan_kernel_llama8b_128k_b4.md): 273.17 MB read + 9.57 MB written for 272.9 MB of summaries.
+SCAN_TRAFFIC_RATIO = (273.17 + 9.57) / 272.9
 # What is stored and multiplied (the line's `dtype`): K/V pages are bf16; mean keys and mean values keep fp32
 # precision as split bf16 pairs (hi = bf16(x), lo = bf16(x - hi), relative error <= 2^-18), variances are fp32; the
 # contractions run on bf16 tensor-core tiles (mma.sync) with fp32 accumulation, everything else is fp32.
@@ -637,8 +637,8 @@ def main():
                      "launch_us_in_eager_step": scan_eager_us,
                      "traffic": SCAN_TRAFFIC_RATIO * stats_b,
                      "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this launch "
-                                       "configuration (profiles/ckv_scan_kernel_llama8b_128k_b4.md: 272.97 MB + "
-                                       "9.33 - 9.51 MB for 272.9 MB of summaries), scaled by the algorithmic bytes"},
+                                       "configuration (profiles/ckv_scan_kernel_llama8b_128k_b4.md: 273.17 MB + "
+                                       "9.57 MB for 272.9 MB of summaries), scaled by the algorithmic bytes"},
         "clocks": clocks,
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "call": "ckv_step_host on the caller's own stream: the step's q/k_new/v_new are written into one set of pinned staging buffers (inside the timed region), out/sel_ids/sel_cnt come back into pinned buffers; returns when the results are complete in the host buffers"},
