@@ -176,6 +176,13 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   const float *lz = P.lz + (size_t)unit * P.max_blocks * G;
   const __nv_bfloat16 *vmean = P.vmean + (size_t)unit * P.max_blocks * P.row_elems;
   const bool mean_lo = P.row_elems == CKV_ROW_ELEMS;   // the mean-value rows carry lo halves (fp32-precision summaries)
+  // How a selected block's mean term |b| e^{zbar} vbar_b (part of the scan's all-block sum) is taken out again.
+  // vbar_b is the mean of the block's value rows, so with full-precision summaries it is enough to lower the weight
+  // of each of the block's tokens by e^{zbar}: sum_j (p_j - e^{zbar}) v_j = sum_j p_j v_j - |b| e^{zbar} vbar_b up to
+  // the 2^-18 rounding of the stored row, with no row to fetch and no extra product.  bf16 summaries round vbar to
+  // 2^-9, which would leave a visible remainder: they keep the product with the stored rows (remove_means).
+  const bool tok_rm = comp && mean_lo, row_rm = comp && !mean_lo;
+  const float lg_bs = log2f((float)P.bs), lg_last = log2f((float)max(N - (X - 1) * P.bs, 1));
   bool bad = false;
 
   // the scan partials this CTA folds in: partial j of the unit goes to split j % n_active
@@ -256,12 +263,14 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         cp_async16(kb + off, k_pool + so, valid);
         cp_async16(vb + off, v_pool + so, valid);
       }
-      if (comp && r.first) {   // verbatim: hi halves then lo halves, swizzled by block index
+      if (row_rm && r.first) {   // verbatim: hi halves then lo halves, swizzled by block index
         if (mean_lo || lane < 16)
           cp_async16(aux_u32 + 512 * slot + 16 * lane, vmean + (size_t)r.blk * P.row_elems + 8 * lane, true);
         if (lane < G)          // and log2 of the weight of its mean term, for every head
           cp_async4(aux_u32 + kLsOff + (slot * G + lane) * 4, lz + (size_t)lane * P.max_blocks + r.blk);
       }
+      if (tok_rm && lane < G)  // log2 of the block's mean-term weight, per head, beside the page's buffer
+        cp_async4(aux_u32 + kLsOff + (buf * G + lane) * 4, lz + (size_t)lane * P.max_blocks + r.blk);
     }
   };
 
@@ -326,7 +335,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   int si = 0;
   auto take_slot = [&](const PageRef &r) {
     const int slot = si;
-    if (comp && r.first && r.phys >= 0) si = (si + 1) & (kMeanSlots - 1);
+    if (row_rm && r.first && r.phys >= 0) si = (si + 1) & (kMeanSlots - 1);
     return slot;
   };
   PageRef cur{-1, 0, -1, false};
@@ -404,6 +413,11 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
           sv[nt][e] = ok ? sv[nt][e] * sl2 : -CUDART_INF_F;
           tmax = fmaxf(tmax, sv[nt][e]);
         }
+      // log2 of e^{zbar} of the page's block for this lane's head (token-weight removal)
+      float lzt = -CUDART_INF_F;
+      if (tok_rm && hv)
+        lzt = *reinterpret_cast<const float *>(waux + kLsOff + (buf * G + head) * 4) - (cur.blk == X - 1 ? lg_last : lg_bs);
+      tmax = fmaxf(tmax, lzt);
       tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
       tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
       if (tmax > m_ref + CKV_RESCALE_SLACK) {
@@ -413,13 +427,14 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
 #pragma unroll
         for (int t = 0; t < 16; ++t) { acc[t][0] *= sc; acc[t][1] *= sc; }
       }
+      const float wtok = lzt == -CUDART_INF_F ? 0.f : fast_exp2(lzt - m_ref);
       uint32_t ph[2], pl[2];
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
         float p[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          p[e] = sv[nt][e] == -CUDART_INF_F ? 0.f : fast_exp2(sv[nt][e] - m_ref);
+          p[e] = sv[nt][e] == -CUDART_INF_F ? 0.f : fast_exp2(sv[nt][e] - m_ref) - wtok;
           l_acc += p[e];
         }
         ph[nt] = pack_bf16(p[0], p[1]);
@@ -440,7 +455,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
           mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], pl[0], pl[1], v[2], v[3]);
         }
       }
-      if (comp && cur.first) {   // its mean-value row sits in aux slot cur_slot
+      if (row_rm && cur.first) {   // its mean-value row sits in aux slot cur_slot
 #pragma unroll
         for (int j = 0; j < kMeanFlush; ++j)
           if (j == nb) { bb[j] = cur.blk; bsl[j] = cur_slot; }
