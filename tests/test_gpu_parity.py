@@ -434,6 +434,26 @@ def test_decode_loop_small_with_appends():
     decode_loop(d, 36, w.budget_tokens, set(range(36)), all_units(w))
 
 
+@pytest.mark.parametrize("tail_on", [False, True])
+@pytest.mark.parametrize("hq,stat_bf16", [(32, 0), (64, 0), (32, 1)])
+def test_scan_ctas_that_span_many_units(hq, stat_bf16, tail_on):
+    """Many short sequences: 320 units of two to three scan tiles each, so that a scan CTA's range spans three to
+    six units -- more than it stages query rows for -- and its warps change units every few parts.  Every unit of
+    a sample of sequences against the oracle, in both step arrangements."""
+    from paper_2609_26300_b200 import binding
+    w = small(batch=40, num_q_heads=hq, num_kv_heads=8, ctx_min=16 * 40 + 1, ctx=16 * 90 + 5, budget_tokens=16 * 10,
+              decode_steps=0, needles=1)
+    d = setup(w, stat_bf16=stat_bf16)
+    d.ckv.set_tail_mode(binding.CKV_TAIL_ON if tail_on else binding.CKV_TAIL_OFF)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    out, lse, ids, cnt, scores = run_decode(d, w.budget_tokens)
+    lens = d.lens.cpu().numpy()
+    for s in (0, 7, 19, 33, 39):
+        for h in range(w.num_kv_heads):
+            check_unit_decode(d, s, h, int(lens[s]), 0, w.budget_tokens, out, lse, ids, cnt, scores,
+                              stat_bf16=bool(stat_bf16))
+
+
 def test_decode_loop_two_calls_in_tail_mode():
     """ckv_append + ckv_decode with the last block of every sequence left to the scan launch's tail CTAs."""
     w = small(ctx_min=16 * 30 + 1, ctx=16 * 60, decode_steps=20)
