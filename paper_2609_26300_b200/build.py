@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcompkv.so")
 SOURCES = ["ckv_api.cu", "ckv_stats.cu", "ckv_scan.cu", "ckv_select.cu", "ckv_attn.cu", "ckv_attn_mma.cu", "ckv_static.cu", "ckv_diag.cu"]
-NVCC_FLAGS = (["-DCKV_TRACE"] if os.environ.get("CKV_TRACE") else []) + ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
 
