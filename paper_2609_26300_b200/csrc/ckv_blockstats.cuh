@@ -56,6 +56,46 @@ __device__ __forceinline__ void block_stats_finish(const CkvDev &P, int b, float
   if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
 }
 
+// The two passes over a one-page block of bf16 rows held in registers: lane (hw, li) holds the 8 coordinates 8 li ..
+// of the key and value rows hw, hw + 2, ... (rows that do not exist: zeros, and they are skipped).  Leaves the mean
+// key (km), the value sums (vs) and this half warp's squared deviations (sq) for block_stats_finish.  Every caller
+// that has such a block's rows in registers uses this one routine, so the summaries have the same bits whether the
+// rows came from the pool or from a prefill chunk on its way into the pool.
+__device__ __forceinline__ void block_stats_rows16(const uint4 (&kraw)[8], const uint4 (&vraw)[8], bool ok, int cnt,
+                                                   int lane, float (&km)[8], float (&vs)[8], float (&sq)[8]) {
+  const int hw = lane >> 4;
+  const float fc = (float)cnt;
+  float ks[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { ks[i] = 0.f; vs[i] = 0.f; }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    if (ok && hw + 2 * j < cnt) {
+      float a[8], c[8];
+      bf16x8_to_float(kraw[j], a);
+      bf16x8_to_float(vraw[j], c);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
+    vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
+    km[i] = ks[i] / fc;
+    sq[i] = 0.f;
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    if (ok && hw + 2 * j < cnt) {
+      float a[8];
+      bf16x8_to_float(kraw[j], a);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+    }
+  }
+}
+
 // NC: the pools are read-only for the whole kernel (loads may use the non-coherent path).
 // sq_smem: 128 floats of shared memory owned by the calling warp.
 template <typename T, bool NC>
@@ -93,32 +133,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
         kraw[j] = valid ? (NC ? __ldg(kp) : *kp) : zero;
         vraw[j] = valid ? (NC ? __ldg(vp) : *vp) : zero;
       }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (ok && hw + 2 * j < cnt) {
-          float a[8], c[8];
-          bf16x8_to_float(kraw[j], a);
-          bf16x8_to_float(vraw[j], c);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
-        vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
-        km[i] = ks[i] / fc;
-        sq[i] = 0.f;
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (ok && hw + 2 * j < cnt) {
-          float a[8];
-          bf16x8_to_float(kraw[j], a);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
-        }
-      }
+      block_stats_rows16(kraw, vraw, ok, cnt, lane, km, vs, sq);
     }
   }
   if (!done) {

@@ -23,8 +23,10 @@
 // 32 consecutive blocks; the tiles, in (unit, position) order, are split into one contiguous range per scan CTA,
 // one scan CTA per remaining SM.  A producer thread streams the CTA's tiles into a ring of shared-memory stages
 // with cp.async.bulk (two 16 KB copies and the variances per tile), completion on mbarriers.  Each of the seven
-// consumer warps takes every seventh half tile (16 blocks) on its own -- there is no CTA-wide barrier in the
-// loop -- with a per-warp running maximum that is only raised when exceeded by a slack.  A warp writes one
+// consumer warps takes every seventh half tile (16 blocks) on its own and visits only the tiles that hold one of
+// its parts -- there is no CTA-wide barrier in the loop -- with a per-warp running maximum that is only raised
+// when exceeded by a slack.  The query rows and variance weights of the CTA's units are staged in shared memory
+// while the first fills are in flight, so a warp that moves on to another unit sets up from there.  A warp writes one
 // partial per unit its CTA touched; partial (scan CTA c, warp w, unit u) lives in entry (c + 2 u) * 7 + w, unique
 // because the (c, u) pairs that occur form a monotone staircase; the entry behind a unit's last one is free and
 // takes the last block's partial, so a unit's partials are one contiguous run (unit_scan_entries).

@@ -11,6 +11,7 @@
 namespace {
 
 constexpr int kBuildRounds = 8;   // blocks per warp of the build kernel
+constexpr int kPrefillRounds = 4; // blocks per warp of the prefill kernel's register-resident variant
 
 // A warp takes kBuildRounds blocks, eight blocks apart, and asks the L2 for the pages of its next block before it
 // works on the current one: the block routine waits for all rows of a block at once, so without the request every
@@ -101,8 +102,9 @@ __global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T 
 // block's new rows into their pages and then runs the block routine over the block (rows that were already in the
 // cache included), so the new keys and values cross DRAM once on the way in and the summaries come out of the same
 // pass.  The CTA that finishes last stores the new sequence lengths (every warp read the old ones when it started).
-template <typename T>
-__global__ void __launch_bounds__(256) ckv_prefill_kernel(CkvDev P, T *k_pool, T *v_pool,
+// ONE: one-page blocks of bf16 rows (the default layout), the variant whose rows never leave the registers.
+template <typename T, bool ONE>
+__global__ void __launch_bounds__(256, ONE ? 2 : 1) ckv_prefill_kernel(CkvDev P, T *k_pool, T *v_pool,
                                                           const int *__restrict__ page_table, int *seq_lens,
                                                           const T *__restrict__ k_src, const T *__restrict__ v_src,
                                                           const int *__restrict__ new_lens, int src_stride, int batch) {
@@ -113,10 +115,76 @@ __global__ void __launch_bounds__(256) ckv_prefill_kernel(CkvDev P, T *k_pool, T
   const int N = seq_lens[s], M = new_lens[s];
   const int m_eff = N < 0 ? 0 : max(min(min(M, src_stride), cap - N), 0);   // tokens that fit
   if (M > m_eff && blockIdx.x == 0 && threadIdx.x == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
-  const int b = (N >= 0 ? N / P.bs : 0) + blockIdx.x * 8 + warp;
+  // the register-resident variant gives a warp kPrefillRounds blocks, eight blocks apart, and asks the L2 for the
+  // next block's rows of the chunk before it works on the current one (as the build kernel does with its pages)
+  constexpr int kRounds = ONE ? kPrefillRounds : 1;
+#pragma unroll 1
+  for (int rnd = 0; rnd < kRounds; ++rnd) {
+  const int b = (N >= 0 ? N / P.bs : 0) + (blockIdx.x * kRounds + rnd) * 8 + warp;
   if (m_eff > 0 && b <= (N + m_eff - 1) / P.bs) {
     const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
+    if constexpr (ONE) {
+      const int bn = b + 8;
+      if (rnd + 1 < kRounds && bn <= (N + m_eff - 1) / P.bs) {
+        // 16 rows x (K, V) x 256 bytes = 64 lines of 128 bytes: two per lane
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int line = lane + 32 * k, t = (line >> 1) & 15, half = line & 1, kv = line >> 5;
+          const int p = bn * CKV_PAGE + t;
+          if (p >= N && p < N + m_eff) {
+            const T *src = (kv ? v_src : k_src) + (((size_t)s * src_stride + (p - N)) * P.Hkv + h) * CKV_D + half * 64;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(src) : "memory");
+          }
+        }
+      }
+    }
     const int p_lo = max(b * P.bs, N), p_hi = min((b + 1) * P.bs, N + m_eff);
+    bool handled = false;
+    if constexpr (ONE) {
+      {
+        // One-page blocks of bf16 rows (the default layout): the rows go from the chunk into registers in the
+        // layout the block routine works in (rows of the block that were already in the cache come from the page),
+        // the new ones are stored to the page, and the summaries are worked out from the registers -- the chunk
+        // crosses DRAM once and nothing is read back.
+        handled = true;
+        const int hw = lane >> 4, li = lane & 15;
+        const int phys = pt_row[b];
+        const bool ok = phys >= 0 && phys < P.num_pages;
+        const int cnt = min(P.bs, N + m_eff - b * P.bs);
+        const size_t pbase = ok ? ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li : 0;
+        uint4 kraw[8], vraw[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int t = hw + 2 * j, p = b * CKV_PAGE + t;
+          const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+          kraw[j] = zero; vraw[j] = zero;
+          if (ok && t < cnt) {
+            if (p >= p_lo) {
+              const size_t so = (((size_t)s * src_stride + (p - N)) * P.Hkv + h) * CKV_D + 8 * li;
+              kraw[j] = __ldg(reinterpret_cast<const uint4 *>(k_src + so));
+              vraw[j] = __ldg(reinterpret_cast<const uint4 *>(v_src + so));
+            } else {
+              kraw[j] = *reinterpret_cast<const uint4 *>(k_pool + pbase + (size_t)t * CKV_D);
+              vraw[j] = *reinterpret_cast<const uint4 *>(v_pool + pbase + (size_t)t * CKV_D);
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int t = hw + 2 * j, p = b * CKV_PAGE + t;
+          if (ok && t < cnt && p >= p_lo) {
+            *reinterpret_cast<uint4 *>(k_pool + pbase + (size_t)t * CKV_D) = kraw[j];
+            *reinterpret_cast<uint4 *>(v_pool + pbase + (size_t)t * CKV_D) = vraw[j];
+          }
+        }
+        float km[8], vs[8], sq[8];
+        block_stats_rows16(kraw, vraw, ok, cnt, lane, km, vs, sq);
+        const size_t row = (size_t)unit * P.max_blocks + b;
+        block_stats_finish(P, b, (float)cnt, km, vs, sq, sq_smem[warp], P.kmean + row * P.row_elems, P.dbar + row * P.r,
+                           P.vmean + row * P.row_elems, lane, !ok);
+      }
+    }
+    if constexpr (!ONE) {
     constexpr int PIECES = (int)(CKV_D * sizeof(T) / 16);   // 16-byte pieces of a row: 16 (bf16) or 32 (fp32)
     constexpr int PP = PIECES / 16;                          // pieces per lane and row
     bool bad = false;
@@ -152,7 +220,9 @@ __global__ void __launch_bounds__(256) ckv_prefill_kernel(CkvDev P, T *k_pool, T
     const size_t row = (size_t)unit * P.max_blocks + b;
     block_stats_warp<T, false>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * P.row_elems,
                                P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
+    }
   }
+  }   // rounds
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -222,12 +292,17 @@ cudaError_t ckv_launch_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int
   if (batch <= 0 || max_new <= 0) return cudaSuccess;
   const int touched = (max_new + P.bs - 1) / P.bs + 1;   // a chunk that starts inside a block touches one more
   dim3 grid((touched + 7) / 8, batch * P.Hkv);
-  if (c->layout.kv_dtype == CKV_BF16)
-    ckv_prefill_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool, page_table,
-                                                            seq_lens, (const __nv_bfloat16 *)k_src,
-                                                            (const __nv_bfloat16 *)v_src, new_lens, src_stride, batch);
+  const dim3 grid_one((touched + 8 * kPrefillRounds - 1) / (8 * kPrefillRounds), batch * P.Hkv);
+  if (c->layout.kv_dtype == CKV_BF16 && P.ppb == 1)
+    ckv_prefill_kernel<__nv_bfloat16, true><<<grid_one, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
+                                                                  page_table, seq_lens, (const __nv_bfloat16 *)k_src,
+                                                                  (const __nv_bfloat16 *)v_src, new_lens, src_stride, batch);
+  else if (c->layout.kv_dtype == CKV_BF16)
+    ckv_prefill_kernel<__nv_bfloat16, false><<<grid, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
+                                                                   page_table, seq_lens, (const __nv_bfloat16 *)k_src,
+                                                                   (const __nv_bfloat16 *)v_src, new_lens, src_stride, batch);
   else
-    ckv_prefill_kernel<float><<<grid, 256, 0, st>>>(P, (float *)k_pool, (float *)v_pool, page_table, seq_lens,
+    ckv_prefill_kernel<float, false><<<grid, 256, 0, st>>>(P, (float *)k_pool, (float *)v_pool, page_table, seq_lens,
                                                     (const float *)k_src, (const float *)v_src, new_lens, src_stride, batch);
   c->launches++;
   return cudaGetLastError();
