@@ -783,10 +783,17 @@ ScanCfg scan_cfg(const CkvDev &P, int G) {
   const size_t TB = (size_t)P.scan_tile;
   const size_t stage_bytes = TB * 2 * (P.row_elems * 2) + (P.r >= 4 ? TB * P.r * 4 : 0);
   const size_t sw_bytes = (P.r == 4 || P.r == CKV_D) ? 0 : (size_t)kConsumerWarps * P.r * G * 4;   // weight table of the generic path
-  const size_t budget = 220 * 1024 - 8 * 1024 - sw_bytes;   // static shared memory stays below 8 KB
+  // 227 KB per CTA, less the kernel's static shared memory (lengths, barriers, the row of zeros: under 6 KB; staged
+  // query rows and variance weights: 4 units x G x 272 bytes) and a reserve
+  const size_t stat = 6 * 1024 + (size_t)4 * G * (CKV_D * 2 + 16);
+  const size_t budget = 227 * 1024 - stat - 1024 - sw_bytes;
   int stages = (int)(budget / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
-  if (stages < 2) stages = 2;
+  // A consumer warp's next part is at most kConsumerWarps parts ahead of its last one; the ring protocol needs
+  // that distance, in tiles, to be no more than the number of stages (see the consumer loop).
+  const int parts = (int)TB / 16;
+  const int need = (kConsumerWarps + parts - 1) / parts;
+  if (stages < need) stages = 0;   // refused by the launcher (no layout reaches this on a 227 KB part)
   return ScanCfg{stages, stages * stage_bytes + sw_bytes};
 }
 
@@ -794,6 +801,7 @@ template <int G, typename QT>
 cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units, int grid, const CkvNewToken &fresh,
                       int n_tail, cudaStream_t st) {
   const ScanCfg cfg = scan_cfg(c->dev, G);
+  if (cfg.stages == 0) return cudaErrorInvalidConfiguration;
   if (c->dev.r == CKV_D)
     ckv_scan_kernel<G, QT, true, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail);
   else if (c->dev.row_elems == CKV_D) {
