@@ -62,8 +62,10 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 
 constexpr int kMaxCluster = 8;    // splits of a unit that can be one cluster (the portable size; 13 measured far slower)
 
-template <int G, bool DENSE, int W, bool CL>
-__global__ void __launch_bounds__(W * 32, DENSE ? 1 : (W <= 4 ? 3 : 2))
+// RM: the mean terms of the selected blocks are removed with the stored mean-value rows (bf16 summaries); otherwise
+// through the tokens' weights, and the row machinery is not compiled in.
+template <int G, bool DENSE, int W, bool CL, bool RM>
+__global__ void __launch_bounds__(W * 32, DENSE ? 1 : 2)
 ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k_pool,
                     const __nv_bfloat16 *__restrict__ v_pool, const int *__restrict__ page_table,
                     const int *__restrict__ seq_lens, const int *__restrict__ sel_ids,
@@ -181,7 +183,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   // of each of the block's tokens by e^{zbar}: sum_j (p_j - e^{zbar}) v_j = sum_j p_j v_j - |b| e^{zbar} vbar_b up to
   // the 2^-18 rounding of the stored row, with no row to fetch and no extra product.  bf16 summaries round vbar to
   // 2^-9, which would leave a visible remainder: they keep the product with the stored rows (remove_means).
-  const bool tok_rm = comp && mean_lo, row_rm = comp && !mean_lo;
+  const bool tok_rm = !RM && comp, row_rm = RM && comp;
   const float lg_bs = log2f((float)P.bs), lg_last = log2f((float)max(N - (X - 1) * P.bs, 1));
   bool bad = false;
 
@@ -462,7 +464,9 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         ++nb;
       }
     }
-    if (nb == kMeanFlush || (nb > 0 && n + 1 == n_mine)) remove_means();
+    if constexpr (RM) {
+      if (nb == kMeanFlush || (nb > 0 && n + 1 == n_mine)) remove_means();
+    }
     __syncwarp();   // the page buffer (and, after a removal, the mean-value slots) may be overwritten from here on
     cur = nxt;
     cur_slot = nxt_slot;
@@ -638,7 +642,7 @@ bool cluster_fits(int n_splits, cudaStream_t st) {
   attr[0].val.clusterDim.x = n_splits; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   int n = 0;
-  const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, ckv_attn_mma_kernel<G, false, kSparseWarps, true>, &cfg);
+  const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, ckv_attn_mma_kernel<G, false, kSparseWarps, true, true>, &cfg);
   if (e != cudaSuccess) (void)cudaGetLastError();
   cache[n_splits] = (e == cudaSuccess && n > 0) ? 1 : 2;
   return cache[n_splits] == 1;
@@ -651,10 +655,11 @@ cudaError_t launch_g(ckv_ctx *c, bool dense, const void *q, const void *k_pool, 
   const int units = (int)grid.y;
   const __nv_bfloat16 *qp = (const __nv_bfloat16 *)q, *kp = (const __nv_bfloat16 *)k_pool, *vp = (const __nv_bfloat16 *)v_pool;
   if (dense) {
-    ckv_attn_mma_kernel<G, true, kDenseWarps, false><<<grid, kDenseWarps * 32, dyn_smem<kDenseWarps>(), st>>>(
+    ckv_attn_mma_kernel<G, true, kDenseWarps, false, false><<<grid, kDenseWarps * 32, dyn_smem<kDenseWarps>(), st>>>(
         c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
     return cudaGetLastError();
   }
+  const bool rm = c->dev.row_elems == CKV_D;   // bf16 summaries: removal with the stored mean-value rows
   if (cluster_fits<G>((int)grid.x, st)) {   // the unit's splits as one cluster: partials never leave the SMs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -665,24 +670,30 @@ cudaError_t launch_g(ckv_ctx *c, bool dense, const void *q, const void *k_pool, 
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = grid.x; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, ckv_attn_mma_kernel<G, false, kSparseWarps, true>, c->dev, qp, kp, vp, page_table,
+    if (rm)
+      return cudaLaunchKernelEx(&cfg, ckv_attn_mma_kernel<G, false, kSparseWarps, true, true>, c->dev, qp, kp, vp, page_table,
+                                seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
+    return cudaLaunchKernelEx(&cfg, ckv_attn_mma_kernel<G, false, kSparseWarps, true, false>, c->dev, qp, kp, vp, page_table,
                               seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
   }
-  ckv_attn_mma_kernel<G, false, kSparseWarps, false><<<grid, kSparseWarps * 32, dyn_smem<kSparseWarps>(), st>>>(
-      c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
+  if (rm)
+    ckv_attn_mma_kernel<G, false, kSparseWarps, false, true><<<grid, kSparseWarps * 32, dyn_smem<kSparseWarps>(), st>>>(
+        c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
+  else
+    ckv_attn_mma_kernel<G, false, kSparseWarps, false, false><<<grid, kSparseWarps * 32, dyn_smem<kSparseWarps>(), st>>>(
+        c->dev, qp, kp, vp, page_table, seq_lens, sel_ids, sel_cnt, kcap, pps, scan_grid, units, (__nv_bfloat16 *)out, lse);
   return cudaGetLastError();
 }
 
 template <int G>
 cudaError_t configure_g() {
-  cudaError_t e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, true, kDenseWarps, false>,
+  cudaError_t e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, true, kDenseWarps, false, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem<kDenseWarps>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, false>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem<kSparseWarps>());
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, true>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem<kSparseWarps>());
+  const int sm = (int)dyn_smem<kSparseWarps>();
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv_attn_mma_kernel<G, false, kSparseWarps, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
   return e;
 }
 
