@@ -17,42 +17,56 @@ __device__ __forceinline__ void block_stats_finish(const CkvDev &P, int b, float
                                                    __nv_bfloat16 *kmean_row, float *dbar_row,
                                                    __nv_bfloat16 *vmean_row, int lane, bool bad) {
   const int hw = lane >> 4, li = lane & 15;
+  const float inv = 1.0f / fc;
 #pragma unroll
   for (int i = 0; i < 8; ++i) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], 16);
-  if (hw == 0) {
-    store_split8(kmean_row, li, b, km, P.row_elems == CKV_ROW_ELEMS);
-    if (P.r == CKV_D) {
-      // one group per coordinate: the variance row has the mean rows' layout (split bf16 pairs, swizzled chunks),
-      // so that the scan can project it with the same tensor-core product as the mean keys
+  // the two mean rows leave through one store routine: half warp 0 writes the mean key, half warp 1 the mean value
+  {
+    float rowv[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) rowv[i] = hw == 0 ? km[i] : vs[i] * inv;
+    store_split8(hw == 0 ? kmean_row : vmean_row, li, b, rowv, P.row_elems == CKV_ROW_ELEMS);
+  }
+  const int gs = CKV_D / P.r;
+  const int run = P.glayout == 0 ? gs : gs / 2;   // consecutive coordinates of a group (two runs, 64 apart, in layout 1)
+  if (P.r == CKV_D) {
+    // one group per coordinate: the variance row has the mean rows' layout (split bf16 pairs, swizzled chunks),
+    // so that the scan can project it with the same tensor-core product as the mean keys
+    if (hw == 0) {
       float dv[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) dv[i] = sq[i] / fc;
+      for (int i = 0; i < 8; ++i) dv[i] = sq[i] * inv;
       store_split8(reinterpret_cast<__nv_bfloat16 *>(dbar_row), li, b, dv);
-    } else {
+    }
+  } else if (run >= 8) {
+    // grouped variance: average of the per-coordinate population variances of each group (Eq. 8).  A run is a
+    // whole number of lanes: the lane's eight coordinates first, then the lanes of the run, then the second run.
+    float ps = ((sq[0] + sq[1]) + (sq[2] + sq[3])) + ((sq[4] + sq[5]) + (sq[6] + sq[7]));
+    const int w = run >> 3;
+    for (int o = 1; o < w; o <<= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+    if (P.glayout != 0) ps += __shfl_xor_sync(0xffffffffu, ps, 8);
+    const int lg = P.glayout == 0 ? li : (li & 7);
+    if (hw == 0 && (lg & (w - 1)) == 0 && (P.glayout == 0 || li < 8)) dbar_row[lg / w] = ps / (fc * (float)gs);
+  } else {
+    // groups narrower than a lane's eight coordinates: through shared memory
+    if (hw == 0) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) sq_smem[8 * li + i] = sq[i];
     }
-  } else {
-    float vm[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) vm[i] = vs[i] / fc;
-    store_split8(vmean_row, li, b, vm, P.row_elems == CKV_ROW_ELEMS);
-  }
-  __syncwarp();
-  // grouped variance: average of the per-coordinate population variances of each group (Eq. 8)
-  const int gs = CKV_D / P.r;
-  for (int t = lane; t < P.r && P.r != CKV_D; t += 32) {
-    float s = 0.f;
-    if (P.glayout == 0) {
-      for (int i = 0; i < gs; ++i) s += sq_smem[t * gs + i];
-    } else {
-      const int hg = gs / 2;
-      for (int i = 0; i < hg; ++i) s += sq_smem[t * hg + i];
-      for (int i = 0; i < hg; ++i) s += sq_smem[CKV_D / 2 + t * hg + i];
+    __syncwarp();
+    for (int t = lane; t < P.r; t += 32) {
+      float s = 0.f;
+      if (P.glayout == 0) {
+        for (int i = 0; i < gs; ++i) s += sq_smem[t * gs + i];
+      } else {
+        const int hg = gs / 2;
+        for (int i = 0; i < hg; ++i) s += sq_smem[t * hg + i];
+        for (int i = 0; i < hg; ++i) s += sq_smem[CKV_D / 2 + t * hg + i];
+      }
+      dbar_row[t] = s / (fc * (float)gs);
     }
-    dbar_row[t] = s / (fc * (float)gs);
+    __syncwarp();
   }
-  __syncwarp();
   if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
 }
 
@@ -61,37 +75,37 @@ __device__ __forceinline__ void block_stats_finish(const CkvDev &P, int b, float
 // key (km), the value sums (vs) and this half warp's squared deviations (sq) for block_stats_finish.  Every caller
 // that has such a block's rows in registers uses this one routine, so the summaries have the same bits whether the
 // rows came from the pool or from a prefill chunk on its way into the pool.
+// FULL: the caller knows that all 16 rows exist (ok, cnt == 16): the same operations without the per-row tests.
+template <bool FULL = false>
 __device__ __forceinline__ void block_stats_rows16(const uint4 (&kraw)[8], const uint4 (&vraw)[8], bool ok, int cnt,
                                                    int lane, float (&km)[8], float (&vs)[8], float (&sq)[8]) {
   const int hw = lane >> 4;
-  const float fc = (float)cnt;
+  const float inv = 1.0f / (float)cnt;   // the reciprocal every routine of this file divides by (exact for 16-token blocks)
   float ks[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) { ks[i] = 0.f; vs[i] = 0.f; }
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    if (ok && hw + 2 * j < cnt) {
-      float a[8], c[8];
-      bf16x8_to_float(kraw[j], a);
-      bf16x8_to_float(vraw[j], c);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+    if (FULL || (ok && hw + 2 * j < cnt)) {
+      // mixed-precision adds: a bf16 operand widened inside the instruction (exact), the same sum as ks[i] += float(k)
+      add_bf16x8(kraw[j], ks);
+      add_bf16x8(vraw[j], vs);
     }
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
     vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
-    km[i] = ks[i] / fc;
+    km[i] = ks[i] * inv;
     sq[i] = 0.f;
   }
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    if (ok && hw + 2 * j < cnt) {
-      float a[8];
-      bf16x8_to_float(kraw[j], a);
+    if (FULL || (ok && hw + 2 * j < cnt)) {
+      float dv[8];
+      sub_bf16x8(kraw[j], km, dv);   // float(k) - km
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+      for (int i = 0; i < 8; ++i) sq[i] = fmaf(dv[i], dv[i], sq[i]);
     }
   }
 }
@@ -109,7 +123,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
   for (int i = 0; i < 8; ++i) { ks[i] = 0.f; vs[i] = 0.f; }
   const int npages = (cnt + CKV_PAGE - 1) / CKV_PAGE;
   bool bad = false;
-  const float fc = (float)cnt;
+  const float fc = (float)cnt, inv = 1.0f / fc;
   float km[8], sq[8];
   bool done = false;
   if constexpr (sizeof(T) == 2) {
@@ -123,17 +137,26 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
       bad = !ok;
       const size_t base = ok ? ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li : 0;
       uint4 kraw[8], vraw[8];
+      const uint4 *kp = reinterpret_cast<const uint4 *>(k_pool + base + (size_t)hw * CKV_D);
+      const uint4 *vp = reinterpret_cast<const uint4 *>(v_pool + base + (size_t)hw * CKV_D);
+      constexpr int kStep = 2 * CKV_D / 8;   // two rows on, in 16-byte units
+      if (ok && cnt == CKV_PAGE) {   // a full block (all but the last of a sequence): no per-row tests
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int t = hw + 2 * j;
-        const bool valid = ok && t < cnt;
-        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-        const uint4 *kp = reinterpret_cast<const uint4 *>(k_pool + base + (size_t)t * CKV_D);
-        const uint4 *vp = reinterpret_cast<const uint4 *>(v_pool + base + (size_t)t * CKV_D);
-        kraw[j] = valid ? (NC ? __ldg(kp) : *kp) : zero;
-        vraw[j] = valid ? (NC ? __ldg(vp) : *vp) : zero;
+        for (int j = 0; j < 8; ++j) {
+          kraw[j] = NC ? __ldg(kp + j * kStep) : kp[j * kStep];
+          vraw[j] = NC ? __ldg(vp + j * kStep) : vp[j * kStep];
+        }
+        block_stats_rows16<true>(kraw, vraw, true, CKV_PAGE, lane, km, vs, sq);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const bool valid = ok && hw + 2 * j < cnt;
+          const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+          kraw[j] = valid ? (NC ? __ldg(kp + j * kStep) : kp[j * kStep]) : zero;
+          vraw[j] = valid ? (NC ? __ldg(vp + j * kStep) : vp[j * kStep]) : zero;
+        }
+        block_stats_rows16(kraw, vraw, ok, cnt, lane, km, vs, sq);
       }
-      block_stats_rows16(kraw, vraw, ok, cnt, lane, km, vs, sq);
     }
   }
   if (!done) {
@@ -172,7 +195,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
     for (int i = 0; i < 8; ++i) {
       ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
       vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
-      km[i] = ks[i] / fc;
+      km[i] = ks[i] * inv;
       sq[i] = 0.f;
     }
     for (int pg = 0; pg < npages; ++pg) {
@@ -216,7 +239,7 @@ __device__ __forceinline__ void block_stats_warp_staged(const CkvDev &P, const T
 #pragma unroll
   for (int i = 0; i < 8; ++i) { ks[i] = 0.f; vs[i] = 0.f; }
   const int npages = (cnt + CKV_PAGE - 1) / CKV_PAGE;
-  const float fc = (float)cnt;
+  const float fc = (float)cnt, inv = 1.0f / fc;
   bool bad = false;
   auto stage_page = [&](int pg, bool with_v) -> bool {   // false: the page id is bad, nothing staged
     const int phys = pt_row[b * P.ppb + pg];
@@ -254,7 +277,7 @@ __device__ __forceinline__ void block_stats_warp_staged(const CkvDev &P, const T
   for (int i = 0; i < 8; ++i) {
     ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
     vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
-    km[i] = ks[i] / fc;
+    km[i] = ks[i] * inv;
     sq[i] = 0.f;
   }
 #pragma unroll 1

@@ -125,6 +125,44 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4 &u, float (&o)[8]) {
   o[6] = __uint_as_float(u.w << 16); o[7] = __uint_as_float(u.w & 0xffff0000u);
 }
 
+// Mixed-precision adds of sm_100: the bf16 operand is widened inside the instruction (exactly), so the result has the
+// bits of converting first and adding in fp32, at half the instructions.
+__device__ __forceinline__ void split_b32(uint32_t u, uint16_t &lo, uint16_t &hi) {
+  asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(u));
+}
+__device__ __forceinline__ float add_f32_bf16(uint16_t a, float c) {
+  float r;
+  asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(r) : "h"(a), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float sub_f32_bf16(uint16_t a, float c) {   // a - c
+  float r;
+  asm("sub.rn.f32.bf16 %0, %1, %2;" : "=f"(r) : "h"(a), "f"(c));
+  return r;
+}
+// acc[i] += float(u[i]) for the eight bf16 values of u
+__device__ __forceinline__ void add_bf16x8(const uint4 &u, float (&acc)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint16_t lo, hi;
+    split_b32(w[i], lo, hi);
+    acc[2 * i] = add_f32_bf16(lo, acc[2 * i]);
+    acc[2 * i + 1] = add_f32_bf16(hi, acc[2 * i + 1]);
+  }
+}
+// d[i] = float(u[i]) - m[i]
+__device__ __forceinline__ void sub_bf16x8(const uint4 &u, const float (&m)[8], float (&d)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint16_t lo, hi;
+    split_b32(w[i], lo, hi);
+    d[2 * i] = sub_f32_bf16(lo, m[2 * i]);
+    d[2 * i + 1] = sub_f32_bf16(hi, m[2 * i + 1]);
+  }
+}
+
 // Eight consecutive elements as floats.  NC = read-only (non-coherent) path; use NC = false for
 // data the same kernel has just written.
 template <bool NC>
@@ -158,12 +196,12 @@ __device__ __forceinline__ int swz_chunk(int chunk, int block) { return chunk ^ 
 __device__ __forceinline__ void store_split8(__nv_bfloat16 *row, int chunk, int block, const float (&x)[8], bool lo_half = true) {
   uint32_t hi[4], lo[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const __nv_bfloat16 h0 = __float2bfloat16_rn(x[2 * i]), h1 = __float2bfloat16_rn(x[2 * i + 1]);
-    const __nv_bfloat16 l0 = __float2bfloat16_rn(x[2 * i] - __bfloat162float(h0));
-    const __nv_bfloat16 l1 = __float2bfloat16_rn(x[2 * i + 1] - __bfloat162float(h1));
-    hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-    lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+  for (int i = 0; i < 4; ++i) {   // two values per conversion instruction; the halves come back out by shift and mask
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+    hi[i] = *reinterpret_cast<const uint32_t *>(&h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x[2 * i] - __uint_as_float(hi[i] << 16),
+                                                   x[2 * i + 1] - __uint_as_float(hi[i] & 0xffff0000u));
+    lo[i] = *reinterpret_cast<const uint32_t *>(&l);
   }
   const int p = swz_chunk(chunk, block) * 8;
   *reinterpret_cast<uint4 *>(row + p) = make_uint4(hi[0], hi[1], hi[2], hi[3]);

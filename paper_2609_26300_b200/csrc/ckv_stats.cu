@@ -13,11 +13,13 @@ namespace {
 constexpr int kBuildRounds = 8;   // blocks per warp of the build kernel
 constexpr int kPrefillRounds = 4; // blocks per warp of the prefill kernel's register-resident variant
 
-// A warp takes kBuildRounds blocks, eight blocks apart, and asks the L2 for the pages of its next block before it
-// works on the current one: the block routine waits for all rows of a block at once, so without the request every
-// block would cost a full DRAM round trip with nothing else in flight for that warp.
+// A warp takes kBuildRounds blocks, eight blocks apart.  Two CTAs per SM: the block routine holds a block's 16 key and
+// 16 value rows in registers, which does not fit three CTAs' register share without spills, and the kernel was bound
+// by instruction issue, not by DRAM, while it spilled.  With blocks of several pages (read page after page, twice) a
+// warp asks the L2 for the pages of its next block before it works on the current one; with one-page blocks the 16
+// warps of an SM keep enough rows in flight by themselves and the requests only cost instructions.
 template <typename T>
-__global__ void __launch_bounds__(256, 3) ckv_stats_build_kernel(CkvDev P, const T *__restrict__ k_pool,
+__global__ void __launch_bounds__(256, 2) ckv_stats_build_kernel(CkvDev P, const T *__restrict__ k_pool,
                                                               const T *__restrict__ v_pool,
                                                               const int *__restrict__ page_table,
                                                               const int *__restrict__ seq_lens) {
@@ -33,7 +35,7 @@ __global__ void __launch_bounds__(256, 3) ckv_stats_build_kernel(CkvDev P, const
     const int b = (blockIdx.x * kBuildRounds + i) * 8 + warp;
     if (b >= X) return;
     const int bn = b + 8;
-    if (i + 1 < kBuildRounds && bn < X && lane < P.ppb && bn * P.bs + lane * CKV_PAGE < N) {
+    if (P.ppb > 1 && i + 1 < kBuildRounds && bn < X && lane < P.ppb && bn * P.bs + lane * CKV_PAGE < N) {
       const int phys = pt_row[bn * P.ppb + lane];
       if (phys >= 0 && phys < P.num_pages) {
         const size_t off = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D;
@@ -115,29 +117,14 @@ __global__ void __launch_bounds__(256, ONE ? 2 : 1) ckv_prefill_kernel(CkvDev P,
   const int N = seq_lens[s], M = new_lens[s];
   const int m_eff = N < 0 ? 0 : max(min(min(M, src_stride), cap - N), 0);   // tokens that fit
   if (M > m_eff && blockIdx.x == 0 && threadIdx.x == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
-  // the register-resident variant gives a warp kPrefillRounds blocks, eight blocks apart, and asks the L2 for the
-  // next block's rows of the chunk before it works on the current one (as the build kernel does with its pages)
+  // the register-resident variant gives a warp kPrefillRounds blocks, eight blocks apart (L2 requests for the next
+  // block's rows ahead of time made it slower once the block routine had been trimmed: 763 against 728 us)
   constexpr int kRounds = ONE ? kPrefillRounds : 1;
 #pragma unroll 1
   for (int rnd = 0; rnd < kRounds; ++rnd) {
   const int b = (N >= 0 ? N / P.bs : 0) + (blockIdx.x * kRounds + rnd) * 8 + warp;
   if (m_eff > 0 && b <= (N + m_eff - 1) / P.bs) {
     const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
-    if constexpr (ONE) {
-      const int bn = b + 8;
-      if (rnd + 1 < kRounds && bn <= (N + m_eff - 1) / P.bs) {
-        // 16 rows x (K, V) x 256 bytes = 64 lines of 128 bytes: two per lane
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          const int line = lane + 32 * k, t = (line >> 1) & 15, half = line & 1, kv = line >> 5;
-          const int p = bn * CKV_PAGE + t;
-          if (p >= N && p < N + m_eff) {
-            const T *src = (kv ? v_src : k_src) + (((size_t)s * src_stride + (p - N)) * P.Hkv + h) * CKV_D + half * 64;
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(src) : "memory");
-          }
-        }
-      }
-    }
     const int p_lo = max(b * P.bs, N), p_hi = min((b + 1) * P.bs, N + m_eff);
     bool handled = false;
     if constexpr (ONE) {
@@ -153,6 +140,23 @@ __global__ void __launch_bounds__(256, ONE ? 2 : 1) ckv_prefill_kernel(CkvDev P,
         const int cnt = min(P.bs, N + m_eff - b * P.bs);
         const size_t pbase = ok ? ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li : 0;
         uint4 kraw[8], vraw[8];
+        float km[8], vs[8], sq[8];
+        if (ok && cnt == CKV_PAGE && p_lo == b * CKV_PAGE) {
+          // a full block made of new rows only (all but the first and last touched block): no per-row tests
+          const size_t so = (((size_t)s * src_stride + (p_lo + hw - N)) * P.Hkv + h) * CKV_D + 8 * li;
+          const size_t sstep = (size_t)2 * P.Hkv * CKV_D;   // two chunk rows on
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            kraw[j] = __ldg(reinterpret_cast<const uint4 *>(k_src + so + j * sstep));
+            vraw[j] = __ldg(reinterpret_cast<const uint4 *>(v_src + so + j * sstep));
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            *reinterpret_cast<uint4 *>(k_pool + pbase + (size_t)(hw + 2 * j) * CKV_D) = kraw[j];
+            *reinterpret_cast<uint4 *>(v_pool + pbase + (size_t)(hw + 2 * j) * CKV_D) = vraw[j];
+          }
+          block_stats_rows16<true>(kraw, vraw, true, CKV_PAGE, lane, km, vs, sq);
+        } else {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int t = hw + 2 * j, p = b * CKV_PAGE + t;
@@ -177,8 +181,8 @@ __global__ void __launch_bounds__(256, ONE ? 2 : 1) ckv_prefill_kernel(CkvDev P,
             *reinterpret_cast<uint4 *>(v_pool + pbase + (size_t)t * CKV_D) = vraw[j];
           }
         }
-        float km[8], vs[8], sq[8];
         block_stats_rows16(kraw, vraw, ok, cnt, lane, km, vs, sq);
+        }
         const size_t row = (size_t)unit * P.max_blocks + b;
         block_stats_finish(P, b, (float)cnt, km, vs, sq, sq_smem[warp], P.kmean + row * P.row_elems, P.dbar + row * P.r,
                            P.vmean + row * P.row_elems, lane, !ok);
