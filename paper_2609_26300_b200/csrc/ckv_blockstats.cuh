@@ -3,8 +3,10 @@
 //
 // A token row (128 elements) is spread over the 16 lanes of a half warp, 8 consecutive coordinates per lane (one
 // 16-byte load for bf16); the two half warps take alternate rows.  Means and squared deviations are accumulated in
-// fp32 in two passes (mean first, then deviations from it).  Every caller runs this same code, so a block's
-// summary has the same bits whichever way it was produced.
+// fp32 in two passes (mean first, then deviations from it) over the rows of a page held in registers or shared
+// memory; a block of several bf16 pages is read once, page after page, and the pages' (count, mean, squared
+// deviations) are combined with the pairwise update of Chan et al. (combine_pages).  Every caller runs the same
+// operations in the same order, so a block's summary has the same bits whichever way it was produced.
 #ifndef CKV_BLOCKSTATS_CUH_
 #define CKV_BLOCKSTATS_CUH_
 #include "ckv_internal.cuh"
@@ -70,6 +72,29 @@ __device__ __forceinline__ void block_stats_finish(const CkvDev &P, int b, float
   if (bad && lane == 0) atomicOr(P.status, CKV_DEV_BAD_PAGE);
 }
 
+// Running (count, mean key, squared deviations from it, value sums) of the pages seen so far, joined with those of
+// one more page of nb rows: delta = m_b - m_a, m = m_a + delta n_b / n, M2 = M2_a + M2_b + delta^2 n_a n_b / n.
+// Everything is per coordinate and the same in all lanes that hold the coordinate; the first page only initialises.
+__device__ __forceinline__ void combine_pages(float &na, float (&mean)[8], float (&m2)[8], float (&vsum)[8], int nb,
+                                              const float (&mb)[8], const float (&m2b)[8], const float (&vb)[8]) {
+  if (na == 0.f) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { mean[i] = mb[i]; m2[i] = m2b[i]; vsum[i] = vb[i]; }
+    na = (float)nb;
+    return;
+  }
+  const float fb = (float)nb, n = na + fb;
+  const float wb = fb / n, wab = na * wb;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float d = mb[i] - mean[i];
+    mean[i] = fmaf(d, wb, mean[i]);
+    m2[i] = fmaf(d * d, wab, m2[i] + m2b[i]);
+    vsum[i] += vb[i];
+  }
+  na = n;
+}
+
 // The two passes over a one-page block of bf16 rows held in registers: lane (hw, li) holds the 8 coordinates 8 li ..
 // of the key and value rows hw, hw + 2, ... (rows that do not exist: zeros, and they are skipped).  Leaves the mean
 // key (km), the value sums (vs) and this half warp's squared deviations (sq) for block_stats_finish.  Every caller
@@ -111,8 +136,9 @@ __device__ __forceinline__ void block_stats_rows16(const uint4 (&kraw)[8], const
 }
 
 // NC: the pools are read-only for the whole kernel (loads may use the non-coherent path).
+// ONEP: the caller's layout has one-page blocks of bf16 rows, and only that path is compiled (fewer registers).
 // sq_smem: 128 floats of shared memory owned by the calling warp.
-template <typename T, bool NC>
+template <typename T, bool NC, bool ONEP = false>
 __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__restrict__ k_pool,
                                                  const T *__restrict__ v_pool, const int *__restrict__ pt_row,
                                                  int h, int b, int cnt, float *sq_smem, __nv_bfloat16 *kmean_row,
@@ -159,6 +185,65 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
       }
     }
   }
+  if constexpr (sizeof(T) == 2 && !ONEP) {
+    if (!done) {
+      // Several pages of bf16 rows (32- and 64-token blocks): every page goes through the registers once -- its own
+      // two passes, as for a one-page block -- and is joined to the pages before it.  When the caller works on one
+      // block only (the append, the chunked prefill) the L2 is asked for all pages first, so that only the first one
+      // costs a DRAM round trip.  (The build kernel asks for its next block itself.)
+      done = true;
+      if constexpr (!NC) {
+        if (lane < npages) {
+          const int phys = pt_row[b * P.ppb + lane];
+          if (phys >= 0 && phys < P.num_pages) {
+            const size_t off = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D;
+            const unsigned bytes = CKV_PAGE * CKV_D * sizeof(T);
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(k_pool + off), "r"(bytes) : "memory");
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(v_pool + off), "r"(bytes) : "memory");
+          }
+        }
+      }
+      float na = 0.f, m2[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { km[i] = 0.f; m2[i] = 0.f; }
+#pragma unroll 1
+      for (int pg = 0; pg < npages; ++pg) {
+        const int phys = pt_row[b * P.ppb + pg];
+        if (phys < 0 || phys >= P.num_pages) { bad = true; continue; }
+        const size_t base = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+        const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+        const uint4 *kp = reinterpret_cast<const uint4 *>(k_pool + base + (size_t)hw * CKV_D);
+        const uint4 *vp = reinterpret_cast<const uint4 *>(v_pool + base + (size_t)hw * CKV_D);
+        constexpr int kStep = 2 * CKV_D / 8;
+        uint4 kraw[8], vraw[8];
+        float mb[8], vb[8], qb[8];
+        if (ntok == CKV_PAGE) {   // a full page: no per-row tests
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            kraw[j] = NC ? __ldg(kp + j * kStep) : kp[j * kStep];
+            vraw[j] = NC ? __ldg(vp + j * kStep) : vp[j * kStep];
+          }
+          block_stats_rows16<true>(kraw, vraw, true, CKV_PAGE, lane, mb, vb, qb);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const bool valid = hw + 2 * j < ntok;
+            const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+            kraw[j] = valid ? (NC ? __ldg(kp + j * kStep) : kp[j * kStep]) : zero;
+            vraw[j] = valid ? (NC ? __ldg(vp + j * kStep) : vp[j * kStep]) : zero;
+          }
+          block_stats_rows16(kraw, vraw, true, ntok, lane, mb, vb, qb);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) qb[i] += __shfl_xor_sync(0xffffffffu, qb[i], 16);
+        combine_pages(na, km, m2, vs, ntok, mb, qb, vb);
+      }
+      // block_stats_finish adds the two half warps' squared deviations: the joined ones are already complete
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sq[i] = hw == 0 ? m2[i] : 0.f;
+    }
+  }
+  if constexpr (sizeof(T) != 2) {
   if (!done) {
     if constexpr (!NC) {
       // A block of several pages (32- or 64-token blocks) is read page after page, twice: when the caller works on
@@ -215,6 +300,14 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
       }
     }
   }
+  }
+  if constexpr (ONEP) {
+    if (!done) {   // not a one-page block after all: nothing is read, the summary is marked bad
+      bad = true;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { km[i] = 0.f; sq[i] = 0.f; }
+    }
+  }
   block_stats_finish(P, b, fc, km, vs, sq, sq_smem, kmean_row, dbar_row, vmean_row, lane, bad);
 }
 
@@ -256,46 +349,97 @@ __device__ __forceinline__ void block_stats_warp_staged(const CkvDev &P, const T
     __syncwarp();
     return true;
   };
-#pragma unroll 1
-  for (int pg = 0; pg < npages; ++pg) {
-    if (!stage_page(pg, true)) { bad = true; continue; }
-    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
-#pragma unroll 1
-    for (int j = 0; j < 8; ++j) {
-      const int t = hw + 2 * j;
-      if (t < ntok) {
-        float a[8], c[8];
-        load8<false>(sk + t * CKV_D + 8 * li, a);
-        load8<false>(sv + t * CKV_D + 8 * li, c);
+  if constexpr (sizeof(T) == 2) {
+    // bf16 pages: every page is staged once and goes through its own two passes; several pages are joined as in
+    // block_stats_warp (same operations, same order, same bits)
+    float na = 0.f, m2[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+    for (int i = 0; i < 8; ++i) { km[i] = 0.f; m2[i] = 0.f; }
+#pragma unroll 1
+    for (int pg = 0; pg < npages; ++pg) {
+      if (!stage_page(pg, true)) { bad = true; continue; }
+      const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+      const float invp = 1.0f / (float)ntok;
+      float kb[8], vb[8], mb[8], qb[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { kb[i] = 0.f; vb[i] = 0.f; }
+#pragma unroll 1
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          float a[8], c[8];
+          load8<false>(sk + t * CKV_D + 8 * li, a);
+          load8<false>(sv + t * CKV_D + 8 * li, c);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { kb[i] += a[i]; vb[i] += c[i]; }
+        }
       }
-    }
-    __syncwarp();   // the stage may be overwritten
-  }
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
-    vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
-    km[i] = ks[i] * inv;
-    sq[i] = 0.f;
-  }
-#pragma unroll 1
-  for (int pg = 0; pg < npages; ++pg) {
-    if (npages > 1 && !stage_page(pg, false)) continue;   // a one-page block is still staged from the first pass
-    if (npages == 1 && bad) continue;
-    const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
-#pragma unroll 1
-    for (int j = 0; j < 8; ++j) {
-      const int t = hw + 2 * j;
-      if (t < ntok) {
-        float a[8];
-        load8<false>(sk + t * CKV_D + 8 * li, a);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+      for (int i = 0; i < 8; ++i) {
+        kb[i] += __shfl_xor_sync(0xffffffffu, kb[i], 16);
+        vb[i] += __shfl_xor_sync(0xffffffffu, vb[i], 16);
+        mb[i] = kb[i] * invp;
+        qb[i] = 0.f;
       }
+#pragma unroll 1
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          float a[8];
+          load8<false>(sk + t * CKV_D + 8 * li, a);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { const float dv = a[i] - mb[i]; qb[i] = fmaf(dv, dv, qb[i]); }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) qb[i] += __shfl_xor_sync(0xffffffffu, qb[i], 16);
+      combine_pages(na, km, m2, vs, ntok, mb, qb, vb);
+      __syncwarp();   // the stage may be overwritten
     }
-    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sq[i] = hw == 0 ? m2[i] : 0.f;
+  } else {
+#pragma unroll 1
+    for (int pg = 0; pg < npages; ++pg) {
+      if (!stage_page(pg, true)) { bad = true; continue; }
+      const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+#pragma unroll 1
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          float a[8], c[8];
+          load8<false>(sk + t * CKV_D + 8 * li, a);
+          load8<false>(sv + t * CKV_D + 8 * li, c);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { ks[i] += a[i]; vs[i] += c[i]; }
+        }
+      }
+      __syncwarp();   // the stage may be overwritten
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      ks[i] += __shfl_xor_sync(0xffffffffu, ks[i], 16);
+      vs[i] += __shfl_xor_sync(0xffffffffu, vs[i], 16);
+      km[i] = ks[i] * inv;
+      sq[i] = 0.f;
+    }
+#pragma unroll 1
+    for (int pg = 0; pg < npages; ++pg) {
+      if (npages > 1 && !stage_page(pg, false)) continue;   // a one-page block is still staged from the first pass
+      if (npages == 1 && bad) continue;
+      const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+#pragma unroll 1
+      for (int j = 0; j < 8; ++j) {
+        const int t = hw + 2 * j;
+        if (t < ntok) {
+          float a[8];
+          load8<false>(sk + t * CKV_D + 8 * li, a);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { const float dv = a[i] - km[i]; sq[i] = fmaf(dv, dv, sq[i]); }
+        }
+      }
+      __syncwarp();
+    }
   }
   block_stats_finish(P, b, fc, km, vs, sq, sq_smem, kmean_row, dbar_row, vmean_row, lane, bad);
 }

@@ -13,12 +13,13 @@ namespace {
 constexpr int kBuildRounds = 8;   // blocks per warp of the build kernel
 constexpr int kPrefillRounds = 4; // blocks per warp of the prefill kernel's register-resident variant
 
-// A warp takes kBuildRounds blocks, eight blocks apart.  Two CTAs per SM: the block routine holds a block's 16 key and
+// A warp takes kBuildRounds blocks, eight blocks apart.  Two CTAs per SM: the block routine holds a page's 16 key and
 // 16 value rows in registers, which does not fit three CTAs' register share without spills, and the kernel was bound
-// by instruction issue, not by DRAM, while it spilled.  With blocks of several pages (read page after page, twice) a
-// warp asks the L2 for the pages of its next block before it works on the current one; with one-page blocks the 16
-// warps of an SM keep enough rows in flight by themselves and the requests only cost instructions.
-template <typename T>
+// by instruction issue, not by DRAM, while it spilled.  The 16 warps of an SM keep enough rows in flight by
+// themselves: asking the L2 for a warp's next block ahead of time (which paid while the block routine was long) now
+// only costs instructions, and with blocks of several pages it cost a third of the time.
+// ONEP: one-page blocks of bf16 rows (the default layout), compiled without the other paths of the block routine.
+template <typename T, bool ONEP>
 __global__ void __launch_bounds__(256, 2) ckv_stats_build_kernel(CkvDev P, const T *__restrict__ k_pool,
                                                               const T *__restrict__ v_pool,
                                                               const int *__restrict__ page_table,
@@ -29,24 +30,14 @@ __global__ void __launch_bounds__(256, 2) ckv_stats_build_kernel(CkvDev P, const
   const int N = min(seq_lens[s], P.max_blocks * P.bs);
   const int X = (N + P.bs - 1) / P.bs;
   const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
-  constexpr unsigned kPageBytes = CKV_PAGE * CKV_D * sizeof(T);
 #pragma unroll 1
   for (int i = 0; i < kBuildRounds; ++i) {
     const int b = (blockIdx.x * kBuildRounds + i) * 8 + warp;
     if (b >= X) return;
-    const int bn = b + 8;
-    if (P.ppb > 1 && i + 1 < kBuildRounds && bn < X && lane < P.ppb && bn * P.bs + lane * CKV_PAGE < N) {
-      const int phys = pt_row[bn * P.ppb + lane];
-      if (phys >= 0 && phys < P.num_pages) {
-        const size_t off = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D;
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(k_pool + off), "r"(kPageBytes) : "memory");
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(v_pool + off), "r"(kPageBytes) : "memory");
-      }
-    }
     const int cnt = min(P.bs, N - b * P.bs);
     const size_t row = (size_t)unit * P.max_blocks + b;
-    block_stats_warp<T, true>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * P.row_elems,
-                              P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
+    block_stats_warp<T, true, ONEP>(P, k_pool, v_pool, pt_row, h, b, cnt, sq_smem[warp], P.kmean + row * P.row_elems,
+                                    P.dbar + row * P.r, P.vmean + row * P.row_elems, lane);
   }
 }
 
@@ -104,9 +95,10 @@ __global__ void __launch_bounds__(256) ckv_append_kernel(CkvDev P, T *k_pool, T 
 // block's new rows into their pages and then runs the block routine over the block (rows that were already in the
 // cache included), so the new keys and values cross DRAM once on the way in and the summaries come out of the same
 // pass.  The CTA that finishes last stores the new sequence lengths (every warp read the old ones when it started).
-// ONE: one-page blocks of bf16 rows (the default layout), the variant whose rows never leave the registers.
-template <typename T, bool ONE>
-__global__ void __launch_bounds__(256, ONE ? 2 : 1) ckv_prefill_kernel(CkvDev P, T *k_pool, T *v_pool,
+// REG: 1 = one-page blocks of bf16 rows (the default layout), 2 = bf16 blocks of several pages: the variants whose
+// rows never leave the registers; 0 = the general form (fp32 pages).
+template <typename T, int REG>
+__global__ void __launch_bounds__(256, REG ? 2 : 1) ckv_prefill_kernel(CkvDev P, T *k_pool, T *v_pool,
                                                           const int *__restrict__ page_table, int *seq_lens,
                                                           const T *__restrict__ k_src, const T *__restrict__ v_src,
                                                           const int *__restrict__ new_lens, int src_stride, int batch) {
@@ -119,31 +111,31 @@ __global__ void __launch_bounds__(256, ONE ? 2 : 1) ckv_prefill_kernel(CkvDev P,
   if (M > m_eff && blockIdx.x == 0 && threadIdx.x == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
   // the register-resident variant gives a warp kPrefillRounds blocks, eight blocks apart (L2 requests for the next
   // block's rows ahead of time made it slower once the block routine had been trimmed: 763 against 728 us)
-  constexpr int kRounds = ONE ? kPrefillRounds : 1;
+  constexpr int kRounds = REG ? kPrefillRounds : 1;
 #pragma unroll 1
   for (int rnd = 0; rnd < kRounds; ++rnd) {
   const int b = (N >= 0 ? N / P.bs : 0) + (blockIdx.x * kRounds + rnd) * 8 + warp;
   if (m_eff > 0 && b <= (N + m_eff - 1) / P.bs) {
     const int *pt_row = page_table + (size_t)s * P.max_pages_per_seq;
     const int p_lo = max(b * P.bs, N), p_hi = min((b + 1) * P.bs, N + m_eff);
-    bool handled = false;
-    if constexpr (ONE) {
-      {
-        // One-page blocks of bf16 rows (the default layout): the rows go from the chunk into registers in the
-        // layout the block routine works in (rows of the block that were already in the cache come from the page),
-        // the new ones are stored to the page, and the summaries are worked out from the registers -- the chunk
-        // crosses DRAM once and nothing is read back.
-        handled = true;
-        const int hw = lane >> 4, li = lane & 15;
-        const int phys = pt_row[b];
-        const bool ok = phys >= 0 && phys < P.num_pages;
-        const int cnt = min(P.bs, N + m_eff - b * P.bs);
-        const size_t pbase = ok ? ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li : 0;
+    if constexpr (REG != 0) {
+      // bf16 rows: the rows of a page go from the chunk into registers in the layout the block routine works in (rows
+      // of the block that were already in the cache come from the page), the new ones are stored to the page, and the
+      // summaries are worked out from the registers -- the chunk crosses DRAM once and nothing is read back.  A block of
+      // several pages is joined page by page, exactly as the block routine does it (same bits).
+      const int hw = lane >> 4, li = lane & 15;
+      const int cnt = min(P.bs, N + m_eff - b * P.bs);
+      bool bad = false;
+      // page pg of the block: its mean key, value sums and this half warp's squared deviations; false: bad page id
+      auto page = [&](int pg, int ntok, float (&mb)[8], float (&vb)[8], float (&qb)[8]) -> bool {
+        const int phys = pt_row[b * P.ppb + pg];
+        if (phys < 0 || phys >= P.num_pages) return false;
+        const size_t pbase = ((size_t)phys * P.Hkv + h) * CKV_PAGE * CKV_D + 8 * li;
+        const int pfirst = b * P.bs + pg * CKV_PAGE;   // position of the page's first row
         uint4 kraw[8], vraw[8];
-        float km[8], vs[8], sq[8];
-        if (ok && cnt == CKV_PAGE && p_lo == b * CKV_PAGE) {
-          // a full block made of new rows only (all but the first and last touched block): no per-row tests
-          const size_t so = (((size_t)s * src_stride + (p_lo + hw - N)) * P.Hkv + h) * CKV_D + 8 * li;
+        if (ntok == CKV_PAGE && pfirst >= N) {
+          // a full page made of new rows only (all but the first and last touched page): no per-row tests
+          const size_t so = (((size_t)s * src_stride + (pfirst + hw - N)) * P.Hkv + h) * CKV_D + 8 * li;
           const size_t sstep = (size_t)2 * P.Hkv * CKV_D;   // two chunk rows on
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -155,40 +147,65 @@ __global__ void __launch_bounds__(256, ONE ? 2 : 1) ckv_prefill_kernel(CkvDev P,
             *reinterpret_cast<uint4 *>(k_pool + pbase + (size_t)(hw + 2 * j) * CKV_D) = kraw[j];
             *reinterpret_cast<uint4 *>(v_pool + pbase + (size_t)(hw + 2 * j) * CKV_D) = vraw[j];
           }
-          block_stats_rows16<true>(kraw, vraw, true, CKV_PAGE, lane, km, vs, sq);
+          block_stats_rows16<true>(kraw, vraw, true, CKV_PAGE, lane, mb, vb, qb);
         } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int t = hw + 2 * j, p = b * CKV_PAGE + t;
-          const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-          kraw[j] = zero; vraw[j] = zero;
-          if (ok && t < cnt) {
-            if (p >= p_lo) {
-              const size_t so = (((size_t)s * src_stride + (p - N)) * P.Hkv + h) * CKV_D + 8 * li;
-              kraw[j] = __ldg(reinterpret_cast<const uint4 *>(k_src + so));
-              vraw[j] = __ldg(reinterpret_cast<const uint4 *>(v_src + so));
-            } else {
-              kraw[j] = *reinterpret_cast<const uint4 *>(k_pool + pbase + (size_t)t * CKV_D);
-              vraw[j] = *reinterpret_cast<const uint4 *>(v_pool + pbase + (size_t)t * CKV_D);
+          for (int j = 0; j < 8; ++j) {
+            const int t = hw + 2 * j, p = pfirst + t;
+            const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+            kraw[j] = zero; vraw[j] = zero;
+            if (t < ntok) {
+              if (p >= p_lo) {
+                const size_t so = (((size_t)s * src_stride + (p - N)) * P.Hkv + h) * CKV_D + 8 * li;
+                kraw[j] = __ldg(reinterpret_cast<const uint4 *>(k_src + so));
+                vraw[j] = __ldg(reinterpret_cast<const uint4 *>(v_src + so));
+              } else {
+                kraw[j] = *reinterpret_cast<const uint4 *>(k_pool + pbase + (size_t)t * CKV_D);
+                vraw[j] = *reinterpret_cast<const uint4 *>(v_pool + pbase + (size_t)t * CKV_D);
+              }
             }
           }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int t = hw + 2 * j, p = pfirst + t;
+            if (t < ntok && p >= p_lo) {
+              *reinterpret_cast<uint4 *>(k_pool + pbase + (size_t)t * CKV_D) = kraw[j];
+              *reinterpret_cast<uint4 *>(v_pool + pbase + (size_t)t * CKV_D) = vraw[j];
+            }
+          }
+          block_stats_rows16(kraw, vraw, true, ntok, lane, mb, vb, qb);
+        }
+        return true;
+      };
+      float km[8], vs[8], sq[8];
+      if constexpr (REG == 1) {   // one-page blocks (the default layout)
+        if (!page(0, cnt, km, vs, sq)) {
+          bad = true;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { km[i] = 0.f; vs[i] = 0.f; sq[i] = 0.f; }
+        }
+      } else {
+        float na = 0.f, m2[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { km[i] = 0.f; vs[i] = 0.f; m2[i] = 0.f; }
+        const int npages = (cnt + CKV_PAGE - 1) / CKV_PAGE;
+#pragma unroll 1
+        for (int pg = 0; pg < npages; ++pg) {
+          const int ntok = min(CKV_PAGE, cnt - pg * CKV_PAGE);
+          float mb[8], vb[8], qb[8];
+          if (!page(pg, ntok, mb, vb, qb)) { bad = true; continue; }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) qb[i] += __shfl_xor_sync(0xffffffffu, qb[i], 16);
+          combine_pages(na, km, m2, vs, ntok, mb, qb, vb);
         }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int t = hw + 2 * j, p = b * CKV_PAGE + t;
-          if (ok && t < cnt && p >= p_lo) {
-            *reinterpret_cast<uint4 *>(k_pool + pbase + (size_t)t * CKV_D) = kraw[j];
-            *reinterpret_cast<uint4 *>(v_pool + pbase + (size_t)t * CKV_D) = vraw[j];
-          }
-        }
-        block_stats_rows16(kraw, vraw, ok, cnt, lane, km, vs, sq);
-        }
-        const size_t row = (size_t)unit * P.max_blocks + b;
-        block_stats_finish(P, b, (float)cnt, km, vs, sq, sq_smem[warp], P.kmean + row * P.row_elems, P.dbar + row * P.r,
-                           P.vmean + row * P.row_elems, lane, !ok);
+        for (int i = 0; i < 8; ++i) sq[i] = hw == 0 ? m2[i] : 0.f;
       }
+      const size_t row = (size_t)unit * P.max_blocks + b;
+      block_stats_finish(P, b, (float)cnt, km, vs, sq, sq_smem[warp], P.kmean + row * P.row_elems, P.dbar + row * P.r,
+                         P.vmean + row * P.row_elems, lane, bad);
     }
-    if constexpr (!ONE) {
+    if constexpr (REG == 0) {
     constexpr int PIECES = (int)(CKV_D * sizeof(T) / 16);   // 16-byte pieces of a row: 16 (bf16) or 32 (fp32)
     constexpr int PP = PIECES / 16;                          // pieces per lane and row
     bool bad = false;
@@ -279,12 +296,15 @@ cudaError_t ckv_launch_stats_build(ckv_ctx *c, const void *k_pool, const void *v
   const int xmax = (max_len + P.bs - 1) / P.bs;
   if (xmax <= 0 || batch <= 0) return cudaSuccess;
   dim3 grid((xmax + 8 * kBuildRounds - 1) / (8 * kBuildRounds), batch * P.Hkv);
-  if (c->layout.kv_dtype == CKV_BF16)
-    ckv_stats_build_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16 *)k_pool,
-                                                                (const __nv_bfloat16 *)v_pool, page_table, seq_lens);
+  if (c->layout.kv_dtype == CKV_BF16 && P.ppb == 1)
+    ckv_stats_build_kernel<__nv_bfloat16, true><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16 *)k_pool,
+                                                                      (const __nv_bfloat16 *)v_pool, page_table, seq_lens);
+  else if (c->layout.kv_dtype == CKV_BF16)
+    ckv_stats_build_kernel<__nv_bfloat16, false><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16 *)k_pool,
+                                                                       (const __nv_bfloat16 *)v_pool, page_table, seq_lens);
   else
-    ckv_stats_build_kernel<float><<<grid, 256, 0, st>>>(P, (const float *)k_pool, (const float *)v_pool, page_table,
-                                                        seq_lens);
+    ckv_stats_build_kernel<float, false><<<grid, 256, 0, st>>>(P, (const float *)k_pool, (const float *)v_pool, page_table,
+                                                               seq_lens);
   c->launches++;
   return cudaGetLastError();
 }
@@ -298,15 +318,15 @@ cudaError_t ckv_launch_prefill(ckv_ctx *c, void *k_pool, void *v_pool, const int
   dim3 grid((touched + 7) / 8, batch * P.Hkv);
   const dim3 grid_one((touched + 8 * kPrefillRounds - 1) / (8 * kPrefillRounds), batch * P.Hkv);
   if (c->layout.kv_dtype == CKV_BF16 && P.ppb == 1)
-    ckv_prefill_kernel<__nv_bfloat16, true><<<grid_one, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
+    ckv_prefill_kernel<__nv_bfloat16, 1><<<grid_one, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
                                                                   page_table, seq_lens, (const __nv_bfloat16 *)k_src,
                                                                   (const __nv_bfloat16 *)v_src, new_lens, src_stride, batch);
   else if (c->layout.kv_dtype == CKV_BF16)
-    ckv_prefill_kernel<__nv_bfloat16, false><<<grid, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
+    ckv_prefill_kernel<__nv_bfloat16, 2><<<grid_one, 256, 0, st>>>(P, (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
                                                                    page_table, seq_lens, (const __nv_bfloat16 *)k_src,
                                                                    (const __nv_bfloat16 *)v_src, new_lens, src_stride, batch);
   else
-    ckv_prefill_kernel<float, false><<<grid, 256, 0, st>>>(P, (float *)k_pool, (float *)v_pool, page_table, seq_lens,
+    ckv_prefill_kernel<float, 0><<<grid, 256, 0, st>>>(P, (float *)k_pool, (float *)v_pool, page_table, seq_lens,
                                                     (const float *)k_src, (const float *)v_src, new_lens, src_stride, batch);
   c->launches++;
   return cudaGetLastError();
