@@ -139,7 +139,8 @@ void ckv_destroy(ckv_ctx *ctx);
 
 /* Build the summaries of every block of `batch` prefilled sequences from the paged cache
  * (Eq. 8 right half; Sec. 4.2): |b|, mean key, mean value and, per coordinate group, the
- * population variance of the keys around the block mean (two passes, fp32 accumulation).
+ * population variance of the keys around the block mean (fp32: two passes over each 16-token page, mean first and
+ * deviations from it second; the pages of a longer block are joined with the pairwise update of Chan et al.).
  * Sequence s of this call uses summary rows of batch slot s.
  * max_seq_len_host: an upper bound (host) on seq_lens[s], used only to size the grid. */
 int ckv_stats_build(ckv_ctx *ctx, const void *k_pool, const void *v_pool, const int32_t *page_table,

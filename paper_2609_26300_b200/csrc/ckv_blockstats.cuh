@@ -155,8 +155,7 @@ __device__ __forceinline__ void block_stats_warp(const CkvDev &P, const T *__res
   if constexpr (sizeof(T) == 2) {
     if (npages == 1) {
       // One page of bf16 rows (every block of the default 16-token layout): the key rows stay in registers between
-      // the two passes, so the cache is read exactly once.  Same operations in the same order as the general path
-      // below (rows that do not exist contribute exact zeros), hence the same bits.
+      // the two passes, so the cache is read exactly once.
       done = true;
       const int phys = pt_row[b * P.ppb];
       const bool ok = phys >= 0 && phys < P.num_pages;

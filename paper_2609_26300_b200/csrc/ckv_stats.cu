@@ -3,8 +3,9 @@
 // One warp owns one block.  A token row (128 elements) is spread over the 16 lanes of a half
 // warp, 8 consecutive coordinates per lane (one 16-byte load for bf16); the two half warps take
 // alternate rows.  Means and squared deviations are accumulated in fp32 in two passes (mean
-// first, then deviations from it), the second pass re-reading the rows it just touched.
-// Build and append call the same routine, so their results are bit-identical.
+// first, then deviations from it) over a page of rows held in registers; the pages of a longer
+// block are joined pairwise (ckv_blockstats.cuh).  Build, append and chunked prefill run the same
+// operations in the same order, so their results are bit-identical.
 #include "ckv_internal.cuh"
 #include "ckv_blockstats.cuh"
 
