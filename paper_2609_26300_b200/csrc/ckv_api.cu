@@ -169,6 +169,8 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.comp_part = (float *)(wb + R.comp); P.attn_part = (float *)(wb + R.attn);
   P.spin_limit = ckv_pipe::kSpinLimit; P.debug = 0;
   P.scan_tile = layout->stat_bf16 ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE;
+  P.lg_bs = P.bs == 16 ? 4 : (P.bs == 32 ? 5 : 6);
+  P.lg_tile = P.scan_tile == 32 ? 5 : 6;
   c->work = wb; c->work_bytes = work_bytes;
   c->stage_q = R.stage_q; c->stage_knew = R.stage_knew; c->stage_vnew = R.stage_vnew;
   c->stage_out = R.stage_out; c->stage_ids = R.stage_ids; c->stage_cnt = R.stage_cnt;

@@ -95,7 +95,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     if (i < kcap * P.ppb) blk0 = sel_ids[(size_t)unit * kcap + (i >> pshift)];
   }
   const int N = max(min(n_raw, P.max_blocks * P.bs), 0);
-  const int X = (N + P.bs - 1) / P.bs;
+  const int X = (N + P.bs - 1) >> P.lg_bs;
   const int nsel = DENSE ? X : min(cnt_raw, kcap);
   const int total = DENSE ? (N + CKV_PAGE - 1) / CKV_PAGE : nsel * P.ppb;
   const bool comp = !DENSE && nsel < X && !(P.variant & CKV_VARIANT_DROP);

@@ -42,6 +42,9 @@ struct CkvDev {
   int variant;       // ckv_variant bits
   float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
   int scan_tile;     // blocks per scan tile: CKV_SCAN_TILE, or CKV_SCAN_TILE_HS with bf16 summaries
+  int lg_bs, lg_tile;  // log2 of bs and of scan_tile (both powers of two): the kernels' prologues divide by shifting --
+                       // a division by a run-time value is two dozen instructions, and a prologue's time is the fetch of its
+                       // own cold instructions
   int tail;          // 1: the scan launch leaves the last block of every sequence to its tail CTAs (set per step)
   int *unit_done;    // [unit] attention splits finished this step (zero between steps); null = merge is a separate launch
   int *status;       // device status word
@@ -313,7 +316,7 @@ __device__ __forceinline__ float exp2_diff(float a, float b) {
 // sequence (the one a new token lands in) to the launch's tail CTAs, whose partial takes the first entry of that
 // free group.  Either way a unit's entries are contiguous: `first`, and `count` of them (zero for an empty sequence).
 // len_of(i) is the clamped length of sequence i.  Must be called by all 32 lanes of a warp; every lane gets the result.
-__device__ __forceinline__ int ckv_scan_blocks(int n, int bs, int tail) { return max((n + bs - 1) / bs - tail, 0); }
+__device__ __forceinline__ int ckv_scan_blocks(const CkvDev &P, int n) { return max(((n + P.bs - 1) >> P.lg_bs) - P.tail, 0); }   // n >= 0
 template <class LenFn>
 __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of, int units, int unit, int scan_grid,
                                                   int lane, int &first, int &count) {
@@ -321,7 +324,7 @@ __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of,
   unsigned tot = 0, before = 0, mine = 0, n_mine = 0;
   for (int i = lane; i < batch; i += 32) {
     const int n = len_of(i);
-    const unsigned t = (unsigned)((ckv_scan_blocks(n, P.bs, P.tail) + P.scan_tile - 1) / P.scan_tile);
+    const unsigned t = (unsigned)((ckv_scan_blocks(P, n) + P.scan_tile - 1) >> P.lg_tile);
     tot += t;
     if (i < s) before += t;
     if (i == s) { mine = t; n_mine = (unsigned)n; }

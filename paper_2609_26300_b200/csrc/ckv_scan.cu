@@ -61,13 +61,13 @@ __device__ __forceinline__ int seq_len_of(const CkvDev &P, const int *s_len, con
 __device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *s_len, const int *__restrict__ seq_lens, int u) {
   UnitInfo ui;
   ui.N = seq_len_of(P, s_len, seq_lens, u / P.Hkv);
-  ui.X = ckv_scan_blocks(ui.N, P.bs, P.tail);
-  ui.tiles = (ui.X + P.scan_tile - 1) / P.scan_tile;
+  ui.X = ckv_scan_blocks(P, ui.N);
+  ui.tiles = (ui.X + P.scan_tile - 1) >> P.lg_tile;
   return ui;
 }
 
 __device__ __forceinline__ int seq_tiles(const int *s_len, const int *__restrict__ seq_lens, const CkvDev &P, int i) {
-  return (ckv_scan_blocks(seq_len_of(P, s_len, seq_lens, i), P.bs, P.tail) + P.scan_tile - 1) / P.scan_tile;
+  return (ckv_scan_blocks(P, seq_len_of(P, s_len, seq_lens, i)) + P.scan_tile - 1) >> P.lg_tile;
 }
 
 constexpr int kLenCounter = 16;   // word of the status region that counts the CTAs which have read the lengths
@@ -132,11 +132,11 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
   const int u_first = (int)blockIdx.x * 8 + warp;
   // the new row of the warp's first unit does not depend on the lengths: it is requested together with them
   uint4 piece[PP];
-  float qx[G][8];   // this lane's 8 coordinates of the unit's G query rows (rows u G .. u G + G - 1): also independent of the lengths
-  if (u_first < units) {
-#pragma unroll
-    for (int g = 0; g < G; ++g) load8<true>(q + ((size_t)u_first * G + g) * CKV_D + 8 * li, qx[g]);
-  }
+  // the unit's G query rows are read head by head in a rolled loop further down (this routine's time is the fetch
+  // of its own instructions, executed once per launch: a short loop beats unrolled code); the L2 is asked for them
+  // now, while nothing depends on them
+  if (u_first < units && lane < G)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(q + ((size_t)u_first * G + lane) * CKV_D) : "memory");
   if (append && u_first < units) {
     const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + (size_t)u_first * CKV_D);
 #pragma unroll
@@ -148,21 +148,30 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
   __syncthreads();
   auto len_of = [&](int i) { return seq_len_of(P, s_len, seq_lens, i); };
 
+  // The length before the append, from the staged (already incremented and clamped) one; the device array is only
+  // asked where that is ambiguous (an empty or exactly full sequence).
+  auto raw_len = [&](int sq_idx) {
+    const int eff = len_of(sq_idx);
+    return (eff > 0 && eff < cap && sq_idx < kMaxSeqs) ? eff - 1 : seq_lens[sq_idx];
+  };
 #pragma unroll 1
   for (int u = u_first; u < units; u += n_tail * 8) {
     const int s = u / P.Hkv, h = u % P.Hkv;
-    if (u != u_first) {
-#pragma unroll
-      for (int g = 0; g < G; ++g) load8<true>(q + ((size_t)u * G + g) * CKV_D + 8 * li, qx[g]);
-    }
+    const int *pt_row = fresh.page_table + (size_t)s * P.max_pages_per_seq;
+    const int raw = append ? raw_len(s) : -1;
+    const bool room = raw >= 0 && raw < cap;
+    int phys = -1;
+    // the page of the new token is asked for first, and the unit's place among the scan partials (which depends on
+    // the lengths only) is worked out while that entry is on its way
+    if (append && room) phys = pt_row[raw / CKV_PAGE];
+    int first = 0, count = 0;
+    unit_scan_entries(P, len_of, units, u, nscan, lane, first, count);
     if (append) {
-      const int raw = seq_lens[s];
-      if (raw < 0 || raw >= cap) {
+      if (!room) {
         if (lane == 0) atomicOr(P.status, CKV_DEV_SEQ_FULL);
       } else {
-        const int *pt_row = fresh.page_table + (size_t)s * P.max_pages_per_seq;
-        const int phys = pt_row[raw / CKV_PAGE], slot = raw % CKV_PAGE;
-        const int b = raw / P.bs, cnt = raw + 1 - b * P.bs;
+        const int slot = raw % CKV_PAGE;
+        const int b = raw >> P.lg_bs, cnt = raw + 1 - b * P.bs;
         if (phys >= 0 && phys < P.num_pages) {
           if (u != u_first) {
             const uint4 *src = reinterpret_cast<const uint4 *>((lane < 16 ? k_new : v_new) + (size_t)u * CKV_D);
@@ -189,7 +198,7 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
     }
     const int N = len_of(s);
     if (N == 0) continue;   // warp-uniform
-    const int b = (N + P.bs - 1) / P.bs - 1, cnt = N - b * P.bs;
+    const int b = ((N + P.bs - 1) >> P.lg_bs) - 1, cnt = N - b * P.bs;
     const size_t row = (size_t)u * P.max_blocks + b;
     __syncwarp();
     float kx[8], vx[8], dx[8];   // this lane's 8 coordinates of kbar, vbar and of the variance of their group
@@ -207,17 +216,17 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
         dx[i] = drow[P.glayout == 0 ? c >> sh : (c & (CKV_D / 2 - 1)) >> (sh - 1)];
       }
     }
-    int first = 0, count = 0;
-    unit_scan_entries(P, len_of, units, u, nscan, lane, first, count);
     float *part = P.comp_part + (size_t)(first + count - 1) * G * CKV_PART_STRIDE;
     const float logc = logf((float)cnt);
-#pragma unroll
+#pragma unroll 1
     for (int g = 0; g < G; ++g) {
+      float qx[8];   // this lane's 8 coordinates of query row u G + g
+      load8<true>(q + ((size_t)u * G + g) * CKV_D + 8 * li, qx);
       float d = 0.f, sg = 0.f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        d = fmaf(qx[g][i], kx[i], d);
-        const float qs = qx[g][i] * P.scale;
+        d = fmaf(qx[i], kx[i], d);
+        const float qs = qx[i] * P.scale;
         sg = fmaf(qs * qs, dx[i], sg);   // Eq. 8: the squared logit scale is its 1/d
       }
 #pragma unroll

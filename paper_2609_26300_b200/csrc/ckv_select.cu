@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = blockIdx.x, s = unit / P.Hkv;
   const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
-  const int X = (N + P.bs - 1) / P.bs;
+  const int X = (N + P.bs - 1) >> P.lg_bs;
   int *ids = sel_ids + (size_t)unit * kcap;
   const int K = min(kcap, X);
   if (X <= kcap) {   // every block is selected: the step is dense attention

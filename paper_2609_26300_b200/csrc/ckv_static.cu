@@ -62,6 +62,8 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
   P.row_elems = layout->stat_bf16 ? CKV_D : CKV_ROW_ELEMS;
   P.variant = layout->variant; P.half_var = 0.5f;   // the dense pass reads neither
   P.scan_tile = layout->stat_bf16 ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE;
+  P.lg_bs = P.bs == 16 ? 4 : (P.bs == 32 ? 5 : 6);
+  P.lg_tile = P.scan_tile == 32 ? 5 : 6;
 
   // the partials of the largest split count the launch heuristic may pick must fit the fixed array
   const size_t per_split = (size_t)batch * P.Hkv * P.G * CKV_PART_STRIDE * sizeof(float);
