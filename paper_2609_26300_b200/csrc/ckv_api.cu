@@ -32,9 +32,11 @@ int check_layout(const ckv_layout *L) {
   if (!(L->sm_scale >= 0.f) || !isfinite(L->sm_scale)) return CKV_ERR_BAD_LAYOUT;
   if (L->variant & ~(CKV_VARIANT_FIRST_ORDER_MASS | CKV_VARIANT_RANK_BY_MASS | CKV_VARIANT_DROP)) return CKV_ERR_BAD_LAYOUT;
   if (L->stat_bf16 != 0 && L->stat_bf16 != 1) return CKV_ERR_BAD_LAYOUT;
-  // the kernels count the scan tiles (32 blocks each) of a whole step in 32 bits
-  if ((long long)L->max_batch * L->num_kv_heads * ((L->max_blocks_per_seq + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE) >= (1ll << 30))
+  // the kernels divide the count of a step's scan tiles (32 blocks each) with a float reciprocal that is exact below
+  // 2^24 (those many tiles would be half a terabyte of summaries), and unit indices by a multiplication
+  if ((long long)L->max_batch * L->num_kv_heads * ((L->max_blocks_per_seq + CKV_SCAN_TILE - 1) / CKV_SCAN_TILE) >= (1ll << 24))
     return CKV_ERR_BAD_LAYOUT;
+  if ((long long)L->max_batch * L->num_kv_heads * L->num_kv_heads >= (1ll << 32)) return CKV_ERR_BAD_LAYOUT;
   if (L->stat_bf16 == 1 && (L->kv_dtype != CKV_BF16 || L->var_groups == CKV_D)) return CKV_ERR_BAD_LAYOUT;
   return CKV_OK;
 }
@@ -171,6 +173,7 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.scan_tile = layout->stat_bf16 ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE;
   P.lg_bs = P.bs == 16 ? 4 : (P.bs == 32 ? 5 : 6);
   P.lg_tile = P.scan_tile == 32 ? 5 : 6;
+  P.hkv_magic = (unsigned)((1ull << 32) / (unsigned)P.Hkv) + 1u;   // unused when Hkv == 1 (where it wraps)
   c->work = wb; c->work_bytes = work_bytes;
   c->stage_q = R.stage_q; c->stage_knew = R.stage_knew; c->stage_vnew = R.stage_vnew;
   c->stage_out = R.stage_out; c->stage_ids = R.stage_ids; c->stage_cnt = R.stage_cnt;

@@ -82,7 +82,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int head = lane >> 2, qd = lane & 3;
   const bool hv = head < G;
-  const int unit = blockIdx.y, s = unit / P.Hkv, h = unit % P.Hkv;
+  const int unit = blockIdx.y, s = ckv_div_hkv(P, unit), h = unit - s * P.Hkv;
   const int pshift = P.ppb == 1 ? 0 : (P.ppb == 2 ? 1 : 2);
   const int p0 = blockIdx.x * pages_per_split;
 

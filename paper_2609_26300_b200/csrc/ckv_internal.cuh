@@ -42,6 +42,7 @@ struct CkvDev {
   int variant;       // ckv_variant bits
   float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
   int scan_tile;     // blocks per scan tile: CKV_SCAN_TILE, or CKV_SCAN_TILE_HS with bf16 summaries
+  unsigned hkv_magic;  // floor(2^32 / Hkv) + 1: x / Hkv = umulhi(x, hkv_magic) for x < 2^32 / Hkv (ckv_div_hkv)
   int lg_bs, lg_tile;  // log2 of bs and of scan_tile (both powers of two): the kernels' prologues divide by shifting --
                        // a division by a run-time value is two dozen instructions, and a prologue's time is the fetch of its
                        // own cold instructions
@@ -316,11 +317,27 @@ __device__ __forceinline__ float exp2_diff(float a, float b) {
 // sequence (the one a new token lands in) to the launch's tail CTAs, whose partial takes the first entry of that
 // free group.  Either way a unit's entries are contiguous: `first`, and `count` of them (zero for an empty sequence).
 // len_of(i) is the clamped length of sequence i.  Must be called by all 32 lanes of a warp; every lane gets the result.
+//
+// The divisions of this arithmetic are done without the division instruction sequence (about 25 instructions each, and
+// a kernel's prologue costs what its cold instructions cost to fetch):
+// x / Hkv for unit indices (x * Hkv < 2^32, checked at creation) by a multiplication with a host-made constant;
+__device__ __forceinline__ int ckv_div_hkv(const CkvDev &P, int x) {
+  return P.Hkv == 1 ? x : (int)__umulhi((unsigned)x, P.hkv_magic);
+}
+// a / b for tile counts (a, b < 2^24, b >= 1: a step has fewer than 2^24 tiles, checked at creation) by a float
+// reciprocal, exact in both operands, whose quotient is then put right by its remainder.
+__device__ __forceinline__ unsigned ckv_udiv24(unsigned a, unsigned b) {
+  unsigned q = (unsigned)__fdividef((float)a, (float)b);
+  int r = (int)a - (int)(q * b);
+  while (r < 0) { --q; r += (int)b; }
+  while (r >= (int)b) { ++q; r -= (int)b; }
+  return q;
+}
 __device__ __forceinline__ int ckv_scan_blocks(const CkvDev &P, int n) { return max(((n + P.bs - 1) >> P.lg_bs) - P.tail, 0); }   // n >= 0
 template <class LenFn>
 __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of, int units, int unit, int scan_grid,
                                                   int lane, int &first, int &count) {
-  const int batch = units / P.Hkv, s = unit / P.Hkv, h = unit % P.Hkv;
+  const int batch = ckv_div_hkv(P, units), s = ckv_div_hkv(P, unit), h = unit - s * P.Hkv;
   unsigned tot = 0, before = 0, mine = 0, n_mine = 0;
   for (int i = lane; i < batch; i += 32) {
     const int n = len_of(i);
@@ -333,11 +350,10 @@ __device__ __forceinline__ void unit_scan_entries(const CkvDev &P, LenFn len_of,
   before = __reduce_add_sync(0xffffffffu, before);
   mine = __reduce_add_sync(0xffffffffu, mine);
   n_mine = __reduce_add_sync(0xffffffffu, n_mine);
-  // 32-bit arithmetic: ckv_create refuses layouts whose tiles per step would not fit (2^30)
   const unsigned T = tot * (unsigned)P.Hkv, T0 = before * (unsigned)P.Hkv + (unsigned)h * mine;
-  const unsigned tpc = max((T + (unsigned)scan_grid - 1u) / (unsigned)scan_grid, 1u);
-  const int cfirst = (int)(T0 / tpc);
-  const int ccount = mine == 0 ? 0 : (int)((T0 + mine - 1u) / tpc) - cfirst + 1;
+  const unsigned tpc = max(ckv_udiv24(T + (unsigned)scan_grid - 1u, (unsigned)scan_grid), 1u);
+  const int cfirst = (int)ckv_udiv24(T0, tpc);
+  const int ccount = mine == 0 ? 0 : (int)ckv_udiv24(T0 + mine - 1u, tpc) - cfirst + 1;
   first = (cfirst + 2 * unit) * CKV_SCAN_WARPS;
   count = ccount * CKV_SCAN_WARPS + ((P.tail && n_mine > 0) ? 1 : 0);
 }

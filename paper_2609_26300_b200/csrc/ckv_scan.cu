@@ -60,7 +60,7 @@ __device__ __forceinline__ int seq_len_of(const CkvDev &P, const int *s_len, con
 }
 __device__ __forceinline__ UnitInfo unit_info(const CkvDev &P, const int *s_len, const int *__restrict__ seq_lens, int u) {
   UnitInfo ui;
-  ui.N = seq_len_of(P, s_len, seq_lens, u / P.Hkv);
+  ui.N = seq_len_of(P, s_len, seq_lens, ckv_div_hkv(P, u));
   ui.X = ckv_scan_blocks(P, ui.N);
   ui.tiles = (ui.X + P.scan_tile - 1) >> P.lg_tile;
   return ui;
@@ -120,7 +120,7 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
                                        int len_mine, int units, int nscan, const CkvNewToken fresh, int n_tail,
                                        float *smem_f, int smem_bytes) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, hw = lane >> 4, li = lane & 15;
-  const int batch = units / P.Hkv, cap = P.max_blocks * P.bs;
+  const int batch = ckv_div_hkv(P, units), cap = P.max_blocks * P.bs;
   const bool append = fresh.k_new != nullptr;
   const bool lo_half = P.row_elems == CKV_ROW_ELEMS;
   const bool by_mass = (P.variant & CKV_VARIANT_RANK_BY_MASS) != 0;
@@ -156,7 +156,7 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
   };
 #pragma unroll 1
   for (int u = u_first; u < units; u += n_tail * 8) {
-    const int s = u / P.Hkv, h = u % P.Hkv;
+    const int s = ckv_div_hkv(P, u), h = u - s * P.Hkv;
     const int *pt_row = fresh.page_table + (size_t)s * P.max_pages_per_seq;
     const int raw = append ? raw_len(s) : -1;
     const bool room = raw >= 0 && raw < cap;
@@ -287,7 +287,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   float *sw_all = reinterpret_cast<float *>(stage_mem + (size_t)stages * stage_bytes);
 
   // the sequence lengths are requested first; the ring is cleared while they are on their way
-  const int batch = units / P.Hkv;
+  const int batch = ckv_div_hkv(P, units);
   const bool append = fresh.k_new != nullptr;
   const int cap = P.max_blocks * P.bs;
   // length the step works on: one more than stored when a token is being appended (a full sequence keeps its length)
@@ -313,10 +313,10 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   for (int i = tid + kThreads; i < batch && i < kMaxSeqs; i += kThreads) s_len[i] = eff_len(seq_lens[i]);
   __syncthreads();
   if (tid == 0) {
-    // this CTA's range of the tiles (32-bit arithmetic: a step has fewer than 2^30 tiles, checked at creation)
+    // this CTA's range of the tiles (a step has fewer than 2^24 tiles, checked at creation: ckv_udiv24)
     unsigned T = 0;
     for (int i = 0; i < batch; ++i) T += (unsigned)seq_tiles(s_len, seq_lens, P, i) * (unsigned)P.Hkv;
-    const unsigned tpc = (T + (unsigned)nscan - 1u) / (unsigned)nscan;
+    const unsigned tpc = ckv_udiv24(T + (unsigned)nscan - 1u, (unsigned)nscan);
     const unsigned first = (unsigned)bid * tpc;
     const unsigned cnt = first >= T ? 0u : min(T - first, tpc);
     int u0 = 0, tl0 = 0, ulast = 0;
@@ -328,11 +328,12 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         if (t > 0) {
           if (!have_first && first < accum + t * (unsigned)P.Hkv) {
             const unsigned off = first - accum;
-            u0 = i * P.Hkv + (int)(off / t); tl0 = (int)(off % t);
+            const unsigned oq = ckv_udiv24(off, t);
+            u0 = i * P.Hkv + (int)oq; tl0 = (int)(off - oq * t);
             have_first = true;
           }
           if (first + cnt - 1u < accum + t * (unsigned)P.Hkv) {
-            ulast = i * P.Hkv + (int)((first + cnt - 1u - accum) / t);
+            ulast = i * P.Hkv + (int)ckv_udiv24(first + cnt - 1u - accum, t);
             break;
           }
         }
@@ -408,7 +409,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
       for (int idx = tid; idx < kStagedUnits * kPieces; idx += kConsumerWarps * 32) {
         const int k = idx / kPieces, pc = idx % kPieces, uu = s_u0 + k;
         if (uu <= s_ulast && uu < units) {
-          const int s2 = uu / P.Hkv, h2 = uu % P.Hkv;
+          const int s2 = ckv_div_hkv(P, uu), h2 = uu - s2 * P.Hkv;
           const uint4 *src = reinterpret_cast<const uint4 *>(q + ((size_t)s2 * P.Hq + h2 * G) * CKV_D);
           reinterpret_cast<uint4 *>(&s_q[k][0][0])[pc] = __ldg(src + pc);
         }
@@ -509,7 +510,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         if (cur >= 0) { write_partial(cur, true); next_empty = cur + 1; }
         fill_empty_upto(u);
         // per-unit setup: query fragments, variance weights, fresh accumulators
-        const int s = u / P.Hkv, h = u % P.Hkv;
+        const int s = ckv_div_hkv(P, u), h = u - s * P.Hkv;
         const QT *qrow = q + ((size_t)s * P.Hq + h * G + (hv ? head : 0)) * CKV_D;
         const int uk = u - s_u0;
         const bool from_smem = staged && uk < kStagedUnits;

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(kThreads) ckv_select_kernel(CkvDev P, const in
   __shared__ uint32_t s_candk[kThreads];   // the candidates' keys, so that the ranking loop reads no key through an id
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int unit = blockIdx.x, s = unit / P.Hkv;
+  const int unit = blockIdx.x, s = ckv_div_hkv(P, unit);
   const int N = max(min(seq_lens[s], P.max_blocks * P.bs), 0);
   const int X = (N + P.bs - 1) >> P.lg_bs;
   int *ids = sel_ids + (size_t)unit * kcap;

@@ -64,6 +64,7 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
   P.scan_tile = layout->stat_bf16 ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE;
   P.lg_bs = P.bs == 16 ? 4 : (P.bs == 32 ? 5 : 6);
   P.lg_tile = P.scan_tile == 32 ? 5 : 6;
+  P.hkv_magic = (unsigned)((1ull << 32) / (unsigned)P.Hkv) + 1u;   // unused when Hkv == 1 (where it wraps)
 
   // the partials of the largest split count the launch heuristic may pick must fit the fixed array
   const size_t per_split = (size_t)batch * P.Hkv * P.G * CKV_PART_STRIDE * sizeof(float);
