@@ -110,6 +110,9 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     cluster_wait();   // every CTA of the cluster has started
     const uint32_t rank = cluster_rank(), csize = cluster_size();
     const uint32_t recv0 = (uint32_t)__cvta_generic_to_shared(s_recv);
+    // g / csize for a head index g < 8, by counting (a division by the run-time cluster size is two dozen instructions,
+    // at the very end of the kernel's dependent chain)
+    auto div_c = [&](uint32_t g) { uint32_t qd_ = 0; for (uint32_t m = csize; m <= g; m += csize) ++qd_; return qd_; };
     constexpr int NP = (G * CKV_D + W * 32 - 1) / (W * 32);
     if (have) {
 #pragma unroll
@@ -117,14 +120,16 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
         const int idx = tid + it * W * 32;
         if (idx < G * CKV_D) {
           const uint32_t g = idx / CKV_D, c = idx % CKV_D;
-          const uint32_t ent = (g / csize) * csize + rank;
-          st_cluster_f32(cluster_map(recv0 + (ent * CKV_PART_STRIDE + 4 + c) * 4, g % csize), num[it]);
+          const uint32_t gq = div_c(g) * csize;
+          const uint32_t ent = gq + rank;
+          st_cluster_f32(cluster_map(recv0 + (ent * CKV_PART_STRIDE + 4 + c) * 4, g - gq), num[it]);
         }
       }
     }
     if (tid < G) {
-      const uint32_t ent = ((uint32_t)tid / csize) * csize + rank;
-      st_cluster_f32x2(cluster_map(recv0 + ent * kPartBytes, (uint32_t)tid % csize),
+      const uint32_t gq = div_c((uint32_t)tid) * csize;
+      const uint32_t ent = gq + rank;
+      st_cluster_f32x2(cluster_map(recv0 + ent * kPartBytes, (uint32_t)tid - gq),
                        have ? s_M[tid] : -CUDART_INF_F, have ? s_den[tid] : 0.f);
     }
     cluster_sync_all();   // release the stores, acquire everybody else's
@@ -159,7 +164,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
     if (CL) cluster_merge(nullptr, false);   // it still takes part in the cluster's merge, with an empty partial
     return;
   }
-  const int n_active = (total + pages_per_split - 1) / pages_per_split;   // splits of this unit that have pages
+  const int n_active = (int)ckv_udiv24((unsigned)(total + pages_per_split - 1), (unsigned)pages_per_split);   // splits of this unit that have pages
 
   unsigned char *wtiles = smem + (size_t)warp * 2 * kPageBytes;
   const uint32_t wtiles_u32 = (uint32_t)__cvta_generic_to_shared(wtiles);
@@ -365,7 +370,7 @@ ckv_attn_mma_kernel(CkvDev P, const __nv_bfloat16 *__restrict__ q, const __nv_bf
   if (comp) {
     int efirst = 0, n_comp = 0;   // where the unit's scan partials sit
     unit_scan_entries(P, CkvClampedLens{seq_lens, P.max_blocks * P.bs}, units, unit, scan_grid, lane, efirst, n_comp);
-    my_cnt = n_comp > (int)blockIdx.x ? (n_comp - (int)blockIdx.x + n_active - 1) / n_active : 0;
+    my_cnt = n_comp > (int)blockIdx.x ? (int)ckv_udiv24((unsigned)(n_comp - (int)blockIdx.x + n_active - 1), (unsigned)n_active) : 0;
     cp0 = P.comp_part + (size_t)efirst * G * CKV_PART_STRIDE;
   }
 

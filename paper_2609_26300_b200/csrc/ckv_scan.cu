@@ -484,17 +484,19 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
     // before it, hence the two sets of full barriers used by alternate rounds of the ring: together they tell four
     // consecutive fills of a stage apart.
     int it_at = 0;   // tile the (u, tl) walk stands at
+    uint32_t round = 0;   // the tile's place in the ring, kept by stepping (a division per visit would be two dozen instructions)
+    int st = 0;
     for (int pidx = warp; pidx < kParts * count; pidx += kConsumerWarps) {
       const int it = pidx / kParts;
       int half = pidx - it * kParts;
+      st += it - it_at;
+      while (st >= stages) { st -= stages; ++round; }
       for (; it_at < it; ++it_at) {
         if (++tl == ui.tiles) {
           tl = 0;
           do { ++u; } while (u < units && (ui = unit_info(P, s_len, seq_lens, u)).tiles == 0);
         }
       }
-      const uint32_t round = (uint32_t)(it / stages);
-      const int st = it - (int)round * stages;
       // a wait that runs out marks the step invalid (`aborted`); the walk still runs to the end
       if (!aborted) {
         bool fail = *(volatile int *)&s_abort != 0;
