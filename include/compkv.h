@@ -117,7 +117,10 @@ int ckv_last_cuda_error(void);
  * block; the count |b| is implied by seq_lens, so 2d + r 32-bit scalars are stored).
  * stats_bytes: block summaries for max_batch sequences.  workspace_bytes: scratch for one
  * decode step at max_batch (block log-weights, scores, split partials, host staging).
- * Host-only; validates the layout (CKV_ERR_BAD_LAYOUT). */
+ * Host-only; validates the layout (CKV_ERR_BAD_LAYOUT).  Besides the per-field ranges a layout must keep
+ * max_batch * num_kv_heads <= 65535, max_blocks_per_seq * block_size <= 2^30, and
+ * max_batch * num_kv_heads * ceil(max_blocks_per_seq / 32) < 2^24 (the kernels' index arithmetic is exact below that;
+ * summaries of that many blocks would need half a terabyte). */
 int ckv_query_sizes(const ckv_layout *layout, size_t *stats_bytes, size_t *workspace_bytes);
 
 /* Byte offsets, inside the stats buffer, of its three regions (the "selection region" holds
