@@ -67,12 +67,19 @@ def test_sizes_follow_the_summary_layout():
                                  dict(sm_scale=float("nan")), dict(max_blocks_per_seq=0), dict(variant=8),
                                  dict(variant=-1), dict(stat_bf16=2), dict(stat_bf16=1, kv_dtype=binding.CKV_F32),
                                  dict(stat_bf16=1, var_groups=128),
-                                 # more scan tiles per step than the kernels count in 32 bits
-                                 dict(max_batch=1 << 16, max_blocks_per_seq=1 << 21)])
+                                 # more scan tiles per step than the kernels' index arithmetic is exact for (2^24)
+                                 dict(max_batch=1 << 16, max_blocks_per_seq=1 << 21),
+                                 dict(max_batch=64, max_blocks_per_seq=1 << 20)])
 def test_bad_layouts_are_rejected(bad):
     with pytest.raises(binding.CompKVError) as e:
         binding.query_sizes(layout(**bad))
     assert e.value.status == binding.CKV_ERR_BAD_LAYOUT
+
+
+def test_layout_just_below_the_tile_limit_is_accepted():
+    # 64 sequences x 8 KV heads x (2^20 - 32) / 32 tiles = 2^24 - 512 tiles per step
+    stats, work = binding.query_sizes(layout(max_batch=64, max_blocks_per_seq=(1 << 20) - 32))
+    assert stats > 0 and work > 0
 
 
 @pytest.mark.parametrize("ok", [dict(var_groups=1), dict(var_groups=64), dict(var_groups=128), dict(block_size=64),
