@@ -55,6 +55,28 @@ def test_stats_build(bs, r, layout, dtype):
     assert d.ckv.read_status() == 0
 
 
+@pytest.mark.parametrize("bs", [32, 64])
+def test_blocks_of_several_pages_join_their_pages_exactly(bs):
+    """Closed form for the pairwise joining of a block's pages (Eq. 8 over a block longer than a page): every
+    16-token page holds one repeated key row, page p of a block at level p + 1 in every coordinate.  The block mean
+    is then the mean of the levels and the variance their population variance -- ((n^2 - 1) / 12 for levels 1..n, all
+    of it the joining term, since no page has any variance of its own) -- both exactly representable."""
+    w = small(batch=1, num_q_heads=4, num_kv_heads=1, block_size=bs, ctx=bs * 6, decode_steps=0, needles=0,
+              outlier_dims=0, shuffle_pages=False)
+    d = setup(w, var_groups=4)
+    ppb = bs // 16
+    for page in range(d.k_pool.shape[0]):
+        d.k_pool[page] = float(page % ppb + 1)
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    torch.cuda.synchronize()
+    km, db, vm = d.ckv.export_stats()
+    mean = (ppb + 1) / 2.0
+    var = (ppb * ppb - 1) / 12.0
+    assert torch.equal(km[0, 0, :6].cpu(), torch.full((6, 128), mean))
+    assert torch.equal(db[0, 0, :6].cpu(), torch.full((6, 4), var))
+    assert d.ckv.read_status() == 0
+
+
 @pytest.mark.parametrize("bs", [16, 32])
 def test_append_equals_rebuild_bit_for_bit(bs):
     steps = 40   # crosses block boundaries: a filled block, a rollover, a one-token block
