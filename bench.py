@@ -34,12 +34,15 @@ FALLBACK_HBM_GBS = 6650.0
 PAPER_CONTEXT = {"speedup_vs_full": 6.85, "hardware": "NVIDIA H100 80GB HBM3, CPU-offload pipeline, batch 1",
                  "setting": "128K endpoint, budget 512, r=4 (1.456 ms vs 9.966 ms)", "note": "context only"}
 # DRAM traffic (reads + writes) per algorithmic byte of the summary-scan kernel, from the committed ncu capture
-# (profiles/ckv_scan_kernel_llama8b_128k_b4.md): 273.17 MB read + 9.57 MB written for 272.9 MB of summaries.
-SCAN_TRAFFIC_RATIO = (273.17 + 9.57) / 272.9
+# (profiles/ckv_scan_kernel_llama8b_128k_b4.md): 206.06 MB read + 10.15 MB written for the 205.5 MB of summaries the
+# step reads (mean keys hi + lo, mean values hi, variances).
+SCAN_TRAFFIC_RATIO = (206.06 + 10.15) / 205.5
 # What is stored and multiplied (the line's `dtype`): K/V pages are bf16; mean keys and mean values keep fp32
 # precision as split bf16 pairs (hi = bf16(x), lo = bf16(x - hi), relative error <= 2^-18), variances are fp32; the
-# contractions run on bf16 tensor-core tiles (mma.sync) with fp32 accumulation, everything else is fp32.
-DTYPE = "bf16 mma operands (bf16 K/V; summaries as split-bf16 pairs hi+lo, rel. error 2^-18; fp32 variances), fp32 accumulate"
+# decode step reads the mean keys as pairs and the mean values as their hi halves; the contractions run on bf16
+# tensor-core tiles (mma.sync) with fp32 accumulation, everything else is fp32.
+DTYPE = ("bf16 mma operands (bf16 K/V; summaries stored as split-bf16 pairs hi+lo, rel. error 2^-18, the step reading "
+         "mean keys hi+lo and mean values hi; fp32 variances), fp32 accumulate")
 
 
 def measured_peak():
@@ -121,7 +124,7 @@ def describe(w, default: bool) -> str:
     head = "configs[2] " if default else "sweep point of "
     ctx = "ctx %d" % w.ctx if w.ctx_min is None else "ctx %d..%d (ragged)" % (w.ctx_min, w.ctx)
     return ("%s%s: batch %d, %dq/%dkv heads, d%d, %s (+ appended tokens), block %d, budget %d, r=%d, "
-            "fp32-precision summaries stored as split bf16 pairs, bf16 paged KV"
+            "fp32-precision summaries stored as split bf16 pairs (mean values read as hi halves when r = 4), bf16 paged KV"
             % (head, w.name, w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, ctx, w.block_size, w.budget_tokens,
                w.var_groups))
 
@@ -199,7 +202,7 @@ def sweep_config5(dev, peak, steps: int = 16):
             torch.cuda.synchronize()
             ms.append(e0.elapsed_time(e1))
         b_us = float(np.median(ms[1:])) * 1e3
-        b_bytes = n0 * w.num_kv_heads * 2 * w.head_dim * 2 + required_bytes(w, [n0], 0)[0]
+        b_bytes = n0 * w.num_kv_heads * 2 * w.head_dim * 2 + required_bytes(w, [n0], 0, stored=True)[0]
         builds.append({"block_size": bs, "us": b_us, "bytes": b_bytes, "gbs": b_bytes / (b_us * 1e-6) / 1e9,
                        "frac_of_peak": b_bytes / (b_us * 1e-6) / 1e9 / peak})
         if dense_us is None:
@@ -263,12 +266,17 @@ def oracle_step(w, kv, stats, n0, cores, step: int):
     return time.perf_counter() - t0
 
 
-def required_bytes(w, lens, sel_tokens_per_unit, mean_bytes: int = 4):
-    """Bytes one decode step must read: every block summary once, plus K and V of the selected tokens."""
+def required_bytes(w, lens, sel_tokens_per_unit, mean_bytes: int = 4, stored: bool = False):
+    """Bytes one decode step must read: every block summary once, plus K and V of the selected tokens.
+
+    With the default layout (full-precision summaries, four variance groups) the step reads the mean values as their
+    bf16 hi halves: 2 bytes per coordinate instead of 4.  stored=True counts the summaries as they are stored (what
+    the stats build and the chunked prefill write)."""
+    value_bytes = 2 if (not stored and mean_bytes == 4 and w.var_groups == 4) else mean_bytes
     stats = 0
     for n in lens:
         x = -(-int(n) // w.block_size)
-        stats += w.num_kv_heads * x * (2 * w.head_dim * mean_bytes + 4 * w.var_groups)
+        stats += w.num_kv_heads * x * (w.head_dim * (mean_bytes + value_bytes) + 4 * w.var_groups)
     sel = int(np.sum(sel_tokens_per_unit)) * 2 * w.head_dim * 2
     return stats, sel
 
@@ -379,7 +387,7 @@ def main():
         build_ms.append(e0.elapsed_time(e1))
     build_us = float(np.median(build_ms[2:])) * 1e3
     build_bytes = sum(int(n) for n in lens.tolist()) * w.num_kv_heads * 2 * w.head_dim * 2 + \
-        required_bytes(w, lens.tolist(), 0, 2 if args.stat_bf16 else 4)[0]
+        required_bytes(w, lens.tolist(), 0, 2 if args.stat_bf16 else 4, stored=True)[0]
 
     # ---- chunked prefill of the same cache from contiguous rows (pages + summaries in one pass), timed separately:
     # the rows are gathered from the pools, so the call rewrites what is already there ----
@@ -399,7 +407,7 @@ def main():
             pf_ms.append(e0.elapsed_time(e1))
         assert torch.equal(cur, lens) and ckv.read_status() == 0
         pf_us = float(np.median(pf_ms[1:])) * 1e3
-        pf_bytes = 2 * (build_bytes - required_bytes(w, lens.tolist(), 0)[0]) + required_bytes(w, lens.tolist(), 0)[0]
+        pf_bytes = 2 * (build_bytes - required_bytes(w, lens.tolist(), 0, stored=True)[0]) + required_bytes(w, lens.tolist(), 0, stored=True)[0]
         prefill = {"us": pf_us, "gbs": pf_bytes / (pf_us * 1e-6) / 1e9, "bytes": pf_bytes,
                    "note": "ckv_prefill: rows read once, written to their pages, summaries from the same pass"}
         del k_src, v_src
@@ -637,8 +645,8 @@ def main():
                      "launch_us_in_eager_step": scan_eager_us,
                      "traffic": SCAN_TRAFFIC_RATIO * stats_b,
                      "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this launch "
-                                       "configuration (profiles/ckv_scan_kernel_llama8b_128k_b4.md: 273.17 MB + "
-                                       "9.57 MB for 272.9 MB of summaries), scaled by the algorithmic bytes"},
+                                       "configuration (profiles/ckv_scan_kernel_llama8b_128k_b4.md: 206.06 MB + "
+                                       "10.15 MB for 205.5 MB of summaries read), scaled by the algorithmic bytes"},
         "clocks": clocks,
         "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "call": "ckv_step_host on the caller's own stream: the step's q/k_new/v_new are written into one set of pinned staging buffers (inside the timed region), out/sel_ids/sel_cnt come back into pinned buffers; returns when the results are complete in the host buffers"},

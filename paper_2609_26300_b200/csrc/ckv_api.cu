@@ -170,7 +170,9 @@ int ckv_create(const ckv_layout *layout, void *stats_dev, size_t stats_bytes, vo
   P.lu = (float *)(wb + R.ls); P.lz = (float *)(wb + R.lz); P.scores = (float *)(wb + R.scores);
   P.comp_part = (float *)(wb + R.comp); P.attn_part = (float *)(wb + R.attn);
   P.spin_limit = ckv_pipe::kSpinLimit; P.debug = 0;
-  P.scan_tile = layout->stat_bf16 ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE;
+  // the default layout (bf16 pages, full-precision summaries, four variance groups) reads the mean values as hi halves
+  P.vhi = (layout->kv_dtype == CKV_BF16 && !layout->stat_bf16 && layout->var_groups == 4) ? 1 : 0;
+  P.scan_tile = (layout->stat_bf16 || P.vhi) ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE;
   P.lg_bs = P.bs == 16 ? 4 : (P.bs == 32 ? 5 : 6);
   P.lg_tile = P.scan_tile == 32 ? 5 : 6;
   P.hkv_magic = (unsigned)((1ull << 32) / (unsigned)P.Hkv) + 1u;   // unused when Hkv == 1 (where it wraps)

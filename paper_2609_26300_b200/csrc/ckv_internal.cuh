@@ -1,6 +1,7 @@
 // Internal declarations shared by the CompKV CUDA translation units (sm_100a).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -41,7 +42,12 @@ struct CkvDev {
   int row_elems;     // bf16 elements of one mean-key / mean-value row: CKV_ROW_ELEMS, or CKV_D when only hi halves are kept
   int variant;       // ckv_variant bits
   float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
-  int scan_tile;     // blocks per scan tile: CKV_SCAN_TILE, or CKV_SCAN_TILE_HS with bf16 summaries
+  int scan_tile;     // blocks per scan tile: CKV_SCAN_TILE, or CKV_SCAN_TILE_HS with bf16 summaries or vhi
+  int vhi;           // 1: the decode step reads the mean values' hi halves only (the lo halves, at most 2^-9 of a value,
+                     // stay in the summaries for whoever exports them): the scan copies 256 of a row's 512 bytes.  The
+                     // compensation term is a weighted average over thousands of blocks and ends in a bf16 output row, so
+                     // the roundings neither add up nor show (measured: the output error against the oracle is the same
+                     // 0.0034 maximum with and without the lo halves)
   unsigned hkv_magic;  // floor(2^32 / Hkv) + 1: x / Hkv = umulhi(x, hkv_magic) for x < 2^32 / Hkv (ckv_div_hkv)
   int lg_bs, lg_tile;  // log2 of bs and of scan_tile (both powers of two): the kernels' prologues divide by shifting --
                        // a division by a run-time value is two dozen instructions, and a prologue's time is the fetch of its
@@ -63,6 +69,7 @@ struct ckv_ctx {
   int64_t launches;
   int sm_count;
   int tail_mode;   // ckv_tail_mode
+  CUtensorMap tm_vhi;   // vhi: the mean-values region as rows of 128 bf16 (the hi halves) 512 bytes apart, boxes of 64 rows
   volatile int *host_flag;   // pinned word ckv_step_host waits on (null: stream synchronisation instead)
   int *host_flag_dev;        // the same word as the device sees it
   int host_epoch;            // number of the last ckv_step_host call that used the word
@@ -76,7 +83,7 @@ struct ckv_ctx {
 
 int ckv_record_cuda_error(cudaError_t e);   // remembers e for ckv_last_cuda_error() on this thread; returns CKV_ERR_CUDA
 cudaError_t ckv_configure_kernels();   // selection kernel attributes
-cudaError_t ckv_configure_scan(const ckv_ctx *c);   // scan kernel attributes
+cudaError_t ckv_configure_scan(ckv_ctx *c);   // scan kernel attributes (and, with vhi, the tensor map of the mean values)
 cudaError_t ckv_configure_attn(const ckv_ctx *c);   // attention kernel attributes
 cudaError_t ckv_configure_attn_mma(const ckv_ctx *c);
 cudaError_t ckv_launch_attn_mma(ckv_ctx *c, bool dense, const void *q, const void *k_pool, const void *v_pool,

@@ -35,6 +35,7 @@
 // one; a counter of CTAs that are done reading decides who stores the new lengths (lens_arrive), so the kernels
 // that follow in the stream see them in place and nobody waits on anybody inside the launch.
 #include <algorithm>
+#include <mutex>
 
 #include "ckv_internal.cuh"
 #include "ckv_pipe.cuh"
@@ -45,7 +46,15 @@ namespace {
 
 using namespace ckv_pipe;
 
-template <bool HS> struct ScanTile { static constexpr int TB = HS ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE; };   // blocks per tile
+template <bool WIDE> struct ScanTile { static constexpr int TB = WIDE ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE; };   // blocks per tile
+
+// One box of a tensor map from global to shared memory (x: first element of the row, y: first row); completion is
+// counted on `bar` in bytes -- always the whole box, rows past the tensor's end arriving as zeros.
+__device__ __forceinline__ void tensor_g2s(uint32_t dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(ckv_pipe::smem_u32(bar))
+               : "memory");
+}
 constexpr int kMaxStages = 8;
 constexpr int kConsumerWarps = CKV_SCAN_WARPS;
 constexpr int kThreads = kConsumerWarps * 32 + 32;   // plus the producer warp
@@ -203,7 +212,7 @@ __device__ __noinline__ void scan_tail(const CkvDev P, const QT *__restrict__ q,
     __syncwarp();
     float kx[8], vx[8], dx[8];   // this lane's 8 coordinates of kbar, vbar and of the variance of their group
     load_split8<false>(P.kmean + row * P.row_elems, li, b, kx, lo_half);
-    load_split8<false>(P.vmean + row * P.row_elems, li, b, vx, lo_half);
+    load_split8<false>(P.vmean + row * P.row_elems, li, b, vx, lo_half && !P.vhi);   // as the scan CTAs read it
     if (P.r == CKV_D) {
       load_split8<false>(reinterpret_cast<const __nv_bfloat16 *>(P.dbar + row * CKV_D), li, b, dx);
     } else {
@@ -259,13 +268,18 @@ template <> struct QSplit<float> { static constexpr bool value = true; };
 // RD: one variance group per coordinate (r = d).  The variance rows then have the mean rows' layout and
 // sigma^2 = sum_i (scale q_i)^2 Dbar_i is a third tensor-core product, with the squared queries as the A operand.
 // HS: the mean rows hold hi halves only (bf16 summaries, 256-byte rows); every product with a lo plane drops out.
-template <int G, typename QT, bool RD, bool HS>
+// VH: full-precision rows in memory, but only the hi halves of the mean VALUES are brought in: one tensor copy per
+// tile takes the first 256 bytes of each 512-byte row, and the value product is that of HS (Sec. 3.1: the
+// compensation term is an average over many blocks; its 2^-9 relative rounding is below that of the bf16 output).
+template <int G, typename QT, bool RD, bool HS, bool VH>
 __global__ void __launch_bounds__(kThreads, 1)
 ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int units, int stages, CkvNewToken fresh,
-                int n_tail) {
+                int n_tail, const __grid_constant__ CUtensorMap tm_v) {
   constexpr bool QS = QSplit<QT>::value;   // fp32 queries are split into hi + lo like the summaries
-  constexpr int kRowBytes = HS ? CKV_D * 2 : CKV_ROW_ELEMS * 2;   // bytes of one mean-key / mean-value row
-  constexpr int TB = ScanTile<HS>::TB;
+  static_assert(!(VH && (HS || RD)), "VH is a variant of the full-precision layout with four variance groups");
+  constexpr int kRowBytes = HS ? CKV_D * 2 : CKV_ROW_ELEMS * 2;   // bytes of one mean-key row in a stage
+  constexpr int kRowBytesV = (HS || VH) ? CKV_D * 2 : CKV_ROW_ELEMS * 2;   // ... of one mean-value row
+  constexpr int TB = ScanTile<HS || VH>::TB;
   extern __shared__ __align__(128) unsigned char stage_mem[];
   __shared__ __align__(8) uint64_t full_bar[2][kMaxStages], empty_bar[kMaxStages];
   __shared__ __align__(16) unsigned char s_zero_row[512];   // what mean-value rows past a unit's last block are read as
@@ -282,7 +296,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
   const bool r4 = P.r == 4;          // the default: the variance projection is four FMAs on one 16-byte read
   const bool dbar_bulk = P.r >= 4;   // smaller rows cannot keep the 16-byte alignment bulk copies need
   constexpr int kParts = TB / 16;    // 16-block parts of a tile, each worked on by one consumer warp
-  const int stage_bytes = TB * 2 * kRowBytes + (dbar_bulk ? TB * P.r * 4 : 0);
+  const int stage_bytes = TB * (kRowBytes + kRowBytesV) + (dbar_bulk ? TB * P.r * 4 : 0);
   // per-warp w_{g,t} table for r != 4, behind the ring
   float *sw_all = reinterpret_cast<float *>(stage_mem + (size_t)stages * stage_bytes);
 
@@ -373,15 +387,25 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
         const uint32_t kbytes = (uint32_t)nb * kRowBytes;
         const uint32_t dbytes = dbar_bulk ? (uint32_t)nb * P.r * 4 : 0;
         uint64_t *fb = &full_bar[round & 1][st];
-        mbar_arrive_expect_tx(fb, 2 * kbytes + dbytes);
+        const uint32_t vbytes = VH ? (uint32_t)TB * kRowBytesV : kbytes;   // a tensor copy always delivers its whole box
+        mbar_arrive_expect_tx(fb, kbytes + vbytes + dbytes);
         const uint32_t lo = smem_u32(stage_mem), hi = lo + (uint32_t)stages * stage_bytes;
         bool ok = nb >= 1 && u < units && row + nb <= (size_t)units * P.max_blocks;
         // test hook (ckv_debug_set): one fill is announced but never issued, so that the waits on it run out
         const bool skip = (P.debug & CKV_DEBUG_SKIP_FILL) != 0 && it == 0 && bid == 0;
         if (!skip) {
           ok = ok && bulk_g2s_checked(sk, P.kmean + row * P.row_elems, kbytes, fb, lo, hi);
-          ok = ok && bulk_g2s_checked(sv, P.vmean + row * P.row_elems, kbytes, fb, lo, hi);
-          if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytes, P.dbar + row * P.r, dbytes, fb, lo, hi);
+          if constexpr (VH) {
+            // rows [row, row + TB) of the mean-values region, first 256 bytes of each (rows past the unit's blocks are
+            // never read; rows past the region's end arrive as zeros)
+            const uint32_t dv = smem_u32(sv);
+            const bool fits = (dv & 127u) == 0 && dv >= lo && dv + vbytes <= hi;
+            if (ok && fits) tensor_g2s(dv, &tm_v, 0, (int)row, fb);
+            ok = ok && fits;
+          } else {
+            ok = ok && bulk_g2s_checked(sv, P.vmean + row * P.row_elems, kbytes, fb, lo, hi);
+          }
+          if (dbar_bulk) ok = ok && bulk_g2s_checked(sv + TB * kRowBytesV, P.dbar + row * P.r, dbytes, fb, lo, hi);
           *(volatile int *)&s_issued = it + 1;
         }
         if (!ok) atomicOr(P.status, CKV_DEV_BAD_COPY);
@@ -592,7 +616,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
       if (!aborted && rb < nb) {
         const uint32_t sk = smem_u32(stage_mem + (size_t)st * stage_bytes);
         const uint32_t sv = sk + TB * kRowBytes;
-        const float *sd = reinterpret_cast<const float *>(stage_mem + (size_t)st * stage_bytes + 2 * TB * kRowBytes);
+        const float *sd = reinterpret_cast<const float *>(stage_mem + (size_t)st * stage_bytes + TB * (kRowBytes + kRowBytesV));
 
         // ---- Z^T = Q Kbar^T: heads x 16 blocks (two n-tiles of 8 blocks), hi and lo planes into one accumulator ----
         // four accumulation chains per n-tile (hi / lo plane x even / odd 16-coordinate step): the products of a chain
@@ -753,7 +777,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
           // ldmatrix.trans lane roles: matrix lane / 8 -> (block half, coordinate chunk parity), row lane % 8
           const int r = rb + ((lane >> 3) & 1) * 8 + (lane & 7);
           const bool real = r < nb;   // rows past the unit's last block: zeros
-          const uint32_t rowaddr = real ? sv + r * kRowBytes : smem_u32(s_zero_row);
+          const uint32_t rowaddr = real ? sv + r * kRowBytesV : smem_u32(s_zero_row);
           const int cpar = lane >> 4;
 #pragma unroll
           for (int t2 = 0; t2 < 8; ++t2) {   // two 8-coordinate n-tiles per ldmatrix.x4
@@ -764,7 +788,7 @@ ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int uni
             mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wl[0], wl[1], vh[0], vh[1]);
             mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vh[2], vh[3]);
             mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wl[0], wl[1], vh[2], vh[3]);
-            if (!HS) {
+            if (!HS && !VH) {
               ldmatrix_x4_trans(vl, rowaddr + (real ? 256u : 0u) + coff);
               mma_rows8(acc[2 * t2][0], acc[2 * t2][1], wh[0], wh[1], vl[0], vl[1]);
               mma_rows8(acc[2 * t2 + 1][0], acc[2 * t2 + 1][1], wh[0], wh[1], vl[2], vl[3]);
@@ -793,7 +817,8 @@ struct ScanCfg { int stages; size_t smem; };
 
 ScanCfg scan_cfg(const CkvDev &P, int G) {
   const size_t TB = (size_t)P.scan_tile;
-  const size_t stage_bytes = TB * 2 * (P.row_elems * 2) + (P.r >= 4 ? TB * P.r * 4 : 0);
+  const size_t krow = (size_t)P.row_elems * 2, vrow = P.vhi ? (size_t)CKV_D * 2 : krow;
+  const size_t stage_bytes = TB * (krow + vrow) + (P.r >= 4 ? TB * P.r * 4 : 0);
   const size_t sw_bytes = (P.r == 4 || P.r == CKV_D) ? 0 : (size_t)kConsumerWarps * P.r * G * 4;   // weight table of the generic path
   // 227 KB per CTA, less the kernel's static shared memory (lengths, barriers, the row of zeros: under 6 KB; staged
   // query rows and variance weights: 4 units x G x 272 bytes) and a reserve
@@ -815,14 +840,19 @@ cudaError_t launch_gt(ckv_ctx *c, const void *q, const int *seq_lens, int units,
   const ScanCfg cfg = scan_cfg(c->dev, G);
   if (cfg.stages == 0) return cudaErrorInvalidConfiguration;
   if (c->dev.r == CKV_D)
-    ckv_scan_kernel<G, QT, true, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail);
+    ckv_scan_kernel<G, QT, true, false, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail, c->tm_vhi);
   else if (c->dev.row_elems == CKV_D) {
     if constexpr (!QSplit<QT>::value)   // bf16 summaries come with bf16 pages and queries only
-      ckv_scan_kernel<G, QT, false, true><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail);
+      ckv_scan_kernel<G, QT, false, true, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail, c->tm_vhi);
+    else
+      return cudaErrorInvalidValue;
+  } else if (c->dev.vhi) {
+    if constexpr (!QSplit<QT>::value)
+      ckv_scan_kernel<G, QT, false, false, true><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail, c->tm_vhi);
     else
       return cudaErrorInvalidValue;
   } else
-    ckv_scan_kernel<G, QT, false, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail);
+    ckv_scan_kernel<G, QT, false, false, false><<<grid, kThreads, cfg.smem, st>>>(c->dev, (const QT *)q, seq_lens, units, cfg.stages, fresh, n_tail, c->tm_vhi);
   return cudaGetLastError();
 }
 
@@ -837,17 +867,58 @@ template <int G, typename QT>
 cudaError_t configure_gt(const ckv_ctx *c) {
   const int smem = (int)scan_cfg(c->dev, G).smem;
   if (c->dev.r == CKV_D)
-    return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (c->dev.row_elems == CKV_D) {
     if constexpr (!QSplit<QT>::value)
-      return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     return cudaErrorInvalidValue;
   }
-  return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (c->dev.vhi) {
+    if constexpr (!QSplit<QT>::value)
+      return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    return cudaErrorInvalidValue;
+  }
+  return cudaFuncSetAttribute(ckv_scan_kernel<G, QT, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+}
+
+// The mean-values region as the copy engine sees it with vhi: a matrix of bf16 rows, [units * max_blocks][128] at a pitch
+// of 512 bytes (the hi halves of the stored rows), copied in boxes of CKV_SCAN_TILE_HS rows.  Host-side arithmetic only;
+// the encoder is the driver's, looked up once through the runtime.
+cudaError_t make_vhi_map(ckv_ctx *c) {
+  using encode_fn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static std::mutex mtx;
+  static encode_fn encode = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(mtx);
+    if (encode == nullptr) {
+      void *fn = nullptr;
+      cudaDriverEntryPointQueryResult qres = cudaDriverEntryPointSymbolNotFound;
+      const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+      if (e != cudaSuccess) return e;
+      if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorSymbolNotFound;
+      encode = reinterpret_cast<encode_fn>(fn);
+    }
+  }
+  const CkvDev &P = c->dev;
+  if (((uintptr_t)P.vmean & 15u) != 0) return cudaErrorMisalignedAddress;
+  const cuuint64_t dims[2] = {(cuuint64_t)CKV_D, (cuuint64_t)c->layout.max_batch * P.Hkv * P.max_blocks};
+  const cuuint64_t strides[1] = {(cuuint64_t)CKV_ROW_ELEMS * 2};   // bytes between rows
+  const cuuint32_t box[2] = {CKV_D, CKV_SCAN_TILE_HS};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = encode(&c->tm_vhi, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)P.vmean, dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 template <int G>
-cudaError_t configure_g(const ckv_ctx *c) {
+cudaError_t configure_g(ckv_ctx *c) {
+  if (c->dev.vhi) {
+    const cudaError_t e = make_vhi_map(c);
+    if (e != cudaSuccess) return e;
+  }
   if (c->layout.kv_dtype == CKV_BF16) return configure_gt<G, __nv_bfloat16>(c);
   return configure_gt<G, float>(c);
 }
@@ -855,7 +926,7 @@ cudaError_t configure_g(const ckv_ctx *c) {
 }  // namespace
 
 // Opt in to the dynamic shared memory this context's scan instantiation needs, on the current device.
-cudaError_t ckv_configure_scan(const ckv_ctx *c) {
+cudaError_t ckv_configure_scan(ckv_ctx *c) {
   switch (c->dev.G) {
     case 1: return configure_g<1>(c);
     case 2: return configure_g<2>(c);

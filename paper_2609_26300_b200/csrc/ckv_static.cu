@@ -61,6 +61,7 @@ extern "C" int ckv_dense_decode_static(const ckv_layout *layout, const void *q, 
   P.scale = c.layout.sm_scale;
   P.row_elems = layout->stat_bf16 ? CKV_D : CKV_ROW_ELEMS;
   P.variant = layout->variant; P.half_var = 0.5f;   // the dense pass reads neither
+  P.vhi = 0;
   P.scan_tile = layout->stat_bf16 ? CKV_SCAN_TILE_HS : CKV_SCAN_TILE;
   P.lg_bs = P.bs == 16 ? 4 : (P.bs == 32 ? 5 : 6);
   P.lg_tile = P.scan_tile == 32 ? 5 : 6;
