@@ -98,7 +98,10 @@ typedef struct ckv_layout {
   int32_t recent_blocks;      /* mandatory trailing blocks (Sec. 4.2: 2) */
   float   sm_scale;           /* logit scale; 0 means 1/sqrt(head_dim) (Sec. 3.1) */
   int32_t variant;            /* OR of ckv_variant bits; 0 = the method as printed */
-  int32_t stat_bf16;          /* 0: mean keys / mean values kept at fp32 precision (the paper's choice, Sec. 4.3);
+  int32_t stat_bf16;          /* 0: mean keys / mean values kept at fp32 precision (the paper's choice, Sec. 4.3).  A
+                                 decode step reads the mean keys and variances in full; with kv_dtype CKV_BF16 and
+                                 var_groups 4 it reads the mean values at bf16 precision (the compensation term of
+                                 Eq. 12 ends in a bf16 output row; the stored summaries keep their precision);
                                  1: kept as bf16 (half the summary bytes; block scores then differ from the fp32
                                  layout's by up to ~1e-2 relative).  Needs kv_dtype CKV_BF16 and
                                  var_groups < head_dim.  Variances stay fp32. */
