@@ -457,6 +457,7 @@ def main():
     sel_cnt = outputs[3].cpu().numpy()
     lens_now = lens.cpu().numpy()
     stats_b, sel_b = required_bytes(w, lens_now, sel_cnt * w.block_size, 2 if args.stat_bf16 else 4)
+    stats_stored_b = required_bytes(w, lens_now, 0, 2 if args.stat_bf16 else 4, stored=True)[0]
     assert ckv.read_status() == 0
 
     # ---- per-kernel durations (events between the launches), L2 flushed before each step ----
@@ -616,10 +617,15 @@ def main():
         "multi_layer": multi,
         "us_per_step_note": "value: one graph replay per event pair, L2 flushed before it (includes the launch latency "
                             "of the graph); warm_l2: same without the flush; back_to_back: 64 replays queued inside "
-                            "one event pair, no flush (every step still streams 273 MB of summaries through a "
-                            "126 MB L2)",
+                            "one event pair, no flush (every step still streams its summaries, more than the 126 MB L2 holds, "
+                            "through it)",
         "tokens_per_s": rep.aggregate_tokens_per_s(w.batch, us_per_step),
         "required_bytes_per_step": req, "hbm_gbs": step_gbs,
+        "required_bytes_note": "summary bytes the step reads (mean keys hi + lo, variances, and -- default layout -- the "
+                               "mean values' hi halves) + K/V of the selected tokens; with whole summary rows, as the "
+                               "summaries are stored, the count would be required_bytes_whole_rows",
+        "required_bytes_whole_rows": int(stats_stored_b + sel_b),
+        "frac_of_%s_peak_on_whole_rows" % peak_kind: (stats_stored_b + sel_b) / (us_per_step * 1e-6) / 1e9 / peak,
         "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS, "frac_of_%s_peak" % peak_kind: step_gbs / peak,
         "dense_us": dense_us, "dense_gbs": dense_bytes / (dense_us * 1e-6) / 1e9,
         "speedup_vs_dense": dense_us / us_per_step,
