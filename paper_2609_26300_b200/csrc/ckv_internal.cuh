@@ -43,7 +43,7 @@ struct CkvDev {
   int variant;       // ckv_variant bits
   float half_var;    // coefficient of sigma^2 in the estimated log mass: 0.5 (Eq. 9), or 0 for the first-order mass
   int scan_tile;     // blocks per scan tile: CKV_SCAN_TILE, or CKV_SCAN_TILE_HS with bf16 summaries or vhi
-  int vhi;           // 1: the decode step reads the mean values' hi halves only (the lo halves, at most 2^-9 of a value,
+  int vhi;           // 1: the decode step reads the mean values' hi halves only (the lo halves, at most 2^-8 of a value,
                      // stay in the summaries for whoever exports them): the scan copies 256 of a row's 512 bytes.  The
                      // compensation term is a weighted average over thousands of blocks and ends in a bf16 output row, so
                      // the roundings neither add up nor show (measured: the output error against the oracle is the same

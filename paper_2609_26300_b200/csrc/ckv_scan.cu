@@ -270,7 +270,8 @@ template <> struct QSplit<float> { static constexpr bool value = true; };
 // HS: the mean rows hold hi halves only (bf16 summaries, 256-byte rows); every product with a lo plane drops out.
 // VH: full-precision rows in memory, but only the hi halves of the mean VALUES are brought in: one tensor copy per
 // tile takes the first 256 bytes of each 512-byte row, and the value product is that of HS (Sec. 3.1: the
-// compensation term is an average over many blocks; its 2^-9 relative rounding is below that of the bf16 output).
+// compensation term is an average over many blocks; its rounding, at most half a bf16 step per block and of varying sign, is within that of the
+// bf16 output).
 template <int G, typename QT, bool RD, bool HS, bool VH>
 __global__ void __launch_bounds__(kThreads, 1)
 ckv_scan_kernel(CkvDev P, const QT *__restrict__ q, const int *seq_lens, int units, int stages, CkvNewToken fresh,

@@ -286,6 +286,35 @@ def test_exact_ties_go_to_lower_block_ids():
             assert b in got
 
 
+def test_mean_values_read_as_hi_halves_worst_case():
+    """The decode step of the default layout reads the mean values at bf16 precision (their hi halves).  Worst case
+    for that: every block mean sits half a bf16 step above a representable value, in every coordinate and with the
+    same sign (tokens alternate between 1 and 1 + 2^-7, mean 1 + 2^-8), and a small budget leaves most of the mass
+    to the compensation term.  The output may then be off by that half step, 2^-8 relative, on top of the half step
+    of its own bf16 rounding -- no more."""
+    w = small(batch=1, num_q_heads=4, num_kv_heads=1, ctx=16 * 96, decode_steps=0, needles=0, outlier_dims=0,
+              shuffle_pages=False)
+    d = setup(w)
+    d.v_pool[:, :, 0::2, :] = 1.0
+    d.v_pool[:, :, 1::2, :] = 1.0 + 2.0 ** -7
+    d.ckv.stats_build(d.k_pool, d.v_pool, d.table, d.lens, d.max_len)
+    km, db, vm = d.ckv.export_stats()
+    assert torch.equal(vm[0, 0, :96].cpu(), torch.full((96, 128), 1.0 + 2.0 ** -8))   # the stored summaries keep it
+    out, lse, ids, cnt, scores = run_decode(d, 16 * 6)
+    K = d.k_pool[:96, 0].float().reshape(-1, 128).cpu().numpy()
+    V = d.v_pool[:96, 0].float().reshape(-1, 128).cpu().numpy()
+    q = synth.queries(w)[0]
+    st = O.stats(K, V, 16)
+    osc = O.scores(q, st)
+    ref_ids = O.select(osc.S, 6)
+    got = ids[0, 0, :int(cnt[0, 0])].cpu().numpy()
+    same = check_ids(got, ref_ids, osc.S, 6)
+    ref_out, ref_lse = O.sparse(q, K, V, st, ref_ids if same else got)
+    err = rel_inf(out[0].double().cpu().numpy(), ref_out)
+    assert err <= 2.0 ** -8 + 2.0 ** -8 + 1e-4, err
+    assert float(np.abs(lse[0].double().cpu().numpy() - ref_lse).max()) <= 1e-4
+
+
 # ---- edge cases ---------------------------------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("n", [1, 15, 16, 17, 47, 48, 49])
