@@ -963,8 +963,8 @@ int ckv_scan_grid(const ckv_ctx *c, int batch, int max_len) {
 
 // Tail mode pays when the scan is long enough to hide the tail CTAs.  A tail warp's work is a chain of dependent
 // cache misses behind the scan's traffic plus a few thousand instructions run once by a single warp: measured from
-// launch, a round of tail work ends after 15 - 20 us without a new token and after 27 us (idle DRAM, 32K cache) to
-// 45 us (beside a saturating 128K scan) with one, whereas the scan streams about 5 MB per microsecond.  Below that
+// launch, a round of tail work ends after 15 - 20 us without a new token and after 20 - 25 us with one (45 us before
+// the routine's cold instructions were trimmed), whereas the scan streams about 5 MB per microsecond.  Below that
 // size the scan CTAs cover every block and the append is a launch of its own, whose warps all run at once.
 bool ckv_scan_wants_tail(const ckv_ctx *c, int batch, int max_len) {
   if (batch > kMaxSeqs || c->tail_mode == CKV_TAIL_OFF) return false;   // the lengths must fit the staging array
@@ -975,10 +975,12 @@ bool ckv_scan_wants_tail(const ckv_ctx *c, int batch, int max_len) {
   const int n_tail = one_round <= 16 ? std::max(1, one_round) : std::min((units + 15) / 16, std::max(16, c->sm_count / 4));
   const int rounds = (units + 8 * n_tail - 1) / (8 * n_tail);
   const double blocks = (double)units * ((max_len + P.bs - 1) / P.bs);
-  const double bytes = blocks * (2.0 * P.row_elems * 2 + 4.0 * P.r);
-  // scan microseconds: bandwidth-bound at about 5 MB/us, or issue-bound at about 6000 blocks/us (bf16 summaries)
+  const double bytes = blocks * (P.row_elems * 2.0 + (P.vhi ? CKV_D * 2.0 : P.row_elems * 2.0) + 4.0 * P.r);   // what the scan reads
+  // scan microseconds: bandwidth-bound at about 5 MB/us, or issue-bound at about 6000 blocks/us (bf16 summaries).
+  // A round of tail work with a new token ends 20 - 25 us after launch; measured crossover at 128K, 8 KV heads: three
+  // sequences (scan about 30 us) gain a microsecond from tail mode, two (about 20 us) lose four.
   const double scan_us = std::max(bytes / 5.0e6, blocks / 6.0e3);
-  return scan_us >= 40.0 * rounds;
+  return scan_us >= 30.0 * rounds;
 }
 
 cudaError_t ckv_launch_scan(ckv_ctx *c, const void *q, const int *seq_lens, int batch, int max_len,
