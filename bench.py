@@ -299,8 +299,9 @@ def reference_arm(args):
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "configs[2] llama8b_128k_b4: batch 4, 32q/8kv heads, d128, ctx 131072, "
-                                   "block 16, budget 2048", "sample": sample},
+            # the same workload string as the other arm's line (the oracle works on it in fp64; how the CUDA path stores
+            # its summaries is part of that string because it is part of the workload's name there)
+            "config": {"workload": describe(w, True), "sample": sample},
             "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
