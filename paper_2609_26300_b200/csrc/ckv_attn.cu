@@ -466,6 +466,20 @@ cudaError_t ckv_launch_attn(ckv_ctx *c, bool dense, const void *q, const void *k
   // Splits per unit: the dense pass (and the fp32 kernel) get about four CTAs per SM overall; the tensor-core
   // kernel's sparse mode is sized below.  At most CKV_MAX_SPLITS splits.
   int n_splits = (sms * 4 + units - 1) / units;
+  if (dense && mma) {
+    // One 8-warp CTA per SM: the grid runs in waves, and a last wave that is mostly empty costs a whole wave's time
+    // (19 splits of 32 units = 608 CTAs = 4.1 waves took 352 us; 9 or 18 splits, 1.95 and 3.9 waves, 320 us).  Among
+    // 1.5 to 4.2 CTAs per SM, the split count whose last wave is fullest (the larger one on a tie) replaces the
+    // rule above where it fills the waves at least a tenth better and its splits stay long (200 pages): short
+    // splits are bound by their own latency, not by the waves (32K, one sequence: 43 us with 64 splits, 47 with 37).
+    n_splits = min(n_splits, CKV_MAX_SPLITS);
+    auto fill = [&](int n) { const long long ctas = (long long)units * n; return (double)ctas / (double)((ctas + sms - 1) / sms * sms); };
+    const int lo = max(1, (3 * sms + 2 * units - 1) / (2 * units)), hi = min(max(lo, 42 * sms / (10 * units)), CKV_MAX_SPLITS);
+    int best = lo;
+    for (int n = lo; n <= hi; ++n)
+      if (fill(n) >= fill(best)) best = n;
+    if (fill(best) >= 1.1 * fill(n_splits) && total / best >= 200) n_splits = best;
+  }
   if (mma && !dense) {
     // Up to 8 splits of a unit run as one cluster and merge in shared memory.  With so few units that 8 splits each
     // would leave most SMs idle, many short splits (merged through global memory) finish sooner.
